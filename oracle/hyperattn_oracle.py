@@ -1,0 +1,389 @@
+"""CPU oracle for the HyperAttention forward pass (Han et al., arXiv 2310.05869).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain, fp64 statement of what
+the hot path computes.  It shares no code with the CUDA library and must never be
+imported by the product path: only the tests, the smoke check and the benchmark's
+CPU-baseline leg may call it.
+
+Every function names the passage of the paper it follows.  Where the paper is
+silent the reading taken is stated in the docstring (the same readings are listed
+in the design notes of the repository).
+
+Stages (paper notation: Q, K, V are n x d; b block size; m sampled columns;
+r hash bits; P_Q, P_K the sortLSH permutations; M^H the block mask):
+
+  philox4x32_10      counter-based random words (Salmon et al., SC'11) used for
+                     the hash directions and the sampled columns
+  directions         r Gaussian directions of the Hamming-sorted LSH (Def. 1)
+  bucket_ids         sign pattern -> Gray-ordered bucket id (Def. 1, Alg. 1 line 2)
+  stable_argsort     permutations P_Q, P_K (Alg. 1 line 3)
+  sortlsh_mask       the mask M^H (Alg. 1 line 4)
+  sample_indices     l_1..l_m ~ Unif([N]) shared by all rows (Alg. 2 line 4, Sec. 4)
+  exact_attention    D^-1 A V and its causal form (Sec. 1.1, Sec. 3.1)
+  node_forward       block-diagonal part + sampled residual with estimated D
+                     (Alg. 2 lines 7 and 9 without caps, Alg. 3, Sec. 4)
+  causal_forward     recursive split (Alg. 4) carried through to outputs
+  forward            all (batch, head) segments
+  dense_weights      the implied n x n row-stochastic weight matrix (tiny n only)
+
+Parity status: every function here is pinned by the CPU tests (brute force on tiny
+inputs, closed forms, the Fig. 1 example, Monte-Carlo checks, published Philox
+known-answer vectors).  The spectral guarantee Eq. (1) is NOT a pin: the paper
+never gives epsilon a value ("parity unpinned" for Eq. (1) only; nothing on the
+hot path depends on it).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+# --------------------------------------------------------------------------------------
+# Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3")
+# --------------------------------------------------------------------------------------
+_PHILOX_M0 = np.uint64(0xD2511F53)
+_PHILOX_M1 = np.uint64(0xCD9E8D57)
+_PHILOX_W0 = np.uint64(0x9E3779B9)
+_PHILOX_W1 = np.uint64(0xBB67AE85)
+_MASK32 = np.uint64(0xFFFFFFFF)
+_SHIFT32 = np.uint64(32)
+
+DOMAIN_DIRECTIONS = 1
+DOMAIN_SAMPLES = 2
+
+
+def philox4x32_10(counter, key):
+    """Ten rounds of Philox-4x32.  `counter` is (..., 4) and `key` is (2,) of 32-bit words.
+
+    One round: (hi0, lo0) = M0 * c0, (hi1, lo1) = M1 * c2 (32x32 -> 64 bit products);
+    c <- (hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0); the key is bumped by the Weyl
+    constants between rounds.  Returns (..., 4) uint32.
+    """
+    c = np.asarray(counter, dtype=np.uint64) & _MASK32
+    c0, c1, c2, c3 = (c[..., i].copy() for i in range(4))
+    k0 = np.uint64(int(key[0]) & 0xFFFFFFFF)
+    k1 = np.uint64(int(key[1]) & 0xFFFFFFFF)
+    for rnd in range(10):
+        if rnd > 0:
+            k0 = (k0 + _PHILOX_W0) & _MASK32
+            k1 = (k1 + _PHILOX_W1) & _MASK32
+        p0 = _PHILOX_M0 * c0
+        p1 = _PHILOX_M1 * c2
+        hi0, lo0 = p0 >> _SHIFT32, p0 & _MASK32
+        hi1, lo1 = p1 >> _SHIFT32, p1 & _MASK32
+        c0, c1, c2, c3 = hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0
+    return np.stack([c0, c1, c2, c3], axis=-1).astype(np.uint32)
+
+
+def _seed_key(seed):
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    return (seed & 0xFFFFFFFF, seed >> 32)
+
+
+def directions(d, r, seed):
+    """The r random directions of the Hamming-sorted LSH (Def. 1; Alg. 1 line 2).
+
+    The paper cites the construction without printing it; the reading taken is r
+    i.i.d. standard Gaussian directions, one set per call shared by queries, keys,
+    all segments and all recursion nodes.  Entry (k, t) of W (dimension k, direction
+    t) is normal number k*r + t of the stream: Philox call c (counter (c, 0, 0, 1),
+    key = seed) gives words x0..x3; u_i = (x_i + 0.5) / 2^32; Box-Muller on (u0, u1)
+    and on (u2, u3) gives normals 4c .. 4c+3 as (rho cos, rho sin) pairs.  The fp64
+    result is rounded once to fp32 (the precision the directions are stored in).
+    """
+    total = d * r
+    calls = (total + 3) // 4
+    ctr = np.zeros((calls, 4), dtype=np.uint64)
+    ctr[:, 0] = np.arange(calls, dtype=np.uint64)
+    ctr[:, 3] = DOMAIN_DIRECTIONS
+    x = philox4x32_10(ctr, _seed_key(seed)).astype(np.float64)
+    u = (x + 0.5) * 2.0 ** -32
+    z = np.empty((calls, 4), dtype=np.float64)
+    for a in (0, 2):
+        rho = np.sqrt(-2.0 * np.log(u[:, a]))
+        ang = 2.0 * np.pi * u[:, a + 1]
+        z[:, a] = rho * np.cos(ang)
+        z[:, a + 1] = rho * np.sin(ang)
+    return z.reshape(-1)[:total].reshape(d, r).astype(np.float32)
+
+
+def sample_indices(seed, g, node, m, N):
+    """l_0..l_{m-1} i.i.d. uniform on [0, N) with replacement (Alg. 2 line 4), shared by
+    every query row of one (segment g, recursion node) as Sec. 4 prescribes.
+
+    Sample j is word j & 3 of Philox call j >> 2 with counter (j >> 2, g, node, 2);
+    l_j = floor(x * N / 2^32).
+    """
+    if m == 0:
+        return np.zeros(0, dtype=np.int64)
+    calls = (m + 3) // 4
+    ctr = np.zeros((calls, 4), dtype=np.uint64)
+    ctr[:, 0] = np.arange(calls, dtype=np.uint64)
+    ctr[:, 1] = g
+    ctr[:, 2] = node
+    ctr[:, 3] = DOMAIN_SAMPLES
+    x = philox4x32_10(ctr, _seed_key(seed)).reshape(-1)[:m].astype(np.uint64)
+    return ((x * np.uint64(N)) >> _SHIFT32).astype(np.int64)
+
+
+# --------------------------------------------------------------------------------------
+# sortLSH (Def. 1, Alg. 1)
+# --------------------------------------------------------------------------------------
+def gray_rank(g, r):
+    """Position of sign pattern g in the reflected Gray sequence: h with h ^ (h >> 1) = g.
+
+    Def. 1 needs adjacent bucket ids to be sign patterns at Hamming distance one
+    (cyclically); ordering the patterns along the Gray sequence gives exactly that.
+    """
+    g = np.asarray(g, dtype=np.int64)
+    h = g.copy()
+    for s in range(1, r):
+        h ^= g >> s
+    return h
+
+
+def projections(X, W):
+    """<x, w_t> for every row x and direction t, in fp64."""
+    return np.asarray(X, dtype=np.float64) @ np.asarray(W, dtype=np.float64)
+
+
+def bucket_ids(X, W):
+    """Hamming-sorted LSH bucket id of every row (Def. 1; Alg. 1 line 2).
+
+    bit_t = [<x, w_t> > 0] (zero and negative give 0); the pattern g = sum bit_t 2^t is
+    mapped to its Gray rank.  Also returns |<x, w_t>| so a caller can tell which bits
+    sit too close to zero to be decided in lower precision.
+    """
+    p = projections(X, W)
+    r = p.shape[-1]
+    bits = (p > 0.0).astype(np.int64)
+    g = (bits << np.arange(r, dtype=np.int64)).sum(axis=-1)
+    return gray_rank(g, r).astype(np.uint8 if r <= 8 else np.int64), np.abs(p)
+
+
+def stable_argsort(ids):
+    """Permutation of Alg. 1 line 3.  `perm[p]` is the row placed at sorted position p;
+    `rank[i]` (the paper's P(i)) is the sorted position of row i.  Equal bucket ids keep
+    their original order (the paper's condition cannot hold for ties; stability makes
+    the permutation unique)."""
+    ids = np.asarray(ids)
+    perm = np.argsort(ids, kind="stable").astype(np.int64)
+    rank = np.empty_like(perm)
+    rank[perm] = np.arange(perm.size, dtype=np.int64)
+    return perm, rank
+
+
+def sortlsh_mask(rank_q, rank_k, b):
+    """M^H_ij = 1{ floor(P_Q(i)/b) = floor(P_K(j)/b) }  (Alg. 1 line 4)."""
+    bq = np.asarray(rank_q) // b
+    bk = np.asarray(rank_k) // b
+    return (bq[:, None] == bk[None, :]).astype(np.int64)
+
+
+# --------------------------------------------------------------------------------------
+# Exact attention (Sec. 1.1, Sec. 3.1): the definition, also the causal base case
+# --------------------------------------------------------------------------------------
+def exact_attention(Q, K, V, scale, causal=False, rows=None):
+    """Att = D^-1 A V with A = exp(scale * Q K^T); causal keeps entries i >= j
+    (M^C_ij = 1{i >= j}, diagonal included).  Returns (out, lse) with lse = ln D_ii.
+    `rows` restricts the evaluation to some query rows (rows are independent)."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    idx = np.arange(Q.shape[0]) if rows is None else np.asarray(rows, dtype=np.int64)
+    s = scale * (Q[idx] @ K.T)
+    if causal:
+        s = np.where(idx[:, None] >= np.arange(K.shape[0])[None, :], s, -np.inf)
+    mx = s.max(axis=1, keepdims=True)
+    a = np.exp(s - mx)
+    den = a.sum(axis=1, keepdims=True)
+    out = (a @ V) / den
+    lse = (mx + np.log(den))[:, 0]
+    return out, lse
+
+
+# --------------------------------------------------------------------------------------
+# One non-causal HyperAttention problem (Alg. 1-3 as specialised in Sec. 4)
+# --------------------------------------------------------------------------------------
+def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
+    """HyperAttention on N queries x N keys.
+
+    For query row i in sorted block beta = floor(P_Q(i)/b):
+      * masked part: the keys j with floor(P_K(j)/b) = beta, exact exp(s_ij)
+        (Alg. 2, "row-sum of masked entries"; Sec. 4 block-diagonal product);
+      * residual: (N/m) * sum over samples l_t with M^H_{i,l_t} = 0 of exp(s_{i,l_t})
+        (Alg. 2 line 7 without the cap C_i; collisions get weight zero, duplicates
+        count with their multiplicity);
+      * d~_i = masked + residual (Alg. 2 line 9 without the lower cap);
+      * numerator: same weights times the value rows (sampled indices reused for the
+        approximate matrix product, Sec. 4; uniform p = 1/N in Lemma 2 gives weight N/m).
+    out_i = numerator_i / d~_i, lse_i = ln d~_i.  If b >= N the whole problem is one
+    block and nothing is sampled.  Returns (out, lse) for `rows` (default all rows),
+    in original row order.
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    N = K.shape[0]
+    assert Q.shape[0] == N, "the paper pairs the beta-th group of Q with the beta-th group of K"
+    if b >= N:
+        return exact_attention(Q, K, V, scale, causal=False, rows=rows)
+    assert N % b == 0, "N must be a multiple of the block size (or b >= N)"
+    perm_q, rank_q = stable_argsort(ids_q)
+    perm_k, rank_k = stable_argsort(ids_k)
+    samples = np.asarray(samples, dtype=np.int64)
+    m = samples.size
+    want = np.arange(N) if rows is None else np.asarray(rows, dtype=np.int64)
+    out = np.zeros((want.size, V.shape[1]), dtype=np.float64)
+    lse = np.zeros(want.size, dtype=np.float64)
+    blk_of_want = rank_q[want] // b
+    Ks, Vs = K[samples], V[samples]
+    blk_of_sample = rank_k[samples] // b
+    for beta in np.unique(blk_of_want):
+        sel = np.nonzero(blk_of_want == beta)[0]
+        qi = want[sel]
+        J = perm_k[beta * b:(beta + 1) * b]
+        s_blk = scale * (Q[qi] @ K[J].T)
+        mx = s_blk.max(axis=1, keepdims=True)
+        if m > 0:
+            keep = (blk_of_sample != beta).astype(np.float64)          # 1 - M^H_{i, l_t}
+            s_smp = scale * (Q[qi] @ Ks.T)
+            if keep.any():
+                mx = np.maximum(mx, s_smp[:, keep > 0].max(axis=1, keepdims=True))
+            w = (N / m) * keep[None, :] * np.exp(np.where(keep[None, :] > 0, s_smp - mx, -np.inf))
+        a = np.exp(s_blk - mx)
+        den = a.sum(axis=1, keepdims=True)
+        num = a @ V[J]
+        if m > 0:
+            den = den + w.sum(axis=1, keepdims=True)
+            num = num + w @ Vs
+        out[sel] = num / den
+        lse[sel] = (mx + np.log(den))[:, 0]
+    return out, lse
+
+
+# --------------------------------------------------------------------------------------
+# Causal masking by recursion (Alg. 4, Fig. 2), carried through to the outputs
+# --------------------------------------------------------------------------------------
+def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, _node=0):
+    """Causal HyperAttention.  If N <= n0: exact causal attention (the paper recurses
+    until the length falls below a base size and uses an exact kernel there).  Else
+    split in equal halves (Alg. 4 line 2); recurse on (Q1,K1,V1) and (Q2,K2,V2)
+    (line 3); run the non-causal algorithm on (Q2,K1,V1) (line 4); rows of the second
+    half add the two row sums, D~_21 + D~_C22 (line 5), and so their outputs combine
+    with weights proportional to the two estimated row sums ("merging attention
+    outputs", Sec. 4.2).  Recursion nodes are numbered like a binary heap
+    (root 0, children 2v+1 and 2v+2) and the off-diagonal problem of node v draws its
+    samples from stream (g, v).
+    """
+    N = Q.shape[0]
+    want = np.arange(N) if rows is None else np.asarray(rows, dtype=np.int64)
+    if N <= n0:
+        return exact_attention(Q, K, V, scale, causal=True, rows=want)
+    assert N % 2 == 0
+    h = N // 2
+    out = np.zeros((want.size, V.shape[1]), dtype=np.float64)
+    lse = np.zeros(want.size, dtype=np.float64)
+    first = np.nonzero(want < h)[0]
+    second = np.nonzero(want >= h)[0]
+    if first.size:
+        o, l = causal_forward(Q[:h], K[:h], V[:h], ids_q[:h], ids_k[:h], b, m, scale, n0, seed, g,
+                              rows=want[first], _node=2 * _node + 1)
+        out[first], lse[first] = o, l
+    if second.size:
+        r2 = want[second] - h
+        o22, l22 = causal_forward(Q[h:], K[h:], V[h:], ids_q[h:], ids_k[h:], b, m, scale, n0, seed, g,
+                                  rows=r2, _node=2 * _node + 2)
+        mm = m if b < h else 0
+        smp = sample_indices(seed, g, _node, mm, h)
+        o21, l21 = node_forward(Q[h:], K[:h], V[:h], ids_q[h:], ids_k[:h], smp, b, scale, rows=r2)
+        l = np.logaddexp(l21, l22)
+        out[second] = o21 * np.exp(l21 - l)[:, None] + o22 * np.exp(l22 - l)[:, None]
+        lse[second] = l
+    return out, lse
+
+
+def heap_node(level, j):
+    """Heap index of the j-th recursion node of a level (root is level 0)."""
+    return (1 << level) - 1 + j
+
+
+# --------------------------------------------------------------------------------------
+# Whole forward pass
+# --------------------------------------------------------------------------------------
+def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None,
+                    ids_q=None, ids_k=None):
+    """Forward pass of one (batch, head) segment.  `ids_q` / `ids_k` may be injected
+    (e.g. the bucket ids another implementation produced) so that later stages can be
+    compared even when a sign bit at |projection| ~ 0 was decided differently."""
+    Q = np.asarray(Q, dtype=np.float64)
+    n, d = Q.shape
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    if ids_q is None:
+        ids_q, _ = bucket_ids(Q, W)
+    if ids_k is None:
+        ids_k, _ = bucket_ids(K, W)
+    if causal:
+        return causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=rows)
+    mm = m if b < n else 0
+    smp = sample_indices(seed, g, 0, mm, n)
+    return node_forward(Q, K, V, ids_q, ids_k, smp, b, scale, rows=rows)
+
+
+def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None):
+    """Q, K, V: (G, n, d).  Returns out (G, n, d) and lse (G, n), fp64."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    G, n, d = Q.shape
+    W = directions(d, r, seed)
+    out = np.zeros((G, n, d), dtype=np.float64)
+    lse = np.zeros((G, n), dtype=np.float64)
+    for g in range(G):
+        out[g], lse[g] = segment_forward(Q[g], K[g], V[g], W, b, m, causal, n0, seed, g, scale)
+    return out, lse
+
+
+# --------------------------------------------------------------------------------------
+# Dense cross-form (tiny n only): the n x n weight matrix the method implies
+# --------------------------------------------------------------------------------------
+def _dense_unnormalised(Q, K, ids_q, ids_k, samples, b, scale):
+    """(M^H + (N/m) c_j (1 - M^H)) o exp(scale Q K^T), c_j = multiplicity of key j among
+    the samples (Alg. 2 lines 7 and 9 without caps, written as one matrix)."""
+    N = K.shape[0]
+    A = np.exp(scale * (np.asarray(Q, np.float64) @ np.asarray(K, np.float64).T))
+    if b >= N:
+        return A
+    _, rank_q = stable_argsort(ids_q)
+    _, rank_k = stable_argsort(ids_k)
+    M = sortlsh_mask(rank_q, rank_k, b).astype(np.float64)
+    c = np.bincount(np.asarray(samples, dtype=np.int64), minlength=N).astype(np.float64)
+    m = max(len(samples), 1)
+    return (M + (N / m) * c[None, :] * (1.0 - M)) * A
+
+
+def dense_weights(Q, K, ids_q, ids_k, b, m, scale, causal, n0, seed, g, _node=0):
+    """Row-normalised n x n weights W~ with out = W~ V; causal problems are assembled
+    quadrant by quadrant exactly as Fig. 2 / Alg. 4 split the matrix."""
+    def unnorm(Q, K, iq, ik, node):
+        N = Q.shape[0]
+        if N <= n0:
+            A = np.exp(scale * (np.asarray(Q, np.float64) @ np.asarray(K, np.float64).T))
+            return np.tril(A)
+        h = N // 2
+        U = np.zeros((N, N))
+        U[:h, :h] = unnorm(Q[:h], K[:h], iq[:h], ik[:h], 2 * node + 1)
+        U[h:, h:] = unnorm(Q[h:], K[h:], iq[h:], ik[h:], 2 * node + 2)
+        mm = m if b < h else 0
+        smp = sample_indices(seed, g, node, mm, h)
+        U[h:, :h] = _dense_unnormalised(Q[h:], K[:h], iq[h:], ik[:h], smp, b, scale)
+        return U
+
+    if causal:
+        U = unnorm(Q, K, ids_q, ids_k, _node)
+    else:
+        N = Q.shape[0]
+        mm = m if b < N else 0
+        U = _dense_unnormalised(Q, K, ids_q, ids_k, sample_indices(seed, g, 0, mm, N), b, scale)
+    return U / U.sum(axis=1, keepdims=True)

@@ -1,0 +1,354 @@
+"""Pins for the CPU oracle: every stage is checked against something other than itself —
+brute force on tiny inputs, closed forms, the paper's Fig. 1, published Philox vectors,
+Monte-Carlo checks of Def. 1 and of the unbiased row-sum estimator of Alg. 2."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import hyperattn_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ helpers (plain loops)
+def brute_attention(Q, K, V, scale, causal):
+    n, d = Q.shape
+    out = np.zeros((n, V.shape[1]))
+    lse = np.zeros(n)
+    for i in range(n):
+        tot = 0.0
+        acc = [0.0] * V.shape[1]
+        for j in range(K.shape[0]):
+            if causal and j > i:
+                continue
+            s = 0.0
+            for k in range(d):
+                s += Q[i, k] * K[j, k]
+            a = math.exp(scale * s)
+            tot += a
+            for c in range(V.shape[1]):
+                acc[c] += a * V[j, c]
+        out[i] = [x / tot for x in acc]
+        lse[i] = math.log(tot)
+    return out, lse
+
+
+def rand_qkv(rng, n, d):
+    return rng.standard_normal((n, d)), rng.standard_normal((n, d)), rng.standard_normal((n, d))
+
+
+# ------------------------------------------------------------------ O8: random numbers
+def test_philox_known_answers():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) if l.strip() and l[0] != "#"]
+    assert len(rows) == 3
+    for w in rows:
+        v = [int(x, 16) for x in w]
+        got = O.philox4x32_10(np.array(v[0:4]), (v[4], v[5]))
+        assert [int(x) for x in got] == v[6:10]
+
+
+def test_philox_vectorised_matches_scalar_calls():
+    ctr = np.array([[i, 3, 5, 2] for i in range(17)])
+    batch = O.philox4x32_10(ctr, (123, 456))
+    for i in range(17):
+        assert (O.philox4x32_10(ctr[i], (123, 456)) == batch[i]).all()
+
+
+def test_directions_are_standard_normal():
+    from scipy import stats
+    W = O.directions(128, 8, 7).astype(np.float64).reshape(-1)
+    W = np.concatenate([W, O.directions(128, 8, 8).astype(np.float64).reshape(-1)])
+    assert abs(W.mean()) < 4 / math.sqrt(W.size)
+    assert abs(W.var() - 1.0) < 4 * math.sqrt(2.0 / W.size)
+    assert stats.kstest(W, "norm").pvalue > 1e-3
+    # the (cos, sin) pairs of Box-Muller are uncorrelated and both halves are used
+    assert abs(np.corrcoef(W[0::2], W[1::2])[0, 1]) < 0.1
+    # prefix property: entry (k, t) is normal number k*r + t of one stream
+    a = O.directions(4, 3, 5).reshape(-1)
+    b = O.directions(8, 3, 5).reshape(-1)
+    assert (a == b[:12]).all()
+    assert O.directions(64, 7, 0).dtype == np.float32
+
+
+def test_sample_indices_uniform_and_in_range():
+    from scipy import stats
+    N = 96
+    s = np.concatenate([O.sample_indices(11, g, 3, 512, N) for g in range(40)])
+    assert s.min() >= 0 and s.max() < N
+    cnt = np.bincount(s, minlength=N)
+    assert stats.chisquare(cnt).pvalue > 1e-3
+    # streams of different segments / nodes / seeds differ; equal arguments repeat
+    assert (O.sample_indices(1, 2, 3, 64, 1000) == O.sample_indices(1, 2, 3, 64, 1000)).all()
+    assert (O.sample_indices(1, 2, 3, 64, 1000) != O.sample_indices(1, 2, 4, 64, 1000)).any()
+    assert (O.sample_indices(1, 2, 3, 64, 1000) != O.sample_indices(1, 3, 3, 64, 1000)).any()
+    assert (O.sample_indices(1, 2, 3, 64, 1000) != O.sample_indices(2, 2, 3, 64, 1000)).any()
+    # floor(x N / 2^32) by hand for one word
+    x = int(O.philox4x32_10(np.array([1, 2, 3, 2]), (1, 0))[2])
+    assert int(O.sample_indices(1, 2, 3, 8, 1000)[6]) == (x * 1000) >> 32
+    assert O.sample_indices(1, 2, 3, 0, 10).size == 0
+
+
+# ------------------------------------------------------------------ O4: Def. 1
+def test_gray_rank_adjacent_buckets_differ_in_one_sign():
+    for r in range(1, 9):
+        h = O.gray_rank(np.arange(1 << r), r)
+        assert sorted(h.tolist()) == list(range(1 << r))          # a bijection
+        inv = np.empty(1 << r, dtype=np.int64)
+        inv[h] = np.arange(1 << r)                                # bucket id -> sign pattern
+        for x in range(1 << r):
+            assert x ^ (x >> 1) == inv[x]                         # the reflected Gray code
+            diff = int(inv[x] ^ inv[(x + 1) % (1 << r)])
+            assert bin(diff).count("1") == 1                      # cyclic adjacency
+
+
+def test_bucket_bit_order_and_sign_convention():
+    W = np.eye(3, dtype=np.float32)                               # direction t reads coordinate t
+    X = np.array([[1.0, -1.0, -1.0],      # g = 001b = 1 -> h = 1
+                  [1.0, 1.0, -1.0],       # g = 011b = 3 -> h = 2
+                  [-1.0, 1.0, -1.0],      # g = 010b = 2 -> h = 3
+                  [-1.0, -1.0, 1.0],      # g = 100b = 4 -> h = 7
+                  [0.0, -0.0, 1.0]])      # zeros count as "not positive": g = 4 -> h = 7
+    ids, absp = O.bucket_ids(X, W)
+    assert ids.tolist() == [1, 2, 3, 7, 7]
+    assert absp.shape == (5, 3) and absp[4, 0] == 0.0
+
+
+def test_def1_collision_and_adjacency_probabilities():
+    r, d, trials = 4, 6, 12000
+    theta = 0.9
+    x = np.zeros(d); x[0] = 2.0
+    y = np.zeros(d); y[0] = 0.7 * math.cos(theta); y[1] = 0.7 * math.sin(theta)
+    same = adj = 0
+    for seed in range(trials):
+        W = O.directions(d, r, seed)
+        (hx, hy), _ = O.bucket_ids(np.stack([x, y]), W)
+        hx, hy = int(hx), int(hy)
+        same += hx == hy
+        adj += (hy == (hx + 1) % (1 << r)) or (hy == (hx - 1) % (1 << r))
+    p_same = (1 - theta / math.pi) ** r
+    p_adj = (2 * theta / math.pi) * (1 - theta / math.pi) ** (r - 1)
+    for got, p in ((same / trials, p_same), (adj / trials, p_adj)):
+        assert abs(got - p) < 4 * math.sqrt(p * (1 - p) / trials), (got, p)
+
+
+# ------------------------------------------------------------------ O7 / O5: sort and mask
+def test_stable_argsort_against_python_sort():
+    rng = np.random.default_rng(0)
+    for n in (1, 2, 37, 500):
+        ids = rng.integers(0, 9, size=n).astype(np.uint8)
+        perm, rank = O.stable_argsort(ids)
+        expect = [i for _, i in sorted((int(ids[i]), i) for i in range(n))]
+        assert perm.tolist() == expect
+        assert all(rank[perm[p]] == p for p in range(n))
+
+
+def test_fig1_mask():
+    spec = {}
+    for line in open(os.path.join(GOLDEN, "fig1_sortlsh.txt")):
+        if line.strip() and line[0] != "#":
+            k, *v = line.split()
+            spec[k] = v
+    sq = [int(x) - 1 for x in spec["sorted_queries"]]
+    sk = [int(x) - 1 for x in spec["sorted_keys"]]
+    b = int(spec["block"][0])
+    boxed = {tuple(int(t) - 1 for t in e.split("-")) for e in spec["boxed"]}
+    assert len(boxed) == 23
+    # bucket ids that reproduce the printed order (one row per bucket)
+    ids_q = np.empty(9, dtype=np.uint8); ids_q[sq] = np.arange(9)
+    ids_k = np.empty(9, dtype=np.uint8); ids_k[sk] = np.arange(9)
+    perm_q, rank_q = O.stable_argsort(ids_q)
+    perm_k, rank_k = O.stable_argsort(ids_k)
+    assert perm_q.tolist() == sq and perm_k.tolist() == sk
+    M = O.sortlsh_mask(rank_q, rank_k, b)
+    assert M.sum() == 27 and (M.sum(axis=0) == 3).all() and (M.sum(axis=1) == 3).all()
+    assert all(M[i, j] == 1 for i, j in boxed)
+    # the three diagonal blocks of the middle panel
+    for blk in range(3):
+        for i in sq[3 * blk:3 * blk + 3]:
+            assert sorted(np.nonzero(M[i])[0].tolist()) == sorted(sk[3 * blk:3 * blk + 3])
+
+
+# ------------------------------------------------------------------ O1: exact attention
+@pytest.mark.parametrize("causal", [False, True])
+def test_exact_attention_brute_force(causal):
+    rng = np.random.default_rng(1)
+    Q, K, V = rand_qkv(rng, 13, 5)
+    out, lse = O.exact_attention(Q, K, V, 0.37, causal=causal)
+    bo, bl = brute_attention(Q, K, V, 0.37, causal)
+    np.testing.assert_allclose(out, bo, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, bl, rtol=0, atol=1e-12)
+    o2, l2 = O.exact_attention(Q, K, V, 0.37, causal=causal, rows=[12, 0, 5])
+    np.testing.assert_allclose(o2, bo[[12, 0, 5]], atol=1e-12)
+    np.testing.assert_allclose(l2, bl[[12, 0, 5]], atol=1e-12)
+
+
+def test_single_block_is_exact_attention():
+    """b = N (or b > N): the mask is all ones, nothing is sampled."""
+    rng = np.random.default_rng(2)
+    Q, K, V = (x[None] for x in rand_qkv(rng, 24, 4))
+    bo, bl = brute_attention(Q[0], K[0], V[0], 0.5, False)
+    for b in (24, 64):
+        out, lse = O.forward(Q, K, V, b=b, m=8, r=3, seed=4, scale=0.5)
+        np.testing.assert_allclose(out[0], bo, atol=1e-12)
+        np.testing.assert_allclose(lse[0], bl, atol=1e-12)
+
+
+def test_causal_base_case_is_exact_causal_attention():
+    rng = np.random.default_rng(3)
+    Q, K, V = (x[None] for x in rand_qkv(rng, 16, 4))
+    bo, bl = brute_attention(Q[0], K[0], V[0], 0.5, True)
+    out, lse = O.forward(Q, K, V, b=4, m=4, r=3, causal=True, n0=16, seed=4, scale=0.5)
+    np.testing.assert_allclose(out[0], bo, atol=1e-12)
+    np.testing.assert_allclose(lse[0], bl, atol=1e-12)
+
+
+# ------------------------------------------------------------------ O2: causal bookkeeping
+@pytest.mark.parametrize("n,n0", [(32, 4), (32, 8), (48, 12), (64, 2)])
+def test_causal_recursion_with_single_block_nodes_is_exact(n, n0):
+    """With b >= n/2 every off-diagonal problem is one block, so Alg. 4's identity
+    D_C = diag(D_C11, D_21 + D_C22) must give exact causal attention for any depth."""
+    rng = np.random.default_rng(n + n0)
+    Q, K, V = (x[None] for x in rand_qkv(rng, n, 3))
+    bo, bl = brute_attention(Q[0], K[0], V[0], 0.6, True)
+    out, lse = O.forward(Q, K, V, b=n // 2, m=8, r=4, causal=True, n0=n0, seed=1, scale=0.6)
+    np.testing.assert_allclose(out[0], bo, atol=1e-11)
+    np.testing.assert_allclose(lse[0], bl, atol=1e-11)
+
+
+# ------------------------------------------------------------------ residual path: closed forms
+def test_samples_covering_every_key_once_give_exact_attention():
+    """m = N samples hitting each key exactly once: N/m = 1, the off-block sum is complete,
+    so masked + residual is the full row sum and the output is exact attention."""
+    rng = np.random.default_rng(5)
+    N, b = 32, 8
+    Q, K, V = rand_qkv(rng, N, 6)
+    iq = rng.integers(0, 8, N).astype(np.uint8)
+    ik = rng.integers(0, 8, N).astype(np.uint8)
+    out, lse = O.node_forward(Q, K, V, iq, ik, rng.permutation(N), b, 0.4)
+    bo, bl = brute_attention(Q, K, V, 0.4, False)
+    np.testing.assert_allclose(out, bo, atol=1e-12)
+    np.testing.assert_allclose(lse, bl, atol=1e-12)
+
+
+def test_zero_logits_give_counting_closed_form():
+    """Q = 0 makes every attention entry 1: d~_i = b + (N/m) #{t : l_t outside i's block};
+    V = 1 makes every output exactly 1 (weights sum to one)."""
+    rng = np.random.default_rng(6)
+    N, b, m, d = 40, 8, 12, 3
+    K = rng.standard_normal((N, d))
+    iq = rng.integers(0, 16, N).astype(np.uint8)
+    ik = rng.integers(0, 16, N).astype(np.uint8)
+    smp = rng.integers(0, N, m)
+    out, lse = O.node_forward(np.zeros((N, d)), K, np.ones((N, d)), iq, ik, smp, b, 1.0)
+    order_q = sorted(range(N), key=lambda i: (int(iq[i]), i))
+    order_k = sorted(range(N), key=lambda i: (int(ik[i]), i))
+    for i in range(N):
+        beta = order_q.index(i) // b
+        outside = sum(1 for l in smp if order_k.index(int(l)) // b != beta)
+        assert abs(lse[i] - math.log(b + (N / m) * outside)) < 1e-12
+    np.testing.assert_allclose(out, 1.0, atol=1e-12)
+
+
+def test_no_samples_and_all_colliding_samples():
+    rng = np.random.default_rng(7)
+    N, b = 16, 4
+    Q, K, V = rand_qkv(rng, N, 3)
+    ids = np.repeat(np.arange(4), 4).astype(np.uint8)            # blocks = consecutive rows
+    out0, lse0 = O.node_forward(Q, K, V, ids, ids, np.zeros(0, dtype=int), b, 0.5)
+    for blk in range(4):
+        sl = slice(4 * blk, 4 * blk + 4)
+        bo, bl = brute_attention(Q[sl], K[sl], V[sl], 0.5, False)
+        np.testing.assert_allclose(out0[sl], bo, atol=1e-12)
+        np.testing.assert_allclose(lse0[sl], bl, atol=1e-12)
+    # samples all inside block 0: rows of block 0 see no residual at all
+    out1, lse1 = O.node_forward(Q, K, V, ids, ids, np.array([0, 1, 2, 3]), b, 0.5)
+    np.testing.assert_allclose(out1[:4], out0[:4], atol=1e-12)
+    np.testing.assert_allclose(lse1[:4], lse0[:4], atol=1e-12)
+    assert (lse1[4:] > lse0[4:]).all()
+
+
+# ------------------------------------------------------------------ O6: unbiased estimator
+def test_sampled_row_sum_and_numerator_are_unbiased():
+    """Alg. 2 line 7 (uncapped): E[(N/m) sum_t (1 - M_{i,l_t}) A_{i,l_t}] is the off-block row
+    sum; with the same weights on V the numerator's expectation is (A V)_i."""
+    rng = np.random.default_rng(8)
+    N, b, m, d, scale = 24, 6, 5, 3, 0.3
+    Q, K, V = rand_qkv(rng, N, d)
+    iq = rng.integers(0, 8, N).astype(np.uint8)
+    ik = rng.integers(0, 8, N).astype(np.uint8)
+    trials = 6000
+    dens = np.zeros((trials, N))
+    nums = np.zeros((trials, N, d))
+    for t in range(trials):
+        smp = O.sample_indices(t, 0, 0, m, N)
+        out, lse = O.node_forward(Q, K, V, iq, ik, smp, b, scale)
+        dens[t] = np.exp(lse)
+        nums[t] = out * dens[t][:, None]
+    A = np.exp(scale * Q @ K.T)
+    full_den = A.sum(axis=1)
+    full_num = A @ V
+    se_d = dens.std(axis=0, ddof=1) / math.sqrt(trials)
+    se_n = nums.std(axis=0, ddof=1) / math.sqrt(trials)
+    assert (np.abs(dens.mean(axis=0) - full_den) < 4.5 * se_d).all()
+    assert (np.abs(nums.mean(axis=0) - full_num) < 4.5 * se_n + 1e-12).all()
+    assert (se_d > 0).all()                                       # the sampled term is really there
+
+
+# ------------------------------------------------------------------ O3: dense cross-form
+@pytest.mark.parametrize("causal,n0", [(False, 0), (True, 8), (True, 4)])
+def test_dense_weights_are_row_stochastic_and_reproduce_output(causal, n0):
+    rng = np.random.default_rng(9)
+    n, d, b, m, r, seed, scale = 32, 4, 4, 6, 3, 21, 0.45
+    Q, K, V = rand_qkv(rng, n, d)
+    W = O.directions(d, r, seed)
+    iq, _ = O.bucket_ids(Q, W)
+    ik, _ = O.bucket_ids(K, W)
+    Wt = O.dense_weights(Q, K, iq, ik, b, m, scale, causal, n0, seed, g=2)
+    np.testing.assert_allclose(Wt.sum(axis=1), 1.0, atol=1e-12)
+    assert (Wt >= 0).all()
+    if causal:
+        assert np.triu(Wt, 1).max() == 0.0
+    out, lse = O.segment_forward(Q, K, V, W, b, m, causal, n0, seed, g=2, scale=scale)
+    np.testing.assert_allclose(out, Wt @ V, atol=1e-12)
+    # V = ones gives ones
+    out1, _ = O.segment_forward(Q, K, np.ones_like(V), W, b, m, causal, n0, seed, g=2, scale=scale)
+    np.testing.assert_allclose(out1, 1.0, atol=1e-12)
+    # rows can be evaluated in any subset / order
+    rows = np.array([31, 0, 17, 8, 16])
+    o2, l2 = O.segment_forward(Q, K, V, W, b, m, causal, n0, seed, g=2, scale=scale, rows=rows)
+    np.testing.assert_allclose(o2, out[rows], atol=1e-13)
+    np.testing.assert_allclose(l2, lse[rows], atol=1e-13)
+
+
+def test_causal_nodes_use_their_own_sample_streams():
+    """Second-quarter rows of a two-level recursion only see node 1 (left child) and
+    the leaves; last-quarter rows see node 0 and node 2."""
+    rng = np.random.default_rng(10)
+    n, d, b, m, r, seed, scale, n0 = 32, 4, 2, 4, 3, 3, 0.5, 8
+    Q, K, V = rand_qkv(rng, n, d)
+    W = O.directions(d, r, seed)
+    iq, _ = O.bucket_ids(Q, W)
+    ik, _ = O.bucket_ids(K, W)
+    out, lse = O.segment_forward(Q, K, V, W, b, m, True, n0, seed, g=0, scale=scale)
+    # rebuild rows 8..15 by hand: exact causal on [8,16) merged with node 1 on (Q[8:16], K[:8])
+    o22, l22 = O.exact_attention(Q[8:16], K[8:16], V[8:16], scale, causal=True)
+    smp = O.sample_indices(seed, 0, O.heap_node(1, 0), m, 8)
+    o21, l21 = O.node_forward(Q[8:16], K[:8], V[:8], iq[8:16], ik[:8], smp, b, scale)
+    den = np.exp(l21) + np.exp(l22)
+    np.testing.assert_allclose(lse[8:16], np.log(den), atol=1e-12)
+    np.testing.assert_allclose(out[8:16], (o21 * np.exp(l21)[:, None] + o22 * np.exp(l22)[:, None]) / den[:, None],
+                               atol=1e-12)
+
+
+# ------------------------------------------------------------------ O9: permutation invariance
+def test_joint_permutation_of_keys_and_values_single_block():
+    rng = np.random.default_rng(11)
+    Q, K, V = rand_qkv(rng, 20, 4)
+    p = rng.permutation(20)
+    ids = rng.integers(0, 4, 20).astype(np.uint8)
+    a, la = O.node_forward(Q, K, V, ids, ids, [], 20, 0.5)
+    c, lc = O.node_forward(Q, K[p], V[p], ids, ids[p], [], 20, 0.5)
+    np.testing.assert_allclose(a, c, atol=1e-12)
+    np.testing.assert_allclose(la, lc, atol=1e-12)
