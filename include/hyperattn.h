@@ -1,0 +1,178 @@
+/*
+ * hyperattn.h -- C ABI of the B200 (sm_100a) HyperAttention forward library.
+ *
+ * Method: Han, Jayaram, Karbasi, Mirrokni, Woodruff, Zandieh, "HyperAttention:
+ * Long-context Attention in Near-Linear Time" (arXiv 2310.05869).  The library
+ * computes the practical forward pass of Sec. 4 ("Implementation Detail"):
+ *
+ *   1. sortLSH (Def. 1, Alg. 1): every query and key row is hashed by the signs of
+ *      r = hash_bits Gaussian projections, the sign pattern is mapped to its position
+ *      in the reflected Gray sequence (adjacent bucket ids differ in one sign), and
+ *      queries and keys are argsorted (stably) by bucket id.
+ *   2. Exact softmax attention inside the b x b diagonal blocks of the sorted order
+ *      (the mask M^H of Alg. 1 line 4; Sec. 4).
+ *   3. Residual (Alg. 2 lines 4, 7 and 9 without the caps; Alg. 3; Sec. 4): m key
+ *      indices drawn i.i.d. uniformly, shared by all query rows; sampled entries outside
+ *      a row's block enter the row sum and the numerator with weight N/m.
+ *   4. out_i = numerator_i / d~_i, lse_i = ln d~_i.  With causal masking the recursive
+ *      split of Alg. 4 / Fig. 2 is applied: the two diagonal halves recurse down to an
+ *      exact causal base case of n0 rows, the lower-left quadrant is a non-causal
+ *      HyperAttention problem, and the row sums (hence the outputs) of the second half
+ *      are combined (Alg. 4 line 5).
+ *
+ * Conventions common to all entry points
+ *   - q, k, v, out are DEVICE pointers to contiguous [B, H, n, d] tensors, d fastest;
+ *     lse is a DEVICE pointer to [B, H, n] floats (natural logarithm of the estimated
+ *     row sum d~_i of exp(softmax_scale * <q_i, k_j>)).  All must be 16-byte aligned.
+ *   - The caller owns every buffer passed in; the library neither frees nor keeps them.
+ *     `out`/`lse` must not alias an input.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All work
+ *     is enqueued on it; no entry point synchronises unless it says so.
+ *   - Return value: 0 on success, a negative hyperattn_status otherwise.  On a
+ *     host-detected error nothing is launched and no output is written.
+ *   - Shapes: d in {64, 128}; 1 <= hash_bits <= 8; samples >= 0; block >= 1.
+ *     Non-causal: n % block == 0 or block >= n (then the problem is one exact block).
+ *     Causal: n <= n0 (exact causal attention) or n == n0 * 2^L; and the half-size of
+ *     every recursion node must be a multiple of block unless block >= that half-size.
+ *   - Recursion nodes are numbered like a binary heap: the off-diagonal problem of the
+ *     j-th node of level l (root level 0) is node (2^l - 1) + j; it pairs query rows
+ *     [(2j+1)s, (2j+2)s) with key rows [2js, (2j+1)s), s = n / 2^(l+1).  A non-causal
+ *     call has the single node 0 over all rows.
+ *   - Random numbers: Philox4x32-10 keyed by `seed`; directions use counter
+ *     (c, 0, 0, 1), samples of (segment g, node v) use counter (j >> 2, g, v, 2),
+ *     word j & 3, index = floor(word * N / 2^32).
+ */
+#ifndef HYPERATTN_H_
+#define HYPERATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum hyperattn_status {
+  HYPERATTN_OK = 0,
+  HYPERATTN_INVALID_ARGUMENT = -1,   /* null pointer, non-positive size, bad enum */
+  HYPERATTN_UNSUPPORTED_SHAPE = -2,  /* shape rules above violated */
+  HYPERATTN_MISALIGNED = -3,         /* a pointer is not 16-byte aligned, or out aliases an input */
+  HYPERATTN_WORKSPACE_TOO_SMALL = -4,
+  HYPERATTN_CUDA_ERROR = -5,         /* a CUDA runtime call failed */
+  HYPERATTN_DEVICE_TIMEOUT = -6      /* a bounded device-side wait gave up (status word) */
+} hyperattn_status;
+
+typedef enum hyperattn_dtype {
+  HYPERATTN_BF16 = 0,
+  HYPERATTN_FP32 = 1
+} hyperattn_dtype;
+
+/* Optional device buffers that receive the intermediate results of the integer stages
+ * (needed to compare them bit for bit with a reference).  Any member may be NULL.
+ * Let G = B*H, LV = number of levels (1 if non-causal or n <= n0, else L),
+ * NL = rows per (level, segment, side): n if non-causal, n/2 if causal with L >= 1,
+ * NODES = 1 if non-causal, 2^L - 1 if causal (0 if n <= n0).
+ *   q_ids, k_ids : uint8 [G, n]        bucket id of every row (Def. 1)
+ *   perm_q,perm_k: int32 [LV, G, NL]   node j of level l occupies [j*s, (j+1)*s);
+ *                                      entry p = row (relative to the node's first query /
+ *                                      key row) placed at sorted position p (Alg. 1 line 3)
+ *   rank_k       : int32 [LV, G, NL]   inverse of perm_k (the paper's P_K)
+ *   samples      : int32 [G, NODES, m] sampled key indices relative to the node (Alg. 2 line 4)
+ *   near_zero_bits: one uint64 counter, incremented by the number of hash bits whose
+ *                   projection magnitude is below 1e-4 (caller zeroes it) */
+typedef struct hyperattn_debug {
+  uint8_t* q_ids;
+  uint8_t* k_ids;
+  int32_t* perm_q;
+  int32_t* perm_k;
+  int32_t* rank_k;
+  int32_t* samples;
+  unsigned long long* near_zero_bits;
+} hyperattn_debug;
+
+typedef struct hyperattn_params {
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;             /* [B,H,n,d] in out_dtype */
+  float* lse;            /* [B,H,n] */
+  int B, H, n, d;
+  int block;             /* b of Alg. 1 */
+  int samples;           /* m of Alg. 2 */
+  int hash_bits;         /* r of Def. 1 */
+  int causal;            /* 0 / 1 */
+  int n0;                /* exact causal base size (ignored if !causal) */
+  uint64_t seed;
+  int dtype;             /* hyperattn_dtype of q, k, v */
+  int out_dtype;         /* hyperattn_dtype of out (fp32 out with bf16 inputs is allowed) */
+  float softmax_scale;   /* <= 0 selects 1/sqrt(d) */
+  void* workspace;       /* device scratch owned by the caller, or NULL: the library then
+                            uses a private per-device buffer that it grows on demand (the
+                            growing call synchronises the device) and keeps until
+                            hyperattn_release(); calls that share it must not overlap */
+  size_t workspace_bytes;
+  const hyperattn_debug* debug; /* may be NULL */
+  void* stream;
+} hyperattn_params;
+
+/* HyperAttention forward (Alg. 1-4 as specialised in Sec. 4) with bf16 inputs and
+ * output, softmax scale 1/sqrt(d) and the library's private workspace. */
+int hyperattn_forward(const void* q, const void* k, const void* v, void* out, float* lse,
+                      int B, int H, int n, int d, int block, int samples, int hash_bits,
+                      int causal, int n0, uint64_t seed, void* stream);
+
+/* The same computation with every option explicit. */
+int hyperattn_forward_ex(const hyperattn_params* p);
+
+/* The same computation for HOST buffers: q, k, v, out, lse of *p are host pointers (pinned
+ * memory makes the copies asynchronous).  The inputs are copied to a private device staging
+ * area on `stream`, the forward pass runs there, and out / lse are copied back on the same
+ * stream; the caller synchronises the stream before reading them.  The staging area is
+ * grown on demand (that call synchronises the device) and kept until hyperattn_release(). */
+int hyperattn_forward_host(const hyperattn_params* p);
+
+/* Bytes of device scratch hyperattn_forward_ex needs for these shapes (host-side; only the
+ * shape members, dtype and out_dtype of *p are read). */
+int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes);
+
+/* Host-side: writes the d x hash_bits direction matrix of Def. 1's hash (row-major,
+ * entry [k*hash_bits + t] = coordinate k of direction t) that a call with this seed uses. */
+int hyperattn_get_projections(int d, int hash_bits, uint64_t seed, float* host_out);
+
+/* Synchronises `stream` and reports the device status word (0, or
+ * HYPERATTN_DEVICE_TIMEOUT if a kernel's bounded wait gave up since the last query). */
+int hyperattn_last_device_status(void* stream, int* status);
+
+/* Stage timing.  While enabled, every forward call brackets each stage with CUDA events
+ * on its stream and hyperattn_profile_read() (which synchronises those events) returns,
+ * for every stage, the summed device milliseconds and launch count since the last
+ * hyperattn_profile_reset().  Stage indices: */
+enum {
+  HYPERATTN_STAGE_CONVERT = 0, /* fp32 -> bf16 staging copy (fp32 inputs only) */
+  HYPERATTN_STAGE_HASH = 1,    /* Def. 1 hash of Q and K rows + chunk histograms */
+  HYPERATTN_STAGE_SAMPLE = 2,  /* Alg. 2 line 4 */
+  HYPERATTN_STAGE_SORT_SCAN = 3,
+  HYPERATTN_STAGE_SORT_SCATTER = 4, /* Alg. 1 line 3 */
+  HYPERATTN_STAGE_ATTENTION = 5,    /* block + sampled + causal-leaf contractions */
+  HYPERATTN_STAGE_MERGE = 6,        /* Alg. 4 line 5 carried to outputs */
+  HYPERATTN_NUM_STAGES = 7
+};
+typedef struct hyperattn_stage_times {
+  float ms[HYPERATTN_NUM_STAGES];
+  int launches[HYPERATTN_NUM_STAGES];
+  int calls;
+} hyperattn_stage_times;
+int hyperattn_profile_enable(int on);
+int hyperattn_profile_reset(void);
+int hyperattn_profile_read(hyperattn_stage_times* out);
+
+/* Frees the private workspaces and profiling events of every device. */
+int hyperattn_release(void);
+
+const char* hyperattn_status_string(int status);
+int hyperattn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYPERATTN_H_ */

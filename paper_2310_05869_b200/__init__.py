@@ -1,0 +1,15 @@
+"""B200-native HyperAttention forward (arXiv 2310.05869): thin binding over libhyperattn.so."""
+from .binding import (  # noqa: F401
+    HyperAttnError,
+    forward,
+    forward_host,
+    get_projections,
+    last_device_status,
+    lib,
+    profile_enable,
+    profile_read,
+    profile_reset,
+    release,
+    version,
+    workspace_bytes,
+)

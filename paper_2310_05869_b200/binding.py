@@ -1,0 +1,194 @@
+"""ctypes binding of the C-ABI library.  Argument marshalling only: every step of the
+forward pass runs inside the library's CUDA kernels.  PyTorch supplies device memory and the
+current stream.  There is no CPU fallback: if the shared library is missing, loading fails."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhyperattn.so")
+_lib = None
+
+BF16, FP32 = 0, 1
+NUM_STAGES = 7
+STAGE_NAMES = ["convert", "hash", "sample", "sort_scan", "sort_scatter", "attention", "merge"]
+EXPORTS = ["hyperattn_forward", "hyperattn_forward_ex", "hyperattn_forward_host", "hyperattn_workspace_bytes",
+           "hyperattn_get_projections", "hyperattn_last_device_status", "hyperattn_profile_enable",
+           "hyperattn_profile_reset", "hyperattn_profile_read", "hyperattn_release",
+           "hyperattn_status_string", "hyperattn_version"]
+
+
+class HyperAttnError(RuntimeError):
+    pass
+
+
+class _Debug(C.Structure):
+    _fields_ = [("q_ids", C.c_void_p), ("k_ids", C.c_void_p), ("perm_q", C.c_void_p), ("perm_k", C.c_void_p),
+                ("rank_k", C.c_void_p), ("samples", C.c_void_p), ("near_zero_bits", C.c_void_p)]
+
+
+class _Params(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("out", C.c_void_p), ("lse", C.c_void_p),
+                ("B", C.c_int), ("H", C.c_int), ("n", C.c_int), ("d", C.c_int),
+                ("block", C.c_int), ("samples", C.c_int), ("hash_bits", C.c_int), ("causal", C.c_int),
+                ("n0", C.c_int), ("seed", C.c_uint64), ("dtype", C.c_int), ("out_dtype", C.c_int),
+                ("softmax_scale", C.c_float), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("debug", C.POINTER(_Debug)), ("stream", C.c_void_p)]
+
+
+class _StageTimes(C.Structure):
+    _fields_ = [("ms", C.c_float * NUM_STAGES), ("launches", C.c_int * NUM_STAGES), ("calls", C.c_int)]
+
+
+def lib() -> C.CDLL:
+    """Loads libhyperattn.so (built in-tree by paper_2310_05869_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise HyperAttnError(f"{_LIB_PATH} is missing: build it with `python -m paper_2310_05869_b200.build`")
+        L = C.CDLL(_LIB_PATH)
+        L.hyperattn_forward.restype = C.c_int
+        L.hyperattn_forward.argtypes = [C.c_void_p] * 5 + [C.c_int] * 9 + [C.c_uint64, C.c_void_p]
+        for name in ("hyperattn_forward_ex", "hyperattn_forward_host"):
+            getattr(L, name).restype = C.c_int
+            getattr(L, name).argtypes = [C.POINTER(_Params)]
+        L.hyperattn_workspace_bytes.restype = C.c_int
+        L.hyperattn_workspace_bytes.argtypes = [C.POINTER(_Params), C.POINTER(C.c_size_t)]
+        L.hyperattn_get_projections.restype = C.c_int
+        L.hyperattn_get_projections.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_void_p]
+        L.hyperattn_last_device_status.restype = C.c_int
+        L.hyperattn_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
+        L.hyperattn_profile_enable.argtypes = [C.c_int]
+        L.hyperattn_profile_read.argtypes = [C.POINTER(_StageTimes)]
+        L.hyperattn_status_string.restype = C.c_char_p
+        L.hyperattn_status_string.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise HyperAttnError(f"{what}: {lib().hyperattn_status_string(rc).decode()} ({rc})")
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.bfloat16:
+        return BF16
+    if t == torch.float32:
+        return FP32
+    raise HyperAttnError(f"unsupported dtype {t}")
+
+
+def _fill(p: _Params, B, H, n, d, block, samples, hash_bits, causal, n0, seed, dtype, out_dtype, scale):
+    p.B, p.H, p.n, p.d = B, H, n, d
+    p.block, p.samples, p.hash_bits, p.causal, p.n0 = block, samples, hash_bits, int(bool(causal)), n0
+    p.seed = seed
+    p.dtype, p.out_dtype, p.softmax_scale = dtype, out_dtype, float(scale)
+
+
+def _debug_shapes(B, H, n, block, samples, causal, n0):
+    """Shapes of the exported intermediates (see hyperattn_debug in the header)."""
+    G = B * H
+    if not causal:
+        LV, NL, NODES = 1, n, 1
+    elif n <= n0:
+        LV, NL, NODES = 1, n, 0
+    else:
+        L = (n // n0).bit_length() - 1
+        LV, NL, NODES = L, n // 2, (1 << L) - 1
+    return G, LV, NL, NODES
+
+
+def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_dtype=None, scale=0.0,
+            workspace=None, debug=False, stream=None):
+    """HyperAttention forward on CUDA tensors q, k, v of shape [B, H, n, d] (bf16 or fp32).
+    Returns (out, lse) or (out, lse, intermediates) when debug=True."""
+    if not (q.is_cuda and k.is_cuda and v.is_cuda):
+        raise HyperAttnError("q, k, v must be CUDA tensors (there is no CPU path)")
+    q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
+    B, H, n, d = q.shape
+    out_dtype = out_dtype or q.dtype
+    out = torch.empty((B, H, n, d), dtype=out_dtype, device=q.device)
+    lse = torch.empty((B, H, n), dtype=torch.float32, device=q.device)
+    p = _Params()
+    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, seed, _dtype_code(q.dtype), _dtype_code(out_dtype), scale)
+    p.q, p.k, p.v, p.out, p.lse = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr()
+    if workspace is not None:
+        p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    p.stream = stream if stream is not None else torch.cuda.current_stream(q.device).cuda_stream
+    inter = None
+    if debug:
+        G, LV, NL, NODES = _debug_shapes(B, H, n, block, samples, causal, n0)
+        dev = q.device
+        inter = {
+            "q_ids": torch.zeros((G, n), dtype=torch.uint8, device=dev),
+            "k_ids": torch.zeros((G, n), dtype=torch.uint8, device=dev),
+            "perm_q": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
+            "perm_k": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
+            "rank_k": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
+            "samples": torch.full((G, max(NODES, 1), max(samples, 1)), -1, dtype=torch.int32, device=dev),
+            "near_zero_bits": torch.zeros(1, dtype=torch.int64, device=dev),
+        }
+        dbg = _Debug(*(inter[f].data_ptr() for f, _ in _Debug._fields_))
+        p.debug = C.pointer(dbg)
+    with torch.cuda.device(q.device):
+        _check(lib().hyperattn_forward_ex(C.byref(p)), "hyperattn_forward_ex")
+    return (out, lse, inter) if debug else (out, lse)
+
+
+def forward_host(q, k, v, out, lse, block, samples, hash_bits, causal=False, n0=0, seed=0, scale=0.0, stream=None):
+    """Host-buffer entry: q, k, v, out, lse are CPU tensors (pinned for asynchronous copies).
+    Enqueues H2D copies, the forward pass and D2H copies on the stream; the caller synchronises."""
+    B, H, n, d = q.shape
+    p = _Params()
+    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, seed, _dtype_code(q.dtype), _dtype_code(out.dtype), scale)
+    p.q, p.k, p.v, p.out, p.lse = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr()
+    p.stream = stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    _check(lib().hyperattn_forward_host(C.byref(p)), "hyperattn_forward_host")
+
+
+def workspace_bytes(B, H, n, d, block, samples, hash_bits, causal=False, n0=0, dtype=BF16, out_dtype=BF16) -> int:
+    p = _Params()
+    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, 0, dtype, out_dtype, 0.0)
+    nbytes = C.c_size_t(0)
+    _check(lib().hyperattn_workspace_bytes(C.byref(p), C.byref(nbytes)), "hyperattn_workspace_bytes")
+    return int(nbytes.value)
+
+
+def get_projections(d: int, hash_bits: int, seed: int) -> np.ndarray:
+    w = np.zeros((d, hash_bits), dtype=np.float32)
+    _check(lib().hyperattn_get_projections(d, hash_bits, seed, w.ctypes.data), "hyperattn_get_projections")
+    return w
+
+
+def last_device_status(stream=None) -> int:
+    st = C.c_int(0)
+    s = stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    _check(lib().hyperattn_last_device_status(s, C.byref(st)), "hyperattn_last_device_status")
+    return int(st.value)
+
+
+def profile_enable(on: bool):
+    lib().hyperattn_profile_enable(int(on))
+
+
+def profile_reset():
+    lib().hyperattn_profile_reset()
+
+
+def profile_read() -> dict:
+    t = _StageTimes()
+    _check(lib().hyperattn_profile_read(C.byref(t)), "hyperattn_profile_read")
+    return {"calls": t.calls, "ms": {STAGE_NAMES[i]: float(t.ms[i]) for i in range(NUM_STAGES)},
+            "launches": {STAGE_NAMES[i]: int(t.launches[i]) for i in range(NUM_STAGES)}}
+
+
+def release():
+    lib().hyperattn_release()
+
+
+def version() -> int:
+    return int(lib().hyperattn_version())

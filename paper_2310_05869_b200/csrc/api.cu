@@ -1,0 +1,466 @@
+// C ABI of the HyperAttention forward library: argument checks, workspace plan, stage
+// sequencing.  Everything here runs on the host; all arithmetic of the method runs in the
+// kernels of hash.cu, sort.cu, attn_*.cu and merge.cu.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <vector>
+
+#include "../../include/hyperattn.h"
+#include "attn_common.cuh"
+
+namespace hyperattn {
+cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st);
+
+namespace {
+
+constexpr int kVersion = 1;
+constexpr size_t kAlign = 256;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// ---- geometry / validation ---------------------------------------------------------------
+int build_geometry(const hyperattn_params& p, Geometry& g) {
+  if (p.B <= 0 || p.H <= 0 || p.n <= 0 || p.block <= 0 || p.samples < 0) return HYPERATTN_INVALID_ARGUMENT;
+  if (p.dtype != HYPERATTN_BF16 && p.dtype != HYPERATTN_FP32) return HYPERATTN_INVALID_ARGUMENT;
+  if (p.out_dtype != HYPERATTN_BF16 && p.out_dtype != HYPERATTN_FP32) return HYPERATTN_INVALID_ARGUMENT;
+  if (p.d != 64 && p.d != 128) return HYPERATTN_UNSUPPORTED_SHAPE;
+  if (p.hash_bits < 1 || p.hash_bits > 8) return HYPERATTN_UNSUPPORTED_SHAPE;
+  if ((long long)p.B * p.H > (1 << 20)) return HYPERATTN_UNSUPPORTED_SHAPE;
+  if (p.n > (1 << 28)) return HYPERATTN_UNSUPPORTED_SHAPE;
+  std::memset(&g, 0, sizeof(g));
+  g.G = p.B * p.H; g.n = p.n; g.d = p.d; g.b = p.block; g.m = p.samples; g.r = p.hash_bits;
+  if (!p.causal) {
+    g.causal = 0; g.L = 0; g.leaf = p.n; g.unit = p.n;
+    if (p.block < p.n) {
+      if (p.n % p.block) return HYPERATTN_UNSUPPORTED_SHAPE;
+      g.levels = 1; g.nl = p.n; g.nodes = 1; g.sorted = 1;
+    }
+  } else {
+    if (p.n0 <= 0) return HYPERATTN_INVALID_ARGUMENT;
+    g.causal = 1;
+    int L = 0;
+    if (p.n > p.n0) {
+      long long s = p.n0;
+      while (s < p.n) { s *= 2; ++L; }
+      if (s != p.n || L > kMaxLevels) return HYPERATTN_UNSUPPORTED_SHAPE;
+    }
+    g.L = L;
+    g.leaf = L ? p.n0 : p.n;
+    g.unit = g.leaf;
+    if (L) {
+      g.levels = L; g.nl = p.n / 2; g.nodes = (1 << L) - 1;
+      for (int l = 0; l < L; ++l) {
+        const int s = p.n >> (l + 1);
+        if (p.block < s) {
+          if (s % p.block) return HYPERATTN_UNSUPPORTED_SHAPE;
+          g.sorted = 1;
+        }
+      }
+    }
+  }
+  if (g.sorted) {
+    const int bpad = (g.b + 63) / 64 * 64, mpad = (g.m + 63) / 64 * 64;
+    if (bpad + mpad > kMaxNodeKeys) return HYPERATTN_UNSUPPORTED_SHAPE;
+  }
+  g.chunks_per_unit = (g.unit + kSortChunk - 1) / kSortChunk;
+  g.chunks_per_seg = (g.n / g.unit) * g.chunks_per_unit;
+  return HYPERATTN_OK;
+}
+
+struct Plan {
+  size_t q16, k16, v16, ids, hist, offs, perm_q, perm_k, rank_k, samples, part_o, part_lse, total;
+};
+
+Plan make_plan(const Geometry& g, int is_fp32) {
+  Plan pl;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  const size_t tensor16 = (size_t)g.G * g.n * g.d * 2;
+  pl.q16 = take(is_fp32 ? tensor16 : 0);
+  pl.k16 = take(is_fp32 ? tensor16 : 0);
+  pl.v16 = take(is_fp32 ? tensor16 : 0);
+  const size_t lvl_rows = (size_t)g.levels * g.G * g.nl;
+  pl.ids = take(g.sorted ? (size_t)2 * g.G * g.n : 0);
+  pl.hist = take(g.sorted ? (size_t)2 * g.G * g.chunks_per_seg * kBuckets * 4 : 0);
+  const size_t chunks_per_level = g.sorted ? (size_t)(g.nl / g.unit) * g.chunks_per_unit : 0;
+  pl.offs = take((size_t)2 * g.levels * g.G * chunks_per_level * kBuckets * 4);
+  pl.perm_q = take(g.sorted ? lvl_rows * 4 : 0);
+  pl.perm_k = take(g.sorted ? lvl_rows * 4 : 0);
+  pl.rank_k = take(g.sorted ? lvl_rows * 4 : 0);
+  pl.samples = take((size_t)g.G * g.nodes * g.m * 4);
+  const size_t part_rows = g.L ? (size_t)g.G * g.n + lvl_rows : 0;
+  pl.part_o = take(part_rows * g.d * 4);
+  pl.part_lse = take(part_rows * 4);
+  pl.total = off + kAlign;
+  return pl;
+}
+
+// ---- direction matrix (Def. 1): Philox + Box-Muller in fp64, rounded once to fp32 -------------
+void make_directions(int d, int r, uint64_t seed, float* w) {
+  const int total = d * r, calls = (total + 3) / 4;
+  const double two_pi = 6.283185307179586476925286766559;
+  for (int c = 0; c < calls; ++c) {
+    const Philox4 x = philox4x32_10((uint32_t)c, 0u, 0u, kDomainDirections, (uint32_t)seed, (uint32_t)(seed >> 32));
+    double u[4], z[4];
+    for (int i = 0; i < 4; ++i) u[i] = ((double)x.x[i] + 0.5) * (1.0 / 4294967296.0);
+    for (int a = 0; a < 4; a += 2) {
+      const double rho = std::sqrt(-2.0 * std::log(u[a])), ang = two_pi * u[a + 1];
+      z[a] = rho * std::cos(ang);
+      z[a + 1] = rho * std::sin(ang);
+    }
+    for (int i = 0; i < 4; ++i)
+      if (4 * c + i < total) w[4 * c + i] = (float)z[i];
+  }
+}
+
+// ---- per-process state ---------------------------------------------------------------------
+struct DeviceState {
+  void* ws = nullptr; size_t ws_bytes = 0;
+  void* host_stage = nullptr; size_t host_stage_bytes = 0;   // device staging for the host-buffer entry
+  int* status = nullptr;
+};
+struct StageEvents { cudaEvent_t beg, end; int stage; int launches; };
+
+std::mutex g_mu;
+std::map<int, DeviceState> g_dev;
+bool g_profile = false;
+std::vector<StageEvents> g_events;
+std::vector<cudaEvent_t> g_event_pool;
+int g_profile_calls = 0;
+struct { int d = 0, r = 0; uint64_t seed = 0; bool valid = false; float w[128 * 8]; } g_wcache;
+
+cudaEvent_t take_event() {
+  if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct StageScope {
+  cudaStream_t st; int stage; int launches; bool on; cudaEvent_t beg = nullptr;
+  StageScope(cudaStream_t s, int stage_, int launches_) : st(s), stage(stage_), launches(launches_), on(g_profile && launches_ > 0) {
+    if (on) { beg = take_event(); cudaEventRecord(beg, st); }
+  }
+  ~StageScope() {
+    if (on) { cudaEvent_t end = take_event(); cudaEventRecord(end, st); g_events.push_back({beg, end, stage, launches}); }
+  }
+};
+
+int check_ptrs(const hyperattn_params& p) {
+  if (!p.q || !p.k || !p.v || !p.out || !p.lse) return HYPERATTN_INVALID_ARGUMENT;
+  const void* ptrs[5] = {p.q, p.k, p.v, p.out, p.lse};
+  for (const void* x : ptrs)
+    if (reinterpret_cast<uintptr_t>(x) & 15) return HYPERATTN_MISALIGNED;
+  if (p.out == p.q || p.out == p.k || p.out == p.v || (void*)p.lse == p.out) return HYPERATTN_MISALIGNED;
+  if (p.workspace && (reinterpret_cast<uintptr_t>(p.workspace) & 15)) return HYPERATTN_MISALIGNED;
+  return HYPERATTN_OK;
+}
+
+int forward_impl(const hyperattn_params& p) {
+  Geometry g;
+  int rc = build_geometry(p, g);
+  if (rc) return rc;
+  rc = check_ptrs(p);
+  if (rc) return rc;
+  const int is_fp32 = p.dtype == HYPERATTN_FP32;
+  const int out_fp32 = p.out_dtype == HYPERATTN_FP32;
+  const Plan pl = make_plan(g, is_fp32);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceState& ds = g_dev[dev];
+  if (!ds.status) {
+    if (cudaMalloc(&ds.status, 256) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+    if (cudaMemset(ds.status, 0, 256) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  }
+  char* base = nullptr;
+  if (p.workspace) {
+    if (p.workspace_bytes < pl.total) return HYPERATTN_WORKSPACE_TOO_SMALL;
+    base = reinterpret_cast<char*>(p.workspace);
+  } else {
+    if (ds.ws_bytes < pl.total) {
+      cudaDeviceSynchronize();
+      if (ds.ws) cudaFree(ds.ws);
+      ds.ws = nullptr; ds.ws_bytes = 0;
+      if (cudaMalloc(&ds.ws, pl.total) != cudaSuccess) { cudaGetLastError(); return HYPERATTN_CUDA_ERROR; }
+      ds.ws_bytes = pl.total;
+    }
+    base = reinterpret_cast<char*>(ds.ws);
+  }
+  base = reinterpret_cast<char*>(align_up(reinterpret_cast<uintptr_t>(base)));
+
+  Workspace ws;
+  ws.q16 = reinterpret_cast<__nv_bfloat16*>(base + pl.q16);
+  ws.k16 = reinterpret_cast<__nv_bfloat16*>(base + pl.k16);
+  ws.v16 = reinterpret_cast<__nv_bfloat16*>(base + pl.v16);
+  ws.ids = reinterpret_cast<uint8_t*>(base + pl.ids);
+  ws.hist = reinterpret_cast<uint32_t*>(base + pl.hist);
+  ws.offs = reinterpret_cast<uint32_t*>(base + pl.offs);
+  ws.perm_q = reinterpret_cast<int32_t*>(base + pl.perm_q);
+  ws.perm_k = reinterpret_cast<int32_t*>(base + pl.perm_k);
+  ws.rank_k = reinterpret_cast<int32_t*>(base + pl.rank_k);
+  ws.samples = reinterpret_cast<int32_t*>(base + pl.samples);
+  ws.part_o = reinterpret_cast<float*>(base + pl.part_o);
+  ws.part_lse = reinterpret_cast<float*>(base + pl.part_lse);
+  ws.status = ds.status;
+
+  const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.f / std::sqrt((float)p.d);
+  const hyperattn_debug* dbg = p.debug;
+  if (g_profile) ++g_profile_calls;
+  cudaError_t e = cudaSuccess;
+#define HA_CHECK(x) do { e = (x); if (e != cudaSuccess) { std::fprintf(stderr, "hyperattn: %s failed: %s\n", #x, cudaGetErrorString(e)); return HYPERATTN_CUDA_ERROR; } } while (0)
+
+  const __nv_bfloat16 *q16 = reinterpret_cast<const __nv_bfloat16*>(p.q), *k16 = reinterpret_cast<const __nv_bfloat16*>(p.k),
+                      *v16 = reinterpret_cast<const __nv_bfloat16*>(p.v);
+  if (is_fp32) {
+    StageScope sc(st, HYPERATTN_STAGE_CONVERT, 3);
+    const size_t cnt = (size_t)g.G * g.n * g.d;
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.q), ws.q16, cnt, st));
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.k), ws.k16, cnt, st));
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.v), ws.v16, cnt, st));
+    q16 = ws.q16; k16 = ws.k16; v16 = ws.v16;
+  }
+  if (g.sorted) {
+    if (!g_wcache.valid || g_wcache.d != g.d || g_wcache.r != g.r || g_wcache.seed != p.seed) {
+      make_directions(g.d, g.r, p.seed, g_wcache.w);
+      g_wcache.d = g.d; g_wcache.r = g.r; g_wcache.seed = p.seed; g_wcache.valid = true;
+    }
+    {
+      StageScope sc(st, HYPERATTN_STAGE_HASH, 1);
+      HA_CHECK(launch_hash(g, p.q, p.k, is_fp32, g_wcache.w, ws, dbg ? dbg->near_zero_bits : nullptr, st));
+    }
+    {
+      StageScope sc(st, HYPERATTN_STAGE_SAMPLE, g.m > 0 ? 1 : 0);
+      HA_CHECK(launch_samples(g, p.seed, ws, st));
+    }
+    {
+      StageScope sc(st, HYPERATTN_STAGE_SORT_SCAN, 1);
+      HA_CHECK(launch_sort_scan(g, ws, st));
+    }
+    {
+      StageScope sc(st, HYPERATTN_STAGE_SORT_SCATTER, 1);
+      HA_CHECK(launch_sort_scatter(g, ws, st));
+    }
+    if (dbg) {
+      const size_t lvl_bytes = (size_t)g.levels * g.G * g.nl * 4;
+      if (dbg->q_ids) HA_CHECK(cudaMemcpyAsync(dbg->q_ids, ws.ids, (size_t)g.G * g.n, cudaMemcpyDeviceToDevice, st));
+      if (dbg->k_ids) HA_CHECK(cudaMemcpyAsync(dbg->k_ids, ws.ids + (size_t)g.G * g.n, (size_t)g.G * g.n, cudaMemcpyDeviceToDevice, st));
+      if (dbg->perm_q) HA_CHECK(cudaMemcpyAsync(dbg->perm_q, ws.perm_q, lvl_bytes, cudaMemcpyDeviceToDevice, st));
+      if (dbg->perm_k) HA_CHECK(cudaMemcpyAsync(dbg->perm_k, ws.perm_k, lvl_bytes, cudaMemcpyDeviceToDevice, st));
+      if (dbg->rank_k) HA_CHECK(cudaMemcpyAsync(dbg->rank_k, ws.rank_k, lvl_bytes, cudaMemcpyDeviceToDevice, st));
+      if (dbg->samples && g.m > 0)
+        HA_CHECK(cudaMemcpyAsync(dbg->samples, ws.samples, (size_t)g.G * g.nodes * g.m * 4, cudaMemcpyDeviceToDevice, st));
+    }
+  }
+
+  // ---- attention tiles: one launch over leaves and all recursion levels -------------------
+  AttnArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.q = q16; a.k = k16; a.v = v16; a.g = g;
+  a.scale_log2 = scale * 1.4426950408889634f;
+  a.perm_q = ws.perm_q; a.perm_k = ws.perm_k; a.rank_k = ws.rank_k; a.samples = ws.samples;
+  a.part_o = ws.part_o; a.part_lse = ws.part_lse; a.out = p.out; a.lse = p.lse;
+  a.out_fp32 = out_fp32;
+  a.direct = g.L == 0;
+  a.dense_causal = g.causal;
+  a.tiles_per_block = (g.b + kTileQ - 1) / kTileQ;
+  const bool has_leaves = g.causal || !g.sorted;
+  if (has_leaves) {
+    a.tiles_per_leaf = (g.leaf + kTileQ - 1) / kTileQ;
+    a.leaves_per_seg = g.n / g.leaf;
+    a.n_leaf_tiles = g.G * a.leaves_per_seg * a.tiles_per_leaf;
+  }
+  long long tiles = a.n_leaf_tiles;
+  for (int l = 0; l < g.levels; ++l) {
+    int s, q0, k0;
+    node_rows(g, l, 0, s, q0, k0);
+    const int nodes_lvl = g.causal ? (1 << l) : 1;
+    a.level_start[l] = (int)tiles;
+    a.level_sorted[l] = g.b < s;
+    const long long per_node = a.level_sorted[l] ? (long long)(s / g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
+    tiles += per_node * nodes_lvl * g.G;
+    if (tiles > 0x7fffffffLL) return HYPERATTN_UNSUPPORTED_SHAPE;
+  }
+  a.level_start[g.levels] = (int)tiles;
+  a.total_tiles = (int)tiles;
+  {
+    StageScope sc(st, HYPERATTN_STAGE_ATTENTION, 1);
+    HA_CHECK(launch_attention_mma(a, st));
+  }
+  if (g.L) {
+    StageScope sc(st, HYPERATTN_STAGE_MERGE, 1);
+    HA_CHECK(launch_merge(g, ws, p.out, p.lse, out_fp32, st));
+  }
+#undef HA_CHECK
+  return HYPERATTN_OK;
+}
+
+}  // namespace
+}  // namespace hyperattn
+
+using namespace hyperattn;
+
+extern "C" {
+
+int hyperattn_forward_ex(const hyperattn_params* p) {
+  if (!p) return HYPERATTN_INVALID_ARGUMENT;
+  return forward_impl(*p);
+}
+
+int hyperattn_forward(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int n,
+                      int d, int block, int samples, int hash_bits, int causal, int n0, uint64_t seed,
+                      void* stream) {
+  hyperattn_params p;
+  std::memset(&p, 0, sizeof(p));
+  p.q = q; p.k = k; p.v = v; p.out = out; p.lse = lse;
+  p.B = B; p.H = H; p.n = n; p.d = d; p.block = block; p.samples = samples; p.hash_bits = hash_bits;
+  p.causal = causal; p.n0 = n0; p.seed = seed;
+  p.dtype = HYPERATTN_BF16; p.out_dtype = HYPERATTN_BF16; p.softmax_scale = 0.f;
+  p.stream = stream;
+  return forward_impl(p);
+}
+
+int hyperattn_forward_host(const hyperattn_params* hp) {
+  if (!hp) return HYPERATTN_INVALID_ARGUMENT;
+  if (!hp->q || !hp->k || !hp->v || !hp->out || !hp->lse) return HYPERATTN_INVALID_ARGUMENT;
+  Geometry g;
+  int rc = build_geometry(*hp, g);
+  if (rc) return rc;
+  const size_t es = hp->dtype == HYPERATTN_FP32 ? 4 : 2, eo = hp->out_dtype == HYPERATTN_FP32 ? 4 : 2;
+  const size_t elems = (size_t)g.G * g.n * g.d;
+  const size_t in_b = align_up(elems * es), out_b = align_up(elems * eo), lse_b = align_up((size_t)g.G * g.n * 4);
+  const size_t need = 3 * in_b + out_b + lse_b;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  char* stage = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState& ds = g_dev[dev];
+    if (ds.host_stage_bytes < need) {
+      cudaDeviceSynchronize();
+      if (ds.host_stage) cudaFree(ds.host_stage);
+      ds.host_stage = nullptr; ds.host_stage_bytes = 0;
+      if (cudaMalloc(&ds.host_stage, need) != cudaSuccess) { cudaGetLastError(); return HYPERATTN_CUDA_ERROR; }
+      ds.host_stage_bytes = need;
+    }
+    stage = reinterpret_cast<char*>(ds.host_stage);
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(hp->stream);
+  hyperattn_params p = *hp;
+  p.q = stage; p.k = stage + in_b; p.v = stage + 2 * in_b;
+  p.out = stage + 3 * in_b; p.lse = reinterpret_cast<float*>(stage + 3 * in_b + out_b);
+  if (cudaMemcpyAsync(const_cast<void*>(p.q), hp->q, elems * es, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(const_cast<void*>(p.k), hp->k, elems * es, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(const_cast<void*>(p.v), hp->v, elems * es, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return HYPERATTN_CUDA_ERROR;
+  rc = forward_impl(p);
+  if (rc) return rc;
+  if (cudaMemcpyAsync(hp->out, p.out, elems * eo, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(hp->lse, p.lse, (size_t)g.G * g.n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return HYPERATTN_CUDA_ERROR;
+  return HYPERATTN_OK;
+}
+
+int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes) {
+  if (!p || !bytes) return HYPERATTN_INVALID_ARGUMENT;
+  Geometry g;
+  const int rc = build_geometry(*p, g);
+  if (rc) return rc;
+  *bytes = make_plan(g, p->dtype == HYPERATTN_FP32).total;
+  return HYPERATTN_OK;
+}
+
+int hyperattn_get_projections(int d, int hash_bits, uint64_t seed, float* host_out) {
+  if (!host_out || d <= 0 || d > 128 || hash_bits < 1 || hash_bits > 8) return HYPERATTN_INVALID_ARGUMENT;
+  make_directions(d, hash_bits, seed, host_out);
+  return HYPERATTN_OK;
+}
+
+int hyperattn_last_device_status(void* stream, int* status) {
+  if (!status) return HYPERATTN_INVALID_ARGUMENT;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceState& ds = g_dev[dev];
+  *status = 0;
+  if (!ds.status) return HYPERATTN_OK;
+  int word = 0;
+  if (cudaMemcpy(&word, ds.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  if (word) {
+    *status = HYPERATTN_DEVICE_TIMEOUT;
+    cudaMemset(ds.status, 0, 4);
+  }
+  return HYPERATTN_OK;
+}
+
+int hyperattn_profile_enable(int on) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  g_profile = on != 0;
+  return HYPERATTN_OK;
+}
+
+int hyperattn_profile_reset(void) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  for (auto& ev : g_events) { g_event_pool.push_back(ev.beg); g_event_pool.push_back(ev.end); }
+  g_events.clear();
+  g_profile_calls = 0;
+  return HYPERATTN_OK;
+}
+
+int hyperattn_profile_read(hyperattn_stage_times* out) {
+  if (!out) return HYPERATTN_INVALID_ARGUMENT;
+  std::lock_guard<std::mutex> lock(g_mu);
+  std::memset(out, 0, sizeof(*out));
+  for (auto& ev : g_events) {
+    if (cudaEventSynchronize(ev.end) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ev.beg, ev.end) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+    out->ms[ev.stage] += ms;
+    out->launches[ev.stage] += ev.launches;
+  }
+  out->calls = g_profile_calls;
+  return HYPERATTN_OK;
+}
+
+int hyperattn_release(void) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  int cur = 0;
+  cudaGetDevice(&cur);
+  for (auto& kv : g_dev) {
+    cudaSetDevice(kv.first);
+    cudaDeviceSynchronize();
+    if (kv.second.ws) cudaFree(kv.second.ws);
+    if (kv.second.host_stage) cudaFree(kv.second.host_stage);
+    if (kv.second.status) cudaFree(kv.second.status);
+  }
+  g_dev.clear();
+  for (auto& ev : g_events) { cudaEventDestroy(ev.beg); cudaEventDestroy(ev.end); }
+  g_events.clear();
+  for (auto& e : g_event_pool) cudaEventDestroy(e);
+  g_event_pool.clear();
+  cudaSetDevice(cur);
+  return HYPERATTN_OK;
+}
+
+const char* hyperattn_status_string(int status) {
+  switch (status) {
+    case HYPERATTN_OK: return "ok";
+    case HYPERATTN_INVALID_ARGUMENT: return "invalid argument";
+    case HYPERATTN_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case HYPERATTN_MISALIGNED: return "misaligned or aliasing pointer";
+    case HYPERATTN_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case HYPERATTN_CUDA_ERROR: return "CUDA error";
+    case HYPERATTN_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int hyperattn_version(void) { return kVersion; }
+
+}  // extern "C"

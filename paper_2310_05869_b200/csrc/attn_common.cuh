@@ -1,0 +1,119 @@
+// Tile schedule shared by the attention kernels.
+//
+// One attention tile = 128 query rows against a list of key tiles.  Two kinds:
+//   DENSE  contiguous query rows against a contiguous key range, optionally with the causal
+//          mask M^C_ij = 1{i >= j}: the exact base case of the causal recursion (Alg. 4 read
+//          with a base size), a problem that is a single block (b >= N), and nothing else.
+//   NODE   128 consecutive *sorted* query positions of block beta of a HyperAttention problem:
+//          keys are the b keys of sorted block beta (Alg. 1 line 4 / Sec. 4 block-diagonal
+//          part) followed by the m sampled keys (Alg. 2 line 7), which carry the weight N/m
+//          as an additive log2(N/m) on the logit, or minus infinity when the sampled key
+//          lies in block beta itself (the factor 1 - M^H).
+// All tiles of all recursion levels and all leaves of one forward call form one flat list
+// so that a single launch covers them; heavy (leaf) tiles come first.
+#pragma once
+#include "common.cuh"
+
+namespace hyperattn {
+
+constexpr int kMaxLevels = 24;
+constexpr int kMaxNodeKeys = 2048;   // padded b + padded m must fit the key index table
+
+struct AttnArgs {
+  const __nv_bfloat16 *q, *k, *v;    // [G, n, D]
+  Geometry g;
+  float scale_log2;                  // softmax scale * log2(e)
+  const int32_t *perm_q, *perm_k, *rank_k, *samples;
+  float *part_o, *part_lse;          // partial results (fp32), used when !direct
+  void* out; float* lse;             // final results, used when direct
+  int out_fp32;
+  int direct;
+  // dense (leaf) tiles
+  int dense_causal;
+  int tiles_per_leaf, leaves_per_seg, n_leaf_tiles;
+  // node tiles, per level
+  int level_start[kMaxLevels + 1];   // first tile index of each level (after the leaf tiles)
+  int level_sorted[kMaxLevels];      // 1: sortLSH node tiles; 0: single-block node (dense tiles)
+  int tiles_per_block;               // ceil(b / 128)
+  int total_tiles;
+};
+
+struct TileDesc {
+  int mode;            // 0 dense, 1 node
+  int seg;
+  int nq;              // valid query rows
+  int q0;              // dense: first query row (segment-relative)
+  int k0, nk;          // dense: key range; node: first key row of the node, N
+  int causal;          // dense: apply j_local <= i_local
+  int qk_off;          // dense causal: local index of the tile's first query row relative to k0
+  int qnode0;          // node: first query row of the node (segment-relative)
+  size_t slice;        // node: offset of this node's slice in perm_q / perm_k / rank_k
+  int spos0;           // node: first sorted position of the tile
+  int beta;            // node: block index
+  int node;            // node: heap index
+  size_t orow_base;    // output row index = orow_base + (segment-relative query row + odelta)
+  int odelta;
+  int partial;         // 1: write part_o/part_lse, 0: write out/lse
+};
+
+__device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
+  const Geometry& g = a.g;
+  TileDesc t;
+  t.partial = !a.direct;
+  if (tile < a.n_leaf_tiles) {
+    const int per = g.G * a.leaves_per_seg;
+    const int tt = a.tiles_per_leaf - 1 - tile / per;      // heavy tiles first
+    const int rem = tile % per;
+    t.seg = rem / a.leaves_per_seg;
+    const int leaf = rem % a.leaves_per_seg;
+    t.mode = 0;
+    t.k0 = leaf * g.leaf; t.nk = g.leaf;
+    t.q0 = t.k0 + tt * kTileQ;
+    t.nq = min(kTileQ, g.leaf - tt * kTileQ);
+    t.causal = a.dense_causal;
+    t.qk_off = tt * kTileQ;
+    t.orow_base = (size_t)t.seg * g.n; t.odelta = 0;
+    return t;
+  }
+  int level = 0;
+  while (level + 1 < g.levels && tile >= a.level_start[level + 1]) ++level;
+  int idx = tile - a.level_start[level];
+  int s, q0n, k0n;
+  node_rows(g, level, 0, s, q0n, k0n);
+  const int nodes_lvl = g.causal ? (1 << level) : 1;
+  const size_t region = a.direct ? 0 : (size_t)g.G * g.n + (size_t)level * g.G * g.nl;
+  if (a.level_sorted[level]) {
+    const int tiles_node = (s / g.b) * a.tiles_per_block;
+    const int tn = idx % tiles_node; idx /= tiles_node;
+    const int j = idx % nodes_lvl;
+    t.seg = idx / nodes_lvl;
+    node_rows(g, level, j, s, q0n, k0n);
+    t.mode = 1;
+    t.beta = tn / a.tiles_per_block;
+    const int sub = tn % a.tiles_per_block;
+    t.spos0 = t.beta * g.b + sub * kTileQ;
+    t.nq = min(kTileQ, g.b - sub * kTileQ);
+    t.k0 = k0n; t.nk = s; t.qnode0 = q0n;
+    t.slice = ((size_t)level * g.G + t.seg) * g.nl + (g.causal ? (size_t)j * s : 0);
+    t.node = g.causal ? (1 << level) - 1 + j : 0;
+    t.causal = 0; t.q0 = 0; t.qk_off = 0;
+    if (a.direct) { t.orow_base = (size_t)t.seg * g.n; t.odelta = 0; }
+    else { t.orow_base = region + (size_t)t.seg * g.nl + (size_t)j * s; t.odelta = -q0n; }
+  } else {
+    const int tiles_node = (s + kTileQ - 1) / kTileQ;
+    const int tn = idx % tiles_node; idx /= tiles_node;
+    const int j = idx % nodes_lvl;
+    t.seg = idx / nodes_lvl;
+    node_rows(g, level, j, s, q0n, k0n);
+    t.mode = 0;
+    t.k0 = k0n; t.nk = s;
+    t.q0 = q0n + tn * kTileQ;
+    t.nq = min(kTileQ, s - tn * kTileQ);
+    t.causal = 0; t.qk_off = 0;
+    if (a.direct) { t.orow_base = (size_t)t.seg * g.n; t.odelta = 0; }
+    else { t.orow_base = region + (size_t)t.seg * g.nl + (size_t)j * s; t.odelta = -q0n; }
+  }
+  return t;
+}
+
+}  // namespace hyperattn

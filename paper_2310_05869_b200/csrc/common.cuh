@@ -1,0 +1,94 @@
+// Shared declarations of the HyperAttention forward library (sm_100a).
+// Notation follows the paper: n rows, d head dimension, b block size, m sampled columns,
+// r hash bits, G = B*H independent (batch, head) segments.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace hyperattn {
+
+constexpr int kSortChunk = 2048;      // rows per histogram / scatter chunk
+constexpr int kBuckets = 256;         // 2^r with r <= 8
+constexpr int kTileQ = 128;           // query rows per attention tile
+constexpr int kMaxLevelsMerge = 24;   // deepest causal recursion supported
+
+// ---- Philox4x32-10 (Salmon et al., SC'11); identical on host and device -------------
+struct Philox4 { uint32_t x[4]; };
+
+__host__ __device__ inline void mulhilo32(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
+#ifdef __CUDA_ARCH__
+  lo = a * b;
+  hi = __umulhi(a, b);
+#else
+  uint64_t p = (uint64_t)a * b;
+  lo = (uint32_t)p;
+  hi = (uint32_t)(p >> 32);
+#endif
+}
+
+__host__ __device__ inline Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int rnd = 0; rnd < 10; ++rnd) {
+    if (rnd > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    uint32_t hi0, lo0, hi1, lo1;
+    mulhilo32(0xD2511F53u, c0, hi0, lo0);
+    mulhilo32(0xCD9E8D57u, c2, hi1, lo1);
+    uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+  }
+  Philox4 r; r.x[0] = c0; r.x[1] = c1; r.x[2] = c2; r.x[3] = c3;
+  return r;
+}
+constexpr uint32_t kDomainDirections = 1, kDomainSamples = 2;
+
+// ---- geometry of one forward call, shared by all stages --------------------------------
+// "unit" = the largest row range that never straddles a recursion node: a causal leaf of n0
+// rows, or the whole segment.  Units are cut into chunks of at most kSortChunk rows; one
+// hash CTA produces the ids and the 256-bin histogram of one chunk, one scatter CTA places it.
+struct Geometry {
+  int G, n, d;
+  int b, m, r;
+  int causal;          // 1: causal with L >= 1 levels or a single causal leaf
+  int L;               // number of recursion levels with off-diagonal nodes (0: none)
+  int leaf;            // rows per exact leaf (n if L == 0)
+  int unit;            // rows per unit
+  int chunks_per_unit;
+  int chunks_per_seg;  // (n / unit) * chunks_per_unit
+  int levels;          // sorted levels: L if causal, else 1 (0 if nothing is sorted)
+  int nl;              // sorted rows per (level, segment, side): n/2 causal, n non-causal
+  int nodes;           // off-diagonal nodes per segment (heap-numbered)
+  int sorted;          // 1 if any node needs sortLSH (some node has b < its size)
+};
+
+// node j of level l: size s, first query row, first key row (non-causal: the whole segment)
+__host__ __device__ inline void node_rows(const Geometry& g, int level, int j, int& s, int& q0, int& k0) {
+  if (!g.causal) { s = g.n; q0 = 0; k0 = 0; return; }
+  s = g.n >> (level + 1);
+  q0 = (2 * j + 1) * s;
+  k0 = 2 * j * s;
+}
+
+// ---- stage launchers (each enqueues on `st`; returns cudaGetLastError()) ---------------
+struct Workspace {
+  __nv_bfloat16 *q16, *k16, *v16;  // bf16 staging of fp32 inputs (else null)
+  uint8_t* ids;                    // [2, G, n]
+  uint32_t* hist;                  // [2, G, chunks_per_seg, 256]
+  uint32_t* offs;                  // [2, levels, G, chunks per (level,seg,side), 256]
+  int32_t *perm_q, *perm_k, *rank_k;  // [levels, G, nl]
+  int32_t* samples;                // [G, nodes, m]
+  float *part_o, *part_lse;        // causal partials: leaf [G,n,(d)] then per level [G,n/2,(d)]
+  int* status;                     // device status word
+};
+
+cudaError_t launch_convert(const float* src, __nv_bfloat16* dst, size_t count, cudaStream_t st);
+cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
+                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st);
+cudaError_t launch_samples(const Geometry& g, uint64_t seed, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_merge(const Geometry& g, const Workspace& ws, void* out, float* lse, int out_fp32,
+                         cudaStream_t st);
+
+}  // namespace hyperattn

@@ -1,0 +1,232 @@
+// Stage 1 of sortLSH (Def. 1; Alg. 1 line 2): bucket id of every query and key row.
+//
+//   p_t = <x, w_t>,  bit_t = [p_t > 0],  g = sum_t bit_t 2^t,  id = Gray rank of g.
+//
+// The kernel streams Q and K once (HBM-bound: d*e bytes in, 1 byte out per row) and also
+// leaves a 256-bin histogram per chunk of rows, which is the first pass of the counting
+// argsort (Alg. 1 line 3).
+//
+// bf16 rows: the projection [16 rows x d] . [d x 8] runs on the tensor cores
+// (mma.sync m16n8k16, fp32 accumulate).  Each lane fetches its operands with 128-bit loads;
+// because a dot product does not care in which order the coordinates are visited, the
+// coordinates a lane happens to hold are assigned to MMA k-slots by a fixed permutation and
+// the direction matrix is laid out with the same permutation.  The fp32 directions are split
+// into three bf16 terms (w = w1 + w2 + w3 exactly), so the products are exact and only the
+// fp32 accumulation rounds; signs can differ from an exact evaluation only where |p_t| is
+// within ~1e-5 of zero.
+#include "common.cuh"
+
+namespace hyperattn {
+namespace {
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+// Gray rank: h with h ^ (h >> 1) == g (prefix xor), 8-bit patterns.
+__device__ __forceinline__ uint32_t gray_rank8(uint32_t g) {
+  g ^= g >> 1; g ^= g >> 2; g ^= g >> 4;
+  return g & 0xFFu;
+}
+
+struct HashArgs {
+  const void* x[2];       // Q, K  [G, n, d]
+  float w[128 * 8];       // [d, r] directions, passed by value (<= 4 KB of kernel parameters)
+  uint8_t* ids;           // [2, G, n]
+  uint32_t* hist;         // [2, G, chunks_per_seg, 256]
+  unsigned long long* near_zero;
+  int G, n, r;
+  int unit, chunks_per_unit, chunks_per_seg;
+};
+
+// One CTA = one chunk (<= kSortChunk rows of one side of one segment).
+template <int D>
+__global__ void __launch_bounds__(256) hash_bf16_kernel(const __grid_constant__ HashArgs a) {
+  constexpr int KS = D / 16;             // MMA k-steps
+  constexpr int CPL = D / 32;            // 16-byte chunks per lane per row
+  __shared__ __align__(16) uint8_t s_ids[kSortChunk];
+  __shared__ uint32_t s_hist[kBuckets];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+  int cta = blockIdx.x;
+  const int chunk = cta % a.chunks_per_seg; cta /= a.chunks_per_seg;
+  const int seg = cta % a.G;
+  const int side = cta / a.G;
+  const int unit_idx = chunk / a.chunks_per_unit, cu = chunk % a.chunks_per_unit;
+  const int row0 = unit_idx * a.unit + cu * kSortChunk;
+  const int rows = min(kSortChunk, a.unit - cu * kSortChunk);
+
+  s_hist[tid] = 0;
+
+  // Direction fragments.  k-slot (step s, half h, element e) of lane (gid, tig) holds
+  // coordinate 8*(tig + 4*(s>>1)) + 2*(2*(s&1) + h) + e; column gid is direction gid.
+  uint32_t bw[3][KS][2];
+#pragma unroll
+  for (int s = 0; s < KS; ++s)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float w[2], t1[2], t2[2], t3[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int coord = 8 * (tig + 4 * (s >> 1)) + 2 * (2 * (s & 1) + h) + e;
+        w[e] = (gid < a.r) ? a.w[coord * a.r + gid] : 0.f;
+        t1[e] = __bfloat162float(__float2bfloat16_rn(w[e]));
+        const float r1 = w[e] - t1[e];
+        t2[e] = __bfloat162float(__float2bfloat16_rn(r1));
+        t3[e] = __bfloat162float(__float2bfloat16_rn(r1 - t2[e]));
+      }
+      bw[0][s][h] = pack_bf16(t1[0], t1[1]);
+      bw[1][s][h] = pack_bf16(t2[0], t2[1]);
+      bw[2][s][h] = pack_bf16(t3[0], t3[1]);
+    }
+  __syncthreads();
+
+  const char* base = reinterpret_cast<const char*>(a.x[side]) + ((size_t)seg * a.n + row0) * (D * 2);
+  unsigned nz = 0;
+  const int groups = (rows + 15) >> 4;
+  for (int grp = warp; grp < groups; grp += 8) {
+    const int ra = grp * 16 + gid, rb = ra + 8;
+    uint4 xa[CPL], xb[CPL];
+#pragma unroll
+    for (int h = 0; h < CPL; ++h) {
+      xa[h] = ra < rows ? ldg_stream(base + (size_t)ra * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
+      xb[h] = rb < rows ? ldg_stream(base + (size_t)rb * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
+    }
+    float hi[4] = {0.f, 0.f, 0.f, 0.f}, lo[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      const uint4 va = xa[s >> 1], vb = xb[s >> 1];
+      uint32_t af[4];
+      af[0] = (s & 1) ? va.z : va.x;   // row gid,   half 0
+      af[1] = (s & 1) ? vb.z : vb.x;   // row gid+8, half 0
+      af[2] = (s & 1) ? va.w : va.y;   // row gid,   half 1
+      af[3] = (s & 1) ? vb.w : vb.y;   // row gid+8, half 1
+      mma_bf16_16816(lo, af, bw[2][s][0], bw[2][s][1]);
+      mma_bf16_16816(lo, af, bw[1][s][0], bw[1][s][1]);
+      mma_bf16_16816(hi, af, bw[0][s][0], bw[0][s][1]);
+    }
+    // lane holds p[row gid][2tig], p[gid][2tig+1], p[gid+8][2tig], p[gid+8][2tig+1]
+    float p[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) p[i] = hi[i] + lo[i];
+    uint32_t ga = (p[0] > 0.f ? 1u : 0u) << (2 * tig) | (p[1] > 0.f ? 1u : 0u) << (2 * tig + 1);
+    uint32_t gb = (p[2] > 0.f ? 1u : 0u) << (2 * tig) | (p[3] > 0.f ? 1u : 0u) << (2 * tig + 1);
+    if (a.near_zero) {
+      if (2 * tig < a.r) { nz += (ra < rows && fabsf(p[0]) < 1e-4f); nz += (rb < rows && fabsf(p[2]) < 1e-4f); }
+      if (2 * tig + 1 < a.r) { nz += (ra < rows && fabsf(p[1]) < 1e-4f); nz += (rb < rows && fabsf(p[3]) < 1e-4f); }
+    }
+    ga |= __shfl_xor_sync(0xffffffffu, ga, 1); ga |= __shfl_xor_sync(0xffffffffu, ga, 2);
+    gb |= __shfl_xor_sync(0xffffffffu, gb, 1); gb |= __shfl_xor_sync(0xffffffffu, gb, 2);
+    if (tig == 0 && ra < rows) { const uint32_t id = gray_rank8(ga); s_ids[ra] = (uint8_t)id; atomicAdd(&s_hist[id], 1u); }
+    if (tig == 1 && rb < rows) { const uint32_t id = gray_rank8(gb); s_ids[rb] = (uint8_t)id; atomicAdd(&s_hist[id], 1u); }
+  }
+  if (a.near_zero) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) nz += __shfl_xor_sync(0xffffffffu, nz, o);
+    if (lane == 0 && nz) atomicAdd(a.near_zero, (unsigned long long)nz);
+  }
+  __syncthreads();
+  uint8_t* dst = a.ids + ((size_t)side * a.G + seg) * a.n + row0;
+  if ((rows & 15) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+    for (int i = tid; i < rows / 16; i += 256)
+      reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(s_ids)[i];
+  } else {
+    for (int i = tid; i < rows; i += 256) dst[i] = s_ids[i];
+  }
+  a.hist[(((size_t)side * a.G + seg) * a.chunks_per_seg + chunk) * kBuckets + tid] = s_hist[tid];
+}
+
+// fp32 rows (small problems): one thread per row, plain fp32 FMA in coordinate order.
+__global__ void __launch_bounds__(256) hash_fp32_kernel(const __grid_constant__ HashArgs a, int d) {
+  __shared__ float s_w[128 * 8];
+  __shared__ uint32_t s_hist[kBuckets];
+  const int tid = threadIdx.x;
+  int cta = blockIdx.x;
+  const int chunk = cta % a.chunks_per_seg; cta /= a.chunks_per_seg;
+  const int seg = cta % a.G;
+  const int side = cta / a.G;
+  const int unit_idx = chunk / a.chunks_per_unit, cu = chunk % a.chunks_per_unit;
+  const int row0 = unit_idx * a.unit + cu * kSortChunk;
+  const int rows = min(kSortChunk, a.unit - cu * kSortChunk);
+  s_hist[tid] = 0;
+  for (int i = tid; i < d * a.r; i += 256) s_w[i] = a.w[i];
+  __syncthreads();
+  const float* base = reinterpret_cast<const float*>(a.x[side]) + ((size_t)seg * a.n + row0) * d;
+  uint8_t* dst = a.ids + ((size_t)side * a.G + seg) * a.n + row0;
+  unsigned long long nz = 0;
+  for (int row = tid; row < rows; row += 256) {
+    float p[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    const float4* xr = reinterpret_cast<const float4*>(base + (size_t)row * d);
+    for (int c = 0; c < d / 4; ++c) {
+      const float4 x = xr[c];
+      const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+          if (t < a.r) p[t] = fmaf(xs[e], s_w[(4 * c + e) * a.r + t], p[t]);
+    }
+    uint32_t g = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+      if (t < a.r) { g |= (p[t] > 0.f ? 1u : 0u) << t; nz += fabsf(p[t]) < 1e-4f; }
+    const uint32_t id = gray_rank8(g);
+    dst[row] = (uint8_t)id;
+    atomicAdd(&s_hist[id], 1u);
+  }
+  if (a.near_zero && nz) atomicAdd(a.near_zero, nz);
+  __syncthreads();
+  a.hist[(((size_t)side * a.G + seg) * a.chunks_per_seg + chunk) * kBuckets + tid] = s_hist[tid];
+}
+
+__global__ void convert_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, size_t count4) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 x = src[i];
+    uint2 o;
+    o.x = pack_bf16(x.x, x.y);
+    o.y = pack_bf16(x.z, x.w);
+    dst[i] = o;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_convert(const float* src, __nv_bfloat16* dst, size_t count, cudaStream_t st) {
+  const size_t count4 = count / 4;
+  const int blocks = (int)((count4 + 255) / 256 < 148 * 16 ? (count4 + 255) / 256 : 148 * 16);
+  convert_kernel<<<blocks > 0 ? blocks : 1, 256, 0, st>>>(reinterpret_cast<const float4*>(src),
+                                                         reinterpret_cast<uint2*>(dst), count4);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
+                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st) {
+  HashArgs a;
+  for (int i = 0; i < g.d * g.r; ++i) a.w[i] = w_host[i];
+  a.x[0] = q; a.x[1] = k; a.ids = ws.ids; a.hist = ws.hist; a.near_zero = near_zero;
+  a.G = g.G; a.n = g.n; a.r = g.r;
+  a.unit = g.unit; a.chunks_per_unit = g.chunks_per_unit; a.chunks_per_seg = g.chunks_per_seg;
+  const int grid = 2 * g.G * g.chunks_per_seg;
+  if (is_fp32) hash_fp32_kernel<<<grid, 256, 0, st>>>(a, g.d);
+  else if (g.d == 64) hash_bf16_kernel<64><<<grid, 256, 0, st>>>(a);
+  else hash_bf16_kernel<128><<<grid, 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace hyperattn

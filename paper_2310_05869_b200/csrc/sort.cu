@@ -1,0 +1,189 @@
+// sortLSH permutations (Alg. 1 line 3) and sampled columns (Alg. 2 line 4).
+//
+// The argsort is a stable counting sort: bucket ids have at most 256 values, so one pass of
+//   per-chunk histogram (done by the hash kernel) -> per-node exclusive scan -> stable scatter
+// orders every (level, segment, node, side) slice.  A chunk never straddles a recursion
+// node, so the histogram of a chunk is the same at every level of the causal recursion and
+// only the scan differs per level.  Ties keep the original row order, which makes the
+// permutation unique.
+#include "common.cuh"
+
+namespace hyperattn {
+namespace {
+
+struct SortArgs {
+  const uint8_t* ids;     // [2, G, n]
+  const uint32_t* hist;   // [2, G, chunks_per_seg, 256]
+  uint32_t* offs;         // [2, levels, G, chunks_per_level, 256]
+  int32_t *perm_q, *perm_k, *rank_k;  // [levels, G, nl]
+  Geometry g;
+  int chunks_per_level;   // chunks per (level, segment, side)
+};
+
+// chunk index (within a segment) of the first chunk of node j's query (side 0) or key (side 1) rows
+__device__ __forceinline__ int node_first_chunk(const Geometry& g, int level, int j, int side, int& nchunks, int& s) {
+  int q0, k0;
+  node_rows(g, level, j, s, q0, k0);
+  nchunks = (s / g.unit) * g.chunks_per_unit;
+  return ((side == 0 ? q0 : k0) / g.unit) * g.chunks_per_unit;
+}
+
+// One CTA per (side, level, segment, node): thread v owns bucket v.
+__global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a) {
+  __shared__ uint32_t s_tot[kBuckets];
+  const Geometry& g = a.g;
+  const int v = threadIdx.x;
+  int cta = blockIdx.x;
+  // nodes of all levels are enumerated heap-style: per (side, seg): sum over levels of 2^level
+  const int nodes_per = g.causal ? g.nodes : 1;
+  const int nd = cta % nodes_per; cta /= nodes_per;
+  const int seg = cta % g.G;
+  const int side = cta / g.G;
+  int level = 0, j = nd;
+  if (g.causal) { level = 31 - __clz(nd + 1); j = nd + 1 - (1 << level); }
+  int nchunks, s;
+  const int first = node_first_chunk(g, level, j, side, nchunks, s);
+  const uint32_t* h = a.hist + (((size_t)side * g.G + seg) * g.chunks_per_seg + first) * kBuckets;
+  const int lvl_chunk0 = g.causal ? j * nchunks : 0;
+  uint32_t* o = a.offs + ((((size_t)side * g.levels + level) * g.G + seg) * a.chunks_per_level + lvl_chunk0) * kBuckets;
+  uint32_t run = 0;
+  for (int c = 0; c < nchunks; ++c) {
+    const uint32_t t = h[(size_t)c * kBuckets + v];
+    o[(size_t)c * kBuckets + v] = run;
+    run += t;
+  }
+  // exclusive scan of the bucket totals over v
+  s_tot[v] = run;
+  __syncthreads();
+  for (int off = 1; off < kBuckets; off <<= 1) {
+    const uint32_t add = v >= off ? s_tot[v - off] : 0u;
+    __syncthreads();
+    s_tot[v] += add;
+    __syncthreads();
+  }
+  const uint32_t base = s_tot[v] - run;
+  for (int c = 0; c < nchunks; ++c) o[(size_t)c * kBuckets + v] += base;
+}
+
+// One CTA per (side, level, segment, chunk of the level): stable placement of <= 2048 rows.
+__global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
+  __shared__ uint32_t s_cnt[8][kBuckets];   // per-warp running positions
+  __shared__ uint8_t s_id[kSortChunk];
+  const Geometry& g = a.g;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int cta = blockIdx.x;
+  const int lc = cta % a.chunks_per_level; cta /= a.chunks_per_level;
+  const int seg = cta % g.G; cta /= g.G;
+  const int level = cta % g.levels;
+  const int side = cta / g.levels;
+  // which node and which row range this chunk is
+  int s, q0, k0, j = 0, nchunks_node = a.chunks_per_level;
+  if (g.causal) {
+    s = g.n >> (level + 1);
+    nchunks_node = (s / g.unit) * g.chunks_per_unit;
+    j = lc / nchunks_node;
+  }
+  node_rows(g, level, j, s, q0, k0);
+  const int cn = lc - j * nchunks_node;                  // chunk within the node
+  const int u = cn / g.chunks_per_unit, cu = cn % g.chunks_per_unit;
+  const int local0 = u * g.unit + cu * kSortChunk;       // first row, relative to the node
+  const int rows = min(kSortChunk, g.unit - cu * kSortChunk);
+  const int row0 = (side == 0 ? q0 : k0) + local0;       // first row within the segment
+
+  const uint8_t* ids = a.ids + ((size_t)side * g.G + seg) * g.n + row0;
+  for (int i = tid; i < rows; i += 256) s_id[i] = ids[i];
+  for (int i = tid; i < 8 * kBuckets; i += 256) (&s_cnt[0][0])[i] = 0;
+  __syncthreads();
+  // per-warp histograms of consecutive sub-ranges of 256 rows
+  const int wbeg = warp * (kSortChunk / 8);
+  const int wend = min(rows, wbeg + kSortChunk / 8);
+  for (int i = wbeg + lane; i < wend; i += 32) atomicAdd(&s_cnt[warp][s_id[i]], 1u);
+  __syncthreads();
+  {
+    const uint32_t* o = a.offs + ((((size_t)side * g.levels + level) * g.G + seg) * a.chunks_per_level + lc) * kBuckets;
+    uint32_t run = o[tid];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { const uint32_t t = s_cnt[w][tid]; s_cnt[w][tid] = run; run += t; }
+  }
+  __syncthreads();
+  const size_t slice = ((size_t)level * g.G + seg) * g.nl + (g.causal ? (size_t)j * s : 0);
+  int32_t* perm = (side == 0 ? a.perm_q : a.perm_k) + slice;
+  int32_t* rank = side == 1 ? a.rank_k + slice : nullptr;
+  for (int i0 = wbeg; i0 < wend; i0 += 32) {
+    const int i = i0 + lane;
+    const bool act = i < wend;
+    const uint32_t id = act ? s_id[i] : 0xFFFFFFFFu;
+    const uint32_t peers = __match_any_sync(0xffffffffu, id);
+    const int before = __popc(peers & ((1u << lane) - 1u));
+    uint32_t pos = 0;
+    if (act) pos = s_cnt[warp][id] + before;
+    __syncwarp();
+    if (act && before == 0) s_cnt[warp][id] += __popc(peers);
+    __syncwarp();
+    if (act) {
+      perm[pos] = local0 + i;
+      if (rank) rank[local0 + i] = (int32_t)pos;
+    }
+  }
+}
+
+struct SampleArgs {
+  int32_t* samples;  // [G, nodes, m]
+  Geometry g;
+  uint32_t k0, k1;
+};
+
+__global__ void samples_kernel(SampleArgs a) {
+  const Geometry& g = a.g;
+  const int calls = (g.m + 3) / 4;
+  const size_t total = (size_t)g.G * g.nodes * calls;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % calls);
+    const int nd = (int)((i / calls) % g.nodes);
+    const int seg = (int)(i / ((size_t)calls * g.nodes));
+    const int level = g.causal ? 31 - __clz(nd + 1) : 0;
+    const uint32_t N = g.causal ? (uint32_t)(g.n >> (level + 1)) : (uint32_t)g.n;
+    const Philox4 x = philox4x32_10((uint32_t)c, (uint32_t)seg, (uint32_t)nd, kDomainSamples, a.k0, a.k1);
+    int32_t* dst = a.samples + ((size_t)seg * g.nodes + nd) * g.m;
+#pragma unroll
+    for (int w = 0; w < 4; ++w)
+      if (4 * c + w < g.m) dst[4 * c + w] = (int32_t)__umulhi(x.x[w], N);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_samples(const Geometry& g, uint64_t seed, const Workspace& ws, cudaStream_t st) {
+  if (g.nodes == 0 || g.m == 0) return cudaSuccess;
+  SampleArgs a; a.samples = ws.samples; a.g = g; a.k0 = (uint32_t)seed; a.k1 = (uint32_t)(seed >> 32);
+  const size_t total = (size_t)g.G * g.nodes * ((g.m + 3) / 4);
+  const int blocks = (int)((total + 255) / 256);
+  samples_kernel<<<blocks < 1184 ? blocks : 1184, 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+static SortArgs make_sort_args(const Geometry& g, const Workspace& ws) {
+  SortArgs a;
+  a.ids = ws.ids; a.hist = ws.hist; a.offs = ws.offs;
+  a.perm_q = ws.perm_q; a.perm_k = ws.perm_k; a.rank_k = ws.rank_k;
+  a.g = g;
+  a.chunks_per_level = (g.nl / g.unit) * g.chunks_per_unit;
+  return a;
+}
+
+cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, cudaStream_t st) {
+  if (!g.sorted) return cudaSuccess;
+  const SortArgs a = make_sort_args(g, ws);
+  const int nodes_per = g.causal ? g.nodes : 1;
+  sort_scan_kernel<<<2 * g.G * nodes_per, 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st) {
+  if (!g.sorted) return cudaSuccess;
+  const SortArgs a = make_sort_args(g, ws);
+  sort_scatter_kernel<<<2 * g.levels * g.G * a.chunks_per_level, 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace hyperattn

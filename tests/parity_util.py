@@ -1,0 +1,158 @@
+"""GPU-vs-oracle comparison helpers shared by the parity tests.
+
+Rules (one per stage of the path):
+  ids      bit-exact, except hash bits whose exact projection magnitude is below 1e-4
+           (those are counted; a mismatch on any other bit fails)
+  samples  bit-exact
+  perms    bit-exact given the GPU's own bucket ids (and end to end when no id differs)
+  out/lse  oracle evaluated with the GPU's ids injected: max |err| <= 2e-2, mean |err| <= 2e-3,
+           |d lse| <= 1e-3 * max(|lse|, 1)
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+import torch
+
+from oracle import hyperattn_oracle as O
+from paper_2310_05869_b200 import workloads as WL
+
+OUT_MAX_ABS = 2e-2
+OUT_MEAN_ABS = 2e-3
+LSE_REL = 1e-3
+AMBIGUOUS = 1e-4
+
+
+def to_device(w: WL.Workload, arrs):
+    """numpy inputs -> CUDA tensors [B, H, n, d]."""
+    outs = []
+    for x in arrs:
+        if x.dtype == np.uint16:
+            t = torch.from_numpy(x.view(np.int16)).cuda().view(torch.bfloat16)
+        else:
+            t = torch.from_numpy(x).cuda()
+        outs.append(t.view(w.B, w.H, w.n, w.d))
+    return outs
+
+
+def levels_of(w: WL.Workload):
+    """[(level, node_size)] of the off-diagonal problems; non-causal: one node of n rows."""
+    if not w.causal:
+        return [(0, w.n)] if w.b < w.n else []
+    if w.n <= w.n0:
+        return []
+    L = (w.n // w.n0).bit_length() - 1
+    return [(l, w.n >> (l + 1)) for l in range(L)]
+
+
+def node_ranges(w: WL.Workload, level: int, j: int):
+    if not w.causal:
+        return 0, 0, w.n
+    s = w.n >> (level + 1)
+    return (2 * j + 1) * s, 2 * j * s, s
+
+
+def check_ids(w, Q64, K64, inter, segs=None):
+    """Returns (ambiguous_bits, mismatched_rows); fails on a mismatch that is not ambiguous."""
+    W = O.directions(w.d, w.r, w.seed)
+    G = w.G
+    segs = range(G) if segs is None else segs
+    gq = inter["q_ids"].cpu().numpy()
+    gk = inter["k_ids"].cpu().numpy()
+    amb_total, mism_total = 0, 0
+    for g in segs:
+        for X, got in ((Q64[g], gq[g]), (K64[g], gk[g])):
+            ids, absp = O.bucket_ids(X, W)
+            amb = absp < AMBIGUOUS
+            amb_total += int(amb.sum())
+            bad = np.nonzero(ids != got)[0]
+            mism_total += bad.size
+            for i in bad:
+                # the differing sign bits must all be ambiguous ones
+                g_ref = int(ids[i]) ^ (int(ids[i]) >> 1)
+                g_got = int(got[i]) ^ (int(got[i]) >> 1)
+                diff = g_ref ^ g_got
+                for t in range(w.r):
+                    if diff >> t & 1:
+                        assert amb[i, t], f"segment {g} row {i}: bit {t} differs with |p|={absp[i, t]:.3e}"
+                assert diff >> w.r == 0
+    return amb_total, mism_total
+
+
+def check_samples(w, inter):
+    if w.m == 0:
+        return
+    got = inter["samples"].cpu().numpy()
+    for g in range(w.G):
+        for level, s in levels_of(w):
+            nodes = (1 << level) if w.causal else 1
+            for j in range(nodes):
+                node = O.heap_node(level, j) if w.causal else 0
+                ref = O.sample_indices(w.seed, g, node, w.m, s)
+                assert (got[g, node, :w.m] == ref).all(), (g, level, j)
+
+
+def check_perms(w, inter, segs=None):
+    """Permutations and ranks against the oracle's stable argsort of the GPU's own ids."""
+    gq = inter["q_ids"].cpu().numpy()
+    gk = inter["k_ids"].cpu().numpy()
+    pq = inter["perm_q"].cpu().numpy()
+    pk = inter["perm_k"].cpu().numpy()
+    rk = inter["rank_k"].cpu().numpy()
+    segs = range(w.G) if segs is None else segs
+    for g in segs:
+        for level, s in levels_of(w):
+            if w.b >= s:
+                continue
+            nodes = (1 << level) if w.causal else 1
+            for j in range(nodes):
+                q0, k0, _ = node_ranges(w, level, j)
+                sl = slice(j * s, (j + 1) * s) if w.causal else slice(0, s)
+                perm, _ = O.stable_argsort(gq[g, q0:q0 + s])
+                assert (pq[level, g, sl] == perm).all(), ("perm_q", g, level, j)
+                perm, rank = O.stable_argsort(gk[g, k0:k0 + s])
+                assert (pk[level, g, sl] == perm).all(), ("perm_k", g, level, j)
+                assert (rk[level, g, sl] == rank).all(), ("rank_k", g, level, j)
+
+
+def oracle_rows(w, Q64, K64, V64, g, rows, ids_q=None, ids_k=None):
+    W = O.directions(w.d, w.r, w.seed)
+    return O.segment_forward(Q64[g], K64[g], V64[g], W, w.b, w.m, w.causal, w.n0, w.seed, g,
+                             scale=1.0 / math.sqrt(w.d), rows=rows, ids_q=ids_q, ids_k=ids_k)
+
+
+def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, segs=None, rng_seed=0):
+    """Compares out/lse with the oracle (GPU ids injected when `inter` is given).  With
+    rows_per_seg, a pseudo-random subset of rows plus the rows around every leaf / node
+    boundary is checked."""
+    out = out.float().cpu().numpy().reshape(w.G, w.n, w.d)
+    lse = lse.float().cpu().numpy().reshape(w.G, w.n)
+    gq = inter["q_ids"].cpu().numpy() if inter is not None else None
+    gk = inter["k_ids"].cpu().numpy() if inter is not None else None
+    segs = range(w.G) if segs is None else segs
+    rng = np.random.default_rng(rng_seed)
+    errs, lerrs = [], []
+    for g in segs:
+        if rows_per_seg is None or rows_per_seg >= w.n:
+            rows = np.arange(w.n)
+        else:
+            rows = set(rng.choice(w.n, size=rows_per_seg, replace=False).tolist())
+            if w.causal and w.n > w.n0:
+                for edge in range(0, w.n + 1, w.n0):
+                    rows.update(x for x in (edge - 1, edge, edge + 127, edge + 128) if 0 <= x < w.n)
+            rows.update((0, w.n - 1))
+            rows = np.array(sorted(rows))
+        ref_o, ref_l = oracle_rows(w, Q64, K64, V64, g, rows,
+                                   None if gq is None else gq[g], None if gk is None else gk[g])
+        errs.append(np.abs(out[g, rows] - ref_o))
+        lerrs.append(np.abs(lse[g, rows] - ref_l) / np.maximum(np.abs(ref_l), 1.0))
+    err = np.concatenate([e.reshape(-1) for e in errs])
+    lerr = np.concatenate(lerrs)
+    stats = {"max_abs": float(err.max()), "mean_abs": float(err.mean()), "lse_rel": float(lerr.max()),
+             "rows": int(lerr.size)}
+    assert np.isfinite(err).all() and np.isfinite(lerr).all(), stats
+    assert stats["max_abs"] <= OUT_MAX_ABS, stats
+    assert stats["mean_abs"] <= OUT_MEAN_ABS, stats
+    assert stats["lse_rel"] <= LSE_REL, stats
+    return stats

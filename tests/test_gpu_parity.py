@@ -1,0 +1,126 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, stage by stage."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2310_05869_b200 as ha
+from paper_2310_05869_b200 import workloads as WL
+
+import parity_util as PU
+
+pytestmark = pytest.mark.gpu
+
+
+def W(name, B, H, n, d, dtype, b, m, r, causal, n0, kind="gaussian", gen_seed=7, seed=0):
+    return WL.Workload(name, B, H, n, d, dtype, b, m, r, causal, n0, kind, gen_seed, seed)
+
+
+SMALL = [
+    WL.CONFIGS[0],                                                             # the baseline's small config
+    W("bf16_d128_tiles", 2, 2, 2048, 128, "bf16", 256, 256, 7, False, 0, seed=3),
+    W("ragged_b96_m40", 1, 3, 1152, 64, "bf16", 96, 40, 5, False, 0, seed=11),
+    W("single_block_ragged", 1, 2, 300, 64, "bf16", 512, 16, 4, False, 0),
+    W("causal_leaf_only_ragged", 1, 2, 500, 128, "bf16", 64, 16, 4, True, 512),
+    W("causal_two_levels", 1, 2, 2048, 64, "bf16", 128, 64, 6, True, 512, seed=5),
+    W("causal_mixed_sorted_unsorted", 1, 2, 1024, 64, "bf16", 256, 32, 7, True, 128, seed=9),
+    W("causal_heavy_tail", 2, 2, 4096, 128, "bf16", 128, 512, 8, True, 1024, kind="student_t", seed=2),
+    W("clustered_ties", 1, 2, 4096, 64, "bf16", 256, 256, 7, False, 0, kind="clustered"),
+    W("no_samples", 1, 2, 1024, 64, "bf16", 128, 0, 7, False, 0),
+    W("chunk_tail", 1, 2, 4608, 64, "bf16", 256, 128, 7, False, 0),
+    W("causal_chunk_tail", 1, 1, 6144, 64, "bf16", 256, 128, 7, True, 3072),
+    W("fp32_causal", 1, 2, 1024, 128, "fp32", 64, 64, 8, True, 256, seed=4),
+    W("one_bit_small_block", 1, 1, 512, 64, "bf16", 32, 8, 1, False, 0),
+]
+
+
+def run(w, out_dtype=None, debug=True, workspace=None):
+    arrs = WL.make_inputs(w)
+    q, k, v = PU.to_device(w, arrs)
+    res = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, out_dtype=out_dtype,
+                     debug=debug, workspace=workspace)
+    torch.cuda.synchronize()
+    assert ha.last_device_status() == 0
+    Q64, K64, V64 = (WL.as_f64(x) for x in arrs)
+    return res, (Q64, K64, V64)
+
+
+@pytest.mark.parametrize("w", SMALL, ids=[w.name for w in SMALL])
+def test_small_configs_every_stage(w):
+    (out, lse, inter), (Q64, K64, V64) = run(w, out_dtype=torch.float32)
+    sorted_any = any(w.b < s for _, s in PU.levels_of(w))
+    if sorted_any:
+        amb, mism = PU.check_ids(w, Q64, K64, inter)
+        PU.check_samples(w, inter)
+        PU.check_perms(w, inter)
+        stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter)
+        print(w.name, "ambiguous bits", amb, "id mismatches", mism, stats)
+    else:
+        stats = PU.check_outputs(w, Q64, K64, V64, out, lse, None)
+        print(w.name, stats)
+
+
+def test_bf16_output_and_caller_workspace():
+    w = SMALL[1]
+    nbytes = ha.workspace_bytes(w.B, w.H, w.n, w.d, w.b, w.m, w.r, w.causal, w.n0)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    (out, lse, inter), (Q64, K64, V64) = run(w, workspace=ws)
+    assert out.dtype == torch.bfloat16
+    PU.check_outputs(w, Q64, K64, V64, out, lse, inter)
+    (out2, lse2, _), _ = run(w)                       # private workspace: identical result
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+    with pytest.raises(ha.HyperAttnError, match="workspace too small"):
+        run(w, workspace=ws[: nbytes // 2])
+
+
+def test_plain_entry_point_matches_ex():
+    import ctypes as C
+    w = SMALL[5]
+    arrs = WL.make_inputs(w)
+    q, k, v = PU.to_device(w, arrs)
+    out = torch.empty_like(q)
+    lse = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
+    rc = ha.lib().hyperattn_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                    w.B, w.H, w.n, w.d, w.b, w.m, w.r, int(w.causal), w.n0, C.c_uint64(w.seed),
+                                    torch.cuda.current_stream().cuda_stream)
+    assert rc == 0
+    out2, lse2 = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+
+
+def test_host_buffer_entry_point():
+    w = SMALL[2]
+    arrs = WL.make_inputs(w)
+    q, k, v = PU.to_device(w, arrs)
+    out_d, lse_d = ha.forward(q, k, v, w.b, w.m, w.r, seed=w.seed)
+    hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+    ho = torch.empty(q.shape, dtype=torch.bfloat16).pin_memory()
+    hl = torch.empty((w.B, w.H, w.n), dtype=torch.float32).pin_memory()
+    ha.forward_host(hq, hk, hv, ho, hl, w.b, w.m, w.r, seed=w.seed)
+    torch.cuda.synchronize()
+    assert torch.equal(ho, out_d.cpu()) and torch.equal(hl, lse_d.cpu())
+
+
+def test_seed_changes_hash_and_samples_and_repeats():
+    w = SMALL[1]
+    (o1, l1, i1), _ = run(w)
+    (o2, l2, i2), _ = run(w)
+    assert torch.equal(o1, o2) and torch.equal(i1["perm_q"], i2["perm_q"])
+    (o3, _, i3), _ = run(w.scaled(seed=w.seed + 1))
+    assert not torch.equal(i1["q_ids"], i3["q_ids"]) and not torch.equal(i1["samples"], i3["samples"])
+
+
+def test_stage_profile_counts_launches():
+    w = SMALL[5]
+    ha.profile_reset()
+    ha.profile_enable(True)
+    try:
+        run(w, debug=False)
+        run(w, debug=False)
+        prof = ha.profile_read()
+    finally:
+        ha.profile_enable(False)
+        ha.profile_reset()
+    assert prof["calls"] == 2
+    assert prof["launches"]["hash"] == 2 and prof["launches"]["attention"] == 2 and prof["launches"]["merge"] == 2
+    assert all(prof["ms"][s] > 0 for s in ("hash", "sort_scan", "sort_scatter", "attention", "merge"))
