@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the HyperAttention forward pass (one step = one whole forward: hash, sample,
+sort, attention tiles, merge) on synthetic inputs of the baseline's shapes.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5|c1] [--impl reference]
+
+Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e` is the same
+metric through the host-buffer entry point (pinned host memory, copies inside the timed
+region); `roofline` describes the dominant kernel (the attention tiles); `kernels` lists every
+stage with its own bound; `cpu_baseline` is the NumPy oracle timed on the host cores on a
+bounded sample of the same workload (a reported baseline, not a target), together with the
+GPU-vs-oracle error on that sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2310_05869_b200 import workloads as WL  # noqa: E402
+
+WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch of the attention kernel from an ncu capture (see profiles/); None until
+# a capture of that workload exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+# ---------------------------------------------------------------- algorithmic work per forward
+def work_model(w: WL.Workload):
+    """Algorithmic flops / bytes of each stage for one forward (what the method itself has to
+    compute or move, not what a particular kernel happens to do)."""
+    G, n, d, e = w.G, w.n, w.d, (2 if w.dtype == "bf16" else 4)
+    nodes = []  # (count per segment, size)
+    leaves = []
+    if not w.causal:
+        if w.b < n:
+            nodes.append((1, n))
+        else:
+            leaves.append((1, n, False))
+    elif n <= w.n0:
+        leaves.append((1, n, True))
+    else:
+        L = (n // w.n0).bit_length() - 1
+        for l in range(L):
+            nodes.append((1 << l, n >> (l + 1)))
+        leaves.append((n // w.n0, w.n0, True))
+    flops = 0.0
+    sorted_rows = 0
+    for cnt, s in nodes:
+        if w.b < s:
+            flops += cnt * 4.0 * s * (w.b + w.m) * d
+            sorted_rows += cnt * s
+        else:
+            flops += cnt * 4.0 * s * s * d
+    for cnt, s, causal in leaves:
+        flops += cnt * (4.0 * d * s * (s + 1) / 2 if causal else 4.0 * s * s * d)
+    flops *= G
+    any_sorted = sorted_rows > 0
+    hash_bytes = 2.0 * G * n * (d * e + 1) if any_sorted else 0.0
+    sort_bytes = G * sorted_rows * (2 * 1 + 4 + 4 + 4)        # ids of Q and K rows, perm_q, perm_k, rank_k
+    merge_bytes = 0.0
+    if w.causal and n > w.n0:
+        L = (n // w.n0).bit_length() - 1
+        merge_bytes = G * n * ((1 + L / 2.0) * (4 * d + 4) + d * e + 4)
+    dense_flops = G * (4.0 * n * n * d) * (0.5 if w.causal else 1.0)
+    return {"attention_flops": flops, "hash_bytes": hash_bytes, "sort_bytes": float(sort_bytes),
+            "merge_bytes": merge_bytes, "dense_attention_flops": dense_flops}
+
+
+# ---------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------- oracle leg
+def oracle_sample_plan(w: WL.Workload, leg: str):
+    """Which part of the workload the oracle is timed on: whole segments, and for causal
+    workloads a bounded set of query rows per segment (hashing and sorting always cover the
+    whole segment).  leg "baseline" (run once, ~10-30 s of CPU work) or "step" (one step of the
+    reference arm, ~1-2 s)."""
+    def spread(k):
+        k = min(k, w.G)
+        return sorted({(i * (w.G - 1)) // max(k - 1, 1) for i in range(k)})
+    if w.n <= 2048:
+        return {"segments": spread(w.G), "rows": None}
+    if w.causal:
+        return {"segments": spread(4 if leg == "baseline" else 2), "rows": 8192 if leg == "baseline" else 4096}
+    per_seg_cost = w.n / 32768.0
+    k = max(1, int((32 if leg == "baseline" else 4) / per_seg_cost))
+    return {"segments": spread(k), "rows": None}
+
+
+def run_oracle_sample(w: WL.Workload, arrs, plan, ids=None):
+    """Runs the oracle on the planned sample.  Returns (seconds, {seg: (rows, out, lse)})."""
+    from oracle import hyperattn_oracle as O
+    res = {}
+    t0 = time.perf_counter()
+    W = O.directions(w.d, w.r, w.seed)
+    rng = np.random.default_rng(12345)
+    for g in plan["segments"]:
+        Q, K, V = (WL.as_f64(x[g]) for x in arrs)
+        rows = None
+        if plan["rows"] is not None and plan["rows"] < w.n:
+            rows = np.sort(rng.choice(w.n, size=plan["rows"], replace=False))
+        iq = ik = None
+        if ids is not None:
+            iq, ik = ids[0][g], ids[1][g]
+        o, l = O.segment_forward(Q, K, V, W, w.b, w.m, w.causal, w.n0, w.seed, g, scale=1.0 / math.sqrt(w.d),
+                                 rows=rows, ids_q=iq, ids_k=ik)
+        res[g] = (np.arange(w.n) if rows is None else rows, o, l)
+    return time.perf_counter() - t0, res
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def sample_tokens(w, plan):
+    per_seg = w.n if plan["rows"] is None else min(plan["rows"], w.n)
+    return per_seg * len(plan["segments"]) / w.H          # tokens = rows of one head set / H heads
+
+
+def reference_arm(args, w):
+    """The oracle timed on the host cores: each step is the bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    arrs = make_sample_inputs(w)
+    plan = oracle_sample_plan(w, "step")
+    for _ in range(min(args.warmup, 1)):
+        run_oracle_sample(w, arrs, plan)
+    times = []
+    for _ in range(args.steps):
+        dt, _ = run_oracle_sample(w, arrs, plan)
+        times.append(dt)
+    tot = sum(times)
+    toks = sample_tokens(w, plan) * args.steps
+    value = toks / tot
+    desc = describe_sample(w, plan)
+    line = {"impl": "reference", "metric": "forward tokens/s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * tot / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(w),
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": host_threads(), "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def describe_sample(w, plan):
+    rows = "all rows" if plan["rows"] is None else f"{plan['rows']} random rows per segment (hash and sort of the whole segment)"
+    return f"segments {plan['segments']} of {w.G} of workload {w.name}, {rows}; tokens counted as rows/H"
+
+
+def make_sample_inputs(w):
+    return WL.make_inputs(w)
+
+
+def config_dict(w):
+    return {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "d": w.d, "block": w.b, "samples": w.m,
+            "hash_bits": w.r, "causal": w.causal, "n0": w.n0, "input_kind": w.kind,
+            "l2": "inputs exceed L2 (no flush)" if w.G * w.n * w.d * 2 * 3 > 126e6 else "inputs fit L2; 256 MB flush buffer written between steps"}
+
+
+# ---------------------------------------------------------------- GPU arm
+def gpu_arm(args, w):
+    import torch
+    import torch.distributed as dist
+    import paper_2310_05869_b200 as ha
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    peaks = load_peaks()
+
+    # every rank owns its own B*H segments (weak scaling: no exchange between segments)
+    wr = w.scaled(gen_seed=w.gen_seed + 7919 * rank)
+    arrs = WL.make_inputs(wr)
+
+    def dev_tensor(x):
+        if x.dtype == np.uint16:
+            return torch.from_numpy(x.view(np.int16)).to(dev).view(torch.bfloat16).view(w.B, w.H, w.n, w.d)
+        return torch.from_numpy(x).to(dev).view(w.B, w.H, w.n, w.d)
+
+    q, k, v = (dev_tensor(x) for x in arrs)
+    small = w.G * w.n * w.d * 2 * 3 <= 126e6
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        if flush is not None:
+            flush.fill_(1)
+        return ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    for _ in range(max(args.warmup, 3)):
+        out, lse = step()
+    barrier()
+    # ---- timed region: K whole forwards, device time, stage events on ------------------------
+    ha.profile_reset()
+    ha.profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush_ms = 0.0
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        out, lse = step()
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    prof = ha.profile_read()
+    ha.profile_enable(False)
+    ha.profile_reset()
+    if flush is not None:   # subtract the flush writes (timed separately)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.steps):
+            flush.fill_(1)
+        f1.record(stream)
+        torch.cuda.synchronize(dev)
+        flush_ms = f0.elapsed_time(f1)
+    ms_total = max(ms_total - flush_ms, 1e-6)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    tokens = w.B * w.n * args.steps * world
+    value = tokens / (ms_total * 1e-3)
+
+    # ---- end to end through the host-buffer entry point ---------------------------------------
+    hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
+    ho = torch.empty(q.shape, dtype=q.dtype).pin_memory()
+    hl = torch.empty((w.B, w.H, w.n), dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        ha.forward_host(hq, hk, hv, ho, hl, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+    barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        ha.forward_host(hq, hk, hv, ho, hl, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+    e1.record(stream)
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item())
+    es = q.element_size()
+    h2d = 3 * q.numel() * es
+    d2h = ho.numel() * ho.element_size() + hl.numel() * 4
+    e2e = {"value": w.B * w.n * e2e_steps * world / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms / e2e_steps,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+    assert torch.equal(ho.to(dev), out), "host-buffer entry point disagrees with the device entry point"
+    clocks = sampler.stop() if sampler else None
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-stage roofline -----------------------------------------------------------------------
+    wm = work_model(w)
+    calls = max(prof["calls"], 1)
+    stage_ms = {s: prof["ms"][s] / calls for s in prof["ms"]}
+    launches = {s: prof["launches"][s] // calls for s in prof["launches"]}
+    tensor_peak = peaks["bf16_tflops_sustained"]
+    att_ms = stage_ms["attention"]
+    att_tflops = wm["attention_flops"] / (att_ms * 1e-3) / 1e12 if att_ms > 0 else 0.0
+    roofline = {"kernel": "attention tiles (block + sampled + causal leaves)", "bound": "tensor", "achieved": att_tflops,
+                "peak": tensor_peak, "unit": "TFLOP/s", "frac": att_tflops / tensor_peak,
+                "peak_source": f"bf16_tflops_sustained of {peaks['source']}", "ms_per_launch": att_ms,
+                "traffic": NCU_TRAFFIC_BYTES.get(w.name)}
+    kernels = {}
+    for s, key in (("hash", "hash_bytes"), ("merge", "merge_bytes")):
+        if stage_ms[s] > 0:
+            gbs = wm[key] / (stage_ms[s] * 1e-3) / 1e9
+            kernels[s] = {"bound": "hbm", "ms": stage_ms[s], "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": gbs / peaks["hbm_gbs"]}
+    sort_ms = stage_ms["sort_scan"] + stage_ms["sort_scatter"]
+    if sort_ms > 0:
+        gbs = wm["sort_bytes"] / (sort_ms * 1e-3) / 1e9
+        kernels["sort"] = {"bound": "hbm", "ms": sort_ms, "ms_scan": stage_ms["sort_scan"], "ms_scatter": stage_ms["sort_scatter"],
+                           "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"]}
+    kernels["attention"] = {"bound": "tensor", "ms": att_ms, "achieved": att_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
+                            "frac": att_tflops / tensor_peak}
+    kernels["sample"] = {"ms": stage_ms["sample"]}
+    ms_step = ms_total / args.steps
+    dense_ms = wm["dense_attention_flops"] / (tensor_peak * 1e12) * 1e3
+
+    # ---- oracle on the host cores: bounded sample, plus the error of the GPU result on it -----
+    cpu = None
+    if not args.no_cpu_baseline:
+        plan = oracle_sample_plan(w, "baseline")
+        out32, lse32, inter = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed,
+                                         out_dtype=torch.float32, debug=True)
+        torch.cuda.synchronize(dev)
+        any_sorted = w.b < (w.n if not w.causal else w.n // 2) and not (w.causal and w.n <= w.n0)
+        ids = (inter["q_ids"].cpu().numpy(), inter["k_ids"].cpu().numpy()) if any_sorted else None
+        secs, res = run_oracle_sample(w, arrs, plan, ids)
+        o_np = out32.view(w.G, w.n, w.d)
+        l_np = lse32.view(w.G, w.n)
+        errs, lerrs = [], []
+        for g, (rows, ro, rl) in res.items():
+            idx = torch.from_numpy(rows).to(dev)
+            errs.append(np.abs(o_np[g][idx].cpu().numpy() - ro).reshape(-1))
+            lerrs.append(np.abs(l_np[g][idx].cpu().numpy() - rl) / np.maximum(np.abs(rl), 1.0))
+        err = np.concatenate(errs)
+        lerr = np.concatenate(lerrs)
+        cpu = {"value": sample_tokens(w, plan) / secs, "unit": "tokens/s", "cores": host_threads(), "kind": "oracle",
+               "sample": describe_sample(w, plan), "seconds": secs,
+               "gpu_vs_oracle": {"out_max_abs": float(err.max()), "out_mean_abs": float(err.mean()),
+                                 "lse_max_rel": float(lerr.max()), "rows": int(lerr.size),
+                                 "near_zero_hash_bits": int(inter["near_zero_bits"].item())}}
+
+    line = {"metric": "forward tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config_dict(w),
+            "latency_ms": ms_step, "dense_attention_roofline_ms": dense_ms, "speedup_vs_dense_roofline": dense_ms / ms_step,
+            "e2e": e2e, "gpu_launches": sum(launches.values()) * args.steps, "launches_per_step": launches,
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "clocks": clocks,
+            "peaks": peaks}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--n", type=int, default=0, help="override the sequence length (c4 sweep)")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = WL.CONFIGS[WORKLOADS[args.workload]]
+    if args.n:
+        w = w.scaled(n=args.n, name=f"{w.name}_n{args.n}")
+    if args.impl == "reference":
+        reference_arm(args, w)
+    else:
+        gpu_arm(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -71,7 +71,7 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
 }
 
 struct Plan {
-  size_t q16, k16, v16, ids, hist, offs, perm_q, perm_k, rank_k, samples, part_o, part_lse, total;
+  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, part_o, part_lse, total;
 };
 
 Plan make_plan(const Geometry& g, int is_fp32) {
@@ -82,6 +82,8 @@ Plan make_plan(const Geometry& g, int is_fp32) {
   pl.q16 = take(is_fp32 ? tensor16 : 0);
   pl.k16 = take(is_fp32 ? tensor16 : 0);
   pl.v16 = take(is_fp32 ? tensor16 : 0);
+  pl.q16lo = take(is_fp32 ? tensor16 : 0);
+  pl.k16lo = take(is_fp32 ? tensor16 : 0);
   const size_t lvl_rows = (size_t)g.levels * g.G * g.nl;
   pl.ids = take(g.sorted ? (size_t)2 * g.G * g.n : 0);
   pl.hist = take(g.sorted ? (size_t)2 * g.G * g.chunks_per_seg * kBuckets * 4 : 0);
@@ -198,6 +200,8 @@ int forward_impl(const hyperattn_params& p) {
   ws.q16 = reinterpret_cast<__nv_bfloat16*>(base + pl.q16);
   ws.k16 = reinterpret_cast<__nv_bfloat16*>(base + pl.k16);
   ws.v16 = reinterpret_cast<__nv_bfloat16*>(base + pl.v16);
+  ws.q16lo = reinterpret_cast<__nv_bfloat16*>(base + pl.q16lo);
+  ws.k16lo = reinterpret_cast<__nv_bfloat16*>(base + pl.k16lo);
   ws.ids = reinterpret_cast<uint8_t*>(base + pl.ids);
   ws.hist = reinterpret_cast<uint32_t*>(base + pl.hist);
   ws.offs = reinterpret_cast<uint32_t*>(base + pl.offs);
@@ -220,9 +224,9 @@ int forward_impl(const hyperattn_params& p) {
   if (is_fp32) {
     StageScope sc(st, HYPERATTN_STAGE_CONVERT, 3);
     const size_t cnt = (size_t)g.G * g.n * g.d;
-    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.q), ws.q16, cnt, st));
-    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.k), ws.k16, cnt, st));
-    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.v), ws.v16, cnt, st));
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.q), ws.q16, ws.q16lo, cnt, st));
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.k), ws.k16, ws.k16lo, cnt, st));
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.v), ws.v16, nullptr, cnt, st));
     q16 = ws.q16; k16 = ws.k16; v16 = ws.v16;
   }
   if (g.sorted) {
@@ -262,6 +266,7 @@ int forward_impl(const hyperattn_params& p) {
   AttnArgs a;
   std::memset(&a, 0, sizeof(a));
   a.q = q16; a.k = k16; a.v = v16; a.g = g;
+  if (is_fp32) { a.q_lo = ws.q16lo; a.k_lo = ws.k16lo; }
   a.scale_log2 = scale * 1.4426950408889634f;
   a.perm_q = ws.perm_q; a.perm_k = ws.perm_k; a.rank_k = ws.rank_k; a.samples = ws.samples;
   a.part_o = ws.part_o; a.part_lse = ws.part_lse; a.out = p.out; a.lse = p.lse;

@@ -21,6 +21,7 @@ constexpr int kMaxNodeKeys = 2048;   // padded b + padded m must fit the key ind
 
 struct AttnArgs {
   const __nv_bfloat16 *q, *k, *v;    // [G, n, D]
+  const __nv_bfloat16 *q_lo, *k_lo;  // second bf16 term of fp32 inputs (else null)
   Geometry g;
   float scale_log2;                  // softmax scale * log2(e)
   const int32_t *perm_q, *perm_k, *rank_k, *samples;

@@ -63,20 +63,25 @@ __device__ __forceinline__ void gather_tile(uint32_t dst, const __nv_bfloat16* s
   }
 }
 
-template <int D>
+template <int D, bool SPLIT>
 struct Smem {
   static constexpr int kQ = kTileQ * D * 2;
   static constexpr int kKV = TK * D * 2;
-  static constexpr int kTotal = kQ + 4 * kKV + kMaxNodeKeys * 8 + kTileQ * 4;
+  static constexpr int kTotal = (SPLIT ? 2 : 1) * kQ + (SPLIT ? 6 : 4) * kKV + kMaxNodeKeys * 8 + kTileQ * 4;
 };
 
-template <int D>
+// SPLIT: the inputs were fp32 and arrive as two bf16 terms (x = hi + lo up to 2^-17 relative);
+// the logits use Q_hi K_hi + Q_lo K_hi + Q_hi K_lo so that they keep fp32-like accuracy.
+template <int D, bool SPLIT>
 __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant__ AttnArgs a) {
   extern __shared__ __align__(1024) uint8_t smem[];
+  using SM = Smem<D, SPLIT>;
   uint8_t* sQ = smem;
-  uint8_t* sK = sQ + Smem<D>::kQ;                 // [2][TK x D]
-  uint8_t* sV = sK + 2 * Smem<D>::kKV;            // [2][TK x D]
-  int* s_kidx = reinterpret_cast<int*>(sV + 2 * Smem<D>::kKV);
+  uint8_t* sK = sQ + SM::kQ;                      // [2][TK x D]
+  uint8_t* sV = sK + 2 * SM::kKV;                 // [2][TK x D]
+  uint8_t* sQl = sV + 2 * SM::kKV;                // SPLIT only
+  uint8_t* sKl = sQl + (SPLIT ? SM::kQ : 0);      // SPLIT only: [2][TK x D]
+  int* s_kidx = reinterpret_cast<int*>(sKl + (SPLIT ? 2 * SM::kKV : 0));
   float* s_kbias = reinterpret_cast<float*>(s_kidx + kMaxNodeKeys);
   int* s_qrow = reinterpret_cast<int*>(s_kbias + kMaxNodeKeys);
 
@@ -116,6 +121,9 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
   __syncthreads();
 
   const uint32_t uQ = smem_u32(sQ), uK = smem_u32(sK), uV = smem_u32(sV);
+  const uint32_t uQl = smem_u32(sQl), uKl = smem_u32(sKl);
+  const __nv_bfloat16* qls = a.q_lo + (size_t)t.seg * g.n * D;
+  const __nv_bfloat16* kls = a.k_lo + (size_t)t.seg * g.n * D;
   auto qrow_fn = [&](int r) { return s_qrow[r]; };
   auto load_kv = [&](int kt, int stage) {
     auto krow_fn = [&](int r) {
@@ -123,18 +131,20 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
       if (t.mode == 1) return s_kidx[i];
       return i < t.nk ? t.k0 + i : -1;
     };
-    gather_tile<D, TK>(uK + stage * Smem<D>::kKV, ks, krow_fn, tid);
-    gather_tile<D, TK>(uV + stage * Smem<D>::kKV, vs, krow_fn, tid);
+    gather_tile<D, TK>(uK + stage * SM::kKV, ks, krow_fn, tid);
+    gather_tile<D, TK>(uV + stage * SM::kKV, vs, krow_fn, tid);
+    if constexpr (SPLIT) gather_tile<D, TK>(uKl + stage * SM::kKV, kls, krow_fn, tid);
   };
 
   gather_tile<D, kTileQ>(uQ, qs, qrow_fn, tid);
+  if constexpr (SPLIT) gather_tile<D, kTileQ>(uQl, qls, qrow_fn, tid);
   const int ntiles = nkeys / TK;
   load_kv(0, 0);
   cp_async_commit();
 
   // ---- per-warp state: 16 query rows ----------------------------------------------------
   constexpr int KS = D / 16, NO = D / 8;
-  uint32_t qf[KS][4];
+  uint32_t qf[SPLIT ? 1 : KS][4];
   float o[NO][4];
 #pragma unroll
   for (int i = 0; i < NO; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
@@ -147,24 +157,43 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
     cp_async_commit();
     cp_async_wait<1>();
     __syncthreads();
-    if (kt == 0) {
+    if constexpr (!SPLIT) {
+      if (kt == 0) {
 #pragma unroll
-      for (int s = 0; s < KS; ++s)
-        ldmatrix_x4(qf[s], uQ + tile_off<kTileQ>(warp * 16 + (lane & 15), 2 * s + (lane >> 4)));
+        for (int s = 0; s < KS; ++s)
+          ldmatrix_x4(qf[s], uQ + tile_off<kTileQ>(warp * 16 + (lane & 15), 2 * s + (lane >> 4)));
+      }
     }
     // S = Q K^T : 16 x 64 per warp
     float sc[TK / 8][4];
 #pragma unroll
     for (int i = 0; i < TK / 8; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
-    const uint32_t kb = uK + stage * Smem<D>::kKV;
+    const uint32_t kb = uK + stage * SM::kKV;
 #pragma unroll
     for (int s = 0; s < KS; ++s) {
+      uint32_t ql[4];
+      if constexpr (SPLIT) {
+        ldmatrix_x4(qf[0], uQ + tile_off<kTileQ>(warp * 16 + (lane & 15), 2 * s + (lane >> 4)));
+        ldmatrix_x4(ql, uQl + tile_off<kTileQ>(warp * 16 + (lane & 15), 2 * s + (lane >> 4)));
+      }
+      const uint32_t(&qh)[4] = qf[SPLIT ? 0 : s];
 #pragma unroll
       for (int np = 0; np < TK / 16; ++np) {
         uint32_t bf[4];
-        ldmatrix_x4(bf, kb + tile_off<TK>(np * 16 + (lane & 7) + ((lane >> 4) << 3), 2 * s + ((lane >> 3) & 1)));
-        mma_16816(sc[2 * np], qf[s], bf[0], bf[1]);
-        mma_16816(sc[2 * np + 1], qf[s], bf[2], bf[3]);
+        const uint32_t koff = tile_off<TK>(np * 16 + (lane & 7) + ((lane >> 4) << 3), 2 * s + ((lane >> 3) & 1));
+        if constexpr (SPLIT) {
+          uint32_t bl[4];
+          ldmatrix_x4(bl, uKl + stage * SM::kKV + koff);
+          mma_16816(sc[2 * np], qh, bl[0], bl[1]);
+          mma_16816(sc[2 * np + 1], qh, bl[2], bl[3]);
+        }
+        ldmatrix_x4(bf, kb + koff);
+        if constexpr (SPLIT) {
+          mma_16816(sc[2 * np], ql, bf[0], bf[1]);
+          mma_16816(sc[2 * np + 1], ql, bf[2], bf[3]);
+        }
+        mma_16816(sc[2 * np], qh, bf[0], bf[1]);
+        mma_16816(sc[2 * np + 1], qh, bf[2], bf[3]);
       }
     }
     // logits in log2 units, masks
@@ -205,7 +234,7 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
       pf[nt >> 1][(nt & 1) * 2 + 1] = pack2(p2, p3);
     }
     // O += P V
-    const uint32_t vb = uV + stage * Smem<D>::kKV;
+    const uint32_t vb = uV + stage * SM::kKV;
 #pragma unroll
     for (int kk = 0; kk < TK / 16; ++kk) {
 #pragma unroll
@@ -261,17 +290,15 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
 
 cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st) {
   if (a.total_tiles == 0) return cudaSuccess;
-  cudaError_t e;
-  if (a.g.d == 64) {
-    e = cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kTotal);
+  auto go = [&](auto kernel, int smem_bytes) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    attn_mma_kernel<64><<<a.total_tiles, 256, Smem<64>::kTotal, st>>>(a);
-  } else {
-    e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kTotal);
-    if (e != cudaSuccess) return e;
-    attn_mma_kernel<128><<<a.total_tiles, 256, Smem<128>::kTotal, st>>>(a);
-  }
-  return cudaGetLastError();
+    kernel<<<a.total_tiles, 256, smem_bytes, st>>>(a);
+    return cudaGetLastError();
+  };
+  const bool split = a.q_lo != nullptr;
+  if (a.g.d == 64) return split ? go(attn_mma_kernel<64, true>, Smem<64, true>::kTotal) : go(attn_mma_kernel<64, false>, Smem<64, false>::kTotal);
+  return split ? go(attn_mma_kernel<128, true>, Smem<128, true>::kTotal) : go(attn_mma_kernel<128, false>, Smem<128, false>::kTotal);
 }
 
 }  // namespace hyperattn

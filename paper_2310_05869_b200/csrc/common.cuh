@@ -73,6 +73,7 @@ __host__ __device__ inline void node_rows(const Geometry& g, int level, int j, i
 // ---- stage launchers (each enqueues on `st`; returns cudaGetLastError()) ---------------
 struct Workspace {
   __nv_bfloat16 *q16, *k16, *v16;  // bf16 staging of fp32 inputs (else null)
+  __nv_bfloat16 *q16lo, *k16lo;    // second bf16 term of fp32 Q, K: x ~= x16 + x16lo
   uint8_t* ids;                    // [2, G, n]
   uint32_t* hist;                  // [2, G, chunks_per_seg, 256]
   uint32_t* offs;                  // [2, levels, G, chunks per (level,seg,side), 256]
@@ -82,7 +83,7 @@ struct Workspace {
   int* status;                     // device status word
 };
 
-cudaError_t launch_convert(const float* src, __nv_bfloat16* dst, size_t count, cudaStream_t st);
+cudaError_t launch_convert(const float* src, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t count, cudaStream_t st);
 cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
                         const Workspace& ws, unsigned long long* near_zero, cudaStream_t st);
 cudaError_t launch_samples(const Geometry& g, uint64_t seed, const Workspace& ws, cudaStream_t st);

@@ -195,23 +195,28 @@ __global__ void __launch_bounds__(256) hash_fp32_kernel(const __grid_constant__ 
   a.hist[(((size_t)side * a.G + seg) * a.chunks_per_seg + chunk) * kBuckets + tid] = s_hist[tid];
 }
 
-__global__ void convert_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, size_t count4) {
+// fp32 -> bf16 staging; `lo` (optional) receives the rounding remainder as a second bf16 term
+__global__ void convert_kernel(const float4* __restrict__ src, uint2* __restrict__ hi, uint2* __restrict__ lo,
+                               size_t count4) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count4; i += (size_t)gridDim.x * blockDim.x) {
     const float4 x = src[i];
-    uint2 o;
-    o.x = pack_bf16(x.x, x.y);
-    o.y = pack_bf16(x.z, x.w);
-    dst[i] = o;
+    const float xs[4] = {x.x, x.y, x.z, x.w};
+    float h[4], l[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { h[e] = __bfloat162float(__float2bfloat16_rn(xs[e])); l[e] = xs[e] - h[e]; }
+    hi[i] = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
+    if (lo) lo[i] = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
   }
 }
 
 }  // namespace
 
-cudaError_t launch_convert(const float* src, __nv_bfloat16* dst, size_t count, cudaStream_t st) {
+cudaError_t launch_convert(const float* src, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t count, cudaStream_t st) {
   const size_t count4 = count / 4;
-  const int blocks = (int)((count4 + 255) / 256 < 148 * 16 ? (count4 + 255) / 256 : 148 * 16);
-  convert_kernel<<<blocks > 0 ? blocks : 1, 256, 0, st>>>(reinterpret_cast<const float4*>(src),
-                                                         reinterpret_cast<uint2*>(dst), count4);
+  const size_t want = (count4 + 255) / 256;
+  const int blocks = (int)(want < 148 * 16 ? (want ? want : 1) : 148 * 16);
+  convert_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<uint2*>(hi),
+                                         reinterpret_cast<uint2*>(lo), count4);
   return cudaGetLastError();
 }
 
