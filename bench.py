@@ -402,12 +402,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--n", type=int, default=0, help="override the sequence length (c4 sweep)")
+    ap.add_argument("--heads", type=int, default=0, help="override H (smaller cases for profiler captures)")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = WL.CONFIGS[WORKLOADS[args.workload]]
     if args.n:
         w = w.scaled(n=args.n, name=f"{w.name}_n{args.n}")
+    if args.heads:
+        w = w.scaled(H=args.heads, name=f"{w.name}_h{args.heads}")
     if args.impl == "reference":
         reference_arm(args, w)
     else:
