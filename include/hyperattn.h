@@ -140,7 +140,9 @@ int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes);
 int hyperattn_get_projections(int d, int hash_bits, uint64_t seed, float* host_out);
 
 /* Synchronises `stream` and reports the device status word (0, or
- * HYPERATTN_DEVICE_TIMEOUT if a kernel's bounded wait gave up since the last query). */
+ * HYPERATTN_DEVICE_TIMEOUT if a kernel's bounded wait gave up since the last query) and
+ * clears it.  While the word is set, attention tiles of later launches return without
+ * computing, so a caller that saw a timeout must not use the outputs written since. */
 int hyperattn_last_device_status(void* stream, int* status);
 
 /* Stage timing.  While enabled, every forward call brackets each stage with CUDA events

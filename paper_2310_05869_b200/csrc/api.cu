@@ -13,6 +13,7 @@
 
 namespace hyperattn {
 cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st);
+cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st);
 
 namespace {
 
@@ -62,7 +63,7 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
     }
   }
   if (g.sorted) {
-    const int bpad = (g.b + 63) / 64 * 64, mpad = (g.m + 63) / 64 * 64;
+    const int bpad = (g.b + 127) / 128 * 128, mpad = (g.m + 127) / 128 * 128;
     if (bpad + mpad > kMaxNodeKeys) return HYPERATTN_UNSUPPORTED_SHAPE;
   }
   g.chunks_per_unit = (g.unit + kSortChunk - 1) / kSortChunk;
@@ -295,7 +296,9 @@ int forward_impl(const hyperattn_params& p) {
   a.total_tiles = (int)tiles;
   {
     StageScope sc(st, HYPERATTN_STAGE_ATTENTION, 1);
-    HA_CHECK(launch_attention_mma(a, st));
+    // bf16 inputs: tcgen05 path; fp32 inputs: split-bf16 logits on the warp-level MMA path
+    if (is_fp32) HA_CHECK(launch_attention_mma(a, st));
+    else HA_CHECK(launch_attention_tc(a, ws.status, st));
   }
   if (g.L) {
     StageScope sc(st, HYPERATTN_STAGE_MERGE, 1);

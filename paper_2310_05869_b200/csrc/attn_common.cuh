@@ -17,7 +17,7 @@
 namespace hyperattn {
 
 constexpr int kMaxLevels = 24;
-constexpr int kMaxNodeKeys = 2048;   // padded b + padded m must fit the key index table
+constexpr int kMaxNodeKeys = 1536;   // b and m, each rounded up to 128, must fit the key index table
 
 struct AttnArgs {
   const __nv_bfloat16 *q, *k, *v;    // [G, n, D]
