@@ -64,7 +64,7 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
   }
   if (g.sorted) {
     const int bpad = (g.b + 127) / 128 * 128, mpad = (g.m + 127) / 128 * 128;
-    if (bpad + mpad > kMaxNodeKeys) return HYPERATTN_UNSUPPORTED_SHAPE;
+    if (2 * bpad + mpad > kMaxNodeKeys) return HYPERATTN_UNSUPPORTED_SHAPE;
   }
   g.chunks_per_unit = (g.unit + kSortChunk - 1) / kSortChunk;
   g.chunks_per_seg = (g.n / g.unit) * g.chunks_per_unit;
@@ -280,8 +280,10 @@ int forward_impl(const hyperattn_params& p) {
     a.tiles_per_leaf = (g.leaf + kTileQ - 1) / kTileQ;
     a.leaves_per_seg = g.n / g.leaf;
     a.n_leaf_tiles = g.G * a.leaves_per_seg * a.tiles_per_leaf;
+    a.pairs_per_leaf = (a.tiles_per_leaf + 1) / 2;
+    a.n_leaf_pairs = g.G * a.leaves_per_seg * a.pairs_per_leaf;
   }
-  long long tiles = a.n_leaf_tiles;
+  long long tiles = a.n_leaf_tiles, pairs = a.n_leaf_pairs;
   for (int l = 0; l < g.levels; ++l) {
     int s, q0, k0;
     node_rows(g, l, 0, s, q0, k0);
@@ -291,9 +293,13 @@ int forward_impl(const hyperattn_params& p) {
     const long long per_node = a.level_sorted[l] ? (long long)(s / g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
     tiles += per_node * nodes_lvl * g.G;
     if (tiles > 0x7fffffffLL) return HYPERATTN_UNSUPPORTED_SHAPE;
+    a.level_pair_start[l] = (int)pairs;
+    pairs += ((per_node + 1) / 2) * nodes_lvl * g.G;
   }
   a.level_start[g.levels] = (int)tiles;
   a.total_tiles = (int)tiles;
+  a.level_pair_start[g.levels] = (int)pairs;
+  a.total_pairs = (int)pairs;
   {
     StageScope sc(st, HYPERATTN_STAGE_ATTENTION, 1);
     // bf16 inputs: tcgen05 path; fp32 inputs: split-bf16 logits on the warp-level MMA path

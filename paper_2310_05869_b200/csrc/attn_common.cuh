@@ -17,7 +17,7 @@
 namespace hyperattn {
 
 constexpr int kMaxLevels = 24;
-constexpr int kMaxNodeKeys = 1536;   // b and m, each rounded up to 128, must fit the key index table
+constexpr int kMaxNodeKeys = 2048;   // 2 * (b rounded up to 128) + (m rounded up to 128) must fit the key table
 
 struct AttnArgs {
   const __nv_bfloat16 *q, *k, *v;    // [G, n, D]
@@ -37,6 +37,10 @@ struct AttnArgs {
   int level_sorted[kMaxLevels];      // 1: sortLSH node tiles; 0: single-block node (dense tiles)
   int tiles_per_block;               // ceil(b / 128)
   int total_tiles;
+  // the same schedule in pairs of neighbouring query tiles (tcgen05 path)
+  int pairs_per_leaf, n_leaf_pairs;
+  int level_pair_start[kMaxLevels + 1];
+  int total_pairs;
 };
 
 struct TileDesc {
