@@ -9,7 +9,7 @@ import os
 import numpy as np
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhyperattn.so")
+_LIB_PATH = os.environ.get("HYPERATTN_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhyperattn.so")
 _lib = None
 
 BF16, FP32 = 0, 1

@@ -3,6 +3,7 @@
 // kernels of hash.cu, sort.cu, attn_*.cu and merge.cu.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -294,7 +295,10 @@ int forward_impl(const hyperattn_params& p) {
     tiles += per_node * nodes_lvl * g.G;
     if (tiles > 0x7fffffffLL) return HYPERATTN_UNSUPPORTED_SHAPE;
     a.level_pair_start[l] = (int)pairs;
-    pairs += ((per_node + 1) / 2) * nodes_lvl * g.G;
+    // two query tiles share a CTA when they share their block's keys (even tiles per block),
+    // or when a block is a single tile; other block sizes run one tile per CTA
+    a.level_paired[l] = !a.level_sorted[l] || a.tiles_per_block % 2 == 0 || a.tiles_per_block == 1;
+    pairs += (a.level_paired[l] ? (per_node + 1) / 2 : per_node) * nodes_lvl * g.G;
   }
   a.level_start[g.levels] = (int)tiles;
   a.total_tiles = (int)tiles;
@@ -407,6 +411,7 @@ int hyperattn_last_device_status(void* stream, int* status) {
   int word = 0;
   if (cudaMemcpy(&word, ds.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   if (word) {
+    if (getenv("HYPERATTN_DEBUG")) std::fprintf(stderr, "hyperattn: device status word %d (site of the wait that gave up)\n", word);
     *status = HYPERATTN_DEVICE_TIMEOUT;
     cudaMemset(ds.status, 0, 4);
   }

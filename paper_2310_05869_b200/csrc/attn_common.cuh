@@ -40,6 +40,7 @@ struct AttnArgs {
   // the same schedule in pairs of neighbouring query tiles (tcgen05 path)
   int pairs_per_leaf, n_leaf_pairs;
   int level_pair_start[kMaxLevels + 1];
+  int level_paired[kMaxLevels];      // 1: CTAs of this level own two query tiles, 0: one
   int total_pairs;
 };
 

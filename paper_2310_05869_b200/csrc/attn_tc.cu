@@ -1,7 +1,7 @@
 // Attention tiles on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 inputs.
 //
 // One CTA owns a PAIR of query tiles (2 x 128 rows) that are neighbours in the tile order of
-// their leaf / recursion node, and walks once over the key tiles (128 keys each) that either
+// their leaf / recursion node, and walks once over the key tiles (64 keys each) that either
 // of them needs:
 //     S_i = Q_i K^T      tcgen05.mma, operands in 128B-swizzled shared memory, S_i in TMEM
 //     P_i = exp2(S_i*c + bias - m)   softmax warpgroup i: one thread per query row (TMEM
@@ -10,15 +10,17 @@
 // which covers the block-diagonal part (Sec. 4), the sampled residual with weight N/m
 // (Alg. 2 line 7) and the exact causal leaves (Sec. 3.1) in one loop.  The two query tiles
 // of a 256-row block share every key tile, so K and V are fetched once for 256 rows, and
-// while one warpgroup exponentiates, the tensor pipe works for the other one.  The running
+// every warpgroup has two S buffers in TMEM, so the tensor pipe computes the scores of the
+// next key tile while the warpgroup exponentiates the current one.  The running
 // row maximum is only moved when it grows by more than 2^8 (the accumulators absorb the
 // rest), so O is rarely rescaled; outputs are normalised by the sum of the bf16-rounded
 // weights that the tensor cores actually used, the log-sum-exp by the unrounded sum.  Rows
 // of Q, K, V are gathered from their original places through the sortLSH permutations by
 // three loader warps with 16-byte cp.async copies; nothing permuted is ever written to HBM.
 //
-// Warp roles (384 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
-// warp 8 MMA issue + TMEM allocation (all 512 columns: S0 S1 O0 O1), warps 9-11 loaders.
+// Warp roles (416 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
+// warps 8 and 9 MMA issue for query tile 0 and 1 (warp 8 also allocates TMEM, all 512
+// columns: 2 x 2 S buffers of 64, O0, O1), warps 10-12 loaders.
 // Every mbarrier wait is bounded: on a timeout the CTA raises the device status word,
 // drains its copies, frees its TMEM and returns.
 #include "attn_common.cuh"
@@ -26,10 +28,23 @@
 namespace hyperattn {
 namespace {
 
-constexpr int TK = 128;                 // keys per tile
+constexpr int TK = 64;                  // keys per tile
 constexpr int kLoaderThreads = 96;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
 constexpr float kRescaleThreshold = 8.f;
+#ifndef HA_TAKE_TURNS
+#define HA_TAKE_TURNS 0
+#endif
+
+// Optional per-role cycle counters (compile with -DHA_TC_TIMING; never in the shipped build).
+#ifdef HA_TC_TIMING
+__device__ unsigned long long g_tc_timing[16];
+#define HA_T0(var) const long long var = clock64()
+#define HA_TACC(slot, var) atomicAdd(&g_tc_timing[slot], (unsigned long long)(clock64() - var))
+#else
+#define HA_T0(var)
+#define HA_TACC(slot, var)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -40,10 +55,12 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One potentially-blocking probe: the hardware may park the warp for up to the hinted time (ns)
+// and wakes it when the phase completes, so waiting warps leave the issue slots to the others.
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
   return ok != 0;
 }
 // returns false when the wait gave up (timeout or another thread aborted)
@@ -52,11 +69,15 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+// SLEEP_NS: back-off between probes, so that waiting warps do not take issue slots from the
+// warps that compute (every role waits far more often than it works)
+template <int SLEEP_NS = 32, int SITE = 1>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
   unsigned long long t0 = 0;
   for (unsigned it = 0;; ++it) {
     if (mbar_try(bar, parity)) return true;
-    if ((it & 255u) == 255u) {
+    __nanosleep(SLEEP_NS);
+    if ((it & 63u) == 63u) {
       if (*abort_flag) return false;
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
@@ -64,7 +85,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
   *abort_flag = 1;
-  atomicExch(status, 1);
+  atomicOr(status, 1 << SITE);     // bit mask of the wait sites that gave up
   return false;
 }
 
@@ -103,6 +124,52 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 }
+// issue without waiting; the data is valid only after tmem_ld32_wait on the same registers
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                 "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                 "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+               : "r"(taddr));
+}
+// waits for every outstanding TMEM load of this thread; the registers are listed as
+// read-write operands so that no use of them can be scheduled above the wait
+__device__ __forceinline__ void tmem_ld32_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :: "memory");
+}
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :: "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
                ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
@@ -122,6 +189,15 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
 }
+// 16 bytes of zeros through the same asynchronous path (source size 0), so that they are tracked
+// by the same completion mechanism as the copies around them
+__device__ __forceinline__ void cp_async16_zero(uint32_t dst, const void* any_valid_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, 0;\n" ::"r"(dst), "l"(any_valid_src) : "memory");
+}
+// the executing thread's arrival on the mbarrier happens when all its earlier cp.async have landed
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void st_shared_zero16(uint32_t dst) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};\n" ::"r"(dst), "r"(0) : "memory");
 }
@@ -130,7 +206,10 @@ __device__ __forceinline__ void cp_async_wait_le(int n) {   // wait until at mos
   switch (n) {
     case 0: asm volatile("cp.async.wait_group 0;\n" ::: "memory"); break;
     case 1: asm volatile("cp.async.wait_group 1;\n" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
+    case 2: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
+    case 3: asm volatile("cp.async.wait_group 3;\n" ::: "memory"); break;
+    case 4: asm volatile("cp.async.wait_group 4;\n" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 5;\n" ::: "memory"); break;
   }
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -140,45 +219,64 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-// byte offset of 16-byte chunk c of row `row` in a [128 x D] bf16 tile: D/64 slabs of
-// [128 rows x 128 B], 128-byte swizzle inside each slab (the canonical tcgen05 layout)
+// byte offset of 16-byte chunk c of row `row` in a [ROWS x D] bf16 tile: D/64 slabs of
+// [ROWS rows x 128 B], 128-byte swizzle inside each slab (the canonical tcgen05 layout)
+template <int ROWS>
 __device__ __forceinline__ uint32_t tile_off(int row, int c) {
-  return (uint32_t)((c >> 3) * (128 * 128) + row * 128 + (((c & 7) ^ (row & 7)) << 4));
+  return (uint32_t)((c >> 3) * (ROWS * 128) + row * 128 + (((c & 7) ^ (row & 7)) << 4));
+}
+
+// Rare path of the online softmax: multiply the O columns a row has accumulated so far by
+// alpha (a power of two, so nothing is re-rounded).  Kept out of line: the hot loop should
+// stay small.  All 32 lanes call it together (TMEM accesses are warp-wide).
+__device__ __noinline__ void rescale_row(uint32_t o_addr, int ocols, float alpha) {
+  uint32_t r[16];
+  for (int c = 0; c < ocols; c += 16) {
+    tmem_ld16_issue(o_addr + c, r);
+    tmem_ld16_wait(r);
+#pragma unroll
+    for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+                 ::"r"(o_addr + c), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+  }
+  tmem_wait_st();
 }
 
 template <int D>
 struct Cfg {
-  static constexpr int NS = (D == 64) ? 4 : 2;        // K stages and V stages
-  static constexpr int kTile = 128 * D * 2;           // bytes of one 128-row tile
+  static constexpr int NS = (D == 64) ? 8 : 4;        // K stages and V stages
+  static constexpr int kQTile = 128 * D * 2;          // bytes of one 128-row query tile
+  static constexpr int kTile = TK * D * 2;            // bytes of one key / value tile
   static constexpr int kOffQ = 0;                     // Q0, Q1
-  static constexpr int kOffK = 2 * kTile;
+  static constexpr int kOffK = 2 * kQTile;
   static constexpr int kOffV = kOffK + NS * kTile;
   static constexpr int kOffIdx = kOffV + NS * kTile;              // int [kMaxNodeKeys] key rows
   static constexpr int kOffMask = kOffIdx + kMaxNodeKeys * 4;     // uint32 [2][kMaxNodeKeys/32] masked-column bits
   static constexpr int kOffQrow = kOffMask + 2 * (kMaxNodeKeys / 32) * 4;   // int [2][128]
   static constexpr int kOffBar = kOffQrow + 2 * 128 * 4;
-  static constexpr int kNumBar = 7 + 4 * NS;
+  static constexpr int kNumBar = 13 + 6 * NS;
   static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
   static constexpr int kTotal = kOffMisc + 16;
   static constexpr int kTmemCols = 512;
-  static constexpr int kColS = 0;                     // S_i at kColS + 128 i
-  static constexpr int kColO = 256;                   // O_i at kColO + D i
+  static constexpr int kColO = 256;                   // S buffer b of tile i at 64 (2 i + b); O_i at kColO + D i
 };
 
-// One query tile of the pair.
+// One query tile of the pair.  The key tiles it looks at are two runs of the pair's tile
+// list: [s1, s1 + n1) and [s2, s2 + n2).
 struct QTile {
   int valid;
   int nq;        // valid rows
   int q0;        // dense: first query row (segment-relative)
-  int tt;        // dense causal: index of the diagonal key tile
+  int row0;      // dense causal: local index of the tile's first row (relative to the first key)
   int beta;      // node: block
   int spos0;     // node: first sorted position
+  int s1, n1, s2, n2;
 };
 
 struct PairDesc {
   int mode;            // 0 dense, 1 node
   int seg;
-  QTile qt[2];
   int causal;          // dense
   int k0, nk;          // dense: key range; node: first key row of the node and N
   int qnode0;          // node: first query row of the node
@@ -189,11 +287,10 @@ struct PairDesc {
   size_t orow_base; int odelta; int partial;
 };
 
-__device__ __forceinline__ PairDesc decode_pair(const AttnArgs& a, int pair) {
+__device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDesc& t, QTile& qa, QTile& qb) {
   const Geometry& g = a.g;
-  PairDesc t;
   t.partial = !a.direct;
-  t.qt[0].valid = 1; t.qt[1].valid = 0;
+  qa.valid = 1; qb.valid = 0;
   t.nbA = t.nbB = t.nsmp = 0;
   int s, q0n, k0n;
   if (pair < a.n_leaf_pairs) {
@@ -204,12 +301,17 @@ __device__ __forceinline__ PairDesc decode_pair(const AttnArgs& a, int pair) {
     const int leaf = rem % a.leaves_per_seg;
     t.mode = 0; t.causal = a.dense_causal;
     t.k0 = leaf * g.leaf; t.nk = g.leaf;
+    QTile* qs[2] = {&qa, &qb};
+#pragma unroll
     for (int i = 0; i < 2; ++i) {
       const int tt = 2 * uu + i;
-      t.qt[i].valid = tt < a.tiles_per_leaf;
-      t.qt[i].tt = tt;
-      t.qt[i].q0 = t.k0 + tt * kTileQ;
-      t.qt[i].nq = min(kTileQ, g.leaf - tt * kTileQ);
+      QTile& q = *qs[i];
+      q.valid = tt < a.tiles_per_leaf;
+      q.row0 = tt * kTileQ;
+      q.q0 = t.k0 + tt * kTileQ;
+      q.nq = min(kTileQ, g.leaf - tt * kTileQ);
+      const int lim = t.causal ? min(t.nk, q.row0 + q.nq) : t.nk;
+      q.s1 = 0; q.n1 = q.valid ? (lim + TK - 1) / TK : 0; q.s2 = 0; q.n2 = 0;
     }
     t.orow_base = (size_t)t.seg * g.n; t.odelta = 0;
   } else {
@@ -219,18 +321,22 @@ __device__ __forceinline__ PairDesc decode_pair(const AttnArgs& a, int pair) {
     node_rows(g, level, 0, s, q0n, k0n);
     const int nodes_lvl = g.causal ? (1 << level) : 1;
     const int sorted = a.level_sorted[level];
+    const int paired = a.level_paired[level];
     const int tiles_node = sorted ? (s / g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
-    const int pairs_node = (tiles_node + 1) / 2;
+    const int pairs_node = paired ? (tiles_node + 1) / 2 : tiles_node;
     const int pn = idx % pairs_node; idx /= pairs_node;
     const int j = idx % nodes_lvl;
     t.seg = idx / nodes_lvl;
     node_rows(g, level, j, s, q0n, k0n);
     t.k0 = k0n; t.nk = s; t.qnode0 = q0n; t.causal = 0;
+    t.mode = sorted;
+    QTile* qs[2] = {&qa, &qb};
+#pragma unroll
     for (int i = 0; i < 2; ++i) {
-      const int tn = 2 * pn + i;
-      QTile& q = t.qt[i];
-      q.valid = tn < tiles_node;
-      q.tt = 0;
+      const int tn = paired ? 2 * pn + i : pn;
+      QTile& q = *qs[i];
+      q.valid = tn < tiles_node && (paired || i == 0);
+      q.row0 = 0;
       if (sorted) {
         q.beta = tn / a.tiles_per_block;
         const int sub = tn % a.tiles_per_block;
@@ -240,41 +346,33 @@ __device__ __forceinline__ PairDesc decode_pair(const AttnArgs& a, int pair) {
       } else {
         q.q0 = q0n + tn * kTileQ;
         q.nq = min(kTileQ, s - tn * kTileQ);
+        q.s1 = 0; q.n1 = q.valid ? (s + TK - 1) / TK : 0; q.s2 = 0; q.n2 = 0;
       }
     }
-    t.mode = sorted;
     if (sorted) {
       t.slice = ((size_t)level * g.G + t.seg) * g.nl + (g.causal ? (size_t)j * s : 0);
       t.node = g.causal ? (1 << level) - 1 + j : 0;
       const int bt = (g.b + TK - 1) / TK;
       t.nbA = bt;
-      t.nbB = (t.qt[1].valid && t.qt[1].beta != t.qt[0].beta) ? bt : 0;
+      t.nbB = (qb.valid && qb.beta != qa.beta) ? bt : 0;
       t.nsmp = (g.m + TK - 1) / TK;
+      qa.s1 = 0; qa.n1 = bt; qa.s2 = t.nbA + t.nbB; qa.n2 = t.nsmp;
+      qb.s1 = t.nbB ? t.nbA : 0; qb.n1 = qb.valid ? bt : 0; qb.s2 = t.nbA + t.nbB; qb.n2 = qb.valid ? t.nsmp : 0;
     }
     if (a.direct) { t.orow_base = (size_t)t.seg * g.n; t.odelta = 0; }
     else { t.orow_base = (size_t)g.G * g.n + (size_t)level * g.G * g.nl + (size_t)t.seg * g.nl + (size_t)j * s; t.odelta = -q0n; }
   }
-  if (t.mode == 1) {
-    t.ntiles = t.nbA + t.nbB + t.nsmp;
-  } else {
-    const QTile& last = t.qt[1].valid ? t.qt[1] : t.qt[0];
-    const int lim = t.causal ? min(t.nk, last.tt * kTileQ + last.nq) : t.nk;
-    t.ntiles = (lim + TK - 1) / TK;
-  }
-  return t;
+  t.ntiles = max(qa.s1 + qa.n1, max(qa.s2 + qa.n2, max(qb.s1 + qb.n1, qb.s2 + qb.n2)));
 }
 
-// does query tile i of the pair look at key tile j ?
-__device__ __forceinline__ bool tile_active(const PairDesc& t, int i, int j) {
-  if (!t.qt[i].valid) return false;
-  if (t.mode == 0) return !t.causal || j <= t.qt[i].tt;
-  if (j >= t.nbA + t.nbB) return true;                         // samples: both
-  if (j < t.nbA) return i == 0 || t.nbB == 0;                  // block of tile 0 (shared when nbB == 0)
-  return i == 1;                                               // block of tile 1
+// a-th key tile of a query tile -> index in the pair's tile list
+__device__ __forceinline__ int tile_of(const QTile& q, int a) { return a < q.n1 ? q.s1 + a : q.s2 + (a - q.n1); }
+__device__ __forceinline__ bool uses_tile(const QTile& q, int j) {
+  return (j >= q.s1 && j < q.s1 + q.n1) || (j >= q.s2 && j < q.s2 + q.n2);
 }
 
 template <int D>
-__global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, int* status) {
+__global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   int* s_kidx = reinterpret_cast<int*>(smem + C::kOffIdx);
@@ -287,17 +385,21 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   const uint32_t ubase = smem_u32(smem);
   const uint32_t bar0 = ubase + C::kOffBar;
   const uint32_t bar_q = bar0;
-  auto bar_s = [&](int i) { return bar0 + 8 + 8 * i; };
-  auto bar_p = [&](int i) { return bar0 + 24 + 8 * i; };
-  auto bar_o = [&](int i) { return bar0 + 40 + 8 * i; };
-  auto bar_kfull = [&](int s) { return bar0 + 56 + 8 * s; };
-  auto bar_kempty = [&](int s) { return bar0 + 56 + 8 * (C::NS + s); };
-  auto bar_vfull = [&](int s) { return bar0 + 56 + 8 * (2 * C::NS + s); };
-  auto bar_vempty = [&](int s) { return bar0 + 56 + 8 * (3 * C::NS + s); };
+  auto bar_s = [&](int i, int b) { return bar0 + 8 + 8 * (2 * i + b); };      // S_i buffer b written
+  auto bar_p = [&](int i, int b) { return bar0 + 40 + 8 * (2 * i + b); };     // P_i buffer b written
+  auto bar_o = [&](int i) { return bar0 + 72 + 8 * i; };
+  auto bar_pv = [&](int i) { return bar0 + 88 + 8 * i; };                     // a PV_i finished
+  auto bar_kfull = [&](int s) { return bar0 + 104 + 8 * s; };
+  auto bar_vfull = [&](int s) { return bar0 + 104 + 8 * (C::NS + s); };
+  auto bar_kempty = [&](int i, int s) { return bar0 + 104 + 8 * ((2 + i) * C::NS + s); };     // released by issuer i
+  auto bar_vempty = [&](int i, int s) { return bar0 + 104 + 8 * ((4 + i) * C::NS + s); };
 
   const Geometry& g = a.g;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const PairDesc t = decode_pair(a, blockIdx.x);
+  PairDesc t;
+  QTile qa, qb;
+  decode_pair(a, blockIdx.x, t, qa, qb);
+  HA_T0(tcta);
 
   // A CTA of a launch in which some wait already timed out returns at once (nothing allocated
   // yet), so a stuck launch drains quickly instead of timing out tile after tile.
@@ -309,16 +411,19 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   // ---- setup: barriers, TMEM, row tables ----------------------------------------------------
   if (tid == 0) {
     mbar_init(bar_q, kLoaderThreads);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_s(i), 1); mbar_init(bar_p(i), 128); mbar_init(bar_o(i), 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_o(i), 1);
+      mbar_init(bar_pv(i), 1);
+      for (int b = 0; b < 2; ++b) { mbar_init(bar_s(i, b), 1); mbar_init(bar_p(i, b), 128); }
+    }
     for (int s = 0; s < C::NS; ++s) {
       mbar_init(bar_kfull(s), kLoaderThreads);
       mbar_init(bar_vfull(s), kLoaderThreads);
-      mbar_init(bar_kempty(s), 1);
-      mbar_init(bar_vempty(s), 1);
+      for (int i = 0; i < 2; ++i) { mbar_init(bar_kempty(i, s), 1); mbar_init(bar_vempty(i, s), 1); }
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = tid; i < 2 * MW; i += 384) s_mask[i] = 0;
+  for (int i = tid; i < 2 * MW; i += 416) s_mask[i] = 0;
   if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(C::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -327,19 +432,19 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 
   float wlog = 0.f;  // log2(N/m): weight of a sampled column
   if (t.mode == 1) {
-    const int bpad = t.nbA * TK;
+    const int bcols = t.nbA * TK;
     const int ncols = t.ntiles * TK;
     wlog = g.m > 0 ? log2f((float)t.nk / (float)g.m) : 0.f;
     const int32_t* smp = a.samples + ((size_t)t.seg * g.nodes + t.node) * g.m;
-    for (int i = tid; i < ncols; i += 384) {
+    for (int i = tid; i < ncols; i += 416) {
       int idx = -1;
-      bool masked[2] = {true, true};
+      bool m0 = true, m1 = true;                      // masked for query tile 0 / 1
       if (i < (t.nbA + t.nbB) * TK) {
-        const int which = i >= bpad;                  // 0: block of tile 0, 1: block of tile 1
-        const int c = i - which * bpad;
+        const int which = i >= bcols;                 // 0: block of tile 0, 1: block of tile 1
+        const int c = i - which * bcols;
         if (c < g.b) {
-          idx = t.k0 + a.perm_k[t.slice + (size_t)t.qt[which].beta * g.b + c];
-          masked[0] = masked[1] = false;
+          idx = t.k0 + a.perm_k[t.slice + (size_t)(which ? qb.beta : qa.beta) * g.b + c];
+          m0 = m1 = false;
         }
       } else {
         const int c = i - (t.nbA + t.nbB) * TK;
@@ -347,23 +452,23 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           const int l = smp[c];
           idx = t.k0 + l;
           const int blk = a.rank_k[t.slice + l] / g.b;
-          masked[0] = blk == t.qt[0].beta;            // the factor (1 - M^H) of Alg. 2 line 7
-          masked[1] = t.qt[1].valid && blk == t.qt[1].beta;
+          m0 = blk == qa.beta;                        // the factor (1 - M^H) of Alg. 2 line 7
+          m1 = qb.valid && blk == qb.beta;
         }
       }
       s_kidx[i] = idx;
-      if (masked[0]) atomicOr(&s_mask[i >> 5], 1u << (i & 31));
-      if (masked[1]) atomicOr(&s_mask[MW + (i >> 5)], 1u << (i & 31));
+      if (m0) atomicOr(&s_mask[i >> 5], 1u << (i & 31));
+      if (m1) atomicOr(&s_mask[MW + (i >> 5)], 1u << (i & 31));
     }
     if (tid < 2 * kTileQ) {
-      const int i = tid >> 7, r = tid & 127;
-      const QTile& q = t.qt[i];
+      const int r = tid & 127;
+      const QTile& q = tid < 128 ? qa : qb;
       s_qrow[tid] = (q.valid && r < q.nq) ? t.qnode0 + a.perm_q[t.slice + q.spos0 + r] : -1;
     }
   } else {
     if (tid < 2 * kTileQ) {
-      const int i = tid >> 7, r = tid & 127;
-      const QTile& q = t.qt[i];
+      const int r = tid & 127;
+      const QTile& q = tid < 128 ? qa : qb;
       s_qrow[tid] = (q.valid && r < q.nq) ? q.q0 + r : -1;
     }
   }
@@ -377,109 +482,131 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     // ================= softmax + epilogue of query tile i: thread = query row ==================
     const int i = warp >> 2;
     const int row = tid & 127;
-    const QTile& q = t.qt[i];
+    const QTile q = i ? qb : qa;
+    const int total = q.n1 + q.n2;
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t colS = C::kColS + 128 * i, colO = C::kColO + D * i;
-    float m_ref = -INFINITY, l = 0.f, lr = 0.f;     // l: unrounded row sum, lr: sum of the bf16 weights
+    const uint32_t colO = C::kColO + D * i;
+    float m_ref = -INFINITY;
+    float l0 = 0.f, l1 = 0.f, lr0 = 0.f, lr1 = 0.f;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each)
     bool ok = true;
-    int na = 0;                                     // active tiles seen
-    for (int j = 0; j < ntiles && ok; ++j) {
-      if (!tile_active(t, i, j)) continue;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_s(i), na & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
+    for (int na = 0; na < total && ok; ++na) {
+      const int j = tile_of(q, na);
+      const int buf = na & 1;
+      HA_T0(tw);
+      ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (na >> 1) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
       if (!ok) break;
       tc_fence_after();
+      if (row == 0) HA_TACC(0 + i, tw);
+      HA_T0(tc);
       // mask kind of this (query tile, key tile): uniform over the warpgroup
       bool table = false, dense_mask = false;
       float ubias = 0.f;
       int climit = 0;                               // dense: last visible column of this row
       if (t.mode == 1) {
         const uint32_t* mw = s_mask + i * MW + j * (TK / 32);
-        table = (mw[0] | mw[1] | mw[2] | mw[3]) != 0;
+        table = (mw[0] | mw[1]) != 0;
         ubias = (j < t.nbA + t.nbB) ? 0.f : wlog;
       } else {
-        dense_mask = (j * TK + TK > t.nk) || (t.causal && j == q.tt);
-        climit = t.causal ? min(t.nk - 1, q.tt * kTileQ + row) : t.nk - 1;
+        climit = t.causal ? min(t.nk - 1, q.row0 + row) : t.nk - 1;
+        dense_mask = (j * TK + TK > t.nk) || (t.causal && j * TK + TK - 1 > q.row0);
       }
-      // pass 1: row maximum of the tile
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < TK / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(lane_addr + colS + c * 32, r);
-        if (table) {
-          const uint32_t bits = s_mask[i * MW + j * (TK / 32) + c];
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (!((bits >> e) & 1u)) mx = fmaxf(mx, __uint_as_float(r[e]));
-        } else if (dense_mask) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (j * TK + c * 32 + e <= climit) mx = fmaxf(mx, __uint_as_float(r[e]));
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
-        }
+      // The 64 scores of this row are read from TMEM once; then (1) the row maximum, (2)
+      // exponentials, row sums and the bf16 P written over the first half of the S buffer.
+      // The reference maximum only moves when the tile exceeds it by more than 2^8, and then
+      // by a whole number of octaves, so that what is already accumulated (O and the row
+      // sums) is rescaled exactly.
+      uint32_t ra[32], rb[32];
+      const uint32_t sbase = lane_addr + 64 * (2 * i + buf);
+      tmem_ld32_issue(sbase, ra);
+      tmem_ld32_issue(sbase + 32, rb);
+      const bool masked_tile = table || dense_mask;
+      uint32_t visa = 0xffffffffu, visb = 0xffffffffu;
+      if (table) { visa = ~s_mask[i * MW + j * 2]; visb = ~s_mask[i * MW + j * 2 + 1]; }
+      else if (dense_mask) {
+        const int rel = climit - j * TK;              // columns 0..rel of the tile are visible
+        visa = rel >= 31 ? 0xffffffffu : (rel < 0 ? 0u : ((2u << rel) - 1u));
+        visb = rel >= 63 ? 0xffffffffu : (rel < 32 ? 0u : ((2u << (rel - 32)) - 1u));
       }
-      mx = fmaf(mx, a.scale_log2, ubias);           // scale_log2 > 0: the maximum commutes with it
-      // move the reference maximum only when it grows a lot (or on the first finite value);
-      // the decision is taken per warp so that the TMEM accesses stay convergent
-      const bool grow = mx > m_ref + kRescaleThreshold;
-      if (__any_sync(0xffffffffu, grow)) {
-        if (na > 0) {
-          const float alpha = grow ? exp2f(m_ref - mx) : 1.f;   // 0 when m_ref = -inf
-          l *= alpha; lr *= alpha;
-#pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(lane_addr + colO + c * 32, r);
+      tmem_ld32_wait(ra);
+      tmem_ld32_wait(rb);
+      float m0 = -INFINITY, m1 = -INFINITY;
+      if (masked_tile) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-            tmem_st32(lane_addr + colO + c * 32, r);
-          }
+        for (int e = 0; e < 32; ++e) {
+          if ((visa >> e) & 1u) m0 = fmaxf(m0, __uint_as_float(ra[e]));
+          if ((visb >> e) & 1u) m1 = fmaxf(m1, __uint_as_float(rb[e]));
         }
-        if (grow) m_ref = mx;
-      }
-      const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
-      // pass 2: P = exp2(x - m), row sums, bf16 P over the first half of S's columns
-#pragma unroll 1
-      for (int c = 0; c < TK / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(lane_addr + colS + c * 32, r);
-        uint32_t p[16];
-        uint32_t vis = 0xffffffffu;                 // visible columns of this chunk
-        if (table) vis = ~s_mask[i * MW + j * (TK / 32) + c];
-        else if (dense_mask) {
-          const int rel = climit - (j * TK + c * 32);           // columns 0..rel visible
-          vis = rel >= 31 ? 0xffffffffu : (rel < 0 ? 0u : ((2u << rel) - 1u));
-        }
+      } else {
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
-          float p0 = exp2f(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
-          float p1 = exp2f(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
-          if (table || dense_mask) {
+          m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+          m1 = max3(m1, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+        }
+      }
+      const float xm = fmaf(fmaxf(m0, m1), a.scale_log2, ubias);   // scale_log2 > 0: the maximum commutes with it
+      const bool grow = xm > m_ref + kRescaleThreshold;
+      if (__any_sync(0xffffffffu, grow)) {          // rare; per warp so that TMEM accesses stay convergent
+        float alpha = 1.f;
+        if (grow) {
+          if (m_ref == -INFINITY) { m_ref = xm; alpha = 0.f; }
+          else { const float k = ceilf(xm - m_ref); m_ref += k; alpha = ex2(-k); }
+        }
+        l0 *= alpha; l1 *= alpha; lr0 *= alpha; lr1 *= alpha;
+        // O may only be touched between two PV products: the one of the previous tile must
+        // have finished (the one of this tile cannot start before this tile's P is published)
+        if (na > 0) {
+          // S of tile na+1 is committed after the PV of tile na-1, so its arrival implies that PV;
+          // the last tile has no successor and uses the PV barrier (committed after PV total-2)
+          if (na + 1 < total) ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_s(i, (na + 1) & 1), ((na + 1) >> 1) & 1, s_abort, status));
+          else ok = __all_sync(0xffffffffu, mbar_wait<20, 4>(bar_pv(i), 0, s_abort, status));
+          if (!ok) break;
+          tc_fence_after();
+          rescale_row(lane_addr + colO, D, alpha);
+        }
+      }
+      const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
+      auto chunk_exp = [&](const uint32_t (&r)[32], uint32_t vis, int c) {
+        uint32_t p[16];
+        if (masked_tile) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
+            float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
             if (!((vis >> e) & 1u)) p0 = 0.f;
             if (!((vis >> (e + 1)) & 1u)) p1 = 0.f;
+            l0 += p0; l1 += p1;
+            const uint32_t w = pack2(p0, p1);
+            lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
+            p[e >> 1] = w;
           }
-          l += p0 + p1;
-          const uint32_t w = pack2(p0, p1);
-          lr += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
-          p[e >> 1] = w;
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
+            const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
+            l0 += p0; l1 += p1;
+            const uint32_t w = pack2(p0, p1);
+            lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
+            p[e >> 1] = w;
+          }
         }
-        tmem_st16(lane_addr + colS + c * 16, p);
-      }
+        tmem_st16(sbase + c * 16, p);
+      };
+      chunk_exp(ra, visa, 0);
+      chunk_exp(rb, visb, 1);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_p(i));
-      ++na;
+      mbar_arrive(bar_p(i, buf));
+      if (row == 0) HA_TACC(2 + i, tc);
     }
     // epilogue
     if (q.valid) {
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_o(i), 0, s_abort, status));
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait<20, 5>(bar_o(i), 0, s_abort, status));
       if (ok) {
         tc_fence_after();
         const int qr = s_qrow[i * 128 + row];
-        const float inv = 1.f / lr;
-        const float lse = (m_ref + log2f(l)) * 0.69314718055994531f;
+        const float inv = 1.f / (lr0 + lr1);
+        const float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
         const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
 #pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
@@ -512,128 +639,167 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
       }
     }
-  } else if (warp == 8) {
-    // ================= MMA issue (one lane) ===========================================================
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+  } else if (warp < 10) {
+    // ================= MMA issue: one lane per query tile (warp 8: tile 0, warp 9: tile 1) ===========
+    // Each issuer walks its own key tiles: scores run two tiles ahead of the PV products
+    // (S buffers alternate).  A tcgen05.mma costs the issuing thread and the tensor pipe
+    // about 55-65 cycles whatever its size, and every commit / barrier probe adds to that, so
+    // the two chains are issued by two threads.  Shared K / V stages are released per issuer.
+    const int i = warp - 8;
+    const QTile q = i ? qb : qa;
+    const int total = q.n1 + q.n2;
+    if (lane == 0 && total > 0) {
+      constexpr uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)TK >> 3) << 17) | ((128u >> 4) << 24);
       constexpr uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
-      bool ok = mbar_wait(bar_q, 0, s_abort, status);
-      int done[2] = {0, 0};        // PV steps issued per query tile
-      int pend[2] = {-1, -1};      // key tile whose P_i is awaited
-      int total[2] = {0, 0};
-      for (int j = 0; j < ntiles; ++j) { total[0] += tile_active(t, 0, j); total[1] += tile_active(t, 1, j); }
-      // PV_i of the pending key tile: needs P_i (softmax) and V of that tile
-      auto flush_pv = [&](int i) {
-        const int jp = pend[i];
-        const int s = jp % C::NS;
-        ok = mbar_wait(bar_p(i), done[i] & 1, s_abort, status);
+      HA_T0(tq);
+      bool ok = mbar_wait<20, 6>(bar_q, 0, s_abort, status);
+      fence_async_smem();
+      if (i == 0) HA_TACC(7, tq);
+      HA_T0(tall);
+      int kseen = -1, vseen = -1;           // highest tile index whose K / V arrival has been observed
+      int krel = -1, vrel = -1;             // highest tile index whose K / V stage this issuer has released
+      // Shared-memory descriptors are built once; per MMA only the start-address field (in
+      // 16-byte units, low bits of the descriptor) moves, by compile-time offsets.
+      const uint64_t dq = make_desc(ubase + C::kOffQ + i * C::kQTile, 16, 1024);
+      const uint64_t dk0 = make_desc(ubase + C::kOffK, 16, 1024);
+      const uint64_t dv0 = make_desc(ubase + C::kOffV, TK * 128, 1024);
+      const uint32_t ocol = tmem + C::kColO + D * i;
+      // K / V arrive in tile order; observing tile j means observing every barrier phase up to it
+      auto see_k = [&](int j) {
+        for (int jj = kseen + 1; jj <= j && ok; ++jj) ok = mbar_wait<20, 7>(bar_kfull(jj % C::NS), (jj / C::NS) & 1, s_abort, status);
+        if (ok && j > kseen) { kseen = j; fence_async_smem(); tc_fence_after(); }
+      };
+      auto see_v = [&](int j) {
+        for (int jj = vseen + 1; jj <= j && ok; ++jj) ok = mbar_wait<20, 9>(bar_vfull(jj % C::NS), (jj / C::NS) & 1, s_abort, status);
+        if (ok && j > vseen) { vseen = j; fence_async_smem(); tc_fence_after(); }
+      };
+      // Tiles this query tile does not look at are released when the walk passes them, but only
+      // after they have arrived: a release must never overtake the loader's wait for the
+      // previous release of the same stage (the barrier would wrap around unseen).  Releases go
+      // through tcgen05.commit, so they also stay behind this thread's earlier MMAs.
+      auto skip_k_to = [&](int j) {
+        for (int jj = krel + 1; jj < j && ok; ++jj) { see_k(jj); if (ok) umma_commit(bar_kempty(i, jj % C::NS)); }
+        if (j - 1 > krel) krel = j - 1;
+      };
+      auto skip_v_to = [&](int j) {
+        for (int jj = vrel + 1; jj < j && ok; ++jj) { see_v(jj); if (ok) umma_commit(bar_vempty(i, jj % C::NS)); }
+        if (j - 1 > vrel) vrel = j - 1;
+      };
+      // S of the a-th key tile into buffer a & 1
+      auto issue_s = [&](int a2) {
+        const int j = tile_of(q, a2);
+        const int s = j % C::NS;
+        skip_k_to(j);
+        HA_T0(tk);
+        see_k(j);
+        if (i == 0) HA_TACC(6, tk);
         if (!ok) return;
-        ok = mbar_wait(bar_vfull(s), (jp / C::NS) & 1, s_abort, status);
+        const uint32_t dcol = tmem + 64 * (2 * i + (a2 & 1));
+        const uint64_t dk = dk0 + (uint64_t)((s * C::kTile) >> 4);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          mma_ss(dcol, dq + (uint64_t)(((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4),
+                 dk + (uint64_t)(((ks >> 2) * (TK * 128) + (ks & 3) * 32) >> 4), idesc_s, ks > 0);
+        umma_commit(bar_s(i, a2 & 1));
+        umma_commit(bar_kempty(i, s));
+        krel = j;
+      };
+      // O += P V of the a-th key tile
+      auto issue_pv = [&](int a2) {
+        const int j = tile_of(q, a2);
+        const int s = j % C::NS;
+        skip_v_to(j);
+        HA_T0(tp);
+        ok = mbar_wait<20, 8>(bar_p(i, a2 & 1), (a2 >> 1) & 1, s_abort, status);
+        if (i == 0) HA_TACC(4, tp);
+        if (!ok) return;
+        HA_T0(tv);
+        see_v(j);
+        if (i == 0) HA_TACC(5, tv);
         if (!ok) return;
         tc_fence_after();
+        const uint32_t pcol = tmem + 64 * (2 * i + (a2 & 1));
+        const uint64_t dv = dv0 + (uint64_t)((s * C::kTile) >> 4);
 #pragma unroll
         for (int kk = 0; kk < TK / 16; ++kk)
-          mma_ts(tmem + C::kColO + D * i, tmem + C::kColS + 128 * i + kk * 8,
-                 make_desc(ubase + C::kOffV + s * C::kTile + kk * 2048, 128 * 128, 1024), idesc_o, (done[i] > 0 || kk > 0));
-        ++done[i];
-        pend[i] = -1;
-        // V of tile jp is free once every query tile that uses it has issued its PV
-        const int other = 1 - i;
-        if (!tile_active(t, other, jp) || pend[other] != jp) umma_commit(bar_vempty(s));
-        if (done[i] == total[i]) umma_commit(bar_o(i));
+          mma_ts(ocol, pcol + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_o, (a2 > 0 || kk > 0));
+        if (a2 == total - 2) umma_commit(bar_pv(i));
+        umma_commit(bar_vempty(i, s));
+        vrel = j;
+        if (a2 == total - 1) umma_commit(bar_o(i));
       };
-      for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % C::NS;
-        bool waited_k = false;
-        for (int i = 0; i < 2 && ok; ++i) {
-          if (pend[i] >= 0) flush_pv(i);
-          if (!ok) break;
-          if (!tile_active(t, i, j)) continue;
-          if (!waited_k) {
-            ok = mbar_wait(bar_kfull(s), (j / C::NS) & 1, s_abort, status);
-            if (!ok) break;
-            tc_fence_after();
-            waited_k = true;
-          }
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const uint32_t koff = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
-            mma_ss(tmem + C::kColS + 128 * i, make_desc(ubase + C::kOffQ + i * C::kTile + koff, 16, 1024),
-                   make_desc(ubase + C::kOffK + s * C::kTile + koff, 16, 1024), idesc_s, ks > 0);
-          }
-          umma_commit(bar_s(i));
-          pend[i] = j;
-          // K of tile j is free once the last query tile that uses it has issued its S
-          if (i == 1 || !tile_active(t, 1, j)) umma_commit(bar_kempty(s));
-        }
+      for (int r = 0; r < total + 2 && ok; ++r) {
+        if (r >= 2) issue_pv(r - 2);
+        if (ok && r < total) issue_s(r);
       }
-      for (int i = 0; i < 2 && ok; ++i)
-        if (pend[i] >= 0) flush_pv(i);
+      if (ok) { skip_k_to(ntiles); skip_v_to(ntiles); }
+      if (i == 0) HA_TACC(8, tall);
     }
     __syncwarp();
   } else {
     // ================= loaders: gather rows into swizzled tiles ======================================
-    const int lt = tid - 288;
+    const int lt = tid - 320;
     const __nv_bfloat16* qs = a.q + (size_t)t.seg * g.n * D;
     const __nv_bfloat16* ks = a.k + (size_t)t.seg * g.n * D;
     const __nv_bfloat16* vs = a.v + (size_t)t.seg * g.n * D;
     constexpr int CPR = D / 8;
-    uint32_t pend[3] = {0u, 0u, 0u};
-    int npend = 0;
+    // Copies are never waited for by the loaders: each thread's arrival on the tile's "full"
+    // barrier is attached to its copies (cp.async.mbarrier.arrive.noinc) and happens when
+    // they land.  The consumer (MMA issuer) crosses from the generic to the async proxy with
+    // a proxy fence after it has observed the barrier.
     bool ok = true;
-    auto retire_oldest = [&]() {
-      cp_async_wait_le(npend - 1);
-      fence_async_smem();
-      mbar_arrive(pend[0]);
-      pend[0] = pend[1]; pend[1] = pend[2];
-      --npend;
-    };
-    // kind 0/1: query tile 0/1 (both under one barrier), 2: key tile kt
-    auto gather_rows = [&](uint32_t dst, const __nv_bfloat16* src, int kind, int kt) {
+    auto gather_q = [&](uint32_t dst, int i) {
       for (int c = lt; c < 128 * CPR; c += kLoaderThreads) {
         const int row = c / CPR, cc = c % CPR;
-        int gr;
-        if (kind < 2) gr = s_qrow[kind * 128 + row];
-        else if (t.mode == 1) gr = s_kidx[kt * TK + row];
-        else { const int i = kt * TK + row; gr = i < t.nk ? t.k0 + i : -1; }
-        const uint32_t d = dst + tile_off(row, cc);
-        if (gr >= 0) cp_async16(d, src + (size_t)gr * D + cc * 8);
-        else st_shared_zero16(d);
+        const int gr = s_qrow[i * 128 + row];
+        const uint32_t d = dst + tile_off<128>(row, cc);
+        if (gr >= 0) cp_async16(d, qs + (size_t)gr * D + cc * 8);
+        else cp_async16_zero(d, qs);
       }
     };
-    auto committed = [&](uint32_t full_bar) {
-      cp_async_commit();
-      pend[npend++] = full_bar;
-      if (npend == 3) retire_oldest();
+    auto gather_kv = [&](uint32_t dst, const __nv_bfloat16* src, int kt) {
+      for (int c = lt; c < TK * CPR; c += kLoaderThreads) {
+        const int row = c / CPR, cc = c % CPR;
+        int gr;
+        if (t.mode == 1) gr = s_kidx[kt * TK + row];
+        else { const int i = kt * TK + row; gr = i < t.nk ? t.k0 + i : -1; }
+        const uint32_t d = dst + tile_off<TK>(row, cc);
+        if (gr >= 0) cp_async16(d, src + (size_t)gr * D + cc * 8);
+        else cp_async16_zero(d, src);
+      }
     };
-    gather_rows(ubase + C::kOffQ, qs, 0, 0);
-    gather_rows(ubase + C::kOffQ + C::kTile, qs, 1, 0);
-    committed(bar_q);
+    gather_q(ubase + C::kOffQ, 0);
+    gather_q(ubase + C::kOffQ + C::kQTile, 1);
+    cp_async_arrive_noinc(bar_q);
     for (int j = 0; j < ntiles && ok; ++j) {
       const int s = j % C::NS;
       const int use = j / C::NS;
       if (use > 0) {
-        while (npend) retire_oldest();
-        ok = mbar_wait(bar_kempty(s), (use - 1) & 1, s_abort, status);
+        ok = mbar_wait<100, 10>(bar_kempty(0, s), (use - 1) & 1, s_abort, status);
+        if (ok && qb.valid) ok = mbar_wait<100, 11>(bar_kempty(1, s), (use - 1) & 1, s_abort, status);
         if (!ok) break;
       }
-      gather_rows(ubase + C::kOffK + s * C::kTile, ks, 2, j);
-      committed(bar_kfull(s));
+      gather_kv(ubase + C::kOffK + s * C::kTile, ks, j);
+      cp_async_arrive_noinc(bar_kfull(s));
       if (use > 0) {
-        while (npend) retire_oldest();
-        ok = mbar_wait(bar_vempty(s), (use - 1) & 1, s_abort, status);
+        ok = mbar_wait<100, 12>(bar_vempty(0, s), (use - 1) & 1, s_abort, status);
+        if (ok && qb.valid) ok = mbar_wait<100, 13>(bar_vempty(1, s), (use - 1) & 1, s_abort, status);
         if (!ok) break;
       }
-      gather_rows(ubase + C::kOffV + s * C::kTile, vs, 2, j);
-      committed(bar_vfull(s));
+      gather_kv(ubase + C::kOffV + s * C::kTile, vs, j);
+      cp_async_arrive_noinc(bar_vfull(s));
     }
-    if (ok) { while (npend) retire_oldest(); }
-    cp_async_wait_le(0);
+    cp_async_commit();
+    cp_async_wait_le(0);      // nothing of this thread is in flight when the CTA tears down
   }
 
   // ---- teardown ------------------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
+  if (tid == 0) { HA_TACC(12, tcta); }
+#ifdef HA_TC_TIMING
+  if (tid == 0) { atomicAdd(&g_tc_timing[13], 1ull); atomicAdd(&g_tc_timing[14], (unsigned long long)ntiles); }
+#endif
   if (warp == 8) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
@@ -642,12 +808,20 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 
 }  // namespace
 
+#ifdef HA_TC_TIMING
+extern "C" int hyperattn_debug_tc_timing(unsigned long long* host16, int reset) {
+  if (cudaMemcpyFromSymbol(host16, g_tc_timing, sizeof(unsigned long long) * 16) != cudaSuccess) return -5;
+  if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)); }
+  return 0;
+}
+#endif
+
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st) {
   if (a.total_pairs == 0) return cudaSuccess;
   auto go = [&](auto kernel, int smem_bytes) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    kernel<<<a.total_pairs, 384, smem_bytes, st>>>(a, status);
+    kernel<<<a.total_pairs, 416, smem_bytes, st>>>(a, status);
     return cudaGetLastError();
   };
   if (a.g.d == 64) return go(attn_tc_kernel<64>, Cfg<64>::kTotal);
