@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     profile_read,
     profile_reset,
     release,
+    sortlsh_noalloc,
     version,
     workspace_bytes,
 )

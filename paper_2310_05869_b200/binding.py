@@ -18,7 +18,7 @@ STAGE_NAMES = ["convert", "hash", "sample", "sort_scan", "sort_scatter", "attent
 EXPORTS = ["hyperattn_forward", "hyperattn_forward_ex", "hyperattn_forward_host", "hyperattn_workspace_bytes",
            "hyperattn_get_projections", "hyperattn_last_device_status", "hyperattn_profile_enable",
            "hyperattn_profile_reset", "hyperattn_profile_read", "hyperattn_release",
-           "hyperattn_status_string", "hyperattn_version"]
+           "hyperattn_status_string", "hyperattn_version", "hyperattn_sortlsh_noalloc"]
 
 
 class HyperAttnError(RuntimeError):
@@ -63,6 +63,9 @@ def lib() -> C.CDLL:
         L.hyperattn_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
         L.hyperattn_profile_enable.argtypes = [C.c_int]
         L.hyperattn_profile_read.argtypes = [C.POINTER(_StageTimes)]
+        L.hyperattn_sortlsh_noalloc.restype = C.c_int
+        L.hyperattn_sortlsh_noalloc.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_uint64,
+                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.hyperattn_status_string.restype = C.c_char_p
         L.hyperattn_status_string.argtypes = [C.c_int]
         _lib = L
@@ -148,6 +151,28 @@ def forward_host(q, k, v, out, lse, block, samples, hash_bits, causal=False, n0=
     p.q, p.k, p.v, p.out, p.lse = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr()
     p.stream = stream if stream is not None else torch.cuda.current_stream().cuda_stream
     _check(lib().hyperattn_forward_host(C.byref(p)), "hyperattn_forward_host")
+
+
+NOALLOC_MAX_ROWS = 262144
+
+
+def sortlsh_noalloc(x, hash_bits, seed=0, stream=None):
+    """sortLSH of one CUDA bf16 matrix x[n, d] through the entry point that allocates nothing
+    inside the library (its scratch is a fixed array in the library image; n is capped at
+    NOALLOC_MAX_ROWS).  The three result tensors are allocated here, by the caller.
+    Returns (ids uint8[n], perm int32[n], rank int32[n])."""
+    if not x.is_cuda or x.dtype != torch.bfloat16 or x.dim() != 2:
+        raise HyperAttnError("x must be a 2-D CUDA bf16 tensor")
+    x = x.contiguous()
+    n, d = x.shape
+    ids = torch.empty(n, dtype=torch.uint8, device=x.device)
+    perm = torch.empty(n, dtype=torch.int32, device=x.device)
+    rank = torch.empty(n, dtype=torch.int32, device=x.device)
+    s = stream if stream is not None else torch.cuda.current_stream(x.device).cuda_stream
+    with torch.cuda.device(x.device):
+        _check(lib().hyperattn_sortlsh_noalloc(x.data_ptr(), n, d, hash_bits, seed, ids.data_ptr(), perm.data_ptr(),
+                                               rank.data_ptr(), s), "hyperattn_sortlsh_noalloc")
+    return ids, perm, rank
 
 
 def workspace_bytes(B, H, n, d, block, samples, hash_bits, causal=False, n0=0, dtype=BF16, out_dtype=BF16) -> int:

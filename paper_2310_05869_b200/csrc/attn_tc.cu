@@ -515,6 +515,11 @@ __global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__
       // The reference maximum only moves when the tile exceeds it by more than 2^8, and then
       // by a whole number of octaves, so that what is already accumulated (O and the row
       // sums) is rescaled exactly.
+#ifdef HA_EXP_NO_SOFTMAX
+      tc_fence_before();
+      mbar_arrive(bar_p(i, buf));
+      continue;
+#endif
       uint32_t ra[32], rb[32];
       const uint32_t sbase = lane_addr + 64 * (2 * i + buf);
       tmem_ld32_issue(sbase, ra);
