@@ -33,9 +33,10 @@ from paper_2310_05869_b200 import workloads as WL  # noqa: E402
 WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes per launch of the attention kernel from an ncu capture (see profiles/); None until
-# a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the attention kernel,
+# from the ncu captures summarised under profiles/ (taken on 4 / 8 heads and scaled to the
+# workload's 32 heads: the traffic is proportional to the number of segments).
+NCU_TRAFFIC_BYTES = {"c3_n131k_causal": 8 * 1.758e9, "c2_n32k_d128": 4 * 0.2478e9}
 
 
 def load_peaks():
