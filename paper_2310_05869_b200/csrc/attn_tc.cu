@@ -89,6 +89,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// the slow path of a wait, out of line; SITE tags the wait in the status word
+template <int SITE>
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  return mbar_wait<20, SITE>(bar, parity, abort_flag, status);
+}
+// one probe inline (the common case for the MMA issuers: what they wait for is usually there)
+template <int SITE>
+__device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow<SITE>(bar, parity, abort_flag, status);
+}
+
 // ---- tcgen05 ----------------------------------------------------------------------------
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   uint64_t d = 0;
@@ -108,6 +120,17 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
                ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// the same with descriptors given as (low, high) 32-bit words: only the low word ever changes
+__device__ __forceinline__ void mma_ss2(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}\n"
+               ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_ts2(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}\n"
+               ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -647,97 +670,92 @@ __global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__
   } else if (warp < 10) {
     // ================= MMA issue: one lane per query tile (warp 8: tile 0, warp 9: tile 1) ===========
     // Each issuer walks its own key tiles: scores run two tiles ahead of the PV products
-    // (S buffers alternate).  A tcgen05.mma costs the issuing thread and the tensor pipe
-    // about 55-65 cycles whatever its size, and every commit / barrier probe adds to that, so
-    // the two chains are issued by two threads.  Shared K / V stages are released per issuer.
+    // (S buffers alternate).  A tcgen05.mma occupies the issuing thread and the tensor pipe
+    // for about 55-65 cycles whatever its size, so the two chains are issued by two threads.
+    // The issuer shares its scheduler with two busy softmax warps and has no instruction-level
+    // parallelism of its own, so its loop is kept to a minimum of instructions: descriptors
+    // are two 32-bit words of which only the low one moves, waits are one probe in the common
+    // case, everything unusual lives in out-of-line slow paths.
     const int i = warp - 8;
     const QTile q = i ? qb : qa;
     const int total = q.n1 + q.n2;
     if (lane == 0 && total > 0) {
       constexpr uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)TK >> 3) << 17) | ((128u >> 4) << 24);
       constexpr uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
-      HA_T0(tq);
-      bool ok = mbar_wait<20, 6>(bar_q, 0, s_abort, status);
-      fence_async_smem();
-      if (i == 0) HA_TACC(7, tq);
-      HA_T0(tall);
-      int kseen = -1, vseen = -1;           // highest tile index whose K / V arrival has been observed
-      int krel = -1, vrel = -1;             // highest tile index whose K / V stage this issuer has released
-      // Shared-memory descriptors are built once; per MMA only the start-address field (in
-      // 16-byte units, low bits of the descriptor) moves, by compile-time offsets.
-      const uint64_t dq = make_desc(ubase + C::kOffQ + i * C::kQTile, 16, 1024);
-      const uint64_t dk0 = make_desc(ubase + C::kOffK, 16, 1024);
-      const uint64_t dv0 = make_desc(ubase + C::kOffV, TK * 128, 1024);
+      // descriptor: low word = start address >> 4 | (leading byte offset >> 4) << 16,
+      // high word = stride byte offset >> 4 | version 1 << 14 | 128-byte swizzle 2 << 29
+      constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t dq_lo = ((ubase + C::kOffQ + i * C::kQTile) >> 4) | (1u << 16);
+      const uint32_t dk_lo0 = ((ubase + C::kOffK) >> 4) | (1u << 16);
+      const uint32_t dv_lo0 = ((ubase + C::kOffV) >> 4) | (((uint32_t)(TK * 128) >> 4) << 16);
       const uint32_t ocol = tmem + C::kColO + D * i;
-      // K / V arrive in tile order; observing tile j means observing every barrier phase up to it
-      auto see_k = [&](int j) {
-        for (int jj = kseen + 1; jj <= j && ok; ++jj) ok = mbar_wait<20, 7>(bar_kfull(jj % C::NS), (jj / C::NS) & 1, s_abort, status);
-        if (ok && j > kseen) { kseen = j; fence_async_smem(); tc_fence_after(); }
+      const uint32_t scol = tmem + 64 * 2 * i;
+      HA_T0(tall);
+      bool ok = wait_fast<6>(bar_q, 0, s_abort, status);
+      fence_async_smem();
+      int knext = 0, vnext = 0;             // next tile whose K / V stage this issuer has to observe and release
+      // Tiles this query tile does not look at (the other tile's own block) are released when
+      // the walk passes them, but only after they have arrived: a release must never overtake
+      // the loader's wait for the previous release of the same stage (the barrier would wrap
+      // around unseen).  Releases go through tcgen05.commit, so they also stay behind this
+      // thread's earlier MMAs.
+      auto skip_k = [&](int j) {
+        for (; knext < j && ok; ++knext) {
+          ok = wait_fast<7>(bar_kfull(knext % C::NS), (knext / C::NS) & 1, s_abort, status);
+          if (ok) umma_commit(bar_kempty(i, knext % C::NS));
+        }
       };
-      auto see_v = [&](int j) {
-        for (int jj = vseen + 1; jj <= j && ok; ++jj) ok = mbar_wait<20, 9>(bar_vfull(jj % C::NS), (jj / C::NS) & 1, s_abort, status);
-        if (ok && j > vseen) { vseen = j; fence_async_smem(); tc_fence_after(); }
-      };
-      // Tiles this query tile does not look at are released when the walk passes them, but only
-      // after they have arrived: a release must never overtake the loader's wait for the
-      // previous release of the same stage (the barrier would wrap around unseen).  Releases go
-      // through tcgen05.commit, so they also stay behind this thread's earlier MMAs.
-      auto skip_k_to = [&](int j) {
-        for (int jj = krel + 1; jj < j && ok; ++jj) { see_k(jj); if (ok) umma_commit(bar_kempty(i, jj % C::NS)); }
-        if (j - 1 > krel) krel = j - 1;
-      };
-      auto skip_v_to = [&](int j) {
-        for (int jj = vrel + 1; jj < j && ok; ++jj) { see_v(jj); if (ok) umma_commit(bar_vempty(i, jj % C::NS)); }
-        if (j - 1 > vrel) vrel = j - 1;
-      };
-      // S of the a-th key tile into buffer a & 1
-      auto issue_s = [&](int a2) {
-        const int j = tile_of(q, a2);
-        const int s = j % C::NS;
-        skip_k_to(j);
-        HA_T0(tk);
-        see_k(j);
-        if (i == 0) HA_TACC(6, tk);
-        if (!ok) return;
-        const uint32_t dcol = tmem + 64 * (2 * i + (a2 & 1));
-        const uint64_t dk = dk0 + (uint64_t)((s * C::kTile) >> 4);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-          mma_ss(dcol, dq + (uint64_t)(((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4),
-                 dk + (uint64_t)(((ks >> 2) * (TK * 128) + (ks & 3) * 32) >> 4), idesc_s, ks > 0);
-        umma_commit(bar_s(i, a2 & 1));
-        umma_commit(bar_kempty(i, s));
-        krel = j;
-      };
-      // O += P V of the a-th key tile
-      auto issue_pv = [&](int a2) {
-        const int j = tile_of(q, a2);
-        const int s = j % C::NS;
-        skip_v_to(j);
-        HA_T0(tp);
-        ok = mbar_wait<20, 8>(bar_p(i, a2 & 1), (a2 >> 1) & 1, s_abort, status);
-        if (i == 0) HA_TACC(4, tp);
-        if (!ok) return;
-        HA_T0(tv);
-        see_v(j);
-        if (i == 0) HA_TACC(5, tv);
-        if (!ok) return;
-        tc_fence_after();
-        const uint32_t pcol = tmem + 64 * (2 * i + (a2 & 1));
-        const uint64_t dv = dv0 + (uint64_t)((s * C::kTile) >> 4);
-#pragma unroll
-        for (int kk = 0; kk < TK / 16; ++kk)
-          mma_ts(ocol, pcol + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_o, (a2 > 0 || kk > 0));
-        if (a2 == total - 2) umma_commit(bar_pv(i));
-        umma_commit(bar_vempty(i, s));
-        vrel = j;
-        if (a2 == total - 1) umma_commit(bar_o(i));
+      auto skip_v = [&](int j) {
+        for (; vnext < j && ok; ++vnext) {
+          ok = wait_fast<9>(bar_vfull(vnext % C::NS), (vnext / C::NS) & 1, s_abort, status);
+          if (ok) umma_commit(bar_vempty(i, vnext % C::NS));
+        }
       };
       for (int r = 0; r < total + 2 && ok; ++r) {
-        if (r >= 2) issue_pv(r - 2);
-        if (ok && r < total) issue_s(r);
+        if (r >= 2) {
+          // ---- O += P V of key tile r - 2 ----------------------------------------------------
+          const int a2 = r - 2;
+          const int j = tile_of(q, a2);
+          const int s = j % C::NS;
+          if (j != vnext) skip_v(j);
+          ok = ok && wait_fast<8>(bar_p(i, a2 & 1), (a2 >> 1) & 1, s_abort, status);
+          ok = ok && wait_fast<9>(bar_vfull(s), (j / C::NS) & 1, s_abort, status);
+          if (!ok) break;
+          fence_async_smem();
+          tc_fence_after();
+          const uint32_t pcol = scol + 64 * (a2 & 1);
+          const uint32_t dv_lo = dv_lo0 + (uint32_t)s * (C::kTile >> 4);
+          mma_ts2(ocol, pcol, dv_lo, desc_hi, idesc_o, a2 > 0);
+#pragma unroll
+          for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
+          umma_commit(bar_vempty(i, s));
+          vnext = j + 1;
+          if (a2 >= total - 2) {
+            if (a2 == total - 2) umma_commit(bar_pv(i));
+            else umma_commit(bar_o(i));
+          }
+        }
+        if (r < total) {
+          // ---- S = Q K^T of key tile r into buffer r & 1 -------------------------------------
+          const int j = tile_of(q, r);
+          const int s = j % C::NS;
+          if (j != knext) skip_k(j);
+          ok = ok && wait_fast<7>(bar_kfull(s), (j / C::NS) & 1, s_abort, status);
+          if (!ok) break;
+          fence_async_smem();
+          tc_fence_after();
+          const uint32_t dcol = scol + 64 * (r & 1);
+          const uint32_t dk_lo = dk_lo0 + (uint32_t)s * (C::kTile >> 4);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            mma_ss2(dcol, dq_lo + (((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4),
+                    dk_lo + (((ks >> 2) * (TK * 128) + (ks & 3) * 32) >> 4), desc_hi, idesc_s, ks > 0);
+          umma_commit(bar_s(i, r & 1));
+          umma_commit(bar_kempty(i, s));
+          knext = j + 1;
+        }
       }
-      if (ok) { skip_k_to(ntiles); skip_v_to(ntiles); }
+      if (ok) { skip_k(ntiles); skip_v(ntiles); }
       if (i == 0) HA_TACC(8, tall);
     }
     __syncwarp();
