@@ -54,13 +54,17 @@ struct HashArgs {
   int unit, chunks_per_unit, chunks_per_seg;
 };
 
-// One CTA = one chunk (<= kSortChunk rows of one side of one segment).
+// One CTA = one chunk (<= kSortChunk rows of one side of one segment).  Each warp walks over
+// groups of 16 rows; the loads of the next group are issued before the MMAs of the current
+// one, and the direction fragments live in shared memory (one 8-byte read per MMA) instead
+// of 48 registers, so that two to four CTAs fit an SM and ~128 KB of loads are in flight.
 template <int D>
-__global__ void __launch_bounds__(256) hash_bf16_kernel(const __grid_constant__ HashArgs a) {
+__global__ void __launch_bounds__(256, D == 64 ? 4 : 2) hash_bf16_kernel(const __grid_constant__ HashArgs a) {
   constexpr int KS = D / 16;             // MMA k-steps
   constexpr int CPL = D / 32;            // 16-byte chunks per lane per row
   __shared__ __align__(16) uint8_t s_ids[kSortChunk];
   __shared__ uint32_t s_hist[kBuckets];
+  __shared__ uint2 s_bw[3][KS][32];      // [split][k-step][lane] -> (b0, b1) of that lane
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, tig = lane & 3;
@@ -76,38 +80,48 @@ __global__ void __launch_bounds__(256) hash_bf16_kernel(const __grid_constant__ 
 
   // Direction fragments.  k-slot (step s, half h, element e) of lane (gid, tig) holds
   // coordinate 8*(tig + 4*(s>>1)) + 2*(2*(s&1) + h) + e; column gid is direction gid.
-  uint32_t bw[3][KS][2];
-#pragma unroll
-  for (int s = 0; s < KS; ++s)
+  for (int idx = tid; idx < KS * 32; idx += 256) {
+    const int s = idx >> 5, l = idx & 31;
+    const int lg = l >> 2, lt = l & 3;
+    uint32_t packed[3][2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      float w[2], t1[2], t2[2], t3[2];
+      float t1[2], t2[2], t3[2];
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const int coord = 8 * (tig + 4 * (s >> 1)) + 2 * (2 * (s & 1) + h) + e;
-        w[e] = (gid < a.r) ? a.w[coord * a.r + gid] : 0.f;
-        t1[e] = __bfloat162float(__float2bfloat16_rn(w[e]));
-        const float r1 = w[e] - t1[e];
+        const int coord = 8 * (lt + 4 * (s >> 1)) + 2 * (2 * (s & 1) + h) + e;
+        const float w = (lg < a.r) ? a.w[coord * a.r + lg] : 0.f;
+        t1[e] = __bfloat162float(__float2bfloat16_rn(w));
+        const float r1 = w - t1[e];
         t2[e] = __bfloat162float(__float2bfloat16_rn(r1));
         t3[e] = __bfloat162float(__float2bfloat16_rn(r1 - t2[e]));
       }
-      bw[0][s][h] = pack_bf16(t1[0], t1[1]);
-      bw[1][s][h] = pack_bf16(t2[0], t2[1]);
-      bw[2][s][h] = pack_bf16(t3[0], t3[1]);
+      packed[0][h] = pack_bf16(t1[0], t1[1]);
+      packed[1][h] = pack_bf16(t2[0], t2[1]);
+      packed[2][h] = pack_bf16(t3[0], t3[1]);
     }
+#pragma unroll
+    for (int sp = 0; sp < 3; ++sp) s_bw[sp][s][l] = make_uint2(packed[sp][0], packed[sp][1]);
+  }
   __syncthreads();
 
   const char* base = reinterpret_cast<const char*>(a.x[side]) + ((size_t)seg * a.n + row0) * (D * 2);
   unsigned nz = 0;
   const int groups = (rows + 15) >> 4;
-  for (int grp = warp; grp < groups; grp += 8) {
+  uint4 xa[CPL], xb[CPL];
+  auto load_group = [&](int grp, uint4 (&pa)[CPL], uint4 (&pb)[CPL]) {
     const int ra = grp * 16 + gid, rb = ra + 8;
-    uint4 xa[CPL], xb[CPL];
 #pragma unroll
     for (int h = 0; h < CPL; ++h) {
-      xa[h] = ra < rows ? ldg_stream(base + (size_t)ra * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
-      xb[h] = rb < rows ? ldg_stream(base + (size_t)rb * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
+      pa[h] = (grp < groups && ra < rows) ? ldg_stream(base + (size_t)ra * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
+      pb[h] = (grp < groups && rb < rows) ? ldg_stream(base + (size_t)rb * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
     }
+  };
+  load_group(warp, xa, xb);
+  for (int grp = warp; grp < groups; grp += 8) {
+    const int ra = grp * 16 + gid, rb = ra + 8;
+    uint4 na[CPL], nb[CPL];
+    load_group(grp + 8, na, nb);                      // in flight while this group is multiplied
     float hi[4] = {0.f, 0.f, 0.f, 0.f}, lo[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int s = 0; s < KS; ++s) {
@@ -117,9 +131,10 @@ __global__ void __launch_bounds__(256) hash_bf16_kernel(const __grid_constant__ 
       af[1] = (s & 1) ? vb.z : vb.x;   // row gid+8, half 0
       af[2] = (s & 1) ? va.w : va.y;   // row gid,   half 1
       af[3] = (s & 1) ? vb.w : vb.y;   // row gid+8, half 1
-      mma_bf16_16816(lo, af, bw[2][s][0], bw[2][s][1]);
-      mma_bf16_16816(lo, af, bw[1][s][0], bw[1][s][1]);
-      mma_bf16_16816(hi, af, bw[0][s][0], bw[0][s][1]);
+      const uint2 w3 = s_bw[2][s][lane], w2 = s_bw[1][s][lane], w1 = s_bw[0][s][lane];
+      mma_bf16_16816(lo, af, w3.x, w3.y);
+      mma_bf16_16816(lo, af, w2.x, w2.y);
+      mma_bf16_16816(hi, af, w1.x, w1.y);
     }
     // lane holds p[row gid][2tig], p[gid][2tig+1], p[gid+8][2tig], p[gid+8][2tig+1]
     float p[4];
@@ -135,6 +150,8 @@ __global__ void __launch_bounds__(256) hash_bf16_kernel(const __grid_constant__ 
     gb |= __shfl_xor_sync(0xffffffffu, gb, 1); gb |= __shfl_xor_sync(0xffffffffu, gb, 2);
     if (tig == 0 && ra < rows) { const uint32_t id = gray_rank8(ga); s_ids[ra] = (uint8_t)id; atomicAdd(&s_hist[id], 1u); }
     if (tig == 1 && rb < rows) { const uint32_t id = gray_rank8(gb); s_ids[rb] = (uint8_t)id; atomicAdd(&s_hist[id], 1u); }
+#pragma unroll
+    for (int h = 0; h < CPL; ++h) { xa[h] = na[h]; xb[h] = nb[h]; }
   }
   if (a.near_zero) {
 #pragma unroll
