@@ -18,18 +18,19 @@
 // of Q, K, V are gathered from their original places through the sortLSH permutations by
 // three loader warps with 16-byte cp.async copies; nothing permuted is ever written to HBM.
 //
-// Warp roles (416 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
+// Warp roles (384 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
 // warps 8 and 9 MMA issue for query tile 0 and 1 (warp 8 also allocates TMEM, all 512
-// columns: 2 x 2 S buffers of 64, O0, O1), warps 10-12 loaders.
+// columns: 2 x 2 S buffers of 64, O0, O1), warps 10-11 loaders.
 // Every mbarrier wait is bounded: on a timeout the CTA raises the device status word,
 // drains its copies, frees its TMEM and returns.
+#include <cstdlib>
 #include "attn_common.cuh"
 
 namespace hyperattn {
 namespace {
 
 constexpr int TK = 64;                  // keys per tile
-constexpr int kLoaderThreads = 96;
+constexpr int kLoaderThreads = 64;    // two loader warps: 12 warps per CTA leave 168 registers per thread
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
 constexpr float kRescaleThreshold = 8.f;
 #ifndef HA_TAKE_TURNS
@@ -266,6 +267,29 @@ __device__ __noinline__ void rescale_row(uint32_t o_addr, int ocols, float alpha
   tmem_wait_st();
 }
 
+// one 32-column chunk of a normalised output row to its place (fp32 partial / fp32 out / bf16 out)
+__device__ __forceinline__ void store_row_chunk(const AttnArgs& a, int partial, size_t orow, int D, int col0,
+                                                const uint32_t (&r)[32], float inv) {
+  if (partial || a.out_fp32) {
+    float* dst = (partial ? a.part_o : reinterpret_cast<float*>(a.out)) + orow * D + col0;
+#pragma unroll
+    for (int e = 0; e < 32; e += 4)
+      *reinterpret_cast<float4*>(dst + e) = make_float4(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv,
+                                                        __uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+  } else {
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.out) + orow * D + col0;
+#pragma unroll
+    for (int e = 0; e < 32; e += 8) {
+      uint4 v;
+      v.x = pack2(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+      v.y = pack2(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+      v.z = pack2(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+      v.w = pack2(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+      *reinterpret_cast<uint4*>(dst + e) = v;
+    }
+  }
+}
+
 template <int D>
 struct Cfg {
   static constexpr int NS = (D == 64) ? 8 : 4;        // K stages and V stages
@@ -274,11 +298,12 @@ struct Cfg {
   static constexpr int kOffQ = 0;                     // Q0, Q1
   static constexpr int kOffK = 2 * kQTile;
   static constexpr int kOffV = kOffK + NS * kTile;
-  static constexpr int kOffIdx = kOffV + NS * kTile;              // int [kMaxNodeKeys] key rows
-  static constexpr int kOffMask = kOffIdx + kMaxNodeKeys * 4;     // uint32 [2][kMaxNodeKeys/32] masked-column bits
-  static constexpr int kOffQrow = kOffMask + 2 * (kMaxNodeKeys / 32) * 4;   // int [2][128]
-  static constexpr int kOffBar = kOffQrow + 2 * 128 * 4;
-  static constexpr int kNumBar = 13 + 6 * NS;
+  // row tables, two sets (the loaders build the set of the next work item while this one runs)
+  static constexpr int kOffIdx = kOffV + NS * kTile;              // int [2][kMaxNodeKeys] key rows
+  static constexpr int kOffMask = kOffIdx + 2 * kMaxNodeKeys * 4; // uint32 [2][2][kMaxNodeKeys/32] masked-column bits
+  static constexpr int kOffQrow = kOffMask + 4 * (kMaxNodeKeys / 32) * 4;   // int [2][2][128]
+  static constexpr int kOffBar = kOffQrow + 4 * 128 * 4;
+  static constexpr int kNumBar = 21 + 6 * NS;
   static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
   static constexpr int kTotal = kOffMisc + 16;
   static constexpr int kTmemCols = 512;
@@ -395,34 +420,35 @@ __device__ __forceinline__ bool uses_tile(const QTile& q, int j) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, int* status) {
+__global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
-  int* s_kidx = reinterpret_cast<int*>(smem + C::kOffIdx);
-  uint32_t* s_mask = reinterpret_cast<uint32_t*>(smem + C::kOffMask);     // [2][kMaxNodeKeys/32]
-  int* s_qrow = reinterpret_cast<int*>(smem + C::kOffQrow);               // [2][128]
+  constexpr int MW = kMaxNodeKeys / 32;
+  int* s_kidx_all = reinterpret_cast<int*>(smem + C::kOffIdx);              // [2][kMaxNodeKeys]
+  uint32_t* s_mask_all = reinterpret_cast<uint32_t*>(smem + C::kOffMask);  // [2][2][MW]
+  int* s_qrow_all = reinterpret_cast<int*>(smem + C::kOffQrow);             // [2][2][128]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 4);
-  constexpr int MW = kMaxNodeKeys / 32;
 
   const uint32_t ubase = smem_u32(smem);
   const uint32_t bar0 = ubase + C::kOffBar;
-  const uint32_t bar_q = bar0;
-  auto bar_s = [&](int i, int b) { return bar0 + 8 + 8 * (2 * i + b); };      // S_i buffer b written
-  auto bar_p = [&](int i, int b) { return bar0 + 40 + 8 * (2 * i + b); };     // P_i buffer b written
-  auto bar_o = [&](int i) { return bar0 + 72 + 8 * i; };
-  auto bar_pv = [&](int i) { return bar0 + 88 + 8 * i; };                     // a PV_i finished
-  auto bar_kfull = [&](int s) { return bar0 + 104 + 8 * s; };
-  auto bar_vfull = [&](int s) { return bar0 + 104 + 8 * (C::NS + s); };
-  auto bar_kempty = [&](int i, int s) { return bar0 + 104 + 8 * ((2 + i) * C::NS + s); };     // released by issuer i
-  auto bar_vempty = [&](int i, int s) { return bar0 + 104 + 8 * ((4 + i) * C::NS + s); };
+  const uint32_t bar_q = bar0;                                                // Q tiles of the item landed
+  const uint32_t bar_qfree = bar0 + 8;                                        // both issuers are done with Q
+  auto bar_s = [&](int i, int b) { return bar0 + 16 + 8 * (2 * i + b); };     // S_i buffer b written
+  auto bar_p = [&](int i, int b) { return bar0 + 48 + 8 * (2 * i + b); };     // P_i buffer b written
+  auto bar_o = [&](int i) { return bar0 + 80 + 8 * i; };                      // O_i of the item complete
+  auto bar_pv = [&](int i) { return bar0 + 96 + 8 * i; };                     // PV_i before the last one finished
+  auto bar_ofree = [&](int i) { return bar0 + 112 + 8 * i; };                 // O_i has been read out
+  auto bar_tabfull = [&](int set) { return bar0 + 128 + 8 * set; };           // row tables of a set written
+  auto bar_tabfree = [&](int set) { return bar0 + 144 + 8 * set; };           // softmax warps are done with a set
+  const uint32_t bar_ld = bar0 + 160;                                         // the loader warps among themselves
+  auto bar_kfull = [&](int s) { return bar0 + 168 + 8 * s; };
+  auto bar_vfull = [&](int s) { return bar0 + 168 + 8 * (C::NS + s); };
+  auto bar_kempty = [&](int i, int s) { return bar0 + 168 + 8 * ((2 + i) * C::NS + s); };     // released by issuer i
+  auto bar_vempty = [&](int i, int s) { return bar0 + 168 + 8 * ((4 + i) * C::NS + s); };
 
   const Geometry& g = a.g;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  PairDesc t;
-  QTile qa, qb;
-  decode_pair(a, blockIdx.x, t, qa, qb);
-  HA_T0(tcta);
 
   // A CTA of a launch in which some wait already timed out returns at once (nothing allocated
   // yet), so a stuck launch drains quickly instead of timing out tile after tile.
@@ -431,12 +457,17 @@ __global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__
   if (*s_abort) return;
   __syncthreads();
 
-  // ---- setup: barriers, TMEM, row tables ----------------------------------------------------
+  // ---- setup: barriers, TMEM ---------------------------------------------------------------------
   if (tid == 0) {
     mbar_init(bar_q, kLoaderThreads);
+    mbar_init(bar_qfree, 2);
+    mbar_init(bar_ld, kLoaderThreads);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_o(i), 1);
       mbar_init(bar_pv(i), 1);
+      mbar_init(bar_ofree(i), 128);
+      mbar_init(bar_tabfull(i), kLoaderThreads);
+      mbar_init(bar_tabfree(i), 256);
       for (int b = 0; b < 2; ++b) { mbar_init(bar_s(i, b), 1); mbar_init(bar_p(i, b), 128); }
     }
     for (int s = 0; s < C::NS; ++s) {
@@ -446,226 +477,189 @@ __global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = tid; i < 2 * MW; i += 416) s_mask[i] = 0;
   if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(C::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  __syncthreads();
-
-  float wlog = 0.f;  // log2(N/m): weight of a sampled column
-  if (t.mode == 1) {
-    const int bcols = t.nbA * TK;
-    const int ncols = t.ntiles * TK;
-    wlog = g.m > 0 ? log2f((float)t.nk / (float)g.m) : 0.f;
-    const int32_t* smp = a.samples + ((size_t)t.seg * g.nodes + t.node) * g.m;
-    for (int i = tid; i < ncols; i += 416) {
-      int idx = -1;
-      bool m0 = true, m1 = true;                      // masked for query tile 0 / 1
-      if (i < (t.nbA + t.nbB) * TK) {
-        const int which = i >= bcols;                 // 0: block of tile 0, 1: block of tile 1
-        const int c = i - which * bcols;
-        if (c < g.b) {
-          idx = t.k0 + a.perm_k[t.slice + (size_t)(which ? qb.beta : qa.beta) * g.b + c];
-          m0 = m1 = false;
-        }
-      } else {
-        const int c = i - (t.nbA + t.nbB) * TK;
-        if (c < g.m) {
-          const int l = smp[c];
-          idx = t.k0 + l;
-          const int blk = a.rank_k[t.slice + l] / g.b;
-          m0 = blk == qa.beta;                        // the factor (1 - M^H) of Alg. 2 line 7
-          m1 = qb.valid && blk == qb.beta;
-        }
-      }
-      s_kidx[i] = idx;
-      if (m0) atomicOr(&s_mask[i >> 5], 1u << (i & 31));
-      if (m1) atomicOr(&s_mask[MW + (i >> 5)], 1u << (i & 31));
-    }
-    if (tid < 2 * kTileQ) {
-      const int r = tid & 127;
-      const QTile& q = tid < 128 ? qa : qb;
-      s_qrow[tid] = (q.valid && r < q.nq) ? t.qnode0 + a.perm_q[t.slice + q.spos0 + r] : -1;
-    }
-  } else {
-    if (tid < 2 * kTileQ) {
-      const int r = tid & 127;
-      const QTile& q = tid < 128 ? qa : qb;
-      s_qrow[tid] = (q.valid && r < q.nq) ? q.q0 + r : -1;
-    }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  const int ntiles = t.ntiles;
 
+  // The CTA is persistent: it walks over work items (pairs of query tiles) blockIdx.x,
+  // blockIdx.x + gridDim.x, ...  Every role runs the same item loop at its own pace; what
+  // they hand to each other across items is described at the barriers above.  All phase
+  // counters keep running across items.
   if (warp < 8) {
     // ================= softmax + epilogue of query tile i: thread = query row ==================
     const int i = warp >> 2;
     const int row = tid & 127;
-    const QTile q = i ? qb : qa;
-    const int total = q.n1 + q.n2;
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t colO = C::kColO + D * i;
-    float m_ref = -INFINITY;
-    float l0 = 0.f, l1 = 0.f, lr0 = 0.f, lr1 = 0.f;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each)
+    int ga = 0;                                       // key tiles this warpgroup has processed so far (all items)
+    int vi = 0;                                       // items in which this query tile existed
     bool ok = true;
-    for (int na = 0; na < total && ok; ++na) {
-      const int j = tile_of(q, na);
-      const int buf = na & 1;
-      HA_T0(tw);
-      ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (na >> 1) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
+    int it = 0;
+    for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+      PairDesc t; QTile qa, qb;
+      decode_pair(a, item, t, qa, qb);
+      const QTile q = i ? qb : qa;
+      const int total = q.n1 + q.n2;
+      const int set = it & 1;
+      const uint32_t* s_mask = s_mask_all + (set * 2 + i) * MW;
+      const int* s_qrow = s_qrow_all + (set * 2 + i) * 128;
+      // the tables of this item (also for a warpgroup without a tile: it may not run ahead)
+      ok = __all_sync(0xffffffffu, mbar_wait<20, 14>(bar_tabfull(set), (it >> 1) & 1, s_abort, status));
       if (!ok) break;
-      tc_fence_after();
-      if (row == 0) HA_TACC(0 + i, tw);
-      HA_T0(tc);
-      // mask kind of this (query tile, key tile): uniform over the warpgroup
-      bool table = false, dense_mask = false;
-      float ubias = 0.f;
-      int climit = 0;                               // dense: last visible column of this row
-      if (t.mode == 1) {
-        const uint32_t* mw = s_mask + i * MW + j * (TK / 32);
-        table = (mw[0] | mw[1]) != 0;
-        ubias = (j < t.nbA + t.nbB) ? 0.f : wlog;
-      } else {
-        climit = t.causal ? min(t.nk - 1, q.row0 + row) : t.nk - 1;
-        dense_mask = (j * TK + TK > t.nk) || (t.causal && j * TK + TK - 1 > q.row0);
-      }
-      // The 64 scores of this row are read from TMEM once; then (1) the row maximum, (2)
-      // exponentials, row sums and the bf16 P written over the first half of the S buffer.
-      // The reference maximum only moves when the tile exceeds it by more than 2^8, and then
-      // by a whole number of octaves, so that what is already accumulated (O and the row
-      // sums) is rescaled exactly.
-#ifdef HA_EXP_NO_SOFTMAX
-      tc_fence_before();
-      mbar_arrive(bar_p(i, buf));
-      continue;
-#endif
-      uint32_t ra[32], rb[32];
-      const uint32_t sbase = lane_addr + 64 * (2 * i + buf);
-      tmem_ld32_issue(sbase, ra);
-      tmem_ld32_issue(sbase + 32, rb);
-      const bool masked_tile = table || dense_mask;
-      uint32_t visa = 0xffffffffu, visb = 0xffffffffu;
-      if (table) { visa = ~s_mask[i * MW + j * 2]; visb = ~s_mask[i * MW + j * 2 + 1]; }
-      else if (dense_mask) {
-        const int rel = climit - j * TK;              // columns 0..rel of the tile are visible
-        visa = rel >= 31 ? 0xffffffffu : (rel < 0 ? 0u : ((2u << rel) - 1u));
-        visb = rel >= 63 ? 0xffffffffu : (rel < 32 ? 0u : ((2u << (rel - 32)) - 1u));
-      }
-      tmem_ld32_wait(ra);
-      tmem_ld32_wait(rb);
-      float m0 = -INFINITY, m1 = -INFINITY;
-      if (masked_tile) {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          if ((visa >> e) & 1u) m0 = fmaxf(m0, __uint_as_float(ra[e]));
-          if ((visb >> e) & 1u) m1 = fmaxf(m1, __uint_as_float(rb[e]));
+      const float wlog = (t.mode == 1 && g.m > 0) ? log2f((float)t.nk / (float)g.m) : 0.f;   // log2(N/m): weight of a sampled column
+      float m_ref = -INFINITY;
+      float l0 = 0.f, l1 = 0.f, lr0 = 0.f, lr1 = 0.f;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each)
+      for (int na = 0; na < total && ok; ++na) {
+        const int j = tile_of(q, na);
+        const int gw = ga + na;
+        const int buf = gw & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (gw >> 1) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
+        if (!ok) break;
+        tc_fence_after();
+        // mask kind of this (query tile, key tile): uniform over the warpgroup
+        bool table = false, dense_mask = false;
+        float ubias = 0.f;
+        int climit = 0;                               // dense: last visible column of this row
+        if (t.mode == 1) {
+          table = (s_mask[j * 2] | s_mask[j * 2 + 1]) != 0;
+          ubias = (j < t.nbA + t.nbB) ? 0.f : wlog;
+        } else {
+          climit = t.causal ? min(t.nk - 1, q.row0 + row) : t.nk - 1;
+          dense_mask = (j * TK + TK > t.nk) || (t.causal && j * TK + TK - 1 > q.row0);
         }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
-          m1 = max3(m1, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+        // The 64 scores of this row are read from TMEM once; then (1) the row maximum, (2)
+        // exponentials, row sums and the bf16 P written over the first half of the S buffer.
+        // The reference maximum only moves when the tile exceeds it by more than 2^8, and then
+        // by a whole number of octaves, so that what is already accumulated (O and the row
+        // sums) is rescaled exactly.
+        uint32_t ra[32], rb[32];
+        const uint32_t sbase = lane_addr + 64 * (2 * i + buf);
+        tmem_ld32_issue(sbase, ra);
+        tmem_ld32_issue(sbase + 32, rb);
+        const bool masked_tile = table || dense_mask;
+        uint32_t visa = 0xffffffffu, visb = 0xffffffffu;
+        if (table) { visa = ~s_mask[j * 2]; visb = ~s_mask[j * 2 + 1]; }
+        else if (dense_mask) {
+          const int rel = climit - j * TK;              // columns 0..rel of the tile are visible
+          visa = rel >= 31 ? 0xffffffffu : (rel < 0 ? 0u : ((2u << rel) - 1u));
+          visb = rel >= 63 ? 0xffffffffu : (rel < 32 ? 0u : ((2u << (rel - 32)) - 1u));
         }
-      }
-      const float xm = fmaf(fmaxf(m0, m1), a.scale_log2, ubias);   // scale_log2 > 0: the maximum commutes with it
-      const bool grow = xm > m_ref + kRescaleThreshold;
-      if (__any_sync(0xffffffffu, grow)) {          // rare; per warp so that TMEM accesses stay convergent
-        float alpha = 1.f;
-        if (grow) {
-          if (m_ref == -INFINITY) { m_ref = xm; alpha = 0.f; }
-          else { const float k = ceilf(xm - m_ref); m_ref += k; alpha = ex2(-k); }
-        }
-        l0 *= alpha; l1 *= alpha; lr0 *= alpha; lr1 *= alpha;
-        // O may only be touched between two PV products: the one of the previous tile must
-        // have finished (the one of this tile cannot start before this tile's P is published)
-        if (na > 0) {
-          // S of tile na+1 is committed after the PV of tile na-1, so its arrival implies that PV;
-          // the last tile has no successor and uses the PV barrier (committed after PV total-2)
-          if (na + 1 < total) ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_s(i, (na + 1) & 1), ((na + 1) >> 1) & 1, s_abort, status));
-          else ok = __all_sync(0xffffffffu, mbar_wait<20, 4>(bar_pv(i), 0, s_abort, status));
-          if (!ok) break;
-          tc_fence_after();
-          rescale_row(lane_addr + colO, D, alpha);
-        }
-      }
-      const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
-      auto chunk_exp = [&](const uint32_t (&r)[32], uint32_t vis, int c) {
-        uint32_t p[16];
+        tmem_ld32_wait(ra);
+        tmem_ld32_wait(rb);
+        float m0 = -INFINITY, m1 = -INFINITY;
         if (masked_tile) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
-            float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
-            if (!((vis >> e) & 1u)) p0 = 0.f;
-            if (!((vis >> (e + 1)) & 1u)) p1 = 0.f;
-            l0 += p0; l1 += p1;
-            const uint32_t w = pack2(p0, p1);
-            lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
-            p[e >> 1] = w;
+          for (int e = 0; e < 32; ++e) {
+            if ((visa >> e) & 1u) m0 = fmaxf(m0, __uint_as_float(ra[e]));
+            if ((visb >> e) & 1u) m1 = fmaxf(m1, __uint_as_float(rb[e]));
           }
         } else {
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
-            const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
-            l0 += p0; l1 += p1;
-            const uint32_t w = pack2(p0, p1);
-            lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
-            p[e >> 1] = w;
+            m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            m1 = max3(m1, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
           }
         }
-        tmem_st16(sbase + c * 16, p);
-      };
-      chunk_exp(ra, visa, 0);
-      chunk_exp(rb, visb, 1);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_p(i, buf));
-      if (row == 0) HA_TACC(2 + i, tc);
-    }
-    // epilogue
-    if (q.valid) {
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait<20, 5>(bar_o(i), 0, s_abort, status));
-      if (ok) {
+        const float xm = fmaf(fmaxf(m0, m1), a.scale_log2, ubias);   // scale_log2 > 0: the maximum commutes with it
+        const bool grow = xm > m_ref + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, grow)) {          // rare; per warp so that TMEM accesses stay convergent
+          float alpha = 1.f;
+          if (grow) {
+            if (m_ref == -INFINITY) { m_ref = xm; alpha = 0.f; }
+            else { const float k = ceilf(xm - m_ref); m_ref += k; alpha = ex2(-k); }
+          }
+          l0 *= alpha; l1 *= alpha; lr0 *= alpha; lr1 *= alpha;
+          // O may only be touched between two PV products: the one of the previous tile must
+          // have finished (the one of this tile cannot start before this tile's P is published)
+          if (na > 0) {
+            // S of tile na+1 is committed after the PV of tile na-1, so its arrival implies that PV;
+            // the last tile has no successor and uses the PV barrier (committed after PV total-2)
+            if (na + 1 < total) ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_s(i, (gw + 1) & 1), ((gw + 1) >> 1) & 1, s_abort, status));
+            else ok = __all_sync(0xffffffffu, mbar_wait<20, 4>(bar_pv(i), vi & 1, s_abort, status));
+            if (!ok) break;
+            tc_fence_after();
+            rescale_row(lane_addr + colO, D, alpha);
+          }
+        }
+        const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
+        auto chunk_exp = [&](const uint32_t (&r)[32], uint32_t vis, int c) {
+          uint32_t p[16];
+          if (masked_tile) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
+              float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
+              if (!((vis >> e) & 1u)) p0 = 0.f;
+              if (!((vis >> (e + 1)) & 1u)) p1 = 0.f;
+              l0 += p0; l1 += p1;
+              const uint32_t w = pack2(p0, p1);
+              lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
+              p[e >> 1] = w;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
+              const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
+              l0 += p0; l1 += p1;
+              const uint32_t w = pack2(p0, p1);
+              lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
+              p[e >> 1] = w;
+            }
+          }
+          tmem_st16(sbase + c * 16, p);
+        };
+        chunk_exp(ra, visa, 0);
+        chunk_exp(rb, visb, 1);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p(i, buf));
+      }
+      if (!ok) break;
+      // epilogue: normalise, log-sum-exp, rows back to their original places
+      if (q.valid) {
+        ok = __all_sync(0xffffffffu, mbar_wait<20, 5>(bar_o(i), vi & 1, s_abort, status));
+        if (!ok) break;
         tc_fence_after();
-        const int qr = s_qrow[i * 128 + row];
+        const int qr = s_qrow[row];
         const float inv = 1.f / (lr0 + lr1);
         const float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
         const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
-#pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(lane_addr + colO + c * 32, r);
+        if (D == 64) {
+          // read everything, free O for the next item at once, then write
+          uint32_t r0[32], r1[32];
+          tmem_ld32_issue(lane_addr + colO, r0);
+          tmem_ld32_issue(lane_addr + colO + 32, r1);
+          tmem_ld32_wait(r0);
+          tmem_ld32_wait(r1);
+          tc_fence_before();
+          mbar_arrive(bar_ofree(i));
           if (qr >= 0) {
-            if (t.partial || a.out_fp32) {
-              float* dst = (t.partial ? a.part_o : reinterpret_cast<float*>(a.out)) + orow * D + c * 32;
-#pragma unroll
-              for (int e = 0; e < 32; e += 4)
-                *reinterpret_cast<float4*>(dst + e) = make_float4(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv,
-                                                                  __uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-            } else {
-              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.out) + orow * D + c * 32;
-#pragma unroll
-              for (int e = 0; e < 32; e += 8) {
-                uint4 v;
-                v.x = pack2(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-                v.y = pack2(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-                v.z = pack2(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-                v.w = pack2(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-                *reinterpret_cast<uint4*>(dst + e) = v;
-              }
-            }
+            store_row_chunk(a, t.partial, orow, D, 0, r0, inv);
+            store_row_chunk(a, t.partial, orow, D, 32, r1, inv);
+          }
+        } else {
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(lane_addr + colO + c * 32, r);
+            if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar_ofree(i)); }
+            if (qr >= 0) store_row_chunk(a, t.partial, orow, D, c * 32, r, inv);
           }
         }
         if (qr >= 0) {
           if (t.partial) a.part_lse[orow] = lse;
           else a.lse[orow] = lse;
         }
+        ++vi;
       }
+      mbar_arrive(bar_tabfree(set));
+      ga += total;
     }
   } else if (warp < 10) {
     // ================= MMA issue: one lane per query tile (warp 8: tile 0, warp 9: tile 1) ===========
@@ -677,9 +671,7 @@ __global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__
     // are two 32-bit words of which only the low one moves, waits are one probe in the common
     // case, everything unusual lives in out-of-line slow paths.
     const int i = warp - 8;
-    const QTile q = i ? qb : qa;
-    const int total = q.n1 + q.n2;
-    if (lane == 0 && total > 0) {
+    if (lane == 0) {
       constexpr uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)TK >> 3) << 17) | ((128u >> 4) << 24);
       constexpr uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
       // descriptor: low word = start address >> 4 | (leading byte offset >> 4) << 16,
@@ -690,127 +682,237 @@ __global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__
       const uint32_t dv_lo0 = ((ubase + C::kOffV) >> 4) | (((uint32_t)(TK * 128) >> 4) << 16);
       const uint32_t ocol = tmem + C::kColO + D * i;
       const uint32_t scol = tmem + 64 * 2 * i;
-      HA_T0(tall);
-      bool ok = wait_fast<6>(bar_q, 0, s_abort, status);
-      fence_async_smem();
-      int knext = 0, vnext = 0;             // next tile whose K / V stage this issuer has to observe and release
-      // Tiles this query tile does not look at (the other tile's own block) are released when
-      // the walk passes them, but only after they have arrived: a release must never overtake
-      // the loader's wait for the previous release of the same stage (the barrier would wrap
-      // around unseen).  Releases go through tcgen05.commit, so they also stay behind this
-      // thread's earlier MMAs.
-      auto skip_k = [&](int j) {
-        for (; knext < j && ok; ++knext) {
+      bool ok = true;
+      int gbase = 0;                        // global index (all items) of the item's first key tile
+      int knext = 0, vnext = 0;             // next global tile whose K / V stage this issuer has to observe and release
+      int ga = 0;                           // key tiles issued so far for this query tile (all items)
+      int vi = 0;                           // items in which this query tile existed
+      // Tiles this query tile does not look at (the other tile's own block, or everything when
+      // the tile does not exist) are released when the walk passes them, but only after they
+      // have arrived: a release must never overtake the loader's wait for the previous
+      // release of the same stage (the barrier would wrap around unseen).  Releases go through
+      // tcgen05.commit, so they also stay behind this thread's earlier MMAs.
+      auto skip_k = [&](int gj) {
+        for (; knext < gj && ok; ++knext) {
           ok = wait_fast<7>(bar_kfull(knext % C::NS), (knext / C::NS) & 1, s_abort, status);
           if (ok) umma_commit(bar_kempty(i, knext % C::NS));
         }
       };
-      auto skip_v = [&](int j) {
-        for (; vnext < j && ok; ++vnext) {
+      auto skip_v = [&](int gj) {
+        for (; vnext < gj && ok; ++vnext) {
           ok = wait_fast<9>(bar_vfull(vnext % C::NS), (vnext / C::NS) & 1, s_abort, status);
           if (ok) umma_commit(bar_vempty(i, vnext % C::NS));
         }
       };
-      for (int r = 0; r < total + 2 && ok; ++r) {
-        if (r >= 2) {
-          // ---- O += P V of key tile r - 2 ----------------------------------------------------
-          const int a2 = r - 2;
-          const int j = tile_of(q, a2);
-          const int s = j % C::NS;
-          if (j != vnext) skip_v(j);
-          ok = ok && wait_fast<8>(bar_p(i, a2 & 1), (a2 >> 1) & 1, s_abort, status);
-          ok = ok && wait_fast<9>(bar_vfull(s), (j / C::NS) & 1, s_abort, status);
-          if (!ok) break;
-          fence_async_smem();
-          tc_fence_after();
-          const uint32_t pcol = scol + 64 * (a2 & 1);
-          const uint32_t dv_lo = dv_lo0 + (uint32_t)s * (C::kTile >> 4);
-          mma_ts2(ocol, pcol, dv_lo, desc_hi, idesc_o, a2 > 0);
+      int it = 0;
+      for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+        PairDesc t; QTile qa, qb;
+        decode_pair(a, item, t, qa, qb);
+        const QTile q = i ? qb : qa;
+        const int total = q.n1 + q.n2;
+        // Q of this item (an issuer without a tile waits too: it may not run ahead of the others)
+        ok = wait_fast<6>(bar_q, it & 1, s_abort, status);
+        if (!ok) break;
+        fence_async_smem();
+        if (total == 0) mbar_arrive(bar_qfree);
+        for (int r = 0; r < total + 2 && ok; ++r) {
+          if (r >= 2) {
+            // ---- O += P V of key tile r - 2 ----------------------------------------------------
+            const int a2 = r - 2;
+            const int gj = gbase + tile_of(q, a2);
+            const int s = gj % C::NS;
+            const int gw = ga + a2;
+            if (gj != vnext) skip_v(gj);
+            ok = ok && wait_fast<8>(bar_p(i, gw & 1), (gw >> 1) & 1, s_abort, status);
+            ok = ok && wait_fast<9>(bar_vfull(s), (gj / C::NS) & 1, s_abort, status);
+            // the first product of an item overwrites O: the previous item's O must have been read
+            if (a2 == 0 && vi > 0) ok = ok && wait_fast<15>(bar_ofree(i), (vi - 1) & 1, s_abort, status);
+            if (!ok) break;
+            fence_async_smem();
+            tc_fence_after();
+            const uint32_t pcol = scol + 64 * (gw & 1);
+            const uint32_t dv_lo = dv_lo0 + (uint32_t)s * (C::kTile >> 4);
+            mma_ts2(ocol, pcol, dv_lo, desc_hi, idesc_o, a2 > 0);
 #pragma unroll
-          for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
-          umma_commit(bar_vempty(i, s));
-          vnext = j + 1;
-          if (a2 >= total - 2) {
-            if (a2 == total - 2) umma_commit(bar_pv(i));
-            else umma_commit(bar_o(i));
+            for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
+            umma_commit(bar_vempty(i, s));
+            vnext = gj + 1;
+            // one PV-barrier phase per item (waited for only by the rare rescale of the last tile)
+            if (a2 == (total >= 2 ? total - 2 : 0)) umma_commit(bar_pv(i));
+            if (a2 == total - 1) umma_commit(bar_o(i));
+          }
+          if (r < total) {
+            // ---- S = Q K^T of key tile r into buffer (ga + r) & 1 -----------------------------------
+            const int gj = gbase + tile_of(q, r);
+            const int s = gj % C::NS;
+            const int gw = ga + r;
+            if (gj != knext) skip_k(gj);
+            ok = ok && wait_fast<7>(bar_kfull(s), (gj / C::NS) & 1, s_abort, status);
+            if (!ok) break;
+            fence_async_smem();
+            tc_fence_after();
+            const uint32_t dcol = scol + 64 * (gw & 1);
+            const uint32_t dk_lo = dk_lo0 + (uint32_t)s * (C::kTile >> 4);
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+              mma_ss2(dcol, dq_lo + (((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4),
+                      dk_lo + (((ks >> 2) * (TK * 128) + (ks & 3) * 32) >> 4), desc_hi, idesc_s, ks > 0);
+            umma_commit(bar_s(i, gw & 1));
+            umma_commit(bar_kempty(i, s));
+            knext = gj + 1;
+            if (r == total - 1) umma_commit(bar_qfree);     // nothing of this item reads Q any more
           }
         }
-        if (r < total) {
-          // ---- S = Q K^T of key tile r into buffer r & 1 -------------------------------------
-          const int j = tile_of(q, r);
-          const int s = j % C::NS;
-          if (j != knext) skip_k(j);
-          ok = ok && wait_fast<7>(bar_kfull(s), (j / C::NS) & 1, s_abort, status);
-          if (!ok) break;
-          fence_async_smem();
-          tc_fence_after();
-          const uint32_t dcol = scol + 64 * (r & 1);
-          const uint32_t dk_lo = dk_lo0 + (uint32_t)s * (C::kTile >> 4);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks)
-            mma_ss2(dcol, dq_lo + (((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4),
-                    dk_lo + (((ks >> 2) * (TK * 128) + (ks & 3) * 32) >> 4), desc_hi, idesc_s, ks > 0);
-          umma_commit(bar_s(i, r & 1));
-          umma_commit(bar_kempty(i, s));
-          knext = j + 1;
-        }
+        if (!ok) break;
+        skip_k(gbase + t.ntiles);
+        skip_v(gbase + t.ntiles);
+        gbase += t.ntiles;
+        ga += total;
+        vi += q.valid;
       }
-      if (ok) { skip_k(ntiles); skip_v(ntiles); }
-      if (i == 0) HA_TACC(8, tall);
     }
     __syncwarp();
   } else {
-    // ================= loaders: gather rows into swizzled tiles ======================================
+    // ================= loaders: row tables of the next item, then gathers into swizzled tiles ========
     const int lt = tid - 320;
-    const __nv_bfloat16* qs = a.q + (size_t)t.seg * g.n * D;
-    const __nv_bfloat16* ks = a.k + (size_t)t.seg * g.n * D;
-    const __nv_bfloat16* vs = a.v + (size_t)t.seg * g.n * D;
     constexpr int CPR = D / 8;
     // Copies are never waited for by the loaders: each thread's arrival on the tile's "full"
     // barrier is attached to its copies (cp.async.mbarrier.arrive.noinc) and happens when
     // they land.  The consumer (MMA issuer) crosses from the generic to the async proxy with
     // a proxy fence after it has observed the barrier.
     bool ok = true;
-    auto gather_q = [&](uint32_t dst, int i) {
-      for (int c = lt; c < 128 * CPR; c += kLoaderThreads) {
-        const int row = c / CPR, cc = c % CPR;
-        const int gr = s_qrow[i * 128 + row];
-        const uint32_t d = dst + tile_off<128>(row, cc);
-        if (gr >= 0) cp_async16(d, qs + (size_t)gr * D + cc * 8);
-        else cp_async16_zero(d, qs);
-      }
+    int gbase = 0;
+    int it = 0;
+    int nsync = 0;                                    // loader-only synchronisations so far (bounded, like every wait here)
+    auto loader_sync = [&]() {
+      mbar_arrive(bar_ld);
+      ok = mbar_wait<20, 18>(bar_ld, nsync & 1, s_abort, status);
+      ++nsync;
     };
-    auto gather_kv = [&](uint32_t dst, const __nv_bfloat16* src, int kt) {
-      for (int c = lt; c < TK * CPR; c += kLoaderThreads) {
-        const int row = c / CPR, cc = c % CPR;
-        int gr;
-        if (t.mode == 1) gr = s_kidx[kt * TK + row];
-        else { const int i = kt * TK + row; gr = i < t.nk ? t.k0 + i : -1; }
-        const uint32_t d = dst + tile_off<TK>(row, cc);
-        if (gr >= 0) cp_async16(d, src + (size_t)gr * D + cc * 8);
-        else cp_async16_zero(d, src);
-      }
-    };
-    gather_q(ubase + C::kOffQ, 0);
-    gather_q(ubase + C::kOffQ + C::kQTile, 1);
-    cp_async_arrive_noinc(bar_q);
-    for (int j = 0; j < ntiles && ok; ++j) {
-      const int s = j % C::NS;
-      const int use = j / C::NS;
-      if (use > 0) {
-        ok = mbar_wait<100, 10>(bar_kempty(0, s), (use - 1) & 1, s_abort, status);
-        if (ok && qb.valid) ok = mbar_wait<100, 11>(bar_kempty(1, s), (use - 1) & 1, s_abort, status);
+    for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+      PairDesc t; QTile qa, qb;
+      decode_pair(a, item, t, qa, qb);
+      const int set = it & 1;
+      int* s_kidx = s_kidx_all + set * kMaxNodeKeys;
+      uint32_t* s_mask = s_mask_all + set * 2 * MW;
+      int* s_qrow = s_qrow_all + set * 2 * 128;
+      // ---- row tables (the softmax warps must be done with this set: item it - 2) --------------
+      if (it >= 2) {
+        ok = mbar_wait<100, 16>(bar_tabfree(set), ((it >> 1) - 1) & 1, s_abort, status);
         if (!ok) break;
       }
-      gather_kv(ubase + C::kOffK + s * C::kTile, ks, j);
-      cp_async_arrive_noinc(bar_kfull(s));
-      if (use > 0) {
-        ok = mbar_wait<100, 12>(bar_vempty(0, s), (use - 1) & 1, s_abort, status);
-        if (ok && qb.valid) ok = mbar_wait<100, 13>(bar_vempty(1, s), (use - 1) & 1, s_abort, status);
+      for (int c = lt; c < 2 * MW; c += kLoaderThreads) s_mask[c] = 0;
+      loader_sync();
+      if (!ok) break;
+      if (t.mode == 1) {
+        const int bcols = t.nbA * TK;
+        const int ncols = t.ntiles * TK;
+        const int32_t* smp = a.samples + ((size_t)t.seg * g.nodes + t.node) * g.m;
+        for (int c0 = lt; c0 < ncols; c0 += kLoaderThreads) {
+          int idx = -1;
+          bool m0 = true, m1 = true;                      // masked for query tile 0 / 1
+          if (c0 < (t.nbA + t.nbB) * TK) {
+            const int which = c0 >= bcols;                // 0: block of tile 0, 1: block of tile 1
+            const int c = c0 - which * bcols;
+            if (c < g.b) {
+              idx = t.k0 + a.perm_k[t.slice + (size_t)(which ? qb.beta : qa.beta) * g.b + c];
+              m0 = m1 = false;
+            }
+          } else {
+            const int c = c0 - (t.nbA + t.nbB) * TK;
+            if (c < g.m) {
+              const int l = smp[c];
+              idx = t.k0 + l;
+              const int blk = a.rank_k[t.slice + l] / g.b;
+              m0 = blk == qa.beta;                        // the factor (1 - M^H) of Alg. 2 line 7
+              m1 = qb.valid && blk == qb.beta;
+            }
+          }
+          s_kidx[c0] = idx;
+          if (m0) atomicOr(&s_mask[c0 >> 5], 1u << (c0 & 31));
+          if (m1) atomicOr(&s_mask[MW + (c0 >> 5)], 1u << (c0 & 31));
+        }
+      }
+      for (int c = lt; c < 2 * kTileQ; c += kLoaderThreads) {
+        const int r = c & 127;
+        const QTile& q = c < 128 ? qa : qb;
+        int v = -1;
+        if (q.valid && r < q.nq) v = t.mode == 1 ? t.qnode0 + a.perm_q[t.slice + q.spos0 + r] : q.q0 + r;
+        s_qrow[c] = v;
+      }
+      loader_sync();                                      // the loaders themselves read the tables below
+      if (!ok) break;
+      mbar_arrive(bar_tabfull(set));
+      // ---- Q (the issuers must be done with the previous item's Q) ----------------------------
+      if (it >= 1) {
+        ok = mbar_wait<100, 17>(bar_qfree, (it - 1) & 1, s_abort, status);
         if (!ok) break;
       }
-      gather_kv(ubase + C::kOffV + s * C::kTile, vs, j);
-      cp_async_arrive_noinc(bar_vfull(s));
+      const __nv_bfloat16* qs = a.q + (size_t)t.seg * g.n * D;
+      const __nv_bfloat16* ks = a.k + (size_t)t.seg * g.n * D;
+      const __nv_bfloat16* vs = a.v + (size_t)t.seg * g.n * D;
+      // (indices first, copies second: the loaders have few warps, so every gather keeps many
+      // independent chunks in flight instead of one dependent index -> address -> copy chain)
+      {
+        constexpr int PER = 8;                                   // chunks per thread per step
+        static_assert((2 * 128 * CPR) % (kLoaderThreads * PER) == 0, "query tile gather must divide evenly");
+#pragma unroll 1
+        for (int c0 = lt; c0 < 2 * 128 * CPR; c0 += kLoaderThreads * PER) {
+          int gr[PER];
+#pragma unroll
+          for (int k = 0; k < PER; ++k) gr[k] = s_qrow[(c0 + k * kLoaderThreads) / CPR];
+#pragma unroll
+          for (int k = 0; k < PER; ++k) {
+            const int c = c0 + k * kLoaderThreads;
+            const int i = c / (128 * CPR);
+            const int row = (c / CPR) & 127, cc = c % CPR;
+            const uint32_t d = ubase + C::kOffQ + i * C::kQTile + tile_off<128>(row, cc);
+            if (gr[k] >= 0) cp_async16(d, qs + (size_t)gr[k] * D + cc * 8);
+            else cp_async16_zero(d, qs);
+          }
+        }
+      }
+      cp_async_arrive_noinc(bar_q);
+      // ---- K / V tiles through the stage ring ----------------------------------------------------
+      auto gather_kv = [&](uint32_t dst, const __nv_bfloat16* src, int kt) {
+        constexpr int PER = TK * CPR / kLoaderThreads;           // 8 (d = 64) or 16 (d = 128) chunks per thread
+        static_assert(PER * kLoaderThreads == TK * CPR, "key tile gather must divide evenly");
+        int gr[PER];
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+          const int row = (lt + k * kLoaderThreads) / CPR;
+          if (t.mode == 1) gr[k] = s_kidx[kt * TK + row];
+          else { const int r = kt * TK + row; gr[k] = r < t.nk ? t.k0 + r : -1; }
+        }
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+          const int c = lt + k * kLoaderThreads;
+          const int row = c / CPR, cc = c % CPR;
+          const uint32_t d = dst + tile_off<TK>(row, cc);
+          if (gr[k] >= 0) cp_async16(d, src + (size_t)gr[k] * D + cc * 8);
+          else cp_async16_zero(d, src);
+        }
+      };
+      for (int j = 0; j < t.ntiles && ok; ++j) {
+        const int gj = gbase + j;
+        const int s = gj % C::NS;
+        const int use = gj / C::NS;
+        if (use > 0) {
+          ok = mbar_wait<100, 10>(bar_kempty(0, s), (use - 1) & 1, s_abort, status);
+          ok = ok && mbar_wait<100, 11>(bar_kempty(1, s), (use - 1) & 1, s_abort, status);
+          if (!ok) break;
+        }
+        gather_kv(ubase + C::kOffK + s * C::kTile, ks, j);
+        cp_async_arrive_noinc(bar_kfull(s));
+        if (use > 0) {
+          ok = mbar_wait<100, 12>(bar_vempty(0, s), (use - 1) & 1, s_abort, status);
+          ok = ok && mbar_wait<100, 13>(bar_vempty(1, s), (use - 1) & 1, s_abort, status);
+          if (!ok) break;
+        }
+        gather_kv(ubase + C::kOffV + s * C::kTile, vs, j);
+        cp_async_arrive_noinc(bar_vfull(s));
+      }
+      gbase += t.ntiles;
     }
     cp_async_commit();
     cp_async_wait_le(0);      // nothing of this thread is in flight when the CTA tears down
@@ -819,10 +921,6 @@ __global__ void __launch_bounds__(416, 1) attn_tc_kernel(const __grid_constant__
   // ---- teardown ------------------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
-  if (tid == 0) { HA_TACC(12, tcta); }
-#ifdef HA_TC_TIMING
-  if (tid == 0) { atomicAdd(&g_tc_timing[13], 1ull); atomicAdd(&g_tc_timing[14], (unsigned long long)ntiles); }
-#endif
   if (warp == 8) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
@@ -844,7 +942,10 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
   auto go = [&](auto kernel, int smem_bytes) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    kernel<<<a.total_pairs, 416, smem_bytes, st>>>(a, status);
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
+    int grid = a.total_pairs < sms ? a.total_pairs : sms;     // persistent: one CTA per SM walks the item list
+    kernel<<<grid, 384, smem_bytes, st>>>(a, status);
     return cudaGetLastError();
   };
   if (a.g.d == 64) return go(attn_tc_kernel<64>, Cfg<64>::kTotal);
