@@ -39,7 +39,7 @@ constexpr float kRescaleThreshold = 8.f;
 
 // Optional per-role cycle counters (compile with -DHA_TC_TIMING; never in the shipped build).
 #ifdef HA_TC_TIMING
-__device__ unsigned long long g_tc_timing[16];
+__device__ unsigned long long g_tc_timing[24];
 #define HA_T0(var) const long long var = clock64()
 #define HA_TACC(slot, var) atomicAdd(&g_tc_timing[slot], (unsigned long long)(clock64() - var))
 #else
@@ -449,6 +449,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 
   const Geometry& g = a.g;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  HA_T0(t_cta);
 
   // A CTA of a launch in which some wait already timed out returns at once (nothing allocated
   // yet), so a stuck launch drains quickly instead of timing out tile after tile.
@@ -509,8 +510,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       const uint32_t* s_mask = s_mask_all + (set * 2 + i) * MW;
       const int* s_qrow = s_qrow_all + (set * 2 + i) * 128;
       // the tables of this item (also for a warpgroup without a tile: it may not run ahead)
+      HA_T0(tt);
       ok = __all_sync(0xffffffffu, mbar_wait<20, 14>(bar_tabfull(set), (it >> 1) & 1, s_abort, status));
       if (!ok) break;
+      if (row == 0 && i == 0) HA_TACC(9, tt);
       const float wlog = (t.mode == 1 && g.m > 0) ? log2f((float)t.nk / (float)g.m) : 0.f;   // log2(N/m): weight of a sampled column
       float m_ref = -INFINITY;
       float l0 = 0.f, l1 = 0.f, lr0 = 0.f, lr1 = 0.f;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each)
@@ -518,8 +521,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         const int j = tile_of(q, na);
         const int gw = ga + na;
         const int buf = gw & 1;
+        HA_T0(tw);
         ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (gw >> 1) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
         if (!ok) break;
+        if (row == 0 && i == 0) HA_TACC(0, tw);
+        HA_T0(tc);
         tc_fence_after();
         // mask kind of this (query tile, key tile): uniform over the warpgroup
         bool table = false, dense_mask = false;
@@ -551,6 +557,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
         tmem_ld32_wait(ra);
         tmem_ld32_wait(rb);
+        if (row == 0 && i == 0) HA_TACC(16, tc);
+        HA_T0(tm);
         float m0 = -INFINITY, m1 = -INFINITY;
         if (masked_tile) {
 #pragma unroll
@@ -570,7 +578,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         if (__any_sync(0xffffffffu, grow)) {          // rare; per warp so that TMEM accesses stay convergent
           float alpha = 1.f;
           if (grow) {
-            if (m_ref == -INFINITY) { m_ref = xm; alpha = 0.f; }
+            // first tile: leave head room for the weight log2(N/m) that the sampled columns will
+            // add, so that reaching them does not move the reference again (any reference within
+            // 2^8 of the true maximum serves; a higher one only shifts the exponents)
+            if (m_ref == -INFINITY) { m_ref = xm + (wlog - ubias); alpha = 0.f; }
             else { const float k = ceilf(xm - m_ref); m_ref += k; alpha = ex2(-k); }
           }
           l0 *= alpha; l1 *= alpha; lr0 *= alpha; lr1 *= alpha;
@@ -587,6 +598,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           }
         }
         const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
+        if (row == 0 && i == 0) HA_TACC(17, tm);
+        HA_T0(tx);
         auto chunk_exp = [&](const uint32_t (&r)[32], uint32_t vis, int c) {
           uint32_t p[16];
           if (masked_tile) {
@@ -616,11 +629,18 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         };
         chunk_exp(ra, visa, 0);
         chunk_exp(rb, visb, 1);
+        if (row == 0 && i == 0) HA_TACC(18, tx);
+        HA_T0(ts);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p(i, buf));
+        if (row == 0 && i == 0) { HA_TACC(2, tc); HA_TACC(19, ts); }
+#ifdef HA_TC_TIMING
+        if (row == 0 && i == 0) atomicAdd(&g_tc_timing[20], 1ull);
+#endif
       }
       if (!ok) break;
+      HA_T0(te);
       // epilogue: normalise, log-sum-exp, rows back to their original places
       if (q.valid) {
         ok = __all_sync(0xffffffffu, mbar_wait<20, 5>(bar_o(i), vi & 1, s_abort, status));
@@ -659,6 +679,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         ++vi;
       }
       mbar_arrive(bar_tabfree(set));
+      if (row == 0 && i == 0) HA_TACC(15, te);
       ga += total;
     }
   } else if (warp < 10) {
@@ -705,14 +726,20 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
       };
       int it = 0;
+      HA_T0(tloop);
       for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
         PairDesc t; QTile qa, qb;
         decode_pair(a, item, t, qa, qb);
         const QTile q = i ? qb : qa;
         const int total = q.n1 + q.n2;
+#ifdef HA_TC_TIMING
+        if (i == 0) atomicAdd(&g_tc_timing[14], (unsigned long long)t.ntiles);
+#endif
         // Q of this item (an issuer without a tile waits too: it may not run ahead of the others)
+        HA_T0(tq);
         ok = wait_fast<6>(bar_q, it & 1, s_abort, status);
         if (!ok) break;
+        if (i == 0) HA_TACC(7, tq);
         fence_async_smem();
         if (total == 0) mbar_arrive(bar_qfree);
         for (int r = 0; r < total + 2 && ok; ++r) {
@@ -723,8 +750,12 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             const int s = gj % C::NS;
             const int gw = ga + a2;
             if (gj != vnext) skip_v(gj);
+            HA_T0(tp);
             ok = ok && wait_fast<8>(bar_p(i, gw & 1), (gw >> 1) & 1, s_abort, status);
+            if (i == 0) HA_TACC(4, tp);
+            HA_T0(tv);
             ok = ok && wait_fast<9>(bar_vfull(s), (gj / C::NS) & 1, s_abort, status);
+            if (i == 0) HA_TACC(5, tv);
             // the first product of an item overwrites O: the previous item's O must have been read
             if (a2 == 0 && vi > 0) ok = ok && wait_fast<15>(bar_ofree(i), (vi - 1) & 1, s_abort, status);
             if (!ok) break;
@@ -747,7 +778,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             const int s = gj % C::NS;
             const int gw = ga + r;
             if (gj != knext) skip_k(gj);
+            HA_T0(tk);
             ok = ok && wait_fast<7>(bar_kfull(s), (gj / C::NS) & 1, s_abort, status);
+            if (i == 0) HA_TACC(6, tk);
             if (!ok) break;
             fence_async_smem();
             tc_fence_after();
@@ -770,6 +803,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         ga += total;
         vi += q.valid;
       }
+      if (i == 0) { HA_TACC(8, tloop); HA_TACC(12, t_cta); }
+#ifdef HA_TC_TIMING
+      if (i == 0) atomicAdd(&g_tc_timing[13], 1ull);
+#endif
     }
     __syncwarp();
   } else {
@@ -797,52 +834,88 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       uint32_t* s_mask = s_mask_all + set * 2 * MW;
       int* s_qrow = s_qrow_all + set * 2 * 128;
       // ---- row tables (the softmax warps must be done with this set: item it - 2) --------------
+      HA_T0(ttab);
       if (it >= 2) {
         ok = mbar_wait<100, 16>(bar_tabfree(set), ((it >> 1) - 1) & 1, s_abort, status);
         if (!ok) break;
       }
-      for (int c = lt; c < 2 * MW; c += kLoaderThreads) s_mask[c] = 0;
-      loader_sync();
-      if (!ok) break;
+      // Every global load of a batch is issued before the first one is used: the two loader
+      // warps have no other way to hide the latency of these dependent lookups.  A warp covers
+      // 32 consecutive columns per step, so one ballot yields a whole word of the mask tables.
       if (t.mode == 1) {
+        constexpr int UB = 4;
         const int bcols = t.nbA * TK;
+        const int nblk = (t.nbA + t.nbB) * TK;            // columns of the block part (multiple of 64)
         const int ncols = t.ntiles * TK;
         const int32_t* smp = a.samples + ((size_t)t.seg * g.nodes + t.node) * g.m;
-        for (int c0 = lt; c0 < ncols; c0 += kLoaderThreads) {
-          int idx = -1;
-          bool m0 = true, m1 = true;                      // masked for query tile 0 / 1
-          if (c0 < (t.nbA + t.nbB) * TK) {
-            const int which = c0 >= bcols;                // 0: block of tile 0, 1: block of tile 1
-            const int c = c0 - which * bcols;
-            if (c < g.b) {
-              idx = t.k0 + a.perm_k[t.slice + (size_t)(which ? qb.beta : qa.beta) * g.b + c];
-              m0 = m1 = false;
-            }
-          } else {
-            const int c = c0 - (t.nbA + t.nbB) * TK;
-            if (c < g.m) {
-              const int l = smp[c];
-              idx = t.k0 + l;
-              const int blk = a.rank_k[t.slice + l] / g.b;
-              m0 = blk == qa.beta;                        // the factor (1 - M^H) of Alg. 2 line 7
-              m1 = qb.valid && blk == qb.beta;
+        const int32_t* pk = a.perm_k + t.slice;
+        const int32_t* rk = a.rank_k + t.slice;
+        // block columns: nothing masked inside the block; padding columns are masked for both tiles
+        for (int c00 = lt; c00 < nblk; c00 += kLoaderThreads * UB) {
+          int idx[UB];
+#pragma unroll
+          for (int u = 0; u < UB; ++u) {
+            const int c0 = c00 + u * kLoaderThreads;
+            idx[u] = -1;
+            if (c0 < nblk) {
+              const int which = c0 >= bcols;
+              const int c = c0 - which * bcols;
+              if (c < g.b) idx[u] = pk[(size_t)(which ? qb.beta : qa.beta) * g.b + c];
             }
           }
-          s_kidx[c0] = idx;
-          if (m0) atomicOr(&s_mask[c0 >> 5], 1u << (c0 & 31));
-          if (m1) atomicOr(&s_mask[MW + (c0 >> 5)], 1u << (c0 & 31));
+#pragma unroll
+          for (int u = 0; u < UB; ++u) {
+            const int c0 = c00 + u * kLoaderThreads;
+            if (c0 - lane < nblk) {                       // warp-uniform (nblk is a multiple of 32)
+              const unsigned pad = __ballot_sync(0xffffffffu, idx[u] < 0);
+              s_kidx[c0] = idx[u] < 0 ? -1 : t.k0 + idx[u];
+              if (lane == 0) { s_mask[c0 >> 5] = pad; s_mask[MW + (c0 >> 5)] = pad; }
+            }
+          }
+        }
+        // sampled columns: masked where the sample falls into the tile's own block (the factor
+        // (1 - M^H) of Alg. 2 line 7)
+        for (int c00 = nblk + lt; c00 < ncols; c00 += kLoaderThreads * UB) {
+          int l[UB], blk[UB];
+#pragma unroll
+          for (int u = 0; u < UB; ++u) {
+            const int c = c00 + u * kLoaderThreads - nblk;
+            l[u] = (c00 + u * kLoaderThreads < ncols && c < g.m) ? smp[c] : -1;
+          }
+#pragma unroll
+          for (int u = 0; u < UB; ++u) blk[u] = l[u] >= 0 ? rk[l[u]] / g.b : -1;
+#pragma unroll
+          for (int u = 0; u < UB; ++u) {
+            const int c0 = c00 + u * kLoaderThreads;
+            if (c0 - lane < ncols) {
+              const bool m0 = l[u] < 0 || blk[u] == qa.beta;
+              const bool m1 = l[u] < 0 || (qb.valid && blk[u] == qb.beta);
+              const unsigned w0 = __ballot_sync(0xffffffffu, m0);
+              const unsigned w1 = __ballot_sync(0xffffffffu, m1);
+              s_kidx[c0] = l[u] < 0 ? -1 : t.k0 + l[u];
+              if (lane == 0) { s_mask[c0 >> 5] = w0; s_mask[MW + (c0 >> 5)] = w1; }
+            }
+          }
         }
       }
-      for (int c = lt; c < 2 * kTileQ; c += kLoaderThreads) {
-        const int r = c & 127;
-        const QTile& q = c < 128 ? qa : qb;
-        int v = -1;
-        if (q.valid && r < q.nq) v = t.mode == 1 ? t.qnode0 + a.perm_q[t.slice + q.spos0 + r] : q.q0 + r;
-        s_qrow[c] = v;
+      {
+        constexpr int UQ = 2 * kTileQ / kLoaderThreads;
+        int v[UQ];
+#pragma unroll
+        for (int u = 0; u < UQ; ++u) {
+          const int c = lt + u * kLoaderThreads;
+          const int r = c & 127;
+          const QTile& q = c < 128 ? qa : qb;
+          v[u] = -1;
+          if (q.valid && r < q.nq) v[u] = t.mode == 1 ? t.qnode0 + a.perm_q[t.slice + q.spos0 + r] : q.q0 + r;
+        }
+#pragma unroll
+        for (int u = 0; u < UQ; ++u) s_qrow[lt + u * kLoaderThreads] = v[u];
       }
       loader_sync();                                      // the loaders themselves read the tables below
       if (!ok) break;
       mbar_arrive(bar_tabfull(set));
+      if (lt == 0) HA_TACC(10, ttab);
       // ---- Q (the issuers must be done with the previous item's Q) ----------------------------
       if (it >= 1) {
         ok = mbar_wait<100, 17>(bar_qfree, (it - 1) & 1, s_abort, status);
@@ -897,20 +970,28 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         const int gj = gbase + j;
         const int s = gj % C::NS;
         const int use = gj / C::NS;
+        HA_T0(tle);
         if (use > 0) {
           ok = mbar_wait<100, 10>(bar_kempty(0, s), (use - 1) & 1, s_abort, status);
           ok = ok && mbar_wait<100, 11>(bar_kempty(1, s), (use - 1) & 1, s_abort, status);
           if (!ok) break;
         }
+        if (lt == 0) HA_TACC(11, tle);
+        HA_T0(tgk);
         gather_kv(ubase + C::kOffK + s * C::kTile, ks, j);
         cp_async_arrive_noinc(bar_kfull(s));
+        if (lt == 0) HA_TACC(3, tgk);
+        HA_T0(tle2);
         if (use > 0) {
           ok = mbar_wait<100, 12>(bar_vempty(0, s), (use - 1) & 1, s_abort, status);
           ok = ok && mbar_wait<100, 13>(bar_vempty(1, s), (use - 1) & 1, s_abort, status);
           if (!ok) break;
         }
+        if (lt == 0) HA_TACC(11, tle2);
+        HA_T0(tgv);
         gather_kv(ubase + C::kOffV + s * C::kTile, vs, j);
         cp_async_arrive_noinc(bar_vfull(s));
+        if (lt == 0) HA_TACC(1, tgv);
       }
       gbase += t.ntiles;
     }
@@ -931,8 +1012,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 
 #ifdef HA_TC_TIMING
 extern "C" int hyperattn_debug_tc_timing(unsigned long long* host16, int reset) {
-  if (cudaMemcpyFromSymbol(host16, g_tc_timing, sizeof(unsigned long long) * 16) != cudaSuccess) return -5;
-  if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)); }
+  if (cudaMemcpyFromSymbol(host16, g_tc_timing, sizeof(unsigned long long) * 24) != cudaSuccess) return -5;
+  if (reset) { unsigned long long z[24] = {0}; cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)); }
   return 0;
 }
 #endif
