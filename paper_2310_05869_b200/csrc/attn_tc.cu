@@ -12,7 +12,7 @@
 // of a 256-row block share every key tile, so K and V are fetched once for 256 rows, and
 // every warpgroup has two S buffers in TMEM, so the tensor pipe computes the scores of the
 // next key tile while the warpgroup exponentiates the current one.  The running
-// row maximum is only moved when it grows by more than 2^8 (the accumulators absorb the
+// row maximum is only moved when it grows by more than 2^32 (the accumulators absorb the
 // rest), so O is rarely rescaled; outputs are normalised by the sum of the bf16-rounded
 // weights that the tensor cores actually used, the log-sum-exp by the unrounded sum.  Rows
 // of Q, K, V are gathered from their original places through the sortLSH permutations by
@@ -32,7 +32,7 @@ namespace {
 constexpr int TK = 64;                  // keys per tile
 constexpr int kLoaderThreads = 64;    // two loader warps: 12 warps per CTA leave 168 registers per thread
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
-constexpr float kRescaleThreshold = 8.f;
+constexpr float kRescaleThreshold = 32.f;   // octaves the scores may exceed the reference before it moves
 #ifndef HA_TAKE_TURNS
 #define HA_TAKE_TURNS 0
 #endif
@@ -193,6 +193,33 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// packed pairs of fp32 (one instruction, two lanes)
+__device__ __forceinline__ uint64_t pack_u2(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi) { return pack_u2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a); hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
@@ -516,7 +543,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       if (row == 0 && i == 0) HA_TACC(9, tt);
       const float wlog = (t.mode == 1 && g.m > 0) ? log2f((float)t.nk / (float)g.m) : 0.f;   // log2(N/m): weight of a sampled column
       float m_ref = -INFINITY;
-      float l0 = 0.f, l1 = 0.f, lr0 = 0.f, lr1 = 0.f;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each)
+      uint64_t l01 = 0, lr01 = 0;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each, packed)
       for (int na = 0; na < total && ok; ++na) {
         const int j = tile_of(q, na);
         const int gw = ga + na;
@@ -540,7 +567,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
         // The 64 scores of this row are read from TMEM once; then (1) the row maximum, (2)
         // exponentials, row sums and the bf16 P written over the first half of the S buffer.
-        // The reference maximum only moves when the tile exceeds it by more than 2^8, and then
+        // The reference maximum only moves when the tile exceeds it by more than 2^32, and then
         // by a whole number of octaves, so that what is already accumulated (O and the row
         // sums) is rescaled exactly.
         uint32_t ra[32], rb[32];
@@ -559,20 +586,24 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         tmem_ld32_wait(rb);
         if (row == 0 && i == 0) HA_TACC(16, tc);
         HA_T0(tm);
-        float m0 = -INFINITY, m1 = -INFINITY;
+        // masked columns become -inf once, here: they then drop out of the maximum and
+        // exponentiate to zero without further tests
         if (masked_tile) {
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            if ((visa >> e) & 1u) m0 = fmaxf(m0, __uint_as_float(ra[e]));
-            if ((visb >> e) & 1u) m1 = fmaxf(m1, __uint_as_float(rb[e]));
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
-            m1 = max3(m1, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+            if (!((visa >> e) & 1u)) ra[e] = 0xff800000u;
+            if (!((visb >> e) & 1u)) rb[e] = 0xff800000u;
           }
         }
+        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+          m1 = max3(m1, __uint_as_float(ra[e + 2]), __uint_as_float(ra[e + 3]));
+          m2 = max3(m2, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+          m3 = max3(m3, __uint_as_float(rb[e + 2]), __uint_as_float(rb[e + 3]));
+        }
+        m0 = fmaxf(m0, m2); m1 = fmaxf(m1, m3);
         const float xm = fmaf(fmaxf(m0, m1), a.scale_log2, ubias);   // scale_log2 > 0: the maximum commutes with it
         const bool grow = xm > m_ref + kRescaleThreshold;
         if (__any_sync(0xffffffffu, grow)) {          // rare; per warp so that TMEM accesses stay convergent
@@ -580,11 +611,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           if (grow) {
             // first tile: leave head room for the weight log2(N/m) that the sampled columns will
             // add, so that reaching them does not move the reference again (any reference within
-            // 2^8 of the true maximum serves; a higher one only shifts the exponents)
+            // 2^32 below the true maximum serves; a higher one only shifts the exponents)
             if (m_ref == -INFINITY) { m_ref = xm + (wlog - ubias); alpha = 0.f; }
             else { const float k = ceilf(xm - m_ref); m_ref += k; alpha = ex2(-k); }
           }
-          l0 *= alpha; l1 *= alpha; lr0 *= alpha; lr1 *= alpha;
+          { const uint64_t al2 = pack_f2(alpha, alpha); l01 = fmul2(l01, al2); lr01 = fmul2(lr01, al2); }
           // O may only be touched between two PV products: the one of the previous tile must
           // have finished (the one of this tile cannot start before this tile's P is published)
           if (na > 0) {
@@ -600,35 +631,24 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
         if (row == 0 && i == 0) HA_TACC(17, tm);
         HA_T0(tx);
-        auto chunk_exp = [&](const uint32_t (&r)[32], uint32_t vis, int c) {
+        // packed fp32 arithmetic (two lanes per instruction) for the scaling and the two row sums
+        const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2), off2 = pack_f2(off, off);
+        auto chunk_exp = [&](const uint32_t (&r)[32], int c) {
           uint32_t p[16];
-          if (masked_tile) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
-              float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
-              if (!((vis >> e) & 1u)) p0 = 0.f;
-              if (!((vis >> (e + 1)) & 1u)) p1 = 0.f;
-              l0 += p0; l1 += p1;
-              const uint32_t w = pack2(p0, p1);
-              lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
-              p[e >> 1] = w;
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              const float p0 = ex2(fmaf(__uint_as_float(r[e]), a.scale_log2, off));
-              const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, off));
-              l0 += p0; l1 += p1;
-              const uint32_t w = pack2(p0, p1);
-              lr0 += __uint_as_float(w << 16); lr1 += __uint_as_float(w & 0xffff0000u);
-              p[e >> 1] = w;
-            }
+          for (int e = 0; e < 32; e += 2) {
+            float x0, x1;
+            unpack_f2(ffma2(pack_u2(r[e], r[e + 1]), sc2, off2), x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            l01 = fadd2(l01, pack_f2(p0, p1));
+            const uint32_t w = pack2(p0, p1);
+            lr01 = fadd2(lr01, pack_u2(w << 16, w & 0xffff0000u));
+            p[e >> 1] = w;
           }
           tmem_st16(sbase + c * 16, p);
         };
-        chunk_exp(ra, visa, 0);
-        chunk_exp(rb, visb, 1);
+        chunk_exp(ra, 0);
+        chunk_exp(rb, 1);
         if (row == 0 && i == 0) HA_TACC(18, tx);
         HA_T0(ts);
         tmem_wait_st();
@@ -647,6 +667,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         if (!ok) break;
         tc_fence_after();
         const int qr = s_qrow[row];
+        float l0, l1, lr0, lr1;
+        unpack_f2(l01, l0, l1);
+        unpack_f2(lr01, lr0, lr1);
         const float inv = 1.f / (lr0 + lr1);
         const float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
         const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
