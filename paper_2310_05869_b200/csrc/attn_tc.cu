@@ -15,22 +15,33 @@
 // row maximum is only moved when it grows by more than 2^32 (the accumulators absorb the
 // rest), so O is rarely rescaled; outputs are normalised by the sum of the bf16-rounded
 // weights that the tensor cores actually used, the log-sum-exp by the unrounded sum.  Rows
-// of Q, K, V are gathered from their original places through the sortLSH permutations by
-// three loader warps with 16-byte cp.async copies; nothing permuted is ever written to HBM.
+// of Q, K, V come from their original places: tiles of consecutive rows (causal leaves) as
+// one TMA box per 64 columns, tiles of sorted or sampled rows gathered through the sortLSH
+// permutations with 16-byte cp.async copies into the same 128B-swizzled operand layout;
+// nothing permuted is ever written to HBM.  (The TMA row gather, tile::gather4, was measured
+// at about 100 cycles of issue per four rows and warp: too slow for this.)
 //
 // Warp roles (384 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
 // warps 8 and 9 MMA issue for query tile 0 and 1 (warp 8 also allocates TMEM, all 512
-// columns: 2 x 2 S buffers of 64, O0, O1), warps 10-11 loaders.
+// columns: 2 x 2 S buffers of 64, O0, O1), warp 10 prepares work items (row tables of the
+// NEXT item while this one computes, then its Q tiles), warp 11 streams K / V tiles through
+// the stage ring, across item boundaries.
 // Every mbarrier wait is bounded: on a timeout the CTA raises the device status word,
 // drains its copies, frees its TMEM and returns.
 #include <cstdlib>
+#include <cuda.h>
 #include "attn_common.cuh"
 
 namespace hyperattn {
 namespace {
 
+// tensor maps of Q, K, V as [G * n rows x d] bf16 tensors, 128-byte swizzle; box = 64 columns x
+// 128 rows (Q) or 64 rows (K, V): one slab of an operand tile
+struct alignas(64) TmaMaps {
+  CUtensorMap q, k, v;
+};
+
 constexpr int TK = 64;                  // keys per tile
-constexpr int kLoaderThreads = 64;    // two loader warps: 12 warps per CTA leave 168 registers per thread
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
 constexpr float kRescaleThreshold = 32.f;   // octaves the scores may exceed the reference before it moves
 #ifndef HA_TAKE_TURNS
@@ -39,7 +50,7 @@ constexpr float kRescaleThreshold = 32.f;   // octaves the scores may exceed the
 
 // Optional per-role cycle counters (compile with -DHA_TC_TIMING; never in the shipped build).
 #ifdef HA_TC_TIMING
-__device__ unsigned long long g_tc_timing[24];
+__device__ unsigned long long g_tc_timing[32];
 #define HA_T0(var) const long long var = clock64()
 #define HA_TACC(slot, var) atomicAdd(&g_tc_timing[slot], (unsigned long long)(clock64() - var))
 #else
@@ -240,30 +251,33 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
 }
-// 16 bytes of zeros through the same asynchronous path (source size 0), so that they are tracked
-// by the same completion mechanism as the copies around them
-__device__ __forceinline__ void cp_async16_zero(uint32_t dst, const void* any_valid_src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, 0;\n" ::"r"(dst), "l"(any_valid_src) : "memory");
-}
 // the executing thread's arrival on the mbarrier happens when all its earlier cp.async have landed
 __device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void st_shared_zero16(uint32_t dst) {
-  asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};\n" ::"r"(dst), "r"(0) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_le(int n) {   // wait until at most n groups are pending
-  switch (n) {
-    case 0: asm volatile("cp.async.wait_group 0;\n" ::: "memory"); break;
-    case 1: asm volatile("cp.async.wait_group 1;\n" ::: "memory"); break;
-    case 2: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
-    case 3: asm volatile("cp.async.wait_group 3;\n" ::: "memory"); break;
-    case 4: asm volatile("cp.async.wait_group 4;\n" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 5;\n" ::: "memory"); break;
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// One TMA box (64 columns x the map's box rows, starting at column x, row y) into a
+// 128B-swizzled slab; completion is counted in bytes on the mbarrier.
+__device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// announces bytes to the current phase without arriving
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Teardown only: waits (bounded, whatever the abort flag says) until a phase that this warp
+// armed has received all its bytes, so that no copy is in flight into the CTA's shared
+// memory when it exits.
+__device__ __noinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  const unsigned long long t0 = global_ns();
+  for (unsigned it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return;
+    if ((it & 15u) == 15u && global_ns() - t0 > kWaitLimitNs) return;
   }
 }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
@@ -330,7 +344,7 @@ struct Cfg {
   static constexpr int kOffMask = kOffIdx + 2 * kMaxNodeKeys * 4; // uint32 [2][2][kMaxNodeKeys/32] masked-column bits
   static constexpr int kOffQrow = kOffMask + 4 * (kMaxNodeKeys / 32) * 4;   // int [2][2][128]
   static constexpr int kOffBar = kOffQrow + 4 * 128 * 4;
-  static constexpr int kNumBar = 21 + 6 * NS;
+  static constexpr int kNumBar = 21 + 6 * NS;          // (slot 20 unused)
   static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
   static constexpr int kTotal = kOffMisc + 16;
   static constexpr int kTmemCols = 512;
@@ -447,7 +461,7 @@ __device__ __forceinline__ bool uses_tile(const QTile& q, int j) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, int* status) {
+__global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TmaMaps maps, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   constexpr int MW = kMaxNodeKeys / 32;
@@ -468,7 +482,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   auto bar_ofree = [&](int i) { return bar0 + 112 + 8 * i; };                 // O_i has been read out
   auto bar_tabfull = [&](int set) { return bar0 + 128 + 8 * set; };           // row tables of a set written
   auto bar_tabfree = [&](int set) { return bar0 + 144 + 8 * set; };           // softmax warps are done with a set
-  const uint32_t bar_ld = bar0 + 160;                                         // the loader warps among themselves
   auto bar_kfull = [&](int s) { return bar0 + 168 + 8 * s; };
   auto bar_vfull = [&](int s) { return bar0 + 168 + 8 * (C::NS + s); };
   auto bar_kempty = [&](int i, int s) { return bar0 + 168 + 8 * ((2 + i) * C::NS + s); };     // released by issuer i
@@ -487,20 +500,19 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 
   // ---- setup: barriers, TMEM ---------------------------------------------------------------------
   if (tid == 0) {
-    mbar_init(bar_q, kLoaderThreads);
+    mbar_init(bar_q, 32);
     mbar_init(bar_qfree, 2);
-    mbar_init(bar_ld, kLoaderThreads);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_o(i), 1);
       mbar_init(bar_pv(i), 1);
       mbar_init(bar_ofree(i), 128);
-      mbar_init(bar_tabfull(i), kLoaderThreads);
-      mbar_init(bar_tabfree(i), 256);
+      mbar_init(bar_tabfull(i), 1);
+      mbar_init(bar_tabfree(i), 257);                   // 256 softmax threads + the K / V streamer
       for (int b = 0; b < 2; ++b) { mbar_init(bar_s(i, b), 1); mbar_init(bar_p(i, b), 128); }
     }
     for (int s = 0; s < C::NS; ++s) {
-      mbar_init(bar_kfull(s), kLoaderThreads);
-      mbar_init(bar_vfull(s), kLoaderThreads);
+      mbar_init(bar_kfull(s), 32);
+      mbar_init(bar_vfull(s), 32);
       for (int i = 0; i < 2; ++i) { mbar_init(bar_kempty(i, s), 1); mbar_init(bar_vempty(i, s), 1); }
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -832,53 +844,47 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 #endif
     }
     __syncwarp();
-  } else {
-    // ================= loaders: row tables of the next item, then gathers into swizzled tiles ========
-    const int lt = tid - 320;
-    constexpr int CPR = D / 8;
-    // Copies are never waited for by the loaders: each thread's arrival on the tile's "full"
-    // barrier is attached to its copies (cp.async.mbarrier.arrive.noinc) and happens when
-    // they land.  The consumer (MMA issuer) crosses from the generic to the async proxy with
-    // a proxy fence after it has observed the barrier.
+  } else if (warp == 10) {
+    constexpr int CPR = D / 8;                             // 16-byte chunks per row
+    // ================= item preparer: row tables of an item, then its Q tiles ========================
+    // Runs one item ahead of the K / V streamer where it can: a table set becomes free when the
+    // softmax warps and the streamer are done with the item before the previous one, so the
+    // dependent global lookups below overlap with the computation of the item in between.
     bool ok = true;
-    int gbase = 0;
     int it = 0;
-    int nsync = 0;                                    // loader-only synchronisations so far (bounded, like every wait here)
-    auto loader_sync = [&]() {
-      mbar_arrive(bar_ld);
-      ok = mbar_wait<20, 18>(bar_ld, nsync & 1, s_abort, status);
-      ++nsync;
-    };
     for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+      HA_T0(tdec);
       PairDesc t; QTile qa, qb;
       decode_pair(a, item, t, qa, qb);
+      if (lane == 0) HA_TACC(26, tdec);
       const int set = it & 1;
       int* s_kidx = s_kidx_all + set * kMaxNodeKeys;
       uint32_t* s_mask = s_mask_all + set * 2 * MW;
       int* s_qrow = s_qrow_all + set * 2 * 128;
-      // ---- row tables (the softmax warps must be done with this set: item it - 2) --------------
       HA_T0(ttab);
       if (it >= 2) {
         ok = mbar_wait<100, 16>(bar_tabfree(set), ((it >> 1) - 1) & 1, s_abort, status);
         if (!ok) break;
       }
-      // Every global load of a batch is issued before the first one is used: the two loader
-      // warps have no other way to hide the latency of these dependent lookups.  A warp covers
-      // 32 consecutive columns per step, so one ballot yields a whole word of the mask tables.
+      if (lane == 0) HA_TACC(21, ttab);
+      const int segrow = t.seg * g.n;                       // row coordinate of the segment's first row
+      // Key rows as tensor-map row coordinates.  Every global load of a batch is issued before
+      // the first one is used; the warp covers 32 consecutive columns per step, so one ballot
+      // yields a whole word of the mask tables.  Padding columns point at a valid row (they are
+      // masked, so that row only has to be finite) and are masked for both tiles.
       if (t.mode == 1) {
-        constexpr int UB = 4;
+        constexpr int UB = 8;
         const int bcols = t.nbA * TK;
         const int nblk = (t.nbA + t.nbB) * TK;            // columns of the block part (multiple of 64)
         const int ncols = t.ntiles * TK;
         const int32_t* smp = a.samples + ((size_t)t.seg * g.nodes + t.node) * g.m;
         const int32_t* pk = a.perm_k + t.slice;
         const int32_t* rk = a.rank_k + t.slice;
-        // block columns: nothing masked inside the block; padding columns are masked for both tiles
-        for (int c00 = lt; c00 < nblk; c00 += kLoaderThreads * UB) {
+        for (int c00 = lane; c00 < nblk; c00 += 32 * UB) {
           int idx[UB];
 #pragma unroll
           for (int u = 0; u < UB; ++u) {
-            const int c0 = c00 + u * kLoaderThreads;
+            const int c0 = c00 + u * 32;
             idx[u] = -1;
             if (c0 < nblk) {
               const int which = c0 >= bcols;
@@ -888,138 +894,194 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           }
 #pragma unroll
           for (int u = 0; u < UB; ++u) {
-            const int c0 = c00 + u * kLoaderThreads;
+            const int c0 = c00 + u * 32;
             if (c0 - lane < nblk) {                       // warp-uniform (nblk is a multiple of 32)
               const unsigned pad = __ballot_sync(0xffffffffu, idx[u] < 0);
-              s_kidx[c0] = idx[u] < 0 ? -1 : t.k0 + idx[u];
+              s_kidx[c0] = segrow + (idx[u] < 0 ? 0 : t.k0 + idx[u]);
               if (lane == 0) { s_mask[c0 >> 5] = pad; s_mask[MW + (c0 >> 5)] = pad; }
             }
           }
         }
         // sampled columns: masked where the sample falls into the tile's own block (the factor
         // (1 - M^H) of Alg. 2 line 7)
-        for (int c00 = nblk + lt; c00 < ncols; c00 += kLoaderThreads * UB) {
+        for (int c00 = nblk + lane; c00 < ncols; c00 += 32 * UB) {
           int l[UB], blk[UB];
 #pragma unroll
           for (int u = 0; u < UB; ++u) {
-            const int c = c00 + u * kLoaderThreads - nblk;
-            l[u] = (c00 + u * kLoaderThreads < ncols && c < g.m) ? smp[c] : -1;
+            const int c = c00 + u * 32 - nblk;
+            l[u] = (c00 + u * 32 < ncols && c < g.m) ? smp[c] : -1;
           }
 #pragma unroll
           for (int u = 0; u < UB; ++u) blk[u] = l[u] >= 0 ? rk[l[u]] / g.b : -1;
 #pragma unroll
           for (int u = 0; u < UB; ++u) {
-            const int c0 = c00 + u * kLoaderThreads;
+            const int c0 = c00 + u * 32;
             if (c0 - lane < ncols) {
               const bool m0 = l[u] < 0 || blk[u] == qa.beta;
               const bool m1 = l[u] < 0 || (qb.valid && blk[u] == qb.beta);
               const unsigned w0 = __ballot_sync(0xffffffffu, m0);
               const unsigned w1 = __ballot_sync(0xffffffffu, m1);
-              s_kidx[c0] = l[u] < 0 ? -1 : t.k0 + l[u];
+              s_kidx[c0] = segrow + (l[u] < 0 ? 0 : t.k0 + l[u]);
               if (lane == 0) { s_mask[c0 >> 5] = w0; s_mask[MW + (c0 >> 5)] = w1; }
             }
           }
         }
       }
-      {
-        constexpr int UQ = 2 * kTileQ / kLoaderThreads;
-        int v[UQ];
+      if (lane == 0) HA_TACC(23, ttab);
+      // query rows of both tiles: lane l owns rows 4l .. 4l+3
+      int qr[2][4];
 #pragma unroll
-        for (int u = 0; u < UQ; ++u) {
-          const int c = lt + u * kLoaderThreads;
-          const int r = c & 127;
-          const QTile& q = c < 128 ? qa : qb;
-          v[u] = -1;
-          if (q.valid && r < q.nq) v[u] = t.mode == 1 ? t.qnode0 + a.perm_q[t.slice + q.spos0 + r] : q.q0 + r;
+      for (int i = 0; i < 2; ++i) {
+        const QTile& q = i ? qb : qa;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int r = 4 * lane + k;
+          qr[i][k] = -1;
+          if (q.valid && r < q.nq) qr[i][k] = t.mode == 1 ? t.qnode0 + a.perm_q[t.slice + q.spos0 + r] : q.q0 + r;
         }
-#pragma unroll
-        for (int u = 0; u < UQ; ++u) s_qrow[lt + u * kLoaderThreads] = v[u];
       }
-      loader_sync();                                      // the loaders themselves read the tables below
-      if (!ok) break;
-      mbar_arrive(bar_tabfull(set));
-      if (lt == 0) HA_TACC(10, ttab);
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+        *reinterpret_cast<int4*>(s_qrow + i * 128 + 4 * lane) = make_int4(qr[i][0], qr[i][1], qr[i][2], qr[i][3]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tabfull(set));       // (release: the table writes of all lanes are ordered before it by the warp barrier)
+      if (lane == 0) HA_TACC(10, ttab);
       // ---- Q (the issuers must be done with the previous item's Q) ----------------------------
       if (it >= 1) {
         ok = mbar_wait<100, 17>(bar_qfree, (it - 1) & 1, s_abort, status);
         if (!ok) break;
       }
-      const __nv_bfloat16* qs = a.q + (size_t)t.seg * g.n * D;
-      const __nv_bfloat16* ks = a.k + (size_t)t.seg * g.n * D;
-      const __nv_bfloat16* vs = a.v + (size_t)t.seg * g.n * D;
-      // (indices first, copies second: the loaders have few warps, so every gather keeps many
-      // independent chunks in flight instead of one dependent index -> address -> copy chain)
-      {
-        constexpr int PER = 8;                                   // chunks per thread per step
-        static_assert((2 * 128 * CPR) % (kLoaderThreads * PER) == 0, "query tile gather must divide evenly");
-#pragma unroll 1
-        for (int c0 = lt; c0 < 2 * 128 * CPR; c0 += kLoaderThreads * PER) {
-          int gr[PER];
+      if (t.mode == 0) {
+        // consecutive rows: one box per 64 columns and tile (rows past the tile's end are other
+        // rows of the tensor or zeros: their results are never stored)
+        if (lane == 0) {
+          mbar_expect_tx(bar_q, (uint32_t)((qa.valid + qb.valid) * C::kQTile));
 #pragma unroll
-          for (int k = 0; k < PER; ++k) gr[k] = s_qrow[(c0 + k * kLoaderThreads) / CPR];
+          for (int i = 0; i < 2; ++i) {
+            if (!(i ? qb.valid : qa.valid)) continue;
 #pragma unroll
-          for (int k = 0; k < PER; ++k) {
-            const int c = c0 + k * kLoaderThreads;
-            const int i = c / (128 * CPR);
-            const int row = (c / CPR) & 127, cc = c % CPR;
-            const uint32_t d = ubase + C::kOffQ + i * C::kQTile + tile_off<128>(row, cc);
-            if (gr[k] >= 0) cp_async16(d, qs + (size_t)gr[k] * D + cc * 8);
-            else cp_async16_zero(d, qs);
+            for (int sl = 0; sl < D / 64; ++sl)
+              tma_tile(ubase + C::kOffQ + i * C::kQTile + sl * (128 * 128), &maps.q, sl * 64, segrow + (i ? qb.q0 : qa.q0), bar_q);
           }
         }
+        mbar_arrive(bar_q);
+      } else {
+        // gathered rows: lane -> column chunk cc and rows rq, rq + 32 / CPR, ... ; padding rows
+        // fetch the segment's first row (finite values whose results are never stored)
+        const int cc = lane % CPR, rq = lane / CPR;
+        const char* qsrc = reinterpret_cast<const char*>(a.q) + cc * 16;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          if (!(i ? qb.valid : qa.valid)) continue;      // nobody reads the tile of a query tile that does not exist
+          const uint32_t dbase = ubase + C::kOffQ + i * C::kQTile + (cc >> 3) * (128 * 128);
+          const int* rows = s_qrow + i * 128;
+#pragma unroll 4
+          for (int r = rq; r < 128; r += 32 / CPR) {
+            const int v = rows[r];
+            cp_async16(dbase + r * 128 + (((cc & 7) ^ (r & 7)) << 4), qsrc + (size_t)(uint32_t)(segrow + (v < 0 ? 0 : v)) * (D * 2));
+          }
+        }
+        cp_async_arrive_noinc(bar_q);
       }
-      cp_async_arrive_noinc(bar_q);
-      // ---- K / V tiles through the stage ring ----------------------------------------------------
-      auto gather_kv = [&](uint32_t dst, const __nv_bfloat16* src, int kt) {
-        constexpr int PER = TK * CPR / kLoaderThreads;           // 8 (d = 64) or 16 (d = 128) chunks per thread
-        static_assert(PER * kLoaderThreads == TK * CPR, "key tile gather must divide evenly");
-        int gr[PER];
+      if (lane == 0) HA_TACC(25, ttab);
+    }
+    cp_async_commit();
+    cp_async_wait_all();
+    if (it > 0) mbar_drain(bar_q, (it - 1) & 1);
+  } else {
+    constexpr int CPR = D / 8;
+    // ================= K / V streamer: key tiles of all items through the stage ring ====================
+    // Tiles of consecutive rows: lane 0 issues one TMA box per 64 columns.  Gathered tiles: lane ->
+    // column chunk cc and the row quads {4 (rq + k R) .. + 3}, R = 32 / CPR; the four row
+    // coordinates of a quad come with one shared-memory load, and the swizzled destination of
+    // every copy is the lane's base plus a compile-time offset (the swizzle phase (row & 7) of
+    // row e of a quad is 4 (rq & 1) + e for every quad of the lane, R being even).
+    bool ok = true;
+    int gbase = 0;
+    int it = 0;
+    int k_armed = 0, v_armed = 0;                         // tiles whose K / V copies have been issued (all items)
+    constexpr int R = 32 / CPR;                            // row quads covered by the warp per step
+    constexpr int QUADS = (TK / 4) / R;                    // steps per tile
+    const int cc = lane % CPR, rq = lane / CPR;
+    uint32_t doff[4];
 #pragma unroll
-        for (int k = 0; k < PER; ++k) {
-          const int row = (lt + k * kLoaderThreads) / CPR;
-          if (t.mode == 1) gr[k] = s_kidx[kt * TK + row];
-          else { const int r = kt * TK + row; gr[k] = r < t.nk ? t.k0 + r : -1; }
-        }
-#pragma unroll
-        for (int k = 0; k < PER; ++k) {
-          const int c = lt + k * kLoaderThreads;
-          const int row = c / CPR, cc = c % CPR;
-          const uint32_t d = dst + tile_off<TK>(row, cc);
-          if (gr[k] >= 0) cp_async16(d, src + (size_t)gr[k] * D + cc * 8);
-          else cp_async16_zero(d, src);
-        }
-      };
+    for (int e = 0; e < 4; ++e)
+      doff[e] = (uint32_t)((cc >> 3) * (TK * 128) + (4 * rq + e) * 128 + (((cc & 7) ^ ((4 * rq + e) & 7)) << 4));
+    const char* ksrc = reinterpret_cast<const char*>(a.k) + cc * 16;
+    const char* vsrc = reinterpret_cast<const char*>(a.v) + cc * 16;
+    for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+      PairDesc t; QTile qa, qb;
+      decode_pair(a, item, t, qa, qb);
+      const int set = it & 1;
+      const int* s_kidx = s_kidx_all + set * kMaxNodeKeys;
+      ok = mbar_wait<100, 18>(bar_tabfull(set), (it >> 1) & 1, s_abort, status);
+      if (!ok) break;
+      const int segrow = t.seg * g.n;
       for (int j = 0; j < t.ntiles && ok; ++j) {
         const int gj = gbase + j;
         const int s = gj % C::NS;
         const int use = gj / C::NS;
+        int4 rows[QUADS];
+        if (t.mode == 1) {
+#pragma unroll
+          for (int k = 0; k < QUADS; ++k) rows[k] = *reinterpret_cast<const int4*>(s_kidx + j * TK + 4 * (rq + k * R));
+        }
+        auto fill = [&](uint32_t stage, const CUtensorMap* map, const char* src, uint32_t bar) {
+          if (t.mode == 0) {
+            // (rows past the end of the key range are masked by the softmax warps)
+            if (lane == 0) {
+              mbar_expect_tx(bar, C::kTile);
+#pragma unroll
+              for (int sl = 0; sl < D / 64; ++sl) tma_tile(stage + sl * (TK * 128), map, sl * 64, segrow + t.k0 + j * TK, bar);
+            }
+            mbar_arrive(bar);
+          } else {
+#pragma unroll
+            for (int k = 0; k < QUADS; ++k) {
+              const uint32_t d = stage + k * (4 * R * 128);
+              cp_async16(d + doff[0], src + (size_t)(uint32_t)rows[k].x * (D * 2));
+              cp_async16(d + doff[1], src + (size_t)(uint32_t)rows[k].y * (D * 2));
+              cp_async16(d + doff[2], src + (size_t)(uint32_t)rows[k].z * (D * 2));
+              cp_async16(d + doff[3], src + (size_t)(uint32_t)rows[k].w * (D * 2));
+            }
+            cp_async_arrive_noinc(bar);
+          }
+        };
         HA_T0(tle);
         if (use > 0) {
           ok = mbar_wait<100, 10>(bar_kempty(0, s), (use - 1) & 1, s_abort, status);
           ok = ok && mbar_wait<100, 11>(bar_kempty(1, s), (use - 1) & 1, s_abort, status);
           if (!ok) break;
         }
-        if (lt == 0) HA_TACC(11, tle);
+        if (lane == 0) HA_TACC(11, tle);
         HA_T0(tgk);
-        gather_kv(ubase + C::kOffK + s * C::kTile, ks, j);
-        cp_async_arrive_noinc(bar_kfull(s));
-        if (lt == 0) HA_TACC(3, tgk);
+        fill(ubase + C::kOffK + s * C::kTile, &maps.k, ksrc, bar_kfull(s));
+        k_armed = gj + 1;
+        if (lane == 0) HA_TACC(3, tgk);
         HA_T0(tle2);
         if (use > 0) {
           ok = mbar_wait<100, 12>(bar_vempty(0, s), (use - 1) & 1, s_abort, status);
           ok = ok && mbar_wait<100, 13>(bar_vempty(1, s), (use - 1) & 1, s_abort, status);
           if (!ok) break;
         }
-        if (lt == 0) HA_TACC(11, tle2);
+        if (lane == 0) HA_TACC(11, tle2);
         HA_T0(tgv);
-        gather_kv(ubase + C::kOffV + s * C::kTile, vs, j);
-        cp_async_arrive_noinc(bar_vfull(s));
-        if (lt == 0) HA_TACC(1, tgv);
+        fill(ubase + C::kOffV + s * C::kTile, &maps.v, vsrc, bar_vfull(s));
+        v_armed = gj + 1;
+        if (lane == 0) HA_TACC(1, tgv);
       }
+      if (!ok) break;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tabfree(set));       // done reading this item's key rows
       gbase += t.ntiles;
     }
+    // nothing may be in flight into shared memory when the CTA exits (trivially true unless it is giving up)
     cp_async_commit();
-    cp_async_wait_le(0);      // nothing of this thread is in flight when the CTA tears down
+    cp_async_wait_all();
+    for (int s = 0; s < C::NS; ++s) {
+      if (k_armed > s) mbar_drain(bar_kfull(s), ((k_armed - 1 - s) / C::NS) & 1);   // phase of the last tile that used stage s
+      if (v_armed > s) mbar_drain(bar_vfull(s), ((v_armed - 1 - s) / C::NS) & 1);
+    }
   }
 
   // ---- teardown ------------------------------------------------------------------------------------
@@ -1035,21 +1097,57 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 
 #ifdef HA_TC_TIMING
 extern "C" int hyperattn_debug_tc_timing(unsigned long long* host16, int reset) {
-  if (cudaMemcpyFromSymbol(host16, g_tc_timing, sizeof(unsigned long long) * 24) != cudaSuccess) return -5;
-  if (reset) { unsigned long long z[24] = {0}; cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)); }
+  if (cudaMemcpyFromSymbol(host16, g_tc_timing, sizeof(unsigned long long) * 32) != cudaSuccess) return -5;
+  if (reset) { unsigned long long z[32] = {0}; cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)); }
   return 0;
 }
 #endif
 
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// the driver's tensor-map encoder, looked up through the runtime (no link against libcuda)
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// [rows x d] bf16, row-major; one box = 64 columns x box_rows rows (one slab of an operand tile)
+bool encode_rows_map(CUtensorMap* m, const void* base, size_t rows, int d, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st) {
   if (a.total_pairs == 0) return cudaSuccess;
+  const size_t rows = (size_t)a.g.G * a.g.n;
+  if (rows > 0x7fffffffull) return cudaErrorInvalidValue;        // row coordinates are 32-bit
+  TmaMaps maps;
+  if (!encode_rows_map(&maps.q, a.q, rows, a.g.d, 128) || !encode_rows_map(&maps.k, a.k, rows, a.g.d, TK) ||
+      !encode_rows_map(&maps.v, a.v, rows, a.g.d, TK)) return cudaErrorInvalidValue;
   auto go = [&](auto kernel, int smem_bytes) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
     int grid = a.total_pairs < sms ? a.total_pairs : sms;     // persistent: one CTA per SM walks the item list
-    kernel<<<grid, 384, smem_bytes, st>>>(a, status);
+    kernel<<<grid, 384, smem_bytes, st>>>(a, maps, status);
     return cudaGetLastError();
   };
   if (a.g.d == 64) return go(attn_tc_kernel<64>, Cfg<64>::kTotal);
