@@ -500,7 +500,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 
   // ---- setup: barriers, TMEM ---------------------------------------------------------------------
   if (tid == 0) {
-    mbar_init(bar_q, 32);
+    mbar_init(bar_q, 32 + 256);                         // item preparer + softmax threads
     mbar_init(bar_qfree, 2);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_o(i), 1);
@@ -540,6 +540,40 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     int vi = 0;                                       // items in which this query tile existed
     bool ok = true;
     int it = 0;
+    // Gathered Q tiles (sorted rows) are fetched by the 256 softmax threads together, 16-byte
+    // chunks through cp.async: one warp alone is limited by the copies it can keep in flight.
+    // Thread -> column chunk cq of rows rq0, rq0 + 256 / CPR, ...; its arrival on the Q barrier
+    // is attached to its copies.  (Tiles of consecutive rows are one TMA box, issued by the
+    // item preparer; then the arrival here is immediate.)
+    auto gather_q = [&](int nitem, int nit) {
+      PairDesc t; QTile qa, qb;
+      decode_pair(a, nitem, t, qa, qb);
+      bool good = mbar_wait<20, 19>(bar_tabfull(nit & 1), (nit >> 1) & 1, s_abort, status);
+      if (good && nit >= 1) good = mbar_wait<20, 20>(bar_qfree, (nit - 1) & 1, s_abort, status);
+      if (!good) return false;
+      if (t.mode == 1) {
+        constexpr int CPR = D / 8;
+        constexpr int RS = 256 / CPR;                       // rows covered by the 256 threads per step
+        const int cq = tid % CPR, rq0 = tid / CPR;
+        const char* qsrc = reinterpret_cast<const char*>(a.q) + (size_t)t.seg * g.n * (D * 2) + cq * 16;
+        const int* rows = s_qrow_all + (nit & 1) * 2 * 128;
+#pragma unroll
+        for (int ti = 0; ti < 2; ++ti) {
+          if (!(ti ? qb.valid : qa.valid)) continue;       // nobody reads the tile of a query tile that does not exist
+          int v[128 / RS];
+#pragma unroll
+          for (int k = 0; k < 128 / RS; ++k) v[k] = rows[ti * 128 + rq0 + k * RS];
+#pragma unroll
+          for (int k = 0; k < 128 / RS; ++k)               // padding rows: the segment's first row (results never stored)
+            cp_async16(ubase + C::kOffQ + ti * C::kQTile + tile_off<128>(rq0 + k * RS, cq), qsrc + (size_t)(uint32_t)max(v[k], 0) * (D * 2));
+        }
+        cp_async_arrive_noinc(bar_q);
+      } else {
+        mbar_arrive(bar_q);
+      }
+      return true;
+    };
+    if (blockIdx.x < a.total_pairs) ok = __all_sync(0xffffffffu, gather_q(blockIdx.x, 0));
     for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
       PairDesc t; QTile qa, qb;
       decode_pair(a, item, t, qa, qb);
@@ -672,6 +706,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 #endif
       }
       if (!ok) break;
+      // the next item's Q tiles go out before this item's results are written
+      if (item + (int)gridDim.x < a.total_pairs) {
+        ok = __all_sync(0xffffffffu, gather_q(item + gridDim.x, it + 1));
+        if (!ok) break;
+      }
       HA_T0(te);
       // epilogue: normalise, log-sum-exp, rows back to their original places
       if (q.valid) {
@@ -947,10 +986,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       if (lane == 0) mbar_arrive(bar_tabfull(set));       // (release: the table writes of all lanes are ordered before it by the warp barrier)
       if (lane == 0) HA_TACC(10, ttab);
       // ---- Q (the issuers must be done with the previous item's Q) ----------------------------
+      HA_T0(tqf);
       if (it >= 1) {
         ok = mbar_wait<100, 17>(bar_qfree, (it - 1) & 1, s_abort, status);
         if (!ok) break;
       }
+      if (lane == 0) HA_TACC(27, tqf);
+      HA_T0(tqi);
       if (t.mode == 0) {
         // consecutive rows: one box per 64 columns and tile (rows past the tile's end are other
         // rows of the tensor or zeros: their results are never stored)
@@ -966,24 +1008,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
         mbar_arrive(bar_q);
       } else {
-        // gathered rows: lane -> column chunk cc and rows rq, rq + 32 / CPR, ... ; padding rows
-        // fetch the segment's first row (finite values whose results are never stored)
-        const int cc = lane % CPR, rq = lane / CPR;
-        const char* qsrc = reinterpret_cast<const char*>(a.q) + cc * 16;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          if (!(i ? qb.valid : qa.valid)) continue;      // nobody reads the tile of a query tile that does not exist
-          const uint32_t dbase = ubase + C::kOffQ + i * C::kQTile + (cc >> 3) * (128 * 128);
-          const int* rows = s_qrow + i * 128;
-#pragma unroll 4
-          for (int r = rq; r < 128; r += 32 / CPR) {
-            const int v = rows[r];
-            cp_async16(dbase + r * 128 + (((cc & 7) ^ (r & 7)) << 4), qsrc + (size_t)(uint32_t)(segrow + (v < 0 ? 0 : v)) * (D * 2));
-          }
-        }
-        cp_async_arrive_noinc(bar_q);
+        mbar_arrive(bar_q);                               // (the softmax threads gather these tiles)
       }
-      if (lane == 0) HA_TACC(25, ttab);
+      if (lane == 0) { HA_TACC(25, ttab); HA_TACC(28, tqi); }
     }
     cp_async_commit();
     cp_async_wait_all();
