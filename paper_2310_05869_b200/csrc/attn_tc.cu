@@ -308,29 +308,6 @@ __device__ __noinline__ void rescale_row(uint32_t o_addr, int ocols, float alpha
   tmem_wait_st();
 }
 
-// one 32-column chunk of a normalised output row to its place (fp32 partial / fp32 out / bf16 out)
-__device__ __forceinline__ void store_row_chunk(const AttnArgs& a, int partial, size_t orow, int D, int col0,
-                                                const uint32_t (&r)[32], float inv) {
-  if (partial || a.out_fp32) {
-    float* dst = (partial ? a.part_o : reinterpret_cast<float*>(a.out)) + orow * D + col0;
-#pragma unroll
-    for (int e = 0; e < 32; e += 4)
-      *reinterpret_cast<float4*>(dst + e) = make_float4(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv,
-                                                        __uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-  } else {
-    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.out) + orow * D + col0;
-#pragma unroll
-    for (int e = 0; e < 32; e += 8) {
-      uint4 v;
-      v.x = pack2(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-      v.y = pack2(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-      v.z = pack2(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-      v.w = pack2(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-      *reinterpret_cast<uint4*>(dst + e) = v;
-    }
-  }
-}
-
 template <int D>
 struct Cfg {
   static constexpr int NS = (D == 64) ? 8 : 4;        // K stages and V stages
@@ -346,7 +323,16 @@ struct Cfg {
   static constexpr int kOffBar = kOffQrow + 4 * 128 * 4;
   static constexpr int kNumBar = 21 + 6 * NS;          // (slot 20 unused)
   static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
-  static constexpr int kTotal = kOffMisc + 16;
+  // Epilogue staging, one slice of 32 rows x kStageRow bytes per softmax warp: rows leave the
+  // warp as whole 64- or 128-byte pieces instead of 16 bytes per lane and row.  d = 64: eight
+  // slices of 4 KB.  d = 128 (less shared memory to spare): slices of 2 KB, those of query tile
+  // 0 in the item's own key-row table, which nobody reads any more once the item's last K / V
+  // tile has been issued and which is not rebuilt before the softmax warps release the set.
+  static constexpr int kStageRow = (D == 64) ? 128 : 64;
+  static constexpr int kStageWarp = 32 * kStageRow;
+  static constexpr int kOffStage = (kOffMisc + 16 + 127) / 128 * 128;
+  static constexpr int kTotal = kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;
+  static_assert(D == 64 || 4 * kStageWarp <= kMaxNodeKeys * 4, "staging of query tile 0 must fit one key-row table");
   static constexpr int kTmemCols = 512;
   static constexpr int kColO = 256;                   // S buffer b of tile i at 64 (2 i + b); O_i at kColO + D i
 };
@@ -724,26 +710,63 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         const float inv = 1.f / (lr0 + lr1);
         const float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
         const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
-        if (D == 64) {
-          // read everything, free O for the next item at once, then write
-          uint32_t r0[32], r1[32];
-          tmem_ld32_issue(lane_addr + colO, r0);
-          tmem_ld32_issue(lane_addr + colO + 32, r1);
-          tmem_ld32_wait(r0);
-          tmem_ld32_wait(r1);
-          tc_fence_before();
-          mbar_arrive(bar_ofree(i));
-          if (qr >= 0) {
-            store_row_chunk(a, t.partial, orow, D, 0, r0, inv);
-            store_row_chunk(a, t.partial, orow, D, 32, r1, inv);
-          }
-        } else {
+        {
+          // O leaves TMEM in pieces of 16 columns (thread = row), is normalised (and rounded to
+          // bf16 for a bf16 result) and staged in shared memory, XOR-swizzled so that neither
+          // side has bank conflicts; then LPR lanes per row write kStageRow contiguous bytes of
+          // RPI rows per instruction.
+          constexpr int RB = C::kStageRow;
+          constexpr int LPR = RB / 16, RPI = 32 / LPR, NI = 32 / RPI;
+          constexpr int NP = D / 16;
+          const bool f32o = t.partial || a.out_fp32;
+          char* obase = f32o ? reinterpret_cast<char*>(t.partial ? a.part_o : reinterpret_cast<float*>(a.out)) : reinterpret_cast<char*>(a.out);
+          const long long myoff = qr >= 0 ? (long long)(orow * (size_t)(D * (f32o ? 4 : 2))) : -1;
+          long long roff[NI];
+#pragma unroll
+          for (int k = 0; k < NI; ++k) roff[k] = __shfl_sync(0xffffffffu, myoff, RPI * k + lane / LPR);
+          const uint32_t stg = (D == 64) ? ubase + C::kOffStage + warp * C::kStageWarp
+                             : (i == 0 ? ubase + C::kOffIdx + set * (kMaxNodeKeys * 4) : ubase + C::kOffStage) + (warp & 3) * C::kStageWarp;
+          const int xw = (RB == 128) ? (lane & 7) : ((lane >> 1) & 3);       // swizzle of this thread's own row
+          const int crow = lane / LPR, cc = lane % LPR;
+          const int lg_pps = f32o ? (RB == 128 ? 1 : 0) : (RB == 128 ? 2 : 1);   // log2(pieces per staging step)
+          uint32_t r[16];
+          tmem_ld16_issue(lane_addr + colO, r);
 #pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(lane_addr + colO + c * 32, r);
-            if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar_ofree(i)); }
-            if (qr >= 0) store_row_chunk(a, t.partial, orow, D, c * 32, r, inv);
+          for (int pc = 0; pc < NP; ++pc) {
+            tmem_ld16_wait(r);
+            float f[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(r[e]) * inv;
+            if (pc + 1 < NP) tmem_ld16_issue(lane_addr + colO + (pc + 1) * 16, r);
+            else { tc_fence_before(); mbar_arrive(bar_ofree(i)); }           // O has been read: the next item may overwrite it
+            const int pin = pc & ((1 << lg_pps) - 1);
+            const uint32_t srow = stg + lane * RB;
+            if (f32o) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(srow + (((pin * 4 + c) ^ xw) << 4)),
+                             "f"(f[4 * c]), "f"(f[4 * c + 1]), "f"(f[4 * c + 2]), "f"(f[4 * c + 3]) : "memory");
+            } else {
+#pragma unroll
+              for (int c = 0; c < 2; ++c)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(srow + (((pin * 2 + c) ^ xw) << 4)),
+                             "r"(pack2(f[8 * c], f[8 * c + 1])), "r"(pack2(f[8 * c + 2], f[8 * c + 3])),
+                             "r"(pack2(f[8 * c + 4], f[8 * c + 5])), "r"(pack2(f[8 * c + 6], f[8 * c + 7])) : "memory");
+            }
+            if (pin == (1 << lg_pps) - 1) {
+              __syncwarp();
+              const int step = pc >> lg_pps;
+#pragma unroll
+              for (int k = 0; k < NI; ++k) {
+                const int rw = RPI * k + crow;
+                const int xr = (RB == 128) ? (rw & 7) : ((rw >> 1) & 3);
+                uint4 w;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                             : "r"(stg + rw * RB + ((cc ^ xr) << 4)) : "memory");
+                if (roff[k] >= 0) *reinterpret_cast<uint4*>(obase + roff[k] + step * RB + cc * 16) = w;
+              }
+              __syncwarp();
+            }
           }
         }
         if (qr >= 0) {
