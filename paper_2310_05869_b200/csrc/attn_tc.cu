@@ -53,9 +53,15 @@ constexpr float kRescaleThreshold = 32.f;   // octaves the scores may exceed the
 __device__ unsigned long long g_tc_timing[32];
 #define HA_T0(var) const long long var = clock64()
 #define HA_TACC(slot, var) atomicAdd(&g_tc_timing[slot], (unsigned long long)(clock64() - var))
+#define HA_LDECL(name) long long name = 0
+#define HA_LACC(name, var) name += clock64() - var
+#define HA_LFLUSH(slot, name) atomicAdd(&g_tc_timing[slot], (unsigned long long)(name))
 #else
 #define HA_T0(var)
 #define HA_TACC(slot, var)
+#define HA_LDECL(name)
+#define HA_LACC(name, var)
+#define HA_LFLUSH(slot, name)
 #endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -308,35 +314,6 @@ __device__ __noinline__ void rescale_row(uint32_t o_addr, int ocols, float alpha
   tmem_wait_st();
 }
 
-template <int D>
-struct Cfg {
-  static constexpr int NS = (D == 64) ? 8 : 4;        // K stages and V stages
-  static constexpr int kQTile = 128 * D * 2;          // bytes of one 128-row query tile
-  static constexpr int kTile = TK * D * 2;            // bytes of one key / value tile
-  static constexpr int kOffQ = 0;                     // Q0, Q1
-  static constexpr int kOffK = 2 * kQTile;
-  static constexpr int kOffV = kOffK + NS * kTile;
-  // row tables, two sets (the loaders build the set of the next work item while this one runs)
-  static constexpr int kOffIdx = kOffV + NS * kTile;              // int [2][kMaxNodeKeys] key rows
-  static constexpr int kOffMask = kOffIdx + 2 * kMaxNodeKeys * 4; // uint32 [2][2][kMaxNodeKeys/32] masked-column bits
-  static constexpr int kOffQrow = kOffMask + 4 * (kMaxNodeKeys / 32) * 4;   // int [2][2][128]
-  static constexpr int kOffBar = kOffQrow + 4 * 128 * 4;
-  static constexpr int kNumBar = 21 + 6 * NS;          // (slot 20 unused)
-  static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
-  // Epilogue staging, one slice of 32 rows x kStageRow bytes per softmax warp: rows leave the
-  // warp as whole 64- or 128-byte pieces instead of 16 bytes per lane and row.  d = 64: eight
-  // slices of 4 KB.  d = 128 (less shared memory to spare): slices of 2 KB, those of query tile
-  // 0 in the item's own key-row table, which nobody reads any more once the item's last K / V
-  // tile has been issued and which is not rebuilt before the softmax warps release the set.
-  static constexpr int kStageRow = (D == 64) ? 128 : 64;
-  static constexpr int kStageWarp = 32 * kStageRow;
-  static constexpr int kOffStage = (kOffMisc + 16 + 127) / 128 * 128;
-  static constexpr int kTotal = kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;
-  static_assert(D == 64 || 4 * kStageWarp <= kMaxNodeKeys * 4, "staging of query tile 0 must fit one key-row table");
-  static constexpr int kTmemCols = 512;
-  static constexpr int kColO = 256;                   // S buffer b of tile i at 64 (2 i + b); O_i at kColO + D i
-};
-
 // One query tile of the pair.  The key tiles it looks at are two runs of the pair's tile
 // list: [s1, s1 + n1) and [s2, s2 + n2).
 struct QTile {
@@ -360,6 +337,43 @@ struct PairDesc {
   int nbA, nbB, nsmp;  // node: key tiles of block A, of block B (0 if shared), of the samples
   int ntiles;          // key tiles walked
   size_t orow_base; int odelta; int partial;
+};
+
+// what every role needs to know about a work item; decoded once, by the item preparer
+struct ItemDesc {
+  PairDesc t;
+  QTile qa, qb;
+};
+
+template <int D>
+struct Cfg {
+  static constexpr int NS = (D == 64) ? 8 : 4;        // K stages and V stages
+  static constexpr int kQTile = 128 * D * 2;          // bytes of one 128-row query tile
+  static constexpr int kTile = TK * D * 2;            // bytes of one key / value tile
+  static constexpr int kOffQ = 0;                     // Q0, Q1
+  static constexpr int kOffK = 2 * kQTile;
+  static constexpr int kOffV = kOffK + NS * kTile;
+  // row tables, two sets (the loaders build the set of the next work item while this one runs)
+  static constexpr int kOffIdx = kOffV + NS * kTile;              // int [2][kMaxNodeKeys] key rows
+  static constexpr int kOffMask = kOffIdx + 2 * kMaxNodeKeys * 4; // uint32 [2][2][kMaxNodeKeys/32] masked-column bits
+  static constexpr int kOffQrow = kOffMask + 4 * (kMaxNodeKeys / 32) * 4;   // int [2][2][128]
+  static constexpr int kOffBar = kOffQrow + 4 * 128 * 4;
+  static constexpr int kNumBar = 21 + 6 * NS;          // (slot 20 unused)
+  static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
+  // Epilogue staging, one slice of 32 rows x kStageRow bytes per softmax warp: rows leave the
+  // warp as whole 64- or 128-byte pieces instead of 16 bytes per lane and row.  d = 64: eight
+  // slices of 4 KB.  d = 128 (less shared memory to spare): slices of 2 KB, those of query tile
+  // 0 in the item's own key-row table, which nobody reads any more once the item's last K / V
+  // tile has been issued and which is not rebuilt before the softmax warps release the set.
+  static constexpr int kStageRow = (D == 64) ? 128 : 64;
+  static constexpr int kStageWarp = 32 * kStageRow;
+  static constexpr int kDescBytes = (sizeof(ItemDesc) + 15) / 16 * 16;
+  static constexpr int kOffDesc = (kOffMisc + 16 + 15) / 16 * 16;   // ItemDesc [2], one per table set
+  static constexpr int kOffStage = (kOffDesc + 2 * kDescBytes + 127) / 128 * 128;
+  static constexpr int kTotal = kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;
+  static_assert(D == 64 || 4 * kStageWarp <= kMaxNodeKeys * 4, "staging of query tile 0 must fit one key-row table");
+  static constexpr int kTmemCols = 512;
+  static constexpr int kColO = 256;                   // S buffer b of tile i at 64 (2 i + b); O_i at kColO + D i
 };
 
 __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDesc& t, QTile& qa, QTile& qb) {
@@ -531,12 +545,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     // Thread -> column chunk cq of rows rq0, rq0 + 256 / CPR, ...; its arrival on the Q barrier
     // is attached to its copies.  (Tiles of consecutive rows are one TMA box, issued by the
     // item preparer; then the arrival here is immediate.)
-    auto gather_q = [&](int nitem, int nit) {
-      PairDesc t; QTile qa, qb;
-      decode_pair(a, nitem, t, qa, qb);
+    auto gather_q = [&](int nit) {
       bool good = mbar_wait<20, 19>(bar_tabfull(nit & 1), (nit >> 1) & 1, s_abort, status);
       if (good && nit >= 1) good = mbar_wait<20, 20>(bar_qfree, (nit - 1) & 1, s_abort, status);
       if (!good) return false;
+      const ItemDesc& de = *reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + (nit & 1) * C::kDescBytes);
+      const PairDesc& t = de.t;
+      const QTile &qa = de.qa, &qb = de.qb;
       if (t.mode == 1) {
         constexpr int CPR = D / 8;
         constexpr int RS = 256 / CPR;                       // rows covered by the 256 threads per step
@@ -559,12 +574,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       }
       return true;
     };
-    if (blockIdx.x < a.total_pairs) ok = __all_sync(0xffffffffu, gather_q(blockIdx.x, 0));
+    HA_LDECL(a_tab); HA_LDECL(a_ws); HA_LDECL(a_cmp); HA_LDECL(a_epi); HA_LDECL(a_gq); HA_LDECL(a_bo); HA_LDECL(a_tiles);
+    HA_T0(t_role);
+    if (blockIdx.x < a.total_pairs) ok = __all_sync(0xffffffffu, gather_q(0));
     for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
-      PairDesc t; QTile qa, qb;
-      decode_pair(a, item, t, qa, qb);
-      const QTile q = i ? qb : qa;
-      const int total = q.n1 + q.n2;
       const int set = it & 1;
       const uint32_t* s_mask = s_mask_all + (set * 2 + i) * MW;
       const int* s_qrow = s_qrow_all + (set * 2 + i) * 128;
@@ -572,7 +585,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       HA_T0(tt);
       ok = __all_sync(0xffffffffu, mbar_wait<20, 14>(bar_tabfull(set), (it >> 1) & 1, s_abort, status));
       if (!ok) break;
-      if (row == 0 && i == 0) HA_TACC(9, tt);
+      HA_LACC(a_tab, tt);
+      const ItemDesc& de = *reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes);
+      const PairDesc t = de.t;
+      const QTile q = i ? de.qb : de.qa;
+      const int total = q.n1 + q.n2;
       const float wlog = (t.mode == 1 && g.m > 0) ? log2f((float)t.nk / (float)g.m) : 0.f;   // log2(N/m): weight of a sampled column
       float m_ref = -INFINITY;
       uint64_t l01 = 0, lr01 = 0;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each, packed)
@@ -583,7 +600,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         HA_T0(tw);
         ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (gw >> 1) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
         if (!ok) break;
-        if (row == 0 && i == 0) HA_TACC(0, tw);
+        HA_LACC(a_ws, tw);
         HA_T0(tc);
         tc_fence_after();
         // mask kind of this (query tile, key tile): uniform over the warpgroup
@@ -616,8 +633,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
         tmem_ld32_wait(ra);
         tmem_ld32_wait(rb);
-        if (row == 0 && i == 0) HA_TACC(16, tc);
-        HA_T0(tm);
         // masked columns become -inf once, here: they then drop out of the maximum and
         // exponentiate to zero without further tests
         if (masked_tile) {
@@ -661,8 +676,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           }
         }
         const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
-        if (row == 0 && i == 0) HA_TACC(17, tm);
-        HA_T0(tx);
         // packed fp32 arithmetic (two lanes per instruction) for the scaling and the two row sums
         const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2), off2 = pack_f2(off, off);
         auto chunk_exp = [&](const uint32_t (&r)[32], int c) {
@@ -681,27 +694,28 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         };
         chunk_exp(ra, 0);
         chunk_exp(rb, 1);
-        if (row == 0 && i == 0) HA_TACC(18, tx);
-        HA_T0(ts);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p(i, buf));
-        if (row == 0 && i == 0) { HA_TACC(2, tc); HA_TACC(19, ts); }
+        HA_LACC(a_cmp, tc);
 #ifdef HA_TC_TIMING
-        if (row == 0 && i == 0) atomicAdd(&g_tc_timing[20], 1ull);
+        a_tiles += 1;
 #endif
       }
       if (!ok) break;
       // the next item's Q tiles go out before this item's results are written
+      HA_T0(tg);
       if (item + (int)gridDim.x < a.total_pairs) {
-        ok = __all_sync(0xffffffffu, gather_q(item + gridDim.x, it + 1));
+        ok = __all_sync(0xffffffffu, gather_q(it + 1));
         if (!ok) break;
       }
+      HA_LACC(a_gq, tg);
       HA_T0(te);
       // epilogue: normalise, log-sum-exp, rows back to their original places
       if (q.valid) {
         ok = __all_sync(0xffffffffu, mbar_wait<20, 5>(bar_o(i), vi & 1, s_abort, status));
         if (!ok) break;
+        HA_LACC(a_bo, te);
         tc_fence_after();
         const int qr = s_qrow[row];
         float l0, l1, lr0, lr1;
@@ -776,9 +790,15 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         ++vi;
       }
       mbar_arrive(bar_tabfree(set));
-      if (row == 0 && i == 0) HA_TACC(15, te);
+      HA_LACC(a_epi, te);
       ga += total;
     }
+#ifdef HA_TC_TIMING
+    if (row == 0 && i == 0) {
+      HA_LFLUSH(9, a_tab); HA_LFLUSH(0, a_ws); HA_LFLUSH(2, a_cmp); HA_LFLUSH(15, a_epi); HA_LFLUSH(16, a_gq); HA_LFLUSH(17, a_bo);
+      HA_LFLUSH(20, a_tiles); HA_TACC(18, t_role); HA_LFLUSH(19, it);
+    }
+#endif
   } else if (warp < 10) {
     // ================= MMA issue: one lane per query tile (warp 8: tile 0, warp 9: tile 1) ===========
     // Each issuer walks its own key tiles: scores run two tiles ahead of the PV products
@@ -823,20 +843,23 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
       };
       int it = 0;
+      HA_LDECL(b_q); HA_LDECL(b_p); HA_LDECL(b_v); HA_LDECL(b_k);
       HA_T0(tloop);
       for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
-        PairDesc t; QTile qa, qb;
-        decode_pair(a, item, t, qa, qb);
-        const QTile q = i ? qb : qa;
+        ok = wait_fast<22>(bar_tabfull(it & 1), (it >> 1) & 1, s_abort, status);
+        if (!ok) break;
+        const ItemDesc& de = *reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + (it & 1) * C::kDescBytes);
+        const QTile q = i ? de.qb : de.qa;
         const int total = q.n1 + q.n2;
+        const int ntiles = de.t.ntiles;
 #ifdef HA_TC_TIMING
-        if (i == 0) atomicAdd(&g_tc_timing[14], (unsigned long long)t.ntiles);
+        if (i == 0) atomicAdd(&g_tc_timing[14], (unsigned long long)ntiles);
 #endif
         // Q of this item (an issuer without a tile waits too: it may not run ahead of the others)
         HA_T0(tq);
         ok = wait_fast<6>(bar_q, it & 1, s_abort, status);
         if (!ok) break;
-        if (i == 0) HA_TACC(7, tq);
+        HA_LACC(b_q, tq);
         fence_async_smem();
         if (total == 0) mbar_arrive(bar_qfree);
         for (int r = 0; r < total + 2 && ok; ++r) {
@@ -849,10 +872,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             if (gj != vnext) skip_v(gj);
             HA_T0(tp);
             ok = ok && wait_fast<8>(bar_p(i, gw & 1), (gw >> 1) & 1, s_abort, status);
-            if (i == 0) HA_TACC(4, tp);
+            HA_LACC(b_p, tp);
             HA_T0(tv);
             ok = ok && wait_fast<9>(bar_vfull(s), (gj / C::NS) & 1, s_abort, status);
-            if (i == 0) HA_TACC(5, tv);
+            HA_LACC(b_v, tv);
             // the first product of an item overwrites O: the previous item's O must have been read
             if (a2 == 0 && vi > 0) ok = ok && wait_fast<15>(bar_ofree(i), (vi - 1) & 1, s_abort, status);
             if (!ok) break;
@@ -877,7 +900,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             if (gj != knext) skip_k(gj);
             HA_T0(tk);
             ok = ok && wait_fast<7>(bar_kfull(s), (gj / C::NS) & 1, s_abort, status);
-            if (i == 0) HA_TACC(6, tk);
+            HA_LACC(b_k, tk);
             if (!ok) break;
             fence_async_smem();
             tc_fence_after();
@@ -894,13 +917,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           }
         }
         if (!ok) break;
-        skip_k(gbase + t.ntiles);
-        skip_v(gbase + t.ntiles);
-        gbase += t.ntiles;
+        skip_k(gbase + ntiles);
+        skip_v(gbase + ntiles);
+        gbase += ntiles;
         ga += total;
         vi += q.valid;
       }
-      if (i == 0) { HA_TACC(8, tloop); HA_TACC(12, t_cta); }
+      if (i == 0) { HA_TACC(8, tloop); HA_TACC(12, t_cta); HA_LFLUSH(7, b_q); HA_LFLUSH(4, b_p); HA_LFLUSH(5, b_v); HA_LFLUSH(6, b_k); }
 #ifdef HA_TC_TIMING
       if (i == 0) atomicAdd(&g_tc_timing[13], 1ull);
 #endif
@@ -929,6 +952,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         if (!ok) break;
       }
       if (lane == 0) HA_TACC(21, ttab);
+      if (lane == 0) {
+        ItemDesc* de = reinterpret_cast<ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes);
+        de->t = t; de->qa = qa; de->qb = qb;
+      }
       const int segrow = t.seg * g.n;                       // row coordinate of the segment's first row
       // Key rows as tensor-map row coordinates.  Every global load of a batch is issued before
       // the first one is used; the warp covers 32 consecutive columns per step, so one ballot
@@ -1060,12 +1087,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     const char* ksrc = reinterpret_cast<const char*>(a.k) + cc * 16;
     const char* vsrc = reinterpret_cast<const char*>(a.v) + cc * 16;
     for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
-      PairDesc t; QTile qa, qb;
-      decode_pair(a, item, t, qa, qb);
       const int set = it & 1;
       const int* s_kidx = s_kidx_all + set * kMaxNodeKeys;
       ok = mbar_wait<100, 18>(bar_tabfull(set), (it >> 1) & 1, s_abort, status);
       if (!ok) break;
+      const PairDesc t = reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes)->t;
       const int segrow = t.seg * g.n;
       for (int j = 0; j < t.ntiles && ok; ++j) {
         const int gj = gbase + j;
