@@ -297,6 +297,28 @@ __device__ __forceinline__ uint32_t tile_off(int row, int c) {
   return (uint32_t)((c >> 3) * (ROWS * 128) + row * 128 + (((c & 7) ^ (row & 7)) << 4));
 }
 
+// Tiles with masked columns (a minority: the diagonal tiles of a causal leaf, padding, sampled
+// columns that fall into the query tile's own block): the masked scores are overwritten with
+// -inf in TMEM before the tile is read, so that the hot loop carries no mask code at all.
+// vis: one bit per column, 1 = visible.  All 32 lanes call it together.
+__device__ __noinline__ void mask_scores(uint32_t sbase, uint32_t visa, uint32_t visb) {
+  uint32_t r[16];
+#pragma unroll 1
+  for (int gcol = 0; gcol < 4; ++gcol) {
+    const uint32_t vis16 = ((gcol < 2 ? visa : visb) >> (16 * (gcol & 1))) & 0xffffu;
+    if (__all_sync(0xffffffffu, vis16 == 0xffffu)) continue;      // warp-uniform: TMEM accesses stay convergent
+    tmem_ld16_issue(sbase + 16 * gcol, r);
+    tmem_ld16_wait(r);
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      if (!((vis16 >> e) & 1u)) r[e] = 0xff800000u;
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+                 ::"r"(sbase + 16 * gcol), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+  }
+  tmem_wait_st();
+}
+
 // Rare path of the online softmax: multiply the O columns a row has accumulated so far by
 // alpha (a power of two, so nothing is re-rounded).  Kept out of line: the hot loop should
 // stay small.  All 32 lanes call it together (TMEM accesses are warp-wide).
@@ -621,27 +643,22 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         // sums) is rescaled exactly.
         uint32_t ra[32], rb[32];
         const uint32_t sbase = lane_addr + 64 * (2 * i + buf);
+        // masked columns become -inf before the tile is read (out of line, in TMEM): they then
+        // drop out of the maximum and exponentiate to zero without any test in this loop
+        if (table || dense_mask) {
+          uint32_t visa, visb;
+          if (table) { visa = ~s_mask[j * 2]; visb = ~s_mask[j * 2 + 1]; }
+          else {
+            const int rel = climit - j * TK;            // columns 0..rel of the tile are visible
+            visa = rel >= 31 ? 0xffffffffu : (rel < 0 ? 0u : ((2u << rel) - 1u));
+            visb = rel >= 63 ? 0xffffffffu : (rel < 32 ? 0u : ((2u << (rel - 32)) - 1u));
+          }
+          mask_scores(sbase, visa, visb);
+        }
         tmem_ld32_issue(sbase, ra);
         tmem_ld32_issue(sbase + 32, rb);
-        const bool masked_tile = table || dense_mask;
-        uint32_t visa = 0xffffffffu, visb = 0xffffffffu;
-        if (table) { visa = ~s_mask[j * 2]; visb = ~s_mask[j * 2 + 1]; }
-        else if (dense_mask) {
-          const int rel = climit - j * TK;              // columns 0..rel of the tile are visible
-          visa = rel >= 31 ? 0xffffffffu : (rel < 0 ? 0u : ((2u << rel) - 1u));
-          visb = rel >= 63 ? 0xffffffffu : (rel < 32 ? 0u : ((2u << (rel - 32)) - 1u));
-        }
         tmem_ld32_wait(ra);
         tmem_ld32_wait(rb);
-        // masked columns become -inf once, here: they then drop out of the maximum and
-        // exponentiate to zero without further tests
-        if (masked_tile) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            if (!((visa >> e) & 1u)) ra[e] = 0xff800000u;
-            if (!((visb >> e) & 1u)) rb[e] = 0xff800000u;
-          }
-        }
         float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
@@ -991,27 +1008,42 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             }
           }
         }
-        // sampled columns: masked where the sample falls into the tile's own block (the factor
-        // (1 - M^H) of Alg. 2 line 7)
-        for (int c00 = nblk + lane; c00 < ncols; c00 += 32 * UB) {
-          int l[UB], blk[UB];
+        // Sampled columns: masked where the sample falls into the tile's own block (the factor
+        // (1 - M^H) of Alg. 2 line 7).  The samples are an unordered multiset, so the masked ones
+        // (for either query tile) are moved to the end of the sample part: only its last tile(s)
+        // then carry mask bits, every other sampled tile takes the softmax warps' fast path.
+        if (nblk < ncols) {
+          for (int wd = (nblk >> 5) + lane; wd < (ncols >> 5); wd += 32) { s_mask[wd] = 0; s_mask[MW + wd] = 0; }
+          __syncwarp();
+          int nfront = 0, nback = 0;                      // unmasked samples placed from the front, masked ones from the back
+          const unsigned lt_mask = (1u << lane) - 1u;
+          for (int c00 = lane; c00 < ncols - nblk; c00 += 32 * UB) {
+            int l[UB], blk[UB];
 #pragma unroll
-          for (int u = 0; u < UB; ++u) {
-            const int c = c00 + u * 32 - nblk;
-            l[u] = (c00 + u * 32 < ncols && c < g.m) ? smp[c] : -1;
-          }
+            for (int u = 0; u < UB; ++u) {
+              const int c = c00 + u * 32;
+              l[u] = c < g.m ? smp[c] : -1;
+            }
 #pragma unroll
-          for (int u = 0; u < UB; ++u) blk[u] = l[u] >= 0 ? rk[l[u]] / g.b : -1;
+            for (int u = 0; u < UB; ++u) blk[u] = l[u] >= 0 ? rk[l[u]] / g.b : -1;
 #pragma unroll
-          for (int u = 0; u < UB; ++u) {
-            const int c0 = c00 + u * 32;
-            if (c0 - lane < ncols) {
-              const bool m0 = l[u] < 0 || blk[u] == qa.beta;
-              const bool m1 = l[u] < 0 || (qb.valid && blk[u] == qb.beta);
-              const unsigned w0 = __ballot_sync(0xffffffffu, m0);
-              const unsigned w1 = __ballot_sync(0xffffffffu, m1);
-              s_kidx[c0] = segrow + (l[u] < 0 ? 0 : t.k0 + l[u]);
-              if (lane == 0) { s_mask[c0 >> 5] = w0; s_mask[MW + (c0 >> 5)] = w1; }
+            for (int u = 0; u < UB; ++u) {
+              const int c = c00 + u * 32;
+              if (c - lane < ncols - nblk) {              // warp-uniform
+                const bool valid = l[u] >= 0;
+                const bool m0 = !valid || blk[u] == qa.beta;
+                const bool m1 = !valid || (qb.valid && blk[u] == qb.beta);
+                const unsigned bf = __ballot_sync(0xffffffffu, valid && !(m0 || m1));
+                const unsigned bb = __ballot_sync(0xffffffffu, valid && (m0 || m1));
+                int pos;
+                if (!valid) pos = nblk + c;                                             // padding stays where it is (behind all samples)
+                else if (!(m0 || m1)) pos = nblk + nfront + __popc(bf & lt_mask);
+                else pos = nblk + g.m - 1 - (nback + __popc(bb & lt_mask));
+                nfront += __popc(bf); nback += __popc(bb);
+                s_kidx[pos] = segrow + (valid ? t.k0 + l[u] : 0);
+                if (m0) atomicOr(&s_mask[pos >> 5], 1u << (pos & 31));
+                if (m1) atomicOr(&s_mask[MW + (pos >> 5)], 1u << (pos & 31));
+              }
             }
           }
         }
