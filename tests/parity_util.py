@@ -120,6 +120,20 @@ def check_perms(w, inter, segs=None):
                 assert (rk[level, g, sl] == rank).all(), ("rank_k", g, level, j)
 
 
+class LazySegments:
+    """Segment-indexed view of a [G, n, d] input array that widens a segment to fp64 only when
+    it is asked for (the full-size workloads are too large to widen as a whole)."""
+
+    def __init__(self, arr):
+        self.arr = arr
+        self.cache = {}
+
+    def __getitem__(self, g):
+        if g not in self.cache:
+            self.cache[g] = WL.as_f64(self.arr[g])
+        return self.cache[g]
+
+
 def oracle_rows(w, Q64, K64, V64, g, rows, ids_q=None, ids_k=None):
     W = O.directions(w.d, w.r, w.seed)
     return O.segment_forward(Q64[g], K64[g], V64[g], W, w.b, w.m, w.causal, w.n0, w.seed, g,
@@ -156,7 +170,7 @@ def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, seg
     stats = {"max_abs": float(err.max()), "mean_abs": float(err.mean()), "lse_rel": float(lerr.max()),
              "rows": int(lerr.size)}
     assert np.isfinite(err).all() and np.isfinite(lerr).all(), stats
-    vscale = max(1.0, float(np.abs(V64).max()) / 5.12)      # see the module docstring
+    vscale = max(1.0, max(float(np.abs(V64[g]).max()) for g in segs) / 5.12)      # see the module docstring
     stats["value_scale"] = vscale
     assert stats["max_abs"] <= OUT_MAX_ABS * vscale, stats
     assert stats["mean_abs"] <= OUT_MEAN_ABS * vscale, stats

@@ -1,0 +1,35 @@
+"""Parity at the full benchmark sizes, in the launch configuration the benchmark times.
+
+The oracle cannot evaluate these workloads as a whole, so two segments (the first and the
+last (batch, head) pair) are checked per workload: bucket ids and permutations in full, the
+outputs on sampled rows plus the rows around every leaf boundary; every output of every
+segment must be finite."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2310_05869_b200 as ha
+from paper_2310_05869_b200 import workloads as WL
+
+import parity_util as PU
+
+pytestmark = pytest.mark.gpu
+
+FULL = [WL.CONFIGS[1], WL.CONFIGS[2], WL.CONFIGS[3], WL.CONFIGS[4]]
+
+
+@pytest.mark.parametrize("w", FULL, ids=[w.name for w in FULL])
+def test_full_size_sampled_segments(w):
+    arrs = WL.make_inputs(w)
+    q, k, v = PU.to_device(w, arrs)
+    out, lse, inter = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, debug=True)
+    torch.cuda.synchronize()
+    assert ha.last_device_status() == 0
+    assert bool(torch.isfinite(out.float()).all()) and bool(torch.isfinite(lse).all())
+    segs = [0, w.G - 1]
+    Q64, K64, V64 = (PU.LazySegments(x) for x in arrs)
+    amb, mism = PU.check_ids(w, Q64, K64, inter, segs=segs)
+    assert mism <= amb
+    PU.check_perms(w, inter, segs=segs)
+    stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter, rows_per_seg=48, segs=segs, rng_seed=1)
+    print(w.name, stats, "ambiguous hash bits", amb, "rows that differ", mism)
