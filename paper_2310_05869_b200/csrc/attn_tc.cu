@@ -24,8 +24,9 @@
 // Warp roles (384 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
 // warps 8 and 9 MMA issue for query tile 0 and 1 (warp 8 also allocates TMEM, all 512
 // columns: 2 x 2 S buffers of 64, O0, O1), warp 10 prepares work items (row tables of the
-// NEXT item while this one computes, then its Q tiles), warp 11 streams K / V tiles through
-// the stage ring, across item boundaries.
+// NEXT item while this one computes, TMA boxes of Q), warp 11 streams K / V tiles through
+// the stage ring, across item boundaries.  Gathered Q tiles are fetched by the 256 softmax
+// threads, for the next item, right before they write the current item's results.
 // Every mbarrier wait is bounded: on a timeout the CTA raises the device status word,
 // drains its copies, frees its TMEM and returns.
 #include <cstdlib>
@@ -120,26 +121,9 @@ __device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, volatil
 }
 
 // ---- tcgen05 ----------------------------------------------------------------------------
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-  d |= (uint64_t)1 << 46;   // descriptor version of sm_100
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
-  return d;
-}
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
-               ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-// the same with descriptors given as (low, high) 32-bit words: only the low word ever changes
+// tcgen05.mma with shared-memory descriptors given as (low, high) 32-bit words: only the low word ever changes
+// (low word = start address >> 4 | (leading byte offset >> 4) << 16, high word = stride byte offset >> 4 |
+// descriptor version 1 << 14 | 128-byte swizzle 2 << 29); [a_tmem]: the A operand read from TMEM
 __device__ __forceinline__ void mma_ss2(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
   asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
                "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}\n"
@@ -155,16 +139,6 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                 "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                 "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-               : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-}
 // issue without waiting; the data is valid only after tmem_ld32_wait on the same registers
 __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -196,10 +170,6 @@ __device__ __forceinline__ void tmem_ld16_wait(uint32_t (&r)[16]) {
                : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
                  "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
                :: "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
-               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
@@ -242,14 +212,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
                ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
                  "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-               "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
-               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-                 "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-                 "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 
@@ -478,10 +440,6 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
 
 // a-th key tile of a query tile -> index in the pair's tile list
 __device__ __forceinline__ int tile_of(const QTile& q, int a) { return a < q.n1 ? q.s1 + a : q.s2 + (a - q.n1); }
-__device__ __forceinline__ bool uses_tile(const QTile& q, int j) {
-  return (j >= q.s1 && j < q.s1 + q.n1) || (j >= q.s2 && j < q.s2 + q.n2);
-}
-
 template <int D>
 __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TmaMaps maps, int* status) {
   using C = Cfg<D>;
@@ -947,7 +905,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     }
     __syncwarp();
   } else if (warp == 10) {
-    constexpr int CPR = D / 8;                             // 16-byte chunks per row
     // ================= item preparer: row tables of an item, then its Q tiles ========================
     // Runs one item ahead of the K / V streamer where it can: a table set becomes free when the
     // softmax warps and the streamer are done with the item before the previous one, so the
