@@ -229,21 +229,18 @@ def config_dict(w):
 # ---------------------------------------------------------------- GPU arm
 def gpu_arm(args, w):
     import torch
-    import torch.distributed as dist
     import paper_2310_05869_b200 as ha
+    from paper_2310_05869_b200 import ranks as RK
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    info = RK.rank_env()
+    world, rank, local = info.world, info.rank, info.local_rank
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
+    RK.init(info, "nccl", dev)
     peaks = load_peaks()
 
     # every rank owns its own B*H segments (weak scaling: no exchange between segments)
-    wr = w.scaled(gen_seed=w.gen_seed + 7919 * rank)
-    arrs = WL.make_inputs(wr)
+    arrs = WL.make_inputs(RK.rank_workload(w, rank))
 
     def dev_tensor(x):
         if x.dtype == np.uint16:
@@ -261,8 +258,7 @@ def gpu_arm(args, w):
         return ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        RK.barrier(info)
         torch.cuda.synchronize(dev)
 
     sampler = ClockSampler(local) if rank == 0 else None
@@ -293,12 +289,8 @@ def gpu_arm(args, w):
         torch.cuda.synchronize(dev)
         flush_ms = f0.elapsed_time(f1)
     ms_total = max(ms_total - flush_ms, 1e-6)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    tokens = w.B * w.n * args.steps * world
-    value = tokens / (ms_total * 1e-3)
+    ms_total = RK.max_over_ranks(info, ms_total, dev)
+    value = RK.job_throughput(info, w.B * w.n, args.steps, ms_total)
 
     # ---- end to end through the host-buffer entry point ---------------------------------------
     hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
@@ -313,21 +305,17 @@ def gpu_arm(args, w):
         ha.forward_host(hq, hk, hv, ho, hl, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
     e1.record(stream)
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item())
+    e2e_ms = RK.max_over_ranks(info, e0.elapsed_time(e1), dev)
     es = q.element_size()
     h2d = 3 * q.numel() * es
     d2h = ho.numel() * ho.element_size() + hl.numel() * 4
-    e2e = {"value": w.B * w.n * e2e_steps * world / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms / e2e_steps,
+    e2e = {"value": RK.job_throughput(info, w.B * w.n, e2e_steps, e2e_ms), "unit": "tokens/s", "ms_per_step": e2e_ms / e2e_steps,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
     assert torch.equal(ho.to(dev), out), "host-buffer entry point disagrees with the device entry point"
     clocks = sampler.stop() if sampler else None
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        RK.shutdown(info)
         return
 
     # ---- per-stage roofline -----------------------------------------------------------------------
@@ -392,8 +380,7 @@ def gpu_arm(args, w):
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "clocks": clocks,
             "peaks": peaks}
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    RK.shutdown(info)
 
 
 def main():
