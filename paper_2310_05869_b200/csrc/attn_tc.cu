@@ -571,6 +571,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       const QTile q = i ? de.qb : de.qa;
       const int total = q.n1 + q.n2;
       const float wlog = (t.mode == 1 && g.m > 0) ? log2f((float)t.nk / (float)g.m) : 0.f;   // log2(N/m): weight of a sampled column
+      // key tiles of this item with masked columns for this query tile, one bit per tile (an item has at most 32)
+      unsigned tile_masked = 0;
+      if (t.mode == 1) tile_masked = __ballot_sync(0xffffffffu, lane < t.ntiles && (s_mask[2 * lane] | s_mask[2 * lane + 1]) != 0);
       float m_ref = -INFINITY;
       uint64_t l01 = 0, lr01 = 0;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each, packed)
       for (int na = 0; na < total && ok; ++na) {
@@ -584,16 +587,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         HA_T0(tc);
         tc_fence_after();
         // mask kind of this (query tile, key tile): uniform over the warpgroup
-        bool table = false, dense_mask = false;
-        float ubias = 0.f;
-        int climit = 0;                               // dense: last visible column of this row
-        if (t.mode == 1) {
-          table = (s_mask[j * 2] | s_mask[j * 2 + 1]) != 0;
-          ubias = (j < t.nbA + t.nbB) ? 0.f : wlog;
-        } else {
-          climit = t.causal ? min(t.nk - 1, q.row0 + row) : t.nk - 1;
-          dense_mask = (j * TK + TK > t.nk) || (t.causal && j * TK + TK - 1 > q.row0);
-        }
+        const bool table = (tile_masked >> j) & 1u;
+        const float ubias = (t.mode == 1 && j >= t.nbA + t.nbB) ? wlog : 0.f;
+        const bool dense_mask = t.mode != 1 && ((j * TK + TK > t.nk) || (t.causal && j * TK + TK - 1 > q.row0));
         // The 64 scores of this row are read from TMEM once; then (1) the row maximum, (2)
         // exponentials, row sums and the bf16 P written over the first half of the S buffer.
         // The reference maximum only moves when the tile exceeds it by more than 2^32, and then
@@ -607,6 +603,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           uint32_t visa, visb;
           if (table) { visa = ~s_mask[j * 2]; visb = ~s_mask[j * 2 + 1]; }
           else {
+            const int climit = t.causal ? min(t.nk - 1, q.row0 + row) : t.nk - 1;   // last visible column of this row
             const int rel = climit - j * TK;            // columns 0..rel of the tile are visible
             visa = rel >= 31 ? 0xffffffffu : (rel < 0 ? 0u : ((2u << rel) - 1u));
             visb = rel >= 63 ? 0xffffffffu : (rel < 32 ? 0u : ((2u << (rel - 32)) - 1u));
