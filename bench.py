@@ -292,6 +292,19 @@ def gpu_arm(args, w):
     ms_total = RK.max_over_ranks(info, ms_total, dev)
     value = RK.job_throughput(info, w.B * w.n, args.steps, ms_total)
 
+    # ---- per-call latency distribution (outside the timed region: one event pair per call) ------
+    lat_steps = max(5, min(args.steps, 30))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(lat_steps)]
+    for a0, a1 in evs:
+        if flush is not None:
+            flush.fill_(1)
+        a0.record(stream)
+        ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+        a1.record(stream)
+    torch.cuda.synchronize(dev)
+    lat = sorted(a0.elapsed_time(a1) for a0, a1 in evs)
+    latency = {"median_ms": lat[len(lat) // 2], "min_ms": lat[0], "calls": lat_steps}
+
     # ---- end to end through the host-buffer entry point ---------------------------------------
     hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
     ho = torch.empty(q.shape, dtype=q.dtype).pin_memory()
@@ -375,7 +388,7 @@ def gpu_arm(args, w):
     line = {"metric": "forward tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config_dict(w),
-            "latency_ms": ms_step, "dense_attention_roofline_ms": dense_ms, "speedup_vs_dense_roofline": dense_ms / ms_step,
+            "latency_per_call": latency, "latency_ms": ms_step, "dense_attention_roofline_ms": dense_ms, "speedup_vs_dense_roofline": dense_ms / ms_step,
             "e2e": e2e, "gpu_launches": sum(launches.values()) * args.steps, "launches_per_step": launches,
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "clocks": clocks,
             "peaks": peaks}

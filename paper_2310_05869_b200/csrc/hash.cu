@@ -78,6 +78,20 @@ __global__ void __launch_bounds__(256, D == 64 ? 4 : 2) hash_bf16_kernel(const _
 
   s_hist[tid] = 0;
 
+  const char* base = reinterpret_cast<const char*>(a.x[side]) + ((size_t)seg * a.n + row0) * (D * 2);
+  unsigned nz = 0;
+  const int groups = (rows + 15) >> 4;
+  uint4 xa[CPL], xb[CPL];
+  auto load_group = [&](int grp, uint4 (&pa)[CPL], uint4 (&pb)[CPL]) {
+    const int ra = grp * 16 + gid, rb = ra + 8;
+#pragma unroll
+    for (int h = 0; h < CPL; ++h) {
+      pa[h] = (grp < groups && ra < rows) ? ldg_stream(base + (size_t)ra * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
+      pb[h] = (grp < groups && rb < rows) ? ldg_stream(base + (size_t)rb * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  load_group(warp, xa, xb);                           // the first rows are on their way while the fragments are built
+
   // Direction fragments.  k-slot (step s, half h, element e) of lane (gid, tig) holds
   // coordinate 8*(tig + 4*(s>>1)) + 2*(2*(s&1) + h) + e; column gid is direction gid.
   for (int idx = tid; idx < KS * 32; idx += 256) {
@@ -105,19 +119,6 @@ __global__ void __launch_bounds__(256, D == 64 ? 4 : 2) hash_bf16_kernel(const _
   }
   __syncthreads();
 
-  const char* base = reinterpret_cast<const char*>(a.x[side]) + ((size_t)seg * a.n + row0) * (D * 2);
-  unsigned nz = 0;
-  const int groups = (rows + 15) >> 4;
-  uint4 xa[CPL], xb[CPL];
-  auto load_group = [&](int grp, uint4 (&pa)[CPL], uint4 (&pb)[CPL]) {
-    const int ra = grp * 16 + gid, rb = ra + 8;
-#pragma unroll
-    for (int h = 0; h < CPL; ++h) {
-      pa[h] = (grp < groups && ra < rows) ? ldg_stream(base + (size_t)ra * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
-      pb[h] = (grp < groups && rb < rows) ? ldg_stream(base + (size_t)rb * (D * 2) + (tig + 4 * h) * 16) : make_uint4(0, 0, 0, 0);
-    }
-  };
-  load_group(warp, xa, xb);
   for (int grp = warp; grp < groups; grp += 8) {
     const int ra = grp * 16 + gid, rb = ra + 8;
     uint4 na[CPL], nb[CPL];
