@@ -164,6 +164,8 @@ typedef struct hyperattn_stage_times {
   int launches[HYPERATTN_NUM_STAGES];
   int calls;
 } hyperattn_stage_times;
+/* on = 0: off; on = 1: every stage; any other value: only the stages s whose bit
+ * (1 << (s + 1)) is set (fewer events on the stream between the kernels). */
 int hyperattn_profile_enable(int on);
 int hyperattn_profile_reset(void);
 int hyperattn_profile_read(hyperattn_stage_times* out);

@@ -196,8 +196,14 @@ def last_device_status(stream=None) -> int:
     return int(st.value)
 
 
-def profile_enable(on: bool):
-    lib().hyperattn_profile_enable(int(on))
+def profile_enable(on: bool, stages=None):
+    """Stage timing on/off; `stages` (names from STAGE_NAMES) restricts it to those stages."""
+    code = int(bool(on))
+    if on and stages is not None:
+        code = 0
+        for name in stages:
+            code |= 1 << (STAGE_NAMES.index(name) + 1)
+    lib().hyperattn_profile_enable(code)
 
 
 def profile_reset():

@@ -131,6 +131,7 @@ struct StageEvents { cudaEvent_t beg, end; int stage; int launches; };
 std::mutex g_mu;
 std::map<int, DeviceState> g_dev;
 bool g_profile = false;
+unsigned g_profile_mask = ~0u;          // stages that are timed while profiling is on
 std::vector<StageEvents> g_events;
 std::vector<cudaEvent_t> g_event_pool;
 int g_profile_calls = 0;
@@ -145,7 +146,7 @@ cudaEvent_t take_event() {
 
 struct StageScope {
   cudaStream_t st; int stage; int launches; bool on; cudaEvent_t beg = nullptr;
-  StageScope(cudaStream_t s, int stage_, int launches_) : st(s), stage(stage_), launches(launches_), on(g_profile && launches_ > 0) {
+  StageScope(cudaStream_t s, int stage_, int launches_) : st(s), stage(stage_), launches(launches_), on(g_profile && launches_ > 0 && ((g_profile_mask >> stage_) & 1u)) {
     if (on) { beg = take_event(); cudaEventRecord(beg, st); }
   }
   ~StageScope() {
@@ -421,6 +422,7 @@ int hyperattn_last_device_status(void* stream, int* status) {
 int hyperattn_profile_enable(int on) {
   std::lock_guard<std::mutex> lock(g_mu);
   g_profile = on != 0;
+  g_profile_mask = (on == 0 || on == 1) ? ~0u : ((unsigned)on >> 1);
   return HYPERATTN_OK;
 }
 
