@@ -228,7 +228,8 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
     assert Q.shape[0] == N, "the paper pairs the beta-th group of Q with the beta-th group of K"
     if b >= N:
         return exact_attention(Q, K, V, scale, causal=False, rows=rows)
-    assert N % b == 0, "N must be a multiple of the block size (or b >= N)"
+    # N need not be a multiple of b: Alg. 1 line 4 defines the mask through floor(P(i)/b), so the
+    # last sorted block simply has N mod b rows of Q and of K (the slices below end at N)
     perm_q, rank_q = stable_argsort(ids_q)
     perm_k, rank_k = stable_argsort(ids_k)
     samples = np.asarray(samples, dtype=np.int64)

@@ -251,6 +251,51 @@ def test_zero_logits_give_counting_closed_form():
     np.testing.assert_allclose(out, 1.0, atol=1e-12)
 
 
+def test_ragged_last_block_counting_closed_form_and_full_coverage():
+    """N not a multiple of b: the mask of Alg. 1 line 4 is floor(P(i)/b), so the last sorted block
+    has N mod b rows.  Q = 0 gives d~_i = |block of i| + (N/m) #{t : l_t outside i's block};
+    samples covering every key once give exact attention, whatever the block sizes."""
+    rng = np.random.default_rng(16)
+    N, b, m, d = 37, 8, 11, 3                                   # blocks of 8, 8, 8, 8, 5
+    K = rng.standard_normal((N, d))
+    iq = rng.integers(0, 16, N).astype(np.uint8)
+    ik = rng.integers(0, 16, N).astype(np.uint8)
+    smp = rng.integers(0, N, m)
+    out, lse = O.node_forward(np.zeros((N, d)), K, np.ones((N, d)), iq, ik, smp, b, 1.0)
+    order_q = sorted(range(N), key=lambda i: (int(iq[i]), i))
+    order_k = sorted(range(N), key=lambda i: (int(ik[i]), i))
+    for i in range(N):
+        beta = order_q.index(i) // b
+        size = sum(1 for j in range(N) if order_k.index(j) // b == beta)
+        assert size == (5 if beta == 4 else 8)
+        outside = sum(1 for l in smp if order_k.index(int(l)) // b != beta)
+        assert abs(lse[i] - math.log(size + (N / m) * outside)) < 1e-12
+    np.testing.assert_allclose(out, 1.0, atol=1e-12)
+    Q, K, V = rand_qkv(rng, N, 5)
+    out, lse = O.node_forward(Q, K, V, iq, ik, rng.permutation(N), b, 0.4)
+    bo, bl = brute_attention(Q, K, V, 0.4, False)
+    np.testing.assert_allclose(out, bo, atol=1e-12)
+    np.testing.assert_allclose(lse, bl, atol=1e-12)
+
+
+@pytest.mark.parametrize("causal,n,n0,b", [(False, 26, 0, 4), (True, 24, 6, 5)])
+def test_dense_weights_with_ragged_blocks(causal, n, n0, b):
+    """The dense cross-form stays row-stochastic and reproduces the output when block sizes do
+    not divide the node sizes (causal: nodes of 12 and 6 rows with b = 5)."""
+    rng = np.random.default_rng(17)
+    d, m, r, seed, scale = 4, 5, 3, 33, 0.5
+    Q, K, V = rand_qkv(rng, n, d)
+    W = O.directions(d, r, seed)
+    iq, _ = O.bucket_ids(Q, W)
+    ik, _ = O.bucket_ids(K, W)
+    Wt = O.dense_weights(Q, K, iq, ik, b, m, scale, causal, n0, seed, g=1)
+    np.testing.assert_allclose(Wt.sum(axis=1), 1.0, atol=1e-12)
+    if causal:
+        assert np.triu(Wt, 1).max() == 0.0
+    out, _ = O.segment_forward(Q, K, V, W, b, m, causal, n0, seed, g=1, scale=scale)
+    np.testing.assert_allclose(out, Wt @ V, atol=1e-12)
+
+
 def test_no_samples_and_all_colliding_samples():
     rng = np.random.default_rng(7)
     N, b = 16, 4
