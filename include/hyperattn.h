@@ -31,9 +31,9 @@
  *   - Return value: 0 on success, a negative hyperattn_status otherwise.  On a
  *     host-detected error nothing is launched and no output is written.
  *   - Shapes: d in {64, 128}; 1 <= hash_bits <= 8; samples >= 0; block >= 1.
- *     Non-causal: n % block == 0 or block >= n (then the problem is one exact block).
- *     Causal: n <= n0 (exact causal attention) or n == n0 * 2^L; and the half-size of
- *     every recursion node must be a multiple of block unless block >= that half-size.
+ *     block need not divide n (or a recursion node's size): the mask of Alg. 1 line 4 is
+ *     floor(P(i) / block), so the last sorted block is short; block >= n makes the problem one
+ *     exact block.  Causal: n <= n0 (exact causal attention) or n == n0 * 2^L.
  *   - Recursion nodes are numbered like a binary heap: the off-diagonal problem of the
  *     j-th node of level l (root level 0) is node (2^l - 1) + j; it pairs query rows
  *     [(2j+1)s, (2j+2)s) with key rows [2js, (2j+1)s), s = n / 2^(l+1).  A non-causal

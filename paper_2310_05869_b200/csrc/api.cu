@@ -37,7 +37,6 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
   if (!p.causal) {
     g.causal = 0; g.L = 0; g.leaf = p.n; g.unit = p.n;
     if (p.block < p.n) {
-      if (p.n % p.block) return HYPERATTN_UNSUPPORTED_SHAPE;
       g.levels = 1; g.nl = p.n; g.nodes = 1; g.sorted = 1;
     }
   } else {
@@ -56,10 +55,7 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
       g.levels = L; g.nl = p.n / 2; g.nodes = (1 << L) - 1;
       for (int l = 0; l < L; ++l) {
         const int s = p.n >> (l + 1);
-        if (p.block < s) {
-          if (s % p.block) return HYPERATTN_UNSUPPORTED_SHAPE;
-          g.sorted = 1;
-        }
+        if (p.block < s) g.sorted = 1;
       }
     }
   }
@@ -292,7 +288,7 @@ int forward_impl(const hyperattn_params& p) {
     const int nodes_lvl = g.causal ? (1 << l) : 1;
     a.level_start[l] = (int)tiles;
     a.level_sorted[l] = g.b < s;
-    const long long per_node = a.level_sorted[l] ? (long long)(s / g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
+    const long long per_node = a.level_sorted[l] ? (long long)node_blocks(s, g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
     tiles += per_node * nodes_lvl * g.G;
     if (tiles > 0x7fffffffLL) return HYPERATTN_UNSUPPORTED_SHAPE;
     a.level_pair_start[l] = (int)pairs;

@@ -89,7 +89,7 @@ __device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
   const int nodes_lvl = g.causal ? (1 << level) : 1;
   const size_t region = a.direct ? 0 : (size_t)g.G * g.n + (size_t)level * g.G * g.nl;
   if (a.level_sorted[level]) {
-    const int tiles_node = (s / g.b) * a.tiles_per_block;
+    const int tiles_node = node_blocks(s, g.b) * a.tiles_per_block;
     const int tn = idx % tiles_node; idx /= tiles_node;
     const int j = idx % nodes_lvl;
     t.seg = idx / nodes_lvl;
@@ -98,7 +98,7 @@ __device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
     t.beta = tn / a.tiles_per_block;
     const int sub = tn % a.tiles_per_block;
     t.spos0 = t.beta * g.b + sub * kTileQ;
-    t.nq = min(kTileQ, g.b - sub * kTileQ);
+    t.nq = max(0, min(kTileQ, block_len(s, g.b, t.beta) - sub * kTileQ));   // 0: the (short) last block has no such tile
     t.k0 = k0n; t.nk = s; t.qnode0 = q0n;
     t.slice = ((size_t)level * g.G + t.seg) * g.nl + (g.causal ? (size_t)j * s : 0);
     t.node = g.causal ? (1 << level) - 1 + j : 0;

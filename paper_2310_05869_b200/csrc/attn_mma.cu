@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
     for (int i = tid; i < nkeys; i += 256) {
       int idx = -1; float bias = -INFINITY;
       if (i < bpad) {
-        if (i < g.b) { idx = t.k0 + a.perm_k[t.slice + (size_t)t.beta * g.b + i]; bias = 0.f; }
+        if (i < block_len(t.nk, g.b, t.beta)) { idx = t.k0 + a.perm_k[t.slice + (size_t)t.beta * g.b + i]; bias = 0.f; }
       } else if (i - bpad < g.m) {
         const int l = smp[i - bpad];
         idx = t.k0 + l;

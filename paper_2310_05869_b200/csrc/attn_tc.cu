@@ -395,7 +395,7 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
     const int nodes_lvl = g.causal ? (1 << level) : 1;
     const int sorted = a.level_sorted[level];
     const int paired = a.level_paired[level];
-    const int tiles_node = sorted ? (s / g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
+    const int tiles_node = sorted ? node_blocks(s, g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
     const int pairs_node = paired ? (tiles_node + 1) / 2 : tiles_node;
     const int pn = idx % pairs_node; idx /= pairs_node;
     const int j = idx % nodes_lvl;
@@ -414,7 +414,8 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
         q.beta = tn / a.tiles_per_block;
         const int sub = tn % a.tiles_per_block;
         q.spos0 = q.beta * g.b + sub * kTileQ;
-        q.nq = min(kTileQ, g.b - sub * kTileQ);
+        q.nq = min(kTileQ, block_len(s, g.b, q.beta) - sub * kTileQ);
+        if (q.nq <= 0) q.valid = 0;                       // the (short) last block has no such tile
         q.q0 = 0;
       } else {
         q.q0 = q0n + tn * kTileQ;
@@ -425,12 +426,15 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
     if (sorted) {
       t.slice = ((size_t)level * g.G + t.seg) * g.nl + (g.causal ? (size_t)j * s : 0);
       t.node = g.causal ? (1 << level) - 1 + j : 0;
-      const int bt = (g.b + TK - 1) / TK;
+      const int bt = (block_len(s, g.b, qa.beta) + TK - 1) / TK;                                  // key tiles of a block: its own length
+      const int btb = qb.valid ? (block_len(s, g.b, qb.beta) + TK - 1) / TK : 0;
       t.nbA = bt;
-      t.nbB = (qb.valid && qb.beta != qa.beta) ? bt : 0;
+      t.nbB = (qb.valid && qb.beta != qa.beta) ? btb : 0;
       t.nsmp = (g.m + TK - 1) / TK;
-      qa.s1 = 0; qa.n1 = bt; qa.s2 = t.nbA + t.nbB; qa.n2 = t.nsmp;
-      qb.s1 = t.nbB ? t.nbA : 0; qb.n1 = qb.valid ? bt : 0; qb.s2 = t.nbA + t.nbB; qb.n2 = qb.valid ? t.nsmp : 0;
+      // (a query tile that does not exist - the short last block may have fewer tiles - walks no key tiles)
+      if (!qa.valid) { t.nbA = 0; t.nsmp = 0; }
+      qa.s1 = 0; qa.n1 = t.nbA; qa.s2 = t.nbA + t.nbB; qa.n2 = t.nsmp;
+      qb.s1 = t.nbB ? t.nbA : 0; qb.n1 = qb.valid ? (t.nbB ? btb : bt) : 0; qb.s2 = t.nbA + t.nbB; qb.n2 = qb.valid ? t.nsmp : 0;
     }
     if (a.direct) { t.orow_base = (size_t)t.seg * g.n; t.odelta = 0; }
     else { t.orow_base = (size_t)g.G * g.n + (size_t)level * g.G * g.nl + (size_t)t.seg * g.nl + (size_t)j * s; t.odelta = -q0n; }
@@ -889,8 +893,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           }
         }
         if (!ok) break;
-        skip_k(gbase + ntiles);
-        skip_v(gbase + ntiles);
+        // what is left of the item's tiles (all of them for a query tile that does not exist) is
+        // released K, V, K, V ... like the streamer fills them: releasing all K tiles first would
+        // wait for a K tile whose stage the streamer cannot reach before a V tile is released
+        for (int e = min(knext, vnext) + 1; e <= gbase + ntiles && ok; ++e) { skip_k(e); skip_v(e); }
         gbase += ntiles;
         ga += total;
         vi += q.valid;
@@ -949,7 +955,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             if (c0 < nblk) {
               const int which = c0 >= bcols;
               const int c = c0 - which * bcols;
-              if (c < g.b) idx[u] = pk[(size_t)(which ? qb.beta : qa.beta) * g.b + c];
+              if (c < block_len(t.nk, g.b, which ? qb.beta : qa.beta)) idx[u] = pk[(size_t)(which ? qb.beta : qa.beta) * g.b + c];
             }
           }
 #pragma unroll

@@ -62,6 +62,11 @@ struct Geometry {
   int sorted;          // 1 if any node needs sortLSH (some node has b < its size)
 };
 
+// sorted blocks of a node of s rows: ceil(s / b) of them, the last one with the remaining rows
+// (Alg. 1 line 4: row i belongs to block floor(P(i) / b))
+__host__ __device__ inline int node_blocks(int s, int b) { return (s + b - 1) / b; }
+__host__ __device__ inline int block_len(int s, int b, int beta) { return (s - beta * b) < b ? (s - beta * b) : b; }
+
 // node j of level l: size s, first query row, first key row (non-causal: the whole segment)
 __host__ __device__ inline void node_rows(const Geometry& g, int level, int j, int& s, int& q0, int& k0) {
   if (!g.causal) { s = g.n; q0 = 0; k0 = 0; return; }

@@ -30,6 +30,11 @@ SMALL = [
     W("causal_chunk_tail", 1, 1, 6144, 64, "bf16", 256, 128, 7, True, 3072),
     W("fp32_causal", 1, 2, 1024, 128, "fp32", 64, 64, 8, True, 256, seed=4),
     W("one_bit_small_block", 1, 1, 512, 64, "bf16", 32, 8, 1, False, 0),
+    # block sizes that do not divide the node sizes: the last sorted block is short
+    W("ragged_blocks_n1100_b96", 1, 2, 1100, 64, "bf16", 96, 48, 6, False, 0, seed=12),
+    W("ragged_blocks_b300_d128", 1, 2, 2000, 128, "bf16", 300, 100, 7, False, 0, seed=13),
+    W("causal_ragged_blocks", 1, 2, 2048, 64, "bf16", 96, 64, 6, True, 256, seed=14),
+    W("fp32_ragged_blocks", 1, 1, 700, 64, "fp32", 128, 32, 5, False, 0, seed=15),
 ]
 
 
