@@ -35,6 +35,13 @@ SMALL = [
     W("ragged_blocks_b300_d128", 1, 2, 2000, 128, "bf16", 300, 100, 7, False, 0, seed=13),
     W("causal_ragged_blocks", 1, 2, 2048, 64, "bf16", 96, 64, 6, True, 256, seed=14),
     W("fp32_ragged_blocks", 1, 1, 700, 64, "fp32", 128, 32, 5, False, 0, seed=15),
+    # degenerate and extreme shapes
+    W("tiny_n64_b16", 1, 1, 64, 64, "bf16", 16, 8, 3, False, 0, seed=16),
+    W("block_of_one_row", 1, 1, 128, 64, "bf16", 1, 4, 7, False, 0, seed=17),
+    W("more_samples_than_keys", 1, 2, 256, 128, "bf16", 64, 300, 4, False, 0, seed=18),
+    W("causal_six_levels", 1, 1, 4096, 64, "bf16", 32, 16, 6, True, 64, seed=19),
+    W("odd_batch_and_heads", 3, 5, 768, 64, "bf16", 128, 64, 7, False, 0, seed=20),
+    W("causal_leaf_of_one_tile_pair", 2, 1, 1024, 128, "bf16", 128, 128, 8, True, 256, seed=21),
 ]
 
 
