@@ -42,6 +42,10 @@ SMALL = [
     W("causal_six_levels", 1, 1, 4096, 64, "bf16", 32, 16, 6, True, 64, seed=19),
     W("odd_batch_and_heads", 3, 5, 768, 64, "bf16", 128, 64, 7, False, 0, seed=20),
     W("causal_leaf_of_one_tile_pair", 2, 1, 1024, 128, "bf16", 128, 128, 8, True, 256, seed=21),
+    # three query tiles per block: tiles are not paired, the second query tile's roles idle through
+    # items with more key tiles than ring stages
+    W("unpaired_tiles_b384_d128", 1, 2, 3072, 128, "bf16", 384, 128, 7, False, 0, seed=22),
+    W("unpaired_tiles_b640_d64", 1, 1, 5120, 64, "bf16", 640, 256, 7, False, 0, seed=23),
 ]
 
 
