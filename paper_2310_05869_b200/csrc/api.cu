@@ -293,7 +293,9 @@ int forward_impl(const hyperattn_params& p) {
     if (tiles > 0x7fffffffLL) return HYPERATTN_UNSUPPORTED_SHAPE;
     a.level_pair_start[l] = (int)pairs;
     // two query tiles share a CTA when they share their block's keys (even tiles per block),
-    // or when a block is a single tile; other block sizes run one tile per CTA
+    // or when a block is a single tile; other block sizes run one tile per CTA (a pair that
+    // straddles two larger blocks would make each tile's issuer skip more key tiles of the
+    // other's block than the stage ring holds, which the ring's release order does not allow)
     a.level_paired[l] = !a.level_sorted[l] || a.tiles_per_block % 2 == 0 || a.tiles_per_block == 1;
     pairs += (a.level_paired[l] ? (per_node + 1) / 2 : per_node) * nodes_lvl * g.G;
   }
