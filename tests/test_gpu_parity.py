@@ -140,3 +140,28 @@ def test_stage_profile_counts_launches():
     assert prof["calls"] == 2
     assert prof["launches"]["hash"] == 2 and prof["launches"]["attention"] == 2 and prof["launches"]["merge"] == 2
     assert all(prof["ms"][s] > 0 for s in ("hash", "sort_scan", "sort_scatter", "attention", "merge"))
+
+
+def test_forward_can_be_captured_in_a_cuda_graph():
+    """The entry point only enqueues work on the caller's stream (workspace from the stream-ordered
+    pool, no synchronisation), so a forward call can be captured once and replayed."""
+    w = W("graph_capture", 1, 4, 2048, 64, "bf16", 128, 64, 7, True, 512, seed=31)
+    arrs = WL.make_inputs(w)
+    q, k, v = PU.to_device(w, arrs)
+    out, lse = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):                      # warm the pool on the capture stream
+        ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        out2, lse2 = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+    for _ in range(3):
+        out2.zero_()
+        graph.replay()
+    torch.cuda.synchronize()
+    assert ha.last_device_status() == 0
+    assert torch.equal(out2, out) and torch.equal(lse2, lse)
