@@ -59,7 +59,7 @@ struct HashArgs {
 // one, and the direction fragments live in shared memory (one 8-byte read per MMA) instead
 // of 48 registers, so that two to four CTAs fit an SM and ~128 KB of loads are in flight.
 template <int D>
-__global__ void __launch_bounds__(256, D == 64 ? 4 : 2) hash_bf16_kernel(const __grid_constant__ HashArgs a) {
+__global__ void __launch_bounds__(256, D == 64 ? 4 : 3) hash_bf16_kernel(const __grid_constant__ HashArgs a) {
   constexpr int KS = D / 16;             // MMA k-steps
   constexpr int CPL = D / 32;            // 16-byte chunks per lane per row
   __shared__ __align__(16) uint8_t s_ids[kSortChunk];
