@@ -1027,6 +1027,20 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tabfull(set));       // (release: the table writes of all lanes are ordered before it by the warp barrier)
       if (lane == 0) HA_TACC(10, ttab);
+      // Sorted query rows are read once in the whole forward pass, so they come from HBM: ask for
+      // them now (the softmax threads gather them a whole item later) so that they are found in L2.
+      if (t.mode == 1) {
+        const char* qbase = reinterpret_cast<const char*>(a.q) + (size_t)segrow * (D * 2);
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (qr[i][k] >= 0) {
+#pragma unroll
+              for (int ln = 0; ln < D * 2 / 128; ++ln)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(qbase + (size_t)qr[i][k] * (D * 2) + ln * 128));
+            }
+      }
       // ---- Q (the issuers must be done with the previous item's Q) ----------------------------
       HA_T0(tqf);
       if (it >= 1) {
