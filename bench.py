@@ -365,7 +365,7 @@ def gpu_arm(args, w):
                            "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"]}
     kernels["attention"] = {"bound": "tensor", "ms": att_ms, "achieved": att_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
                             "frac": att_tflops / tensor_peak}
-    kernels["sample"] = {"ms": stage_ms["sample"]}
+    kernels["sample"] = {"ms": stage_ms["sample"], "note": "drawn by extra blocks of the sort_scan launch"}
     ms_step = ms_total / args.steps
     dense_ms = wm["dense_attention_flops"] / (tensor_peak * 1e12) * 1e3
 

@@ -152,7 +152,7 @@ int hyperattn_last_device_status(void* stream, int* status);
 enum {
   HYPERATTN_STAGE_CONVERT = 0, /* fp32 -> bf16 staging copy (fp32 inputs only) */
   HYPERATTN_STAGE_HASH = 1,    /* Def. 1 hash of Q and K rows + chunk histograms */
-  HYPERATTN_STAGE_SAMPLE = 2,  /* Alg. 2 line 4 */
+  HYPERATTN_STAGE_SAMPLE = 2,  /* Alg. 2 line 4: drawn inside the SORT_SCAN launch, so always 0 here */
   HYPERATTN_STAGE_SORT_SCAN = 3,
   HYPERATTN_STAGE_SORT_SCATTER = 4, /* Alg. 1 line 3 */
   HYPERATTN_STAGE_ATTENTION = 5,    /* block + sampled + causal-leaf contractions */

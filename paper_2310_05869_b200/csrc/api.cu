@@ -238,12 +238,9 @@ int forward_impl(const hyperattn_params& p) {
       HA_CHECK(launch_hash(g, p.q, p.k, is_fp32, g_wcache.w, ws, dbg ? dbg->near_zero_bits : nullptr, st));
     }
     {
-      StageScope sc(st, HYPERATTN_STAGE_SAMPLE, g.m > 0 ? 1 : 0);
-      HA_CHECK(launch_samples(g, p.seed, ws, st));
-    }
-    {
+      // (the samples of Alg. 2 line 4 are drawn by extra blocks of this launch)
       StageScope sc(st, HYPERATTN_STAGE_SORT_SCAN, 1);
-      HA_CHECK(launch_sort_scan(g, ws, st));
+      HA_CHECK(launch_sort_scan(g, ws, true, p.seed, st));
     }
     {
       StageScope sc(st, HYPERATTN_STAGE_SORT_SCATTER, 1);

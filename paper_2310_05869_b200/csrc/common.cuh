@@ -91,8 +91,7 @@ struct Workspace {
 cudaError_t launch_convert(const float* src, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t count, cudaStream_t st);
 cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
                         const Workspace& ws, unsigned long long* near_zero, cudaStream_t st);
-cudaError_t launch_samples(const Geometry& g, uint64_t seed, const Workspace& ws, cudaStream_t st);
-cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st);
 cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_merge(const Geometry& g, const Workspace& ws, void* out, float* lse, int out_fp32,
                          cudaStream_t st);

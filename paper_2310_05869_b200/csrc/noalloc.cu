@@ -88,7 +88,7 @@ extern "C" int hyperattn_sortlsh_noalloc(const void* x, int n, int d, int hash_b
   // the matrix is hashed as both "queries" and "keys" of a one-segment problem; the key side
   // carries the inverse permutation that callers want
   if (launch_hash(g, x, x, /*is_fp32=*/0, w, ws, nullptr, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
-  if (launch_sort_scan(g, ws, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  if (launch_sort_scan(g, ws, false, 0, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   if (launch_sort_scatter(g, ws, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   if (cudaMemcpyAsync(ids, ws.ids + n, (size_t)n, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   return HYPERATTN_OK;

@@ -28,9 +28,37 @@ __device__ __forceinline__ int node_first_chunk(const Geometry& g, int level, in
   return ((side == 0 ? q0 : k0) / g.unit) * g.chunks_per_unit;
 }
 
-// One CTA per (side, level, segment, node): thread v owns bucket v.
-__global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a) {
+struct SampleArgs {
+  int32_t* samples;  // [G, nodes, m]
+  Geometry g;
+  uint32_t k0, k1;
+};
+
+// Alg. 2 line 4: m i.i.d. uniform key indices per (segment, node); word w of Philox call c is
+// sample 4c + w, mapped to [0, N) by a 64-bit multiply-high.  `block` of `nblocks` blocks of 256 threads.
+__device__ __forceinline__ void samples_body(const SampleArgs& a, int block, int nblocks) {
+  const Geometry& g = a.g;
+  const int calls = (g.m + 3) / 4;
+  const size_t total = (size_t)g.G * g.nodes * calls;
+  for (size_t i = (size_t)block * 256 + threadIdx.x; i < total; i += (size_t)nblocks * 256) {
+    const int c = (int)(i % calls);
+    const int nd = (int)((i / calls) % g.nodes);
+    const int seg = (int)(i / ((size_t)calls * g.nodes));
+    const int level = g.causal ? 31 - __clz(nd + 1) : 0;
+    const uint32_t N = g.causal ? (uint32_t)(g.n >> (level + 1)) : (uint32_t)g.n;
+    const Philox4 x = philox4x32_10((uint32_t)c, (uint32_t)seg, (uint32_t)nd, kDomainSamples, a.k0, a.k1);
+    int32_t* dst = a.samples + ((size_t)seg * g.nodes + nd) * g.m;
+#pragma unroll
+    for (int w = 0; w < 4; ++w)
+      if (4 * c + w < g.m) dst[4 * c + w] = (int32_t)__umulhi(x.x[w], N);
+  }
+}
+
+// One CTA per (side, level, segment, node): thread v owns bucket v.  The launch carries the
+// sampling as extra blocks (both are tiny and independent of each other).
+__global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a, SampleArgs sa, int scan_blocks) {
   __shared__ uint32_t s_tot[kBuckets];
+  if ((int)blockIdx.x >= scan_blocks) { samples_body(sa, blockIdx.x - scan_blocks, gridDim.x - scan_blocks); return; }
   const Geometry& g = a.g;
   const int v = threadIdx.x;
   int cta = blockIdx.x;
@@ -127,40 +155,7 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
   }
 }
 
-struct SampleArgs {
-  int32_t* samples;  // [G, nodes, m]
-  Geometry g;
-  uint32_t k0, k1;
-};
-
-__global__ void samples_kernel(SampleArgs a) {
-  const Geometry& g = a.g;
-  const int calls = (g.m + 3) / 4;
-  const size_t total = (size_t)g.G * g.nodes * calls;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    const int c = (int)(i % calls);
-    const int nd = (int)((i / calls) % g.nodes);
-    const int seg = (int)(i / ((size_t)calls * g.nodes));
-    const int level = g.causal ? 31 - __clz(nd + 1) : 0;
-    const uint32_t N = g.causal ? (uint32_t)(g.n >> (level + 1)) : (uint32_t)g.n;
-    const Philox4 x = philox4x32_10((uint32_t)c, (uint32_t)seg, (uint32_t)nd, kDomainSamples, a.k0, a.k1);
-    int32_t* dst = a.samples + ((size_t)seg * g.nodes + nd) * g.m;
-#pragma unroll
-    for (int w = 0; w < 4; ++w)
-      if (4 * c + w < g.m) dst[4 * c + w] = (int32_t)__umulhi(x.x[w], N);
-  }
-}
-
 }  // namespace
-
-cudaError_t launch_samples(const Geometry& g, uint64_t seed, const Workspace& ws, cudaStream_t st) {
-  if (g.nodes == 0 || g.m == 0) return cudaSuccess;
-  SampleArgs a; a.samples = ws.samples; a.g = g; a.k0 = (uint32_t)seed; a.k1 = (uint32_t)(seed >> 32);
-  const size_t total = (size_t)g.G * g.nodes * ((g.m + 3) / 4);
-  const int blocks = (int)((total + 255) / 256);
-  samples_kernel<<<blocks < 1184 ? blocks : 1184, 256, 0, st>>>(a);
-  return cudaGetLastError();
-}
 
 static SortArgs make_sort_args(const Geometry& g, const Workspace& ws) {
   SortArgs a;
@@ -171,11 +166,20 @@ static SortArgs make_sort_args(const Geometry& g, const Workspace& ws) {
   return a;
 }
 
-cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, cudaStream_t st) {
+// scan of the chunk histograms; with_samples: the same launch also draws the samples (Alg. 2 line 4)
+cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st) {
   if (!g.sorted) return cudaSuccess;
   const SortArgs a = make_sort_args(g, ws);
   const int nodes_per = g.causal ? g.nodes : 1;
-  sort_scan_kernel<<<2 * g.G * nodes_per, 256, 0, st>>>(a);
+  const int scan_blocks = 2 * g.G * nodes_per;
+  SampleArgs sa; sa.samples = ws.samples; sa.g = g; sa.k0 = (uint32_t)seed; sa.k1 = (uint32_t)(seed >> 32);
+  int sample_blocks = 0;
+  if (with_samples && g.nodes > 0 && g.m > 0) {
+    const size_t total = (size_t)g.G * g.nodes * ((g.m + 3) / 4);
+    const size_t blocks = (total + 255) / 256;
+    sample_blocks = (int)(blocks < 1184 ? blocks : 1184);
+  }
+  sort_scan_kernel<<<scan_blocks + sample_blocks, 256, 0, st>>>(a, sa, scan_blocks);
   return cudaGetLastError();
 }
 
