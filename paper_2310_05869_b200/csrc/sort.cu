@@ -74,14 +74,17 @@ __global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a, SampleArgs s
   const uint32_t* h = a.hist + (((size_t)side * g.G + seg) * g.chunks_per_seg + first) * kBuckets;
   const int lvl_chunk0 = g.causal ? j * nchunks : 0;
   uint32_t* o = a.offs + ((((size_t)side * g.levels + level) * g.G + seg) * a.chunks_per_level + lvl_chunk0) * kBuckets;
-  uint32_t run = 0;
-  for (int c = 0; c < nchunks; ++c) {
-    const uint32_t t = h[(size_t)c * kBuckets + v];
-    o[(size_t)c * kBuckets + v] = run;
-    run += t;
+  // pass 1: bucket totals of the node (eight loads in flight: the kernel is all latency)
+  uint32_t tot = 0;
+  for (int c0 = 0; c0 < nchunks; c0 += 8) {
+    uint32_t t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) t[u] = c0 + u < nchunks ? h[(size_t)(c0 + u) * kBuckets + v] : 0u;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) tot += t[u];
   }
   // exclusive scan of the bucket totals over v
-  s_tot[v] = run;
+  s_tot[v] = tot;
   __syncthreads();
   for (int off = 1; off < kBuckets; off <<= 1) {
     const uint32_t add = v >= off ? s_tot[v - off] : 0u;
@@ -89,8 +92,18 @@ __global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a, SampleArgs s
     s_tot[v] += add;
     __syncthreads();
   }
-  const uint32_t base = s_tot[v] - run;
-  for (int c = 0; c < nchunks; ++c) o[(size_t)c * kBuckets + v] += base;
+  // pass 2: first position of bucket v in every chunk = buckets before v + the same bucket in earlier chunks
+  uint32_t run = s_tot[v] - tot;
+  for (int c0 = 0; c0 < nchunks; c0 += 8) {
+    uint32_t t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) t[u] = c0 + u < nchunks ? h[(size_t)(c0 + u) * kBuckets + v] : 0u;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (c0 + u < nchunks) o[(size_t)(c0 + u) * kBuckets + v] = run;
+      run += t[u];
+    }
+  }
 }
 
 // One CTA per (side, level, segment, chunk of the level): stable placement of <= 2048 rows.
