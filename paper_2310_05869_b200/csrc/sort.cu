@@ -153,8 +153,17 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
   for (int i0 = wbeg; i0 < wend; i0 += 32) {
     const int i = i0 + lane;
     const bool act = i < wend;
-    const uint32_t id = act ? s_id[i] : 0xFFFFFFFFu;
-    const uint32_t peers = __match_any_sync(0xffffffffu, id);
+    const uint32_t id = act ? s_id[i] : 0u;
+    // lanes with the same bucket id: one ballot per id bit (ids have at most 8 bits; a generic
+    // match.any costs several times more)
+    uint32_t peers = __ballot_sync(0xffffffffu, act);
+#pragma unroll
+    for (int bit = 0; bit < 8; ++bit) {
+      if (bit < g.r) {                                  // (uniform: ids have r bits)
+        const uint32_t bal = __ballot_sync(0xffffffffu, (id >> bit) & 1u);
+        peers &= ((id >> bit) & 1u) ? bal : ~bal;
+      }
+    }
     const int before = __popc(peers & ((1u << lane) - 1u));
     uint32_t pos = 0;
     if (act) pos = s_cnt[warp][id] + before;
