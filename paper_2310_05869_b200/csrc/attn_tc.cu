@@ -23,7 +23,7 @@
 //
 // Warp roles (384 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
 // warps 8 and 9 MMA issue for query tile 0 and 1 (warp 8 also allocates TMEM, all 512
-// columns: 2 x 2 S buffers of 64, O0, O1), warp 10 prepares work items (row tables of the
+// columns: per query tile two S buffers of 64 - three for d = 64 - then O0, O1), warp 10 prepares work items (row tables of the
 // NEXT item while this one computes, TMA boxes of Q), warp 11 streams K / V tiles through
 // the stage ring, across item boundaries.  Gathered Q tiles are fetched by the 256 softmax
 // threads, for the next item, right before they write the current item's results.
@@ -342,7 +342,8 @@ struct Cfg {
   static constexpr int kOffMask = kOffIdx + 2 * kMaxNodeKeys * 4; // uint32 [2][2][kMaxNodeKeys/32] masked-column bits
   static constexpr int kOffQrow = kOffMask + 4 * (kMaxNodeKeys / 32) * 4;   // int [2][2][128]
   static constexpr int kOffBar = kOffQrow + 4 * 128 * 4;
-  static constexpr int kNumBar = 21 + 6 * NS;          // (slot 20 unused)
+  static constexpr int kSBufs = (D == 64) ? 3 : 2;    // S buffers per query tile (d = 64 leaves TMEM columns for a third)
+  static constexpr int kNumBar = 21 + 6 * NS + 12;
   static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
   // Epilogue staging, one slice of 32 rows x kStageRow bytes per softmax warp: rows leave the
   // warp as whole 64- or 128-byte pieces instead of 16 bytes per lane and row.  d = 64: eight
@@ -357,7 +358,8 @@ struct Cfg {
   static constexpr int kTotal = kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;
   static_assert(D == 64 || 4 * kStageWarp <= kMaxNodeKeys * 4, "staging of query tile 0 must fit one key-row table");
   static constexpr int kTmemCols = 512;
-  static constexpr int kColO = 256;                   // S buffer b of tile i at 64 (2 i + b); O_i at kColO + D i
+  static constexpr int kColO = 64 * 2 * kSBufs;       // S buffer b of tile i at 64 (kSBufs i + b); O_i at kColO + D i
+  static_assert(kColO + 2 * D <= 512, "TMEM columns");
 };
 
 __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDesc& t, QTile& qa, QTile& qb) {
@@ -459,8 +461,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   const uint32_t bar0 = ubase + C::kOffBar;
   const uint32_t bar_q = bar0;                                                // Q tiles of the item landed
   const uint32_t bar_qfree = bar0 + 8;                                        // both issuers are done with Q
-  auto bar_s = [&](int i, int b) { return bar0 + 16 + 8 * (2 * i + b); };     // S_i buffer b written
-  auto bar_p = [&](int i, int b) { return bar0 + 48 + 8 * (2 * i + b); };     // P_i buffer b written
+  auto bar_s = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 3 * i + b); };          // S_i buffer b written
+  auto bar_p = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 6 + 3 * i + b); };      // P_i buffer b written
+  auto bar_pvd = [&](int i) { return bar0 + 16 + 8 * i; };                    // P_i V of a key tile finished (one phase per tile)
   auto bar_o = [&](int i) { return bar0 + 80 + 8 * i; };                      // O_i of the item complete
   auto bar_pv = [&](int i) { return bar0 + 96 + 8 * i; };                     // PV_i before the last one finished
   auto bar_ofree = [&](int i) { return bar0 + 112 + 8 * i; };                 // O_i has been read out
@@ -492,7 +495,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       mbar_init(bar_ofree(i), 128);
       mbar_init(bar_tabfull(i), 1);
       mbar_init(bar_tabfree(i), 257);                   // 256 softmax threads + the K / V streamer
-      for (int b = 0; b < 2; ++b) { mbar_init(bar_s(i, b), 1); mbar_init(bar_p(i, b), 128); }
+      mbar_init(bar_pvd(i), 1);
+      for (int b = 0; b < C::kSBufs; ++b) { mbar_init(bar_s(i, b), 1); mbar_init(bar_p(i, b), 128); }
     }
     for (int s = 0; s < C::NS; ++s) {
       mbar_init(bar_kfull(s), 32);
@@ -583,9 +587,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       for (int na = 0; na < total && ok; ++na) {
         const int j = tile_of(q, na);
         const int gw = ga + na;
-        const int buf = gw & 1;
+        const int buf = gw % C::kSBufs;
         HA_T0(tw);
-        ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (gw >> 1) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
+        ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (gw / C::kSBufs) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
         if (!ok) break;
         HA_LACC(a_ws, tw);
         HA_T0(tc);
@@ -600,7 +604,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         // by a whole number of octaves, so that what is already accumulated (O and the row
         // sums) is rescaled exactly.
         uint32_t ra[32], rb[32];
-        const uint32_t sbase = lane_addr + 64 * (2 * i + buf);
+        const uint32_t sbase = lane_addr + 64 * (C::kSBufs * i + buf);
         // masked columns become -inf before the tile is read (out of line, in TMEM): they then
         // drop out of the maximum and exponentiate to zero without any test in this loop
         if (table || dense_mask) {
@@ -642,10 +646,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           // O may only be touched between two PV products: the one of the previous tile must
           // have finished (the one of this tile cannot start before this tile's P is published)
           if (na > 0) {
-            // S of tile na+1 is committed after the PV of tile na-1, so its arrival implies that PV;
-            // the last tile has no successor and uses the PV barrier (committed after PV total-2)
-            if (na + 1 < total) ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_s(i, (gw + 1) & 1), ((gw + 1) >> 1) & 1, s_abort, status));
-            else ok = __all_sync(0xffffffffu, mbar_wait<20, 4>(bar_pv(i), vi & 1, s_abort, status));
+            ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_pvd(i), (gw - 1) & 1, s_abort, status));
             if (!ok) break;
             tc_fence_after();
             rescale_row(lane_addr + colO, D, alpha);
@@ -795,7 +796,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       const uint32_t dk_lo0 = ((ubase + C::kOffK) >> 4) | (1u << 16);
       const uint32_t dv_lo0 = ((ubase + C::kOffV) >> 4) | (((uint32_t)(TK * 128) >> 4) << 16);
       const uint32_t ocol = tmem + C::kColO + D * i;
-      const uint32_t scol = tmem + 64 * 2 * i;
+      const uint32_t scol = tmem + 64 * C::kSBufs * i;
       bool ok = true;
       int gbase = 0;                        // global index (all items) of the item's first key tile
       int knext = 0, vnext = 0;             // next global tile whose K / V stage this issuer has to observe and release
@@ -838,58 +839,66 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         HA_LACC(b_q, tq);
         fence_async_smem();
         if (total == 0) mbar_arrive(bar_qfree);
+        auto issue_pv = [&](int a2) {
+          // ---- O += P V of key tile a2 ----------------------------------------------------------
+          const int gj = gbase + tile_of(q, a2);
+          const int s = gj % C::NS;
+          const int gw = ga + a2;
+          if (gj != vnext) skip_v(gj);
+          HA_T0(tp);
+          ok = ok && wait_fast<8>(bar_p(i, gw % C::kSBufs), (gw / C::kSBufs) & 1, s_abort, status);
+          HA_LACC(b_p, tp);
+          HA_T0(tv);
+          ok = ok && wait_fast<9>(bar_vfull(s), (gj / C::NS) & 1, s_abort, status);
+          HA_LACC(b_v, tv);
+          // the first product of an item overwrites O: the previous item's O must have been read
+          if (a2 == 0 && vi > 0) ok = ok && wait_fast<15>(bar_ofree(i), (vi - 1) & 1, s_abort, status);
+          if (!ok) return;
+          fence_async_smem();
+          tc_fence_after();
+          const uint32_t pcol = scol + 64 * (gw % C::kSBufs);
+          const uint32_t dv_lo = dv_lo0 + (uint32_t)s * (C::kTile >> 4);
+          mma_ts2(ocol, pcol, dv_lo, desc_hi, idesc_o, a2 > 0);
+#pragma unroll
+          for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
+          umma_commit(bar_vempty(i, s));
+          umma_commit(bar_pvd(i));
+          vnext = gj + 1;
+          if (a2 == total - 1) umma_commit(bar_o(i));
+        };
+        auto issue_s = [&](int r) {
+          // ---- S = Q K^T of key tile r into buffer (ga + r) % kSBufs --------------------------------
+          const int gj = gbase + tile_of(q, r);
+          const int s = gj % C::NS;
+          const int gw = ga + r;
+          if (gj != knext) skip_k(gj);
+          HA_T0(tk);
+          ok = ok && wait_fast<7>(bar_kfull(s), (gj / C::NS) & 1, s_abort, status);
+          HA_LACC(b_k, tk);
+          if (!ok) return;
+          fence_async_smem();
+          tc_fence_after();
+          const uint32_t dcol = scol + 64 * (gw % C::kSBufs);
+          const uint32_t dk_lo = dk_lo0 + (uint32_t)s * (C::kTile >> 4);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            mma_ss2(dcol, dq_lo + (((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4),
+                    dk_lo + (((ks >> 2) * (TK * 128) + (ks & 3) * 32) >> 4), desc_hi, idesc_s, ks > 0);
+          umma_commit(bar_s(i, gw % C::kSBufs));
+          umma_commit(bar_kempty(i, s));
+          knext = gj + 1;
+          if (r == total - 1) umma_commit(bar_qfree);     // nothing of this item reads Q any more
+        };
+        // The S buffer of tile r held P of tile r - kSBufs, so the product P V of that tile must be
+        // issued before the scores of tile r.  Two buffers: P V (r - 2), then S (r).  Three: the
+        // scores go first - they do not wait for the warpgroup - and are ready a tile earlier.
         for (int r = 0; r < total + 2 && ok; ++r) {
-          if (r >= 2) {
-            // ---- O += P V of key tile r - 2 ----------------------------------------------------
-            const int a2 = r - 2;
-            const int gj = gbase + tile_of(q, a2);
-            const int s = gj % C::NS;
-            const int gw = ga + a2;
-            if (gj != vnext) skip_v(gj);
-            HA_T0(tp);
-            ok = ok && wait_fast<8>(bar_p(i, gw & 1), (gw >> 1) & 1, s_abort, status);
-            HA_LACC(b_p, tp);
-            HA_T0(tv);
-            ok = ok && wait_fast<9>(bar_vfull(s), (gj / C::NS) & 1, s_abort, status);
-            HA_LACC(b_v, tv);
-            // the first product of an item overwrites O: the previous item's O must have been read
-            if (a2 == 0 && vi > 0) ok = ok && wait_fast<15>(bar_ofree(i), (vi - 1) & 1, s_abort, status);
-            if (!ok) break;
-            fence_async_smem();
-            tc_fence_after();
-            const uint32_t pcol = scol + 64 * (gw & 1);
-            const uint32_t dv_lo = dv_lo0 + (uint32_t)s * (C::kTile >> 4);
-            mma_ts2(ocol, pcol, dv_lo, desc_hi, idesc_o, a2 > 0);
-#pragma unroll
-            for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
-            umma_commit(bar_vempty(i, s));
-            vnext = gj + 1;
-            // one PV-barrier phase per item (waited for only by the rare rescale of the last tile)
-            if (a2 == (total >= 2 ? total - 2 : 0)) umma_commit(bar_pv(i));
-            if (a2 == total - 1) umma_commit(bar_o(i));
-          }
-          if (r < total) {
-            // ---- S = Q K^T of key tile r into buffer (ga + r) & 1 -----------------------------------
-            const int gj = gbase + tile_of(q, r);
-            const int s = gj % C::NS;
-            const int gw = ga + r;
-            if (gj != knext) skip_k(gj);
-            HA_T0(tk);
-            ok = ok && wait_fast<7>(bar_kfull(s), (gj / C::NS) & 1, s_abort, status);
-            HA_LACC(b_k, tk);
-            if (!ok) break;
-            fence_async_smem();
-            tc_fence_after();
-            const uint32_t dcol = scol + 64 * (gw & 1);
-            const uint32_t dk_lo = dk_lo0 + (uint32_t)s * (C::kTile >> 4);
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks)
-              mma_ss2(dcol, dq_lo + (((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4),
-                      dk_lo + (((ks >> 2) * (TK * 128) + (ks & 3) * 32) >> 4), desc_hi, idesc_s, ks > 0);
-            umma_commit(bar_s(i, gw & 1));
-            umma_commit(bar_kempty(i, s));
-            knext = gj + 1;
-            if (r == total - 1) umma_commit(bar_qfree);     // nothing of this item reads Q any more
+          if (C::kSBufs == 2) {
+            if (r >= 2) issue_pv(r - 2);
+            if (ok && r < total) issue_s(r);
+          } else {
+            if (r < total) issue_s(r);
+            if (ok && r >= 2) issue_pv(r - 2);
           }
         }
         if (!ok) break;
