@@ -10,8 +10,9 @@
 // which covers the block-diagonal part (Sec. 4), the sampled residual with weight N/m
 // (Alg. 2 line 7) and the exact causal leaves (Sec. 3.1) in one loop.  The two query tiles
 // of a 256-row block share every key tile, so K and V are fetched once for 256 rows, and
-// every warpgroup has two S buffers in TMEM, so the tensor pipe computes the scores of the
-// next key tile while the warpgroup exponentiates the current one.  The running
+// every warpgroup has two S buffers in TMEM (three for d = 64, where the columns allow it), so
+// the tensor pipe computes the scores of the next key tiles while the warpgroup exponentiates
+// the current one.  The running
 // row maximum is only moved when it grows by more than 2^32 (the accumulators absorb the
 // rest), so O is rarely rescaled; outputs are normalised by the sum of the bf16-rounded
 // weights that the tensor cores actually used, the log-sum-exp by the unrounded sum.  Rows
