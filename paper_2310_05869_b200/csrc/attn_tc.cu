@@ -464,7 +464,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   const uint32_t bar_qfree = bar0 + 8;                                        // both issuers are done with Q
   auto bar_s = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 3 * i + b); };          // S_i buffer b written
   auto bar_p = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 6 + 3 * i + b); };      // P_i buffer b written
-  auto bar_pvd = [&](int i) { return bar0 + 16 + 8 * i; };                    // P_i V of a key tile finished (one phase per tile)
+  // P_i V of a key tile finished; two barriers per query tile, used alternately: with three S
+  // buffers the scores run up to three tiles ahead of the last finished P V, and a parity wait on a
+  // single barrier cannot tell "one phase behind" from "done"
+  auto bar_pvd = [&](int i, int b) { return bar0 + 16 + 8 * (2 * i + b); };
   auto bar_o = [&](int i) { return bar0 + 80 + 8 * i; };                      // O_i of the item complete
   auto bar_pv = [&](int i) { return bar0 + 96 + 8 * i; };                     // PV_i before the last one finished
   auto bar_ofree = [&](int i) { return bar0 + 112 + 8 * i; };                 // O_i has been read out
@@ -496,7 +499,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       mbar_init(bar_ofree(i), 128);
       mbar_init(bar_tabfull(i), 1);
       mbar_init(bar_tabfree(i), 257);                   // 256 softmax threads + the K / V streamer
-      mbar_init(bar_pvd(i), 1);
+      mbar_init(bar_pvd(i, 0), 1); mbar_init(bar_pvd(i, 1), 1);
       for (int b = 0; b < C::kSBufs; ++b) { mbar_init(bar_s(i, b), 1); mbar_init(bar_p(i, b), 128); }
     }
     for (int s = 0; s < C::NS; ++s) {
@@ -647,7 +650,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           // O may only be touched between two PV products: the one of the previous tile must
           // have finished (the one of this tile cannot start before this tile's P is published)
           if (na > 0) {
-            ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_pvd(i), (gw - 1) & 1, s_abort, status));
+            ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_pvd(i, (gw - 1) & 1), ((gw - 1) >> 1) & 1, s_abort, status));
             if (!ok) break;
             tc_fence_after();
             rescale_row(lane_addr + colO, D, alpha);
@@ -863,7 +866,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 #pragma unroll
           for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
           umma_commit(bar_vempty(i, s));
-          umma_commit(bar_pvd(i));
+          umma_commit(bar_pvd(i, gw & 1));
           vnext = gj + 1;
           if (a2 == total - 1) umma_commit(bar_o(i));
         };

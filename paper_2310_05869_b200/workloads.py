@@ -43,7 +43,7 @@ class Workload:
     r: int
     causal: bool
     n0: int
-    kind: str           # "gaussian" | "clustered" | "student_t"
+    kind: str           # "gaussian" | "clustered" | "student_t" | "ramp"
     gen_seed: int
     seed: int = 0       # the library's seed (hash directions and sampled columns)
 
@@ -89,11 +89,25 @@ def _student_t(rng, G, n, d, dof=3.0, clip=20.0):
     return [np.clip(rng.standard_t(dof, size=(G, n, d)), -clip, clip).astype(np.float32) for _ in range(3)]
 
 
+def _ramp(rng, G, n, d):
+    """Logits that keep growing along the key index: every query is close to one direction u,
+    key j is (j / n) * 24 * sqrt(d) * u plus noise, so the row maxima found while walking the
+    keys in index order rise by hundreds of octaves - a stress case for running-maximum bookkeeping.  Test input
+    only; not one of the paper's workloads."""
+    u = rng.standard_normal((G, 1, d)).astype(np.float32)
+    u /= np.linalg.norm(u, axis=2, keepdims=True)
+    q = (u * np.sqrt(d) * 3.0 + 0.3 * rng.standard_normal((G, n, d))).astype(np.float32)
+    ramp = (np.arange(n, dtype=np.float32) / n)[None, :, None]
+    k = (u * ramp * 24.0 * np.sqrt(d) + 0.3 * rng.standard_normal((G, n, d))).astype(np.float32)
+    v = rng.standard_normal((G, n, d)).astype(np.float32)
+    return [q, k, v]
+
+
 def make_inputs(w: Workload):
     """Returns Q, K, V as numpy arrays of shape (G, n, d): float32 for "fp32" workloads,
     uint16 bf16 bit patterns for "bf16" workloads."""
     rng = np.random.Generator(np.random.PCG64(w.gen_seed))
-    gen = {"gaussian": _gaussian, "clustered": _clustered, "student_t": _student_t}[w.kind]
+    gen = {"gaussian": _gaussian, "clustered": _clustered, "student_t": _student_t, "ramp": _ramp}[w.kind]
     qkv = gen(rng, w.G, w.n, w.d)
     if w.dtype == "bf16":
         return [f32_to_bf16_bits(x) for x in qkv]

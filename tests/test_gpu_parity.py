@@ -46,6 +46,10 @@ SMALL = [
     # items with more key tiles than ring stages
     W("unpaired_tiles_b384_d128", 1, 2, 3072, 128, "bf16", 384, 128, 7, False, 0, seed=22),
     W("unpaired_tiles_b640_d64", 1, 1, 5120, 64, "bf16", 640, 256, 7, False, 0, seed=23),
+    # logits that keep growing along the keys: the running maximum moves (and O is rescaled) again and again
+    W("ramp_rescales_d64", 1, 2, 4096, 64, "bf16", 256, 256, 7, False, 0, kind="ramp", seed=24),
+    W("ramp_rescales_causal_d128", 1, 2, 4096, 128, "bf16", 128, 128, 7, True, 1024, kind="ramp", seed=25),
+    W("ramp_rescales_causal_d64", 1, 2, 8192, 64, "bf16", 256, 64, 7, True, 2048, kind="ramp", seed=26),
 ]
 
 
