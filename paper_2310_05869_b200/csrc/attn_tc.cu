@@ -587,7 +587,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       unsigned tile_masked = 0;
       if (t.mode == 1) tile_masked = __ballot_sync(0xffffffffu, lane < t.ntiles && (s_mask[2 * lane] | s_mask[2 * lane + 1]) != 0);
       float m_ref = -INFINITY;
-      uint64_t l01 = 0, lr01 = 0;   // l: unrounded row sum, lr: sum of the bf16 weights (two partial sums each, packed)
+      uint64_t l01 = 0;             // l: unrounded row sum (two partial sums, packed)
+      float lra = 0.f, lrb = 0.f;   // lr: sum of the bf16 weights (two partial sums; the mixed-precision add takes the bf16 halves as they are)
       for (int na = 0; na < total && ok; ++na) {
         const int j = tile_of(q, na);
         const int gw = ga + na;
@@ -646,7 +647,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             if (m_ref == -INFINITY) { m_ref = xm + (wlog - ubias); alpha = 0.f; }
             else { const float k = ceilf(xm - m_ref); m_ref += k; alpha = ex2(-k); }
           }
-          { const uint64_t al2 = pack_f2(alpha, alpha); l01 = fmul2(l01, al2); lr01 = fmul2(lr01, al2); }
+          { const uint64_t al2 = pack_f2(alpha, alpha); l01 = fmul2(l01, al2); lra *= alpha; lrb *= alpha; }
           // O may only be touched between two PV products: the one of the previous tile must
           // have finished (the one of this tile cannot start before this tile's P is published)
           if (na > 0) {
@@ -668,7 +669,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             const float p0 = ex2(x0), p1 = ex2(x1);
             l01 = fadd2(l01, pack_f2(p0, p1));
             const uint32_t w = pack2(p0, p1);
-            lr01 = fadd2(lr01, pack_u2(w << 16, w & 0xffff0000u));
+            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}" : "+f"(lra), "+f"(lrb) : "r"(w));
             p[e >> 1] = w;
           }
           tmem_st16(sbase + c * 16, p);
@@ -701,7 +702,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         const int qr = s_qrow[row];
         float l0, l1, lr0, lr1;
         unpack_f2(l01, l0, l1);
-        unpack_f2(lr01, lr0, lr1);
+        lr0 = lra; lr1 = lrb;
         const float inv = 1.f / (lr0 + lr1);
         const float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
         const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
