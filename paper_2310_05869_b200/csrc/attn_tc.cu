@@ -10,12 +10,13 @@
 // which covers the block-diagonal part (Sec. 4), the sampled residual with weight N/m
 // (Alg. 2 line 7) and the exact causal leaves (Sec. 3.1) in one loop.  The two query tiles
 // of a 256-row block share every key tile, so K and V are fetched once for 256 rows, and
-// every warpgroup has two S buffers in TMEM (three for d = 64, where the columns allow it), so
-// the tensor pipe computes the scores of the next key tiles while the warpgroup exponentiates
-// the current one.  The running
+// every warpgroup has two S buffers in TMEM, so the tensor pipe computes the scores of the next
+// key tile while the warpgroup exponentiates the current one.  The running
 // row maximum is only moved when it grows by more than 2^32 (the accumulators absorb the
 // rest), so O is rarely rescaled; outputs are normalised by the sum of the bf16-rounded
-// weights that the tensor cores actually used, the log-sum-exp by the unrounded sum.  Rows
+// weights that the tensor cores actually used (d = 64: accumulated by the tensor cores
+// themselves, in an extra column of O whose B operand is a slab of ones; d = 128: in
+// registers), the log-sum-exp by the unrounded sum.  Rows
 // of Q, K, V come from their original places: tiles of consecutive rows (causal leaves) as
 // one TMA box per 64 columns, tiles of sorted or sampled rows gathered through the sortLSH
 // permutations with 16-byte cp.async copies into the same 128B-swizzled operand layout;
@@ -24,7 +25,7 @@
 //
 // Warp roles (384 threads): warps 0-3 and 4-7 softmax + epilogue of query tile 0 and 1,
 // warps 8 and 9 MMA issue for query tile 0 and 1 (warp 8 also allocates TMEM, all 512
-// columns: per query tile two S buffers of 64 - three for d = 64 - then O0, O1), warp 10 prepares work items (row tables of the
+// columns: per query tile two S buffers of 64, then O0, O1), warp 10 prepares work items (row tables of the
 // NEXT item while this one computes, TMA boxes of Q), warp 11 streams K / V tiles through
 // the stage ring, across item boundaries.  Gathered Q tiles are fetched by the 256 softmax
 // threads, for the next item, right before they write the current item's results.
@@ -343,7 +344,14 @@ struct Cfg {
   static constexpr int kOffMask = kOffIdx + 2 * kMaxNodeKeys * 4; // uint32 [2][2][kMaxNodeKeys/32] masked-column bits
   static constexpr int kOffQrow = kOffMask + 4 * (kMaxNodeKeys / 32) * 4;   // int [2][2][128]
   static constexpr int kOffBar = kOffQrow + 4 * 128 * 4;
-  static constexpr int kSBufs = (D == 64) ? 3 : 2;    // S buffers per query tile (d = 64 leaves TMEM columns for a third)
+  static constexpr int kSBufs = 2;                    // S buffers per query tile
+  // d = 64: the P V product is 80 columns wide - behind the 64 columns of V the B operand
+  // continues in a slab of ones, so column 64 of O accumulates the sum of the bf16 weights that
+  // normalises the row (the tensor pipe's floor per product does not depend on N up to 128, so
+  // the extra columns are free and the softmax warps save one add per weight).  d = 128 would
+  // pay for them (N = 144) and keeps the sum in registers.
+  static constexpr bool kOnes = D == 64;
+  static constexpr int kOCols = kOnes ? 80 : D;       // TMEM columns of one O accumulator
   static constexpr int kNumBar = 21 + 6 * NS + 12;
   static constexpr int kOffMisc = kOffBar + 8 * kNumBar;          // tmem slot, abort flag
   // Epilogue staging, one slice of 32 rows x kStageRow bytes per softmax warp: rows leave the
@@ -356,11 +364,13 @@ struct Cfg {
   static constexpr int kDescBytes = (sizeof(ItemDesc) + 15) / 16 * 16;
   static constexpr int kOffDesc = (kOffMisc + 16 + 15) / 16 * 16;   // ItemDesc [2], one per table set
   static constexpr int kOffStage = (kOffDesc + 2 * kDescBytes + 127) / 128 * 128;
-  static constexpr int kTotal = kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;
+  static constexpr int kOffOnes = (kOffStage + ((D == 64) ? 8 : 4) * kStageWarp + 1023) / 1024 * 1024;   // [TK keys x 128 B] of bf16 1.0
+  static constexpr int kTotal = kOnes ? kOffOnes + TK * 128 : kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;
+  static_assert(kTotal <= 232448, "shared memory");
   static_assert(D == 64 || 4 * kStageWarp <= kMaxNodeKeys * 4, "staging of query tile 0 must fit one key-row table");
   static constexpr int kTmemCols = 512;
-  static constexpr int kColO = 64 * 2 * kSBufs;       // S buffer b of tile i at 64 (kSBufs i + b); O_i at kColO + D i
-  static_assert(kColO + 2 * D <= 512, "TMEM columns");
+  static constexpr int kColO = 64 * 2 * kSBufs;       // S buffer b of tile i at 64 (kSBufs i + b); O_i at kColO + kOCols i
+  static_assert(kColO + 2 * kOCols <= 512, "TMEM columns");
 };
 
 __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDesc& t, QTile& qa, QTile& qb) {
@@ -464,9 +474,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   const uint32_t bar_qfree = bar0 + 8;                                        // both issuers are done with Q
   auto bar_s = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 3 * i + b); };          // S_i buffer b written
   auto bar_p = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 6 + 3 * i + b); };      // P_i buffer b written
-  // P_i V of a key tile finished; two barriers per query tile, used alternately: with three S
-  // buffers the scores run up to three tiles ahead of the last finished P V, and a parity wait on a
-  // single barrier cannot tell "one phase behind" from "done"
+  // P_i V of a key tile finished; two barriers per query tile, used alternately, so that the
+  // (rare) waiter can never mistake "one phase behind" for "done" however far the scores run ahead
   auto bar_pvd = [&](int i, int b) { return bar0 + 16 + 8 * (2 * i + b); };
   auto bar_o = [&](int i) { return bar0 + 80 + 8 * i; };                      // O_i of the item complete
   auto bar_pv = [&](int i) { return bar0 + 96 + 8 * i; };                     // PV_i before the last one finished
@@ -509,6 +518,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if constexpr (C::kOnes) {
+    for (int k = tid; k < TK * 128 / 16; k += 384) *reinterpret_cast<uint4*>(smem + C::kOffOnes + 16 * k) = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
+    fence_async_smem();                                 // the tensor pipe reads the slab through the async proxy
+  }
   if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(C::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -527,7 +540,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     const int i = warp >> 2;
     const int row = tid & 127;
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t colO = C::kColO + D * i;
+    const uint32_t colO = C::kColO + C::kOCols * i;
     int ga = 0;                                       // key tiles this warpgroup has processed so far (all items)
     int vi = 0;                                       // items in which this query tile existed
     bool ok = true;
@@ -654,7 +667,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_pvd(i, (gw - 1) & 1), ((gw - 1) >> 1) & 1, s_abort, status));
             if (!ok) break;
             tc_fence_after();
-            rescale_row(lane_addr + colO, D, alpha);
+            rescale_row(lane_addr + colO, C::kOCols, alpha);
           }
         }
         const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
@@ -669,7 +682,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             const float p0 = ex2(x0), p1 = ex2(x1);
             l01 = fadd2(l01, pack_f2(p0, p1));
             const uint32_t w = pack2(p0, p1);
-            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}" : "+f"(lra), "+f"(lrb) : "r"(w));
+            if constexpr (!C::kOnes)
+              asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}" : "+f"(lra), "+f"(lrb) : "r"(w));
             p[e >> 1] = w;
           }
           tmem_st16(sbase + c * 16, p);
@@ -703,6 +717,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         float l0, l1, lr0, lr1;
         unpack_f2(l01, l0, l1);
         lr0 = lra; lr1 = lrb;
+        if constexpr (C::kOnes) {                       // the sum of the bf16 weights sits in column D of O
+          uint32_t sumw;
+          asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];\n\ttcgen05.wait::ld.sync.aligned;\n" : "=r"(sumw) : "r"(lane_addr + colO + D) : "memory");
+          lr0 = __uint_as_float(sumw); lr1 = 0.f;
+        }
         const float inv = 1.f / (lr0 + lr1);
         const float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
         const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
@@ -793,14 +812,18 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     const int i = warp - 8;
     if (lane == 0) {
       constexpr uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)TK >> 3) << 17) | ((128u >> 4) << 24);
-      constexpr uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
+      constexpr uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)C::kOCols >> 3) << 17) | ((128u >> 4) << 24);
       // descriptor: low word = start address >> 4 | (leading byte offset >> 4) << 16,
       // high word = stride byte offset >> 4 | version 1 << 14 | 128-byte swizzle 2 << 29
       constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
       const uint32_t dq_lo = ((ubase + C::kOffQ + i * C::kQTile) >> 4) | (1u << 16);
       const uint32_t dk_lo0 = ((ubase + C::kOffK) >> 4) | (1u << 16);
-      const uint32_t dv_lo0 = ((ubase + C::kOffV) >> 4) | (((uint32_t)(TK * 128) >> 4) << 16);
-      const uint32_t ocol = tmem + C::kColO + D * i;
+      // V descriptors: the leading byte offset is the distance to the next 64 columns of the B
+      // operand - the tile's second slab (d = 128) or the slab of ones (d = 64), whose distance
+      // shrinks by one tile per stage
+      const uint32_t dv_lo0 = ((ubase + C::kOffV) >> 4) | (((uint32_t)(C::kOnes ? C::kOffOnes - C::kOffV : TK * 128) >> 4) << 16);
+      constexpr uint32_t dv_step = (uint32_t)(C::kTile >> 4) - (C::kOnes ? ((uint32_t)(C::kTile >> 4) << 16) : 0u);   // per stage
+      const uint32_t ocol = tmem + C::kColO + C::kOCols * i;
       const uint32_t scol = tmem + 64 * C::kSBufs * i;
       bool ok = true;
       int gbase = 0;                        // global index (all items) of the item's first key tile
@@ -862,7 +885,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           fence_async_smem();
           tc_fence_after();
           const uint32_t pcol = scol + 64 * (gw % C::kSBufs);
-          const uint32_t dv_lo = dv_lo0 + (uint32_t)s * (C::kTile >> 4);
+          const uint32_t dv_lo = dv_lo0 + (uint32_t)s * dv_step;
           mma_ts2(ocol, pcol, dv_lo, desc_hi, idesc_o, a2 > 0);
 #pragma unroll
           for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
