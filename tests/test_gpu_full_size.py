@@ -15,7 +15,10 @@ import parity_util as PU
 
 pytestmark = pytest.mark.gpu
 
-FULL = [WL.CONFIGS[1], WL.CONFIGS[2], WL.CONFIGS[3], WL.CONFIGS[4]]
+# beyond the benchmark sizes: a million rows (eight recursion levels over 256 leaves) and half a million rows of d = 128
+LONG = [WL.Workload("long_n1m_causal", 1, 2, 1048576, 64, "bf16", 256, 256, 7, True, 4096, "gaussian", 1010),
+        WL.Workload("long_n512k_d128", 1, 1, 524288, 128, "bf16", 256, 256, 7, False, 0, "gaussian", 1011)]
+FULL = [WL.CONFIGS[1], WL.CONFIGS[2], WL.CONFIGS[3], WL.CONFIGS[4]] + LONG
 
 
 @pytest.mark.parametrize("w", FULL, ids=[w.name for w in FULL])
