@@ -125,10 +125,15 @@ int hyperattn_forward(const void* q, const void* k, const void* v, void* out, fl
 int hyperattn_forward_ex(const hyperattn_params* p);
 
 /* The same computation for HOST buffers: q, k, v, out, lse of *p are host pointers (pinned
- * memory makes the copies asynchronous).  The inputs are copied to a private device staging
- * area on `stream`, the forward pass runs there, and out / lse are copied back on the same
- * stream; the caller synchronises the stream before reading them.  The staging area is
- * grown on demand (that call synchronises the device) and kept until hyperattn_release(). */
+ * memory makes the copies asynchronous).  The (batch, head) segments are independent, so they
+ * go through a private device staging area in up to eight groups: the copy of the next group to
+ * the device and the copy of the previous group's out / lse back run on two streams of the
+ * library while a group is computed on `stream`.  Everything is ordered after the work already
+ * queued on `stream`, and `stream` is made to wait for the last copy back: the caller
+ * synchronises `stream` before reading the results.  Results are bit-identical to
+ * hyperattn_forward_ex on device copies of the same tensors.  With debug outputs requested the
+ * batch is one group.  The staging area is grown on demand (that call synchronises the device)
+ * and kept, like the two streams, until hyperattn_release(). */
 int hyperattn_forward_host(const hyperattn_params* p);
 
 /* Bytes of device scratch hyperattn_forward_ex needs for these shapes (host-side; only the

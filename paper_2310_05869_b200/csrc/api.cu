@@ -33,6 +33,7 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
   if ((long long)p.B * p.H > (1 << 20)) return HYPERATTN_UNSUPPORTED_SHAPE;
   if (p.n > (1 << 28)) return HYPERATTN_UNSUPPORTED_SHAPE;
   std::memset(&g, 0, sizeof(g));
+  g.seg0 = 0;
   g.G = p.B * p.H; g.n = p.n; g.d = p.d; g.b = p.block; g.m = p.samples; g.r = p.hash_bits;
   if (!p.causal) {
     g.causal = 0; g.L = 0; g.leaf = p.n; g.unit = p.n;
@@ -117,10 +118,14 @@ void make_directions(int d, int r, uint64_t seed, float* w) {
 }
 
 // ---- per-process state ---------------------------------------------------------------------
+constexpr int kHostChunks = 8;          // the host-buffer entry point pipelines copies and compute over this many groups of segments
 struct DeviceState {
   void* ws = nullptr; size_t ws_bytes = 0;
   void* host_stage = nullptr; size_t host_stage_bytes = 0;   // device staging for the host-buffer entry
   int* status = nullptr;
+  // host-buffer entry point: one stream per copy direction, events that order them with the caller's stream
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_end = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
 };
 struct StageEvents { cudaEvent_t beg, end; int stage; int launches; };
 
@@ -160,10 +165,13 @@ int check_ptrs(const hyperattn_params& p) {
   return HYPERATTN_OK;
 }
 
-int forward_impl(const hyperattn_params& p) {
+// seg0: index of the call's first segment in the caller's whole tensor (not 0 when a caller's batch is
+// processed in several calls: the samples of a segment depend on its index)
+int forward_impl(const hyperattn_params& p, int seg0 = 0) {
   Geometry g;
   int rc = build_geometry(p, g);
   if (rc) return rc;
+  g.seg0 = seg0;
   rc = check_ptrs(p);
   if (rc) return rc;
   const int is_fp32 = p.dtype == HYPERATTN_FP32;
@@ -365,18 +373,58 @@ int hyperattn_forward_host(const hyperattn_params* hp) {
     stage = reinterpret_cast<char*>(ds.host_stage);
   }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(hp->stream);
-  hyperattn_params p = *hp;
-  p.q = stage; p.k = stage + in_b; p.v = stage + 2 * in_b;
-  p.out = stage + 3 * in_b; p.lse = reinterpret_cast<float*>(stage + 3 * in_b + out_b);
-  if (cudaMemcpyAsync(const_cast<void*>(p.q), hp->q, elems * es, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(const_cast<void*>(p.k), hp->k, elems * es, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(const_cast<void*>(p.v), hp->v, elems * es, cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return HYPERATTN_CUDA_ERROR;
-  rc = forward_impl(p);
-  if (rc) return rc;
-  if (cudaMemcpyAsync(hp->out, p.out, elems * eo, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      cudaMemcpyAsync(hp->lse, p.lse, (size_t)g.G * g.n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return HYPERATTN_CUDA_ERROR;
+  char* dq = stage; char* dk = stage + in_b; char* dv = stage + 2 * in_b;
+  char* dout = stage + 3 * in_b; char* dlse = stage + 3 * in_b + out_b;
+  // Segments are independent, so the batch goes through in groups: the copy of group c + 1 to the
+  // device and the copy of group c - 1 back run (on streams of their own, PCIe being full duplex)
+  // while group c is computed on the caller's stream.  With debug outputs requested, one group.
+  DeviceState* dsp;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    dsp = &g_dev[dev];
+    if (!dsp->copy_in) {
+      bool good = cudaStreamCreateWithFlags(&dsp->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&dsp->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&dsp->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&dsp->ev_end, cudaEventDisableTiming) == cudaSuccess;
+      for (int c = 0; c < kHostChunks && good; ++c)
+        good = cudaEventCreateWithFlags(&dsp->ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&dsp->ev_done[c], cudaEventDisableTiming) == cudaSuccess;
+      if (!good) { dsp->copy_in = nullptr; return HYPERATTN_CUDA_ERROR; }
+    }
+  }
+  DeviceState& ds = *dsp;
+  const int nchunks = hp->debug ? 1 : (g.G < kHostChunks ? g.G : kHostChunks);
+  const int per = (g.G + nchunks - 1) / nchunks;
+  const size_t seg_in = (size_t)g.n * g.d * es, seg_out = (size_t)g.n * g.d * eo, seg_lse = (size_t)g.n * 4;
+#define HA_HOST(x) do { if ((x) != cudaSuccess) { std::fprintf(stderr, "hyperattn: %s failed\n", #x); return HYPERATTN_CUDA_ERROR; } } while (0)
+  // the staging buffers may still be in use by work queued earlier on the caller's stream
+  HA_HOST(cudaEventRecord(ds.ev_start, st));
+  HA_HOST(cudaStreamWaitEvent(ds.copy_in, ds.ev_start, 0));
+  HA_HOST(cudaStreamWaitEvent(ds.copy_out, ds.ev_start, 0));
+  for (int c = 0, s0 = 0; s0 < g.G; ++c, s0 += per) {
+    const int ns = (g.G - s0) < per ? (g.G - s0) : per;
+    const size_t oi = (size_t)s0 * seg_in, oo = (size_t)s0 * seg_out, ol = (size_t)s0 * seg_lse;
+    HA_HOST(cudaMemcpyAsync(dq + oi, static_cast<const char*>(hp->q) + oi, ns * seg_in, cudaMemcpyHostToDevice, ds.copy_in));
+    HA_HOST(cudaMemcpyAsync(dk + oi, static_cast<const char*>(hp->k) + oi, ns * seg_in, cudaMemcpyHostToDevice, ds.copy_in));
+    HA_HOST(cudaMemcpyAsync(dv + oi, static_cast<const char*>(hp->v) + oi, ns * seg_in, cudaMemcpyHostToDevice, ds.copy_in));
+    HA_HOST(cudaEventRecord(ds.ev_in[c], ds.copy_in));
+    HA_HOST(cudaStreamWaitEvent(st, ds.ev_in[c], 0));
+    hyperattn_params p = *hp;
+    p.B = 1; p.H = ns;
+    p.q = dq + oi; p.k = dk + oi; p.v = dv + oi;
+    p.out = dout + oo; p.lse = reinterpret_cast<float*>(dlse + ol);
+    rc = forward_impl(p, s0);
+    if (rc) return rc;
+    HA_HOST(cudaEventRecord(ds.ev_done[c], st));
+    HA_HOST(cudaStreamWaitEvent(ds.copy_out, ds.ev_done[c], 0));
+    HA_HOST(cudaMemcpyAsync(static_cast<char*>(hp->out) + oo, dout + oo, ns * seg_out, cudaMemcpyDeviceToHost, ds.copy_out));
+    HA_HOST(cudaMemcpyAsync(reinterpret_cast<char*>(hp->lse) + ol, dlse + ol, ns * seg_lse, cudaMemcpyDeviceToHost, ds.copy_out));
+  }
+  // the caller's stream is done when the last results are on the host
+  HA_HOST(cudaEventRecord(ds.ev_end, ds.copy_out));
+  HA_HOST(cudaStreamWaitEvent(st, ds.ev_end, 0));
+#undef HA_HOST
   return HYPERATTN_OK;
 }
 
@@ -454,6 +502,11 @@ int hyperattn_release(void) {
     if (kv.second.ws) cudaFree(kv.second.ws);
     if (kv.second.host_stage) cudaFree(kv.second.host_stage);
     if (kv.second.status) cudaFree(kv.second.status);
+    if (kv.second.copy_in) {
+      cudaStreamDestroy(kv.second.copy_in); cudaStreamDestroy(kv.second.copy_out);
+      cudaEventDestroy(kv.second.ev_start); cudaEventDestroy(kv.second.ev_end);
+      for (int c = 0; c < kHostChunks; ++c) { cudaEventDestroy(kv.second.ev_in[c]); cudaEventDestroy(kv.second.ev_done[c]); }
+    }
   }
   g_dev.clear();
   for (auto& ev : g_events) { cudaEventDestroy(ev.beg); cudaEventDestroy(ev.end); }

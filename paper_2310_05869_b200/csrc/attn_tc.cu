@@ -47,9 +47,6 @@ struct alignas(64) TmaMaps {
 constexpr int TK = 64;                  // keys per tile
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
 constexpr float kRescaleThreshold = 32.f;   // octaves the scores may exceed the reference before it moves
-#ifndef HA_TAKE_TURNS
-#define HA_TAKE_TURNS 0
-#endif
 
 // Optional per-role cycle counters (compile with -DHA_TC_TIMING; never in the shipped build).
 #ifdef HA_TC_TIMING
@@ -478,7 +475,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   // (rare) waiter can never mistake "one phase behind" for "done" however far the scores run ahead
   auto bar_pvd = [&](int i, int b) { return bar0 + 16 + 8 * (2 * i + b); };
   auto bar_o = [&](int i) { return bar0 + 80 + 8 * i; };                      // O_i of the item complete
-  auto bar_pv = [&](int i) { return bar0 + 96 + 8 * i; };                     // PV_i before the last one finished
   auto bar_ofree = [&](int i) { return bar0 + 112 + 8 * i; };                 // O_i has been read out
   auto bar_tabfull = [&](int set) { return bar0 + 128 + 8 * set; };           // row tables of a set written
   auto bar_tabfree = [&](int set) { return bar0 + 144 + 8 * set; };           // softmax warps are done with a set
@@ -504,7 +500,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     mbar_init(bar_qfree, 2);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_o(i), 1);
-      mbar_init(bar_pv(i), 1);
       mbar_init(bar_ofree(i), 128);
       mbar_init(bar_tabfull(i), 1);
       mbar_init(bar_tabfree(i), 257);                   // 256 softmax threads + the K / V streamer

@@ -60,6 +60,7 @@ struct Geometry {
   int nl;              // sorted rows per (level, segment, side): n/2 causal, n non-causal
   int nodes;           // off-diagonal nodes per segment (heap-numbered)
   int sorted;          // 1 if any node needs sortLSH (some node has b < its size)
+  int seg0;            // index, in the caller's tensor, of this call's first segment (the sampling counters carry it)
 };
 
 // sorted blocks of a node of s rows: ceil(s / b) of them, the last one with the remaining rows

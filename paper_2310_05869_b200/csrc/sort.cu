@@ -46,7 +46,7 @@ __device__ __forceinline__ void samples_body(const SampleArgs& a, int block, int
     const int seg = (int)(i / ((size_t)calls * g.nodes));
     const int level = g.causal ? 31 - __clz(nd + 1) : 0;
     const uint32_t N = g.causal ? (uint32_t)(g.n >> (level + 1)) : (uint32_t)g.n;
-    const Philox4 x = philox4x32_10((uint32_t)c, (uint32_t)seg, (uint32_t)nd, kDomainSamples, a.k0, a.k1);
+    const Philox4 x = philox4x32_10((uint32_t)c, (uint32_t)(g.seg0 + seg), (uint32_t)nd, kDomainSamples, a.k0, a.k1);
     int32_t* dst = a.samples + ((size_t)seg * g.nodes + nd) * g.m;
 #pragma unroll
     for (int w = 0; w < 4; ++w)
