@@ -454,7 +454,9 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
 
 // a-th key tile of a query tile -> index in the pair's tile list
 __device__ __forceinline__ int tile_of(const QTile& q, int a) { return a < q.n1 ? q.s1 + a : q.s2 + (a - q.n1); }
-template <int D>
+// GATHER_LATE: the softmax threads fetch the next item's Q tiles after, not before, they write
+// the current item's results (see there).
+template <int D, bool GATHER_LATE>
 __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TmaMaps maps, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -694,9 +696,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 #endif
       }
       if (!ok) break;
-      // the next item's Q tiles go out before this item's results are written
+      // The next item's Q tiles go out before this item's results are written, so that they are
+      // there when the results are - except for fp32 partial results of d = 128 (causal
+      // recursion): those are twice the bytes to stage and store and queue behind the gather's
+      // copies in the load/store unit (measured: 5 % faster with the gather after them, while
+      // bf16 results are 5 % slower that way).
       HA_T0(tg);
-      if (item + (int)gridDim.x < a.total_pairs) {
+      if (!GATHER_LATE && item + (int)gridDim.x < a.total_pairs) {
         ok = __all_sync(0xffffffffu, gather_q(it + 1));
         if (!ok) break;
       }
@@ -784,6 +790,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           else a.lse[orow] = lse;
         }
         ++vi;
+      }
+      if (GATHER_LATE && item + (int)gridDim.x < a.total_pairs) {
+        ok = __all_sync(0xffffffffu, gather_q(it + 1));
+        if (!ok) break;
       }
       mbar_arrive(bar_tabfree(set));
       HA_LACC(a_epi, te);
@@ -1264,8 +1274,9 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
     kernel<<<grid, 384, smem_bytes, st>>>(a, maps, status);
     return cudaGetLastError();
   };
-  if (a.g.d == 64) return go(attn_tc_kernel<64>, Cfg<64>::kTotal);
-  return go(attn_tc_kernel<128>, Cfg<128>::kTotal);
+  if (a.g.d == 64) return go(attn_tc_kernel<64, false>, Cfg<64>::kTotal);
+  if (!a.direct) return go(attn_tc_kernel<128, true>, Cfg<128>::kTotal);
+  return go(attn_tc_kernel<128, false>, Cfg<128>::kTotal);
 }
 
 }  // namespace hyperattn
