@@ -25,6 +25,11 @@ r hash bits; P_Q, P_K the sortLSH permutations; M^H the block mask):
   causal_forward     recursive split (Alg. 4) carried through to outputs
   forward            all (batch, head) segments
   dense_weights      the implied n x n row-stochastic weight matrix (tiny n only)
+  dense_coefficients the matrix C with W~ = rownorm(C o exp(scale Q K^T)) (tiny n only)
+  dense_backward     gradients of (out, lse) with respect to Q, K, V with the sortLSH
+                     permutations and the sampled columns held fixed (tiny n only); the paper
+                     times a backward pass (Sec. 4.2) but never writes it down: this is the
+                     derivative of the forward map as defined above, nothing more
 
 Parity status: every function here is pinned by the CPU tests (brute force on tiny
 inputs, closed forms, the Fig. 1 example, Monte-Carlo checks, published Philox
@@ -388,3 +393,64 @@ def dense_weights(Q, K, ids_q, ids_k, b, m, scale, causal, n0, seed, g, _node=0)
         mm = m if b < N else 0
         U = _dense_unnormalised(Q, K, ids_q, ids_k, sample_indices(seed, g, 0, mm, N), b, scale)
     return U / U.sum(axis=1, keepdims=True)
+
+
+# --------------------------------------------------------------------------------------
+# Backward pass (tiny n only): derivative of the forward map, discrete choices held fixed
+# --------------------------------------------------------------------------------------
+def dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g, _node=0):
+    """C (n x n, entries >= 0) such that the forward pass is out = rownorm(C o A) V,
+    lse = ln rowsum(C o A), A = exp(scale Q K^T).  C depends on Q and K only through the
+    bucket ids: C_ij = 1 on the block mask M^H, (N/m) * multiplicity of j among the
+    samples elsewhere (Alg. 2 lines 7 and 9 without caps), the lower triangle of ones in
+    an exact causal leaf, zero above the diagonal blocks of the recursion (Alg. 4)."""
+    def coeff(N, iq, ik, node):
+        if causal and N <= n0:
+            return np.tril(np.ones((N, N)))
+        if causal:
+            h = N // 2
+            C = np.zeros((N, N))
+            C[:h, :h] = coeff(h, iq[:h], ik[:h], 2 * node + 1)
+            C[h:, h:] = coeff(h, iq[h:], ik[h:], 2 * node + 2)
+            C[h:, :h] = block(h, iq[h:], ik[:h], node)
+            return C
+        return block(N, iq, ik, node)
+
+    def block(N, iq, ik, node):
+        if b >= N:
+            return np.ones((N, N))
+        _, rank_q = stable_argsort(iq)
+        _, rank_k = stable_argsort(ik)
+        M = sortlsh_mask(rank_q, rank_k, b).astype(np.float64)
+        smp = sample_indices(seed, g, node, m, N)
+        c = np.bincount(np.asarray(smp, dtype=np.int64), minlength=N).astype(np.float64)
+        return M + (N / max(m, 1)) * c[None, :] * (1.0 - M)
+
+    return coeff(n, np.asarray(ids_q), np.asarray(ids_k), _node)
+
+
+def dense_backward(Q, K, V, C, scale, d_out, d_lse=None):
+    """Gradients of L = <d_out, out> + <d_lse, lse> for out = P V, P = rownorm(C o A),
+    lse = ln rowsum(C o A), A = exp(scale Q K^T), C constant:
+        dV = P^T d_out
+        dP = d_out V^T
+        dS = P o (dP - rowsum(P o dP) + d_lse)      (softmax Jacobian; d lse_i / d s_ij = P_ij)
+        dQ = scale dS K,   dK = scale dS^T Q.
+    Returns (dQ, dK, dV), fp64."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    d_out = np.asarray(d_out, dtype=np.float64)
+    s = scale * (Q @ K.T)
+    with np.errstate(divide="ignore"):
+        z = s + np.log(C)
+    z = z - z.max(axis=1, keepdims=True)
+    P = np.exp(z)
+    P = P / P.sum(axis=1, keepdims=True)
+    dV = P.T @ d_out
+    dP = d_out @ V.T
+    inner = (P * dP).sum(axis=1, keepdims=True)
+    dS = P * (dP - inner)
+    if d_lse is not None:
+        dS = dS + P * np.asarray(d_lse, dtype=np.float64)[:, None]
+    return scale * (dS @ K), scale * (dS.T @ Q), dV

@@ -397,3 +397,49 @@ def test_joint_permutation_of_keys_and_values_single_block():
     c, lc = O.node_forward(Q, K[p], V[p], ids, ids[p], [], 20, 0.5)
     np.testing.assert_allclose(a, c, atol=1e-12)
     np.testing.assert_allclose(la, lc, atol=1e-12)
+
+
+# ---- backward pass: the derivative of the forward map, discrete choices held fixed --------------
+@pytest.mark.parametrize("causal,n,n0,b,m", [(False, 48, 0, 8, 6), (True, 64, 16, 8, 5), (False, 40, 0, 64, 0), (True, 32, 32, 4, 4)])
+def test_backward_matches_finite_differences_of_the_forward_oracle(causal, n, n0, b, m):
+    """Central differences of the (independently written) forward oracle along random directions,
+    with the bucket ids injected so that the sortLSH permutations do not move."""
+    rng = np.random.default_rng(77 + n + b)
+    d, r, seed, g = 8, 4, 3, 1
+    Q, K, V = (rng.standard_normal((n, d)) for _ in range(3))
+    W = O.directions(d, r, seed)
+    ids_q, _ = O.bucket_ids(Q, W)
+    ids_k, _ = O.bucket_ids(K, W)
+    scale = 0.4
+    G_out = rng.standard_normal((n, d))
+    g_lse = rng.standard_normal(n)
+
+    def loss(Q_, K_, V_):
+        out, lse = O.segment_forward(Q_, K_, V_, W, b, m, causal, n0, seed, g, scale=scale, ids_q=ids_q, ids_k=ids_k)
+        return float((out * G_out).sum() + (lse * g_lse).sum())
+
+    C = O.dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g)
+    dQ, dK, dV = O.dense_backward(Q, K, V, C, scale, G_out, g_lse)
+    eps = 1e-6
+    for X, dX, which in ((Q, dQ, 0), (K, dK, 1), (V, dV, 2)):
+        for _ in range(3):
+            D = rng.standard_normal(X.shape)
+            args_p = [Q, K, V]; args_m = [Q, K, V]
+            args_p[which] = X + eps * D; args_m[which] = X - eps * D
+            fd = (loss(*args_p) - loss(*args_m)) / (2 * eps)
+            an = float((dX * D).sum())
+            assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (which, fd, an)
+
+
+def test_dense_coefficients_reproduce_dense_weights():
+    rng = np.random.default_rng(5)
+    n, d, r, b, m, seed, g = 64, 8, 5, 8, 7, 11, 2
+    Q, K = rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    W = O.directions(d, r, seed)
+    ids_q, _ = O.bucket_ids(Q, W)
+    ids_k, _ = O.bucket_ids(K, W)
+    for causal, n0 in ((False, 0), (True, 16)):
+        C = O.dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g)
+        U = C * np.exp(0.3 * (Q @ K.T))
+        Wt = O.dense_weights(Q, K, ids_q, ids_k, b, m, 0.3, causal, n0, seed, g)
+        assert np.allclose(U / U.sum(axis=1, keepdims=True), Wt, rtol=1e-12, atol=1e-15)
