@@ -64,10 +64,12 @@ def work_model(w: WL.Workload):
     elif n <= w.n0:
         leaves.append((1, n, True))
     else:
-        L = (n // w.n0).bit_length() - 1
+        L = 0
+        while (n >> L) > w.n0:
+            L += 1
         for l in range(L):
             nodes.append((1 << l, n >> (l + 1)))
-        leaves.append((n // w.n0, w.n0, True))
+        leaves.append((1 << L, n >> L, True))
     flops = 0.0
     sorted_rows = 0
     for cnt, s in nodes:
@@ -84,7 +86,9 @@ def work_model(w: WL.Workload):
     sort_bytes = G * sorted_rows * (2 * 1 + 4 + 4 + 4)        # ids of Q and K rows, perm_q, perm_k, rank_k
     merge_bytes = 0.0
     if w.causal and n > w.n0:
-        L = (n // w.n0).bit_length() - 1
+        L = 0
+        while (n >> L) > w.n0:
+            L += 1
         merge_bytes = G * n * ((1 + L / 2.0) * (4 * d + 4) + d * e + 4)
     dense_flops = G * (4.0 * n * n * d) * (0.5 if w.causal else 1.0)
     return {"attention_flops": flops, "hash_bytes": hash_bytes, "sort_bytes": float(sort_bytes),

@@ -33,7 +33,10 @@
  *   - Shapes: d in {64, 128}; 1 <= hash_bits <= 8; samples >= 0; block >= 1.
  *     block need not divide n (or a recursion node's size): the mask of Alg. 1 line 4 is
  *     floor(P(i) / block), so the last sorted block is short; block >= n makes the problem one
- *     exact block.  Causal: n <= n0 (exact causal attention) or n == n0 * 2^L.
+ *     exact block.  Causal: Alg. 4 halves the rows until a part is not longer than n0 (L
+ *     halvings, 2^L exact causal leaves of n / 2^L rows; L = 0 if n <= n0); the halves are
+ *     equal, so 2^L must divide n (n = n0 * 2^L is the common case; n = 100000 with
+ *     n0 = 4096 has 32 leaves of 3125 rows).
  *   - Recursion nodes are numbered like a binary heap: the off-diagonal problem of the
  *     j-th node of level l (root level 0) is node (2^l - 1) + j; it pairs query rows
  *     [(2j+1)s, (2j+2)s) with key rows [2js, (2j+1)s), s = n / 2^(l+1).  A non-causal

@@ -100,7 +100,9 @@ def _debug_shapes(B, H, n, block, samples, causal, n0):
     elif n <= n0:
         LV, NL, NODES = 1, n, 0
     else:
-        L = (n // n0).bit_length() - 1
+        L = 0
+        while (n >> L) > n0:                      # Alg. 4: halve until a part is not longer than n0
+            L += 1
         LV, NL, NODES = L, n // 2, (1 << L) - 1
     return G, LV, NL, NODES
 

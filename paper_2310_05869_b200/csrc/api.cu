@@ -43,14 +43,13 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
   } else {
     if (p.n0 <= 0) return HYPERATTN_INVALID_ARGUMENT;
     g.causal = 1;
+    // Alg. 4 halves the problem until it is not longer than n0: L levels, 2^L equal leaves of
+    // n / 2^L rows (n0 itself when n = n0 2^L); the halves must be equal, so 2^L must divide n
     int L = 0;
-    if (p.n > p.n0) {
-      long long s = p.n0;
-      while (s < p.n) { s *= 2; ++L; }
-      if (s != p.n || L > kMaxLevels) return HYPERATTN_UNSUPPORTED_SHAPE;
-    }
+    while (((long long)p.n >> L) > p.n0 && L <= kMaxLevels) ++L;
+    if (L > kMaxLevels || (p.n & ((1 << L) - 1)) != 0) return HYPERATTN_UNSUPPORTED_SHAPE;
     g.L = L;
-    g.leaf = L ? p.n0 : p.n;
+    g.leaf = p.n >> L;
     g.unit = g.leaf;
     if (L) {
       g.levels = L; g.nl = p.n / 2; g.nodes = (1 << L) - 1;

@@ -46,7 +46,9 @@ def levels_of(w: WL.Workload):
         return [(0, w.n)] if w.b < w.n else []
     if w.n <= w.n0:
         return []
-    L = (w.n // w.n0).bit_length() - 1
+    L = 0
+    while (w.n >> L) > w.n0:
+        L += 1
     return [(l, w.n >> (l + 1)) for l in range(L)]
 
 
@@ -157,7 +159,8 @@ def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, seg
         else:
             rows = set(rng.choice(w.n, size=rows_per_seg, replace=False).tolist())
             if w.causal and w.n > w.n0:
-                for edge in range(0, w.n + 1, w.n0):
+                leaf = w.n >> len(levels_of(w))
+                for edge in range(0, w.n + 1, leaf):
                     rows.update(x for x in (edge - 1, edge, edge + 127, edge + 128) if 0 <= x < w.n)
             rows.update((0, w.n - 1))
             rows = np.array(sorted(rows))

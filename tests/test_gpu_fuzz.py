@@ -20,11 +20,13 @@ def draw(seed: int) -> WL.Workload:
     B, H = int(rng.integers(1, 3)), int(rng.integers(1, 4))
     causal = bool(rng.random() < 0.5)
     if causal:
-        n0 = int(rng.choice([32, 64, 96, 128, 200, 256, 384, 512, 1000]))
-        L = int(rng.integers(0, 5))
-        while n0 << L > 8192:
+        # 2^L leaves of any size: Alg. 4 halves until a part is not longer than n0
+        leaf = int(np.exp(rng.uniform(np.log(3), np.log(1000))))
+        L = int(rng.integers(0, 6))
+        while leaf << L > 8192:
             L -= 1
-        n = n0 << L
+        n = leaf << L
+        n0 = int(rng.integers(leaf, 2 * leaf))
     else:
         n0 = 0
         n = int(np.exp(rng.uniform(np.log(33), np.log(6000))))

@@ -50,6 +50,10 @@ SMALL = [
     W("ramp_rescales_d64", 1, 2, 4096, 64, "bf16", 256, 256, 7, False, 0, kind="ramp", seed=24),
     W("ramp_rescales_causal_d128", 1, 2, 4096, 128, "bf16", 128, 128, 7, True, 1024, kind="ramp", seed=25),
     W("ramp_rescales_causal_d64", 1, 2, 8192, 64, "bf16", 256, 64, 7, True, 2048, kind="ramp", seed=26),
+    # causal lengths that are not n0 * 2^L: Alg. 4 halves until a part is not longer than n0
+    W("causal_leaves_of_125_rows", 1, 2, 4000, 64, "bf16", 96, 64, 6, True, 128, seed=27),
+    W("causal_leaves_of_750_rows_d128", 1, 2, 6000, 128, "bf16", 256, 128, 7, True, 1000, seed=28),
+    W("causal_leaves_of_3_rows", 1, 1, 768, 64, "bf16", 16, 8, 4, True, 5, seed=29),
 ]
 
 

@@ -205,7 +205,7 @@ def test_causal_base_case_is_exact_causal_attention():
 
 
 # ------------------------------------------------------------------ O2: causal bookkeeping
-@pytest.mark.parametrize("n,n0", [(32, 4), (32, 8), (48, 12), (64, 2)])
+@pytest.mark.parametrize("n,n0", [(32, 4), (32, 8), (48, 12), (64, 2), (48, 5), (40, 7), (72, 10)])   # the last three: leaves of 3, 5 and 9 rows (n0 does not divide n)
 def test_causal_recursion_with_single_block_nodes_is_exact(n, n0):
     """With b >= n/2 every off-diagonal problem is one block, so Alg. 4's identity
     D_C = diag(D_C11, D_21 + D_C22) must give exact causal attention for any depth."""
