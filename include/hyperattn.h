@@ -139,6 +139,31 @@ int hyperattn_forward_ex(const hyperattn_params* p);
  * and kept, like the two streams, until hyperattn_release(). */
 int hyperattn_forward_host(const hyperattn_params* p);
 
+/* Backward pass.  The paper times a backward pass (Sec. 4.2) without writing it down; this is the
+ * derivative of the forward map of Alg. 2-4 as computed by hyperattn_forward_ex, with the sortLSH
+ * permutations and the sampled columns held fixed (they are recomputed from q, k and the seed, so
+ * *p must be the forward call's parameters): with P = rownorm(C o exp(scale Q K^T)), C the 0 / 1 /
+ * (N/m) x multiplicity coefficients of the block mask, the samples and the causal recursion,
+ *     dV = P^T dO,  dS = P o (dO V^T - rowsum(dO o O)),  dQ = scale dS K,  dK = scale dS^T Q.
+ *   p->q, k, v       device, bf16 (fp32 inputs: HYPERATTN_UNSUPPORTED_SHAPE)
+ *   p->out, p->lse   device, the forward call's results (read only here), out of p->out_dtype
+ *   dout             device, bf16 [B, H, n, d]: gradient of the loss with respect to out
+ *   dq, dk, dv       device, [B, H, n, d] of grad_dtype (HYPERATTN_BF16 or HYPERATTN_FP32), written;
+ *                    16-byte aligned; must not alias any input
+ * Gradients are accumulated in fp32 (in place for fp32 gradients, in the workspace otherwise) with
+ * global reductions, so the low bits depend on the order in which tiles finish.  Enqueued on
+ * p->stream like the forward pass; p->debug is ignored.  No gradient flows through lse. */
+typedef struct hyperattn_grads {
+  const void* dout;
+  void* dq;
+  void* dk;
+  void* dv;
+  int grad_dtype;
+} hyperattn_grads;
+int hyperattn_backward(const hyperattn_params* p, const hyperattn_grads* grads);
+/* Bytes of device scratch hyperattn_backward needs (host-side, like hyperattn_workspace_bytes). */
+int hyperattn_backward_workspace_bytes(const hyperattn_params* p, int grad_dtype, size_t* bytes);
+
 /* Bytes of device scratch hyperattn_forward_ex needs for these shapes (host-side; only the
  * shape members, dtype and out_dtype of *p are read). */
 int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes);
@@ -165,7 +190,8 @@ enum {
   HYPERATTN_STAGE_SORT_SCATTER = 4, /* Alg. 1 line 3 */
   HYPERATTN_STAGE_ATTENTION = 5,    /* block + sampled + causal-leaf contractions */
   HYPERATTN_STAGE_MERGE = 6,        /* Alg. 4 line 5 carried to outputs */
-  HYPERATTN_NUM_STAGES = 7
+  HYPERATTN_STAGE_BACKWARD = 7,     /* hyperattn_backward: zeroing, <dO, O>, gradient tiles, conversion */
+  HYPERATTN_NUM_STAGES = 8
 };
 typedef struct hyperattn_stage_times {
   float ms[HYPERATTN_NUM_STAGES];

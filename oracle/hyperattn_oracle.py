@@ -429,14 +429,15 @@ def dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g, _node=0):
     return coeff(n, np.asarray(ids_q), np.asarray(ids_k), _node)
 
 
-def dense_backward(Q, K, V, C, scale, d_out, d_lse=None):
+def dense_backward(Q, K, V, C, scale, d_out, d_lse=None, with_term_sizes=False):
     """Gradients of L = <d_out, out> + <d_lse, lse> for out = P V, P = rownorm(C o A),
     lse = ln rowsum(C o A), A = exp(scale Q K^T), C constant:
         dV = P^T d_out
         dP = d_out V^T
         dS = P o (dP - rowsum(P o dP) + d_lse)      (softmax Jacobian; d lse_i / d s_ij = P_ij)
         dQ = scale dS K,   dK = scale dS^T Q.
-    Returns (dQ, dK, dV), fp64."""
+    Returns (dQ, dK, dV), fp64; with_term_sizes adds, per gradient, the sum of the absolute
+    values of the terms behind every entry (a yardstick for rounding errors)."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
@@ -453,4 +454,15 @@ def dense_backward(Q, K, V, C, scale, d_out, d_lse=None):
     dS = P * (dP - inner)
     if d_lse is not None:
         dS = dS + P * np.asarray(d_lse, dtype=np.float64)[:, None]
-    return scale * (dS @ K), scale * (dS.T @ Q), dV
+    grads = (scale * (dS @ K), scale * (dS.T @ Q), dV)
+    if not with_term_sizes:
+        return grads
+    # sums of the absolute values of the terms each gradient entry is made of (what a rounding of
+    # every term by a relative eps can move it by, divided by eps): the two products inside dS
+    # count separately
+    # (delta_i = <dO_i, O_i> counts with the absolute values of ITS terms: a caller that forms it
+    # from a rounded O moves it by eps times that sum, however much the terms cancel)
+    delta_terms = (np.abs(d_out) * np.abs(P @ V)).sum(axis=1, keepdims=True)
+    T = P * (np.abs(dP) + np.abs(inner) + delta_terms)
+    sizes = (scale * (T @ np.abs(K)), scale * (T.T @ np.abs(Q)), P.T @ np.abs(d_out))
+    return grads, sizes

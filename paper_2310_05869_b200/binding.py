@@ -14,8 +14,9 @@ _lib = None
 
 BF16, FP32 = 0, 1
 NUM_STAGES = 7
-STAGE_NAMES = ["convert", "hash", "sample", "sort_scan", "sort_scatter", "attention", "merge"]
+STAGE_NAMES = ["convert", "hash", "sample", "sort_scan", "sort_scatter", "attention", "merge", "backward"]
 EXPORTS = ["hyperattn_forward", "hyperattn_forward_ex", "hyperattn_forward_host", "hyperattn_workspace_bytes",
+           "hyperattn_backward", "hyperattn_backward_workspace_bytes",
            "hyperattn_get_projections", "hyperattn_last_device_status", "hyperattn_profile_enable",
            "hyperattn_profile_reset", "hyperattn_profile_read", "hyperattn_release",
            "hyperattn_status_string", "hyperattn_version", "hyperattn_sortlsh_noalloc"]
@@ -66,6 +67,8 @@ def lib() -> C.CDLL:
         L.hyperattn_sortlsh_noalloc.restype = C.c_int
         L.hyperattn_sortlsh_noalloc.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_uint64,
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.hyperattn_backward.restype = C.c_int
+        L.hyperattn_backward.argtypes = [C.POINTER(_Params), C.POINTER(_Grads)]
         L.hyperattn_status_string.restype = C.c_char_p
         L.hyperattn_status_string.argtypes = [C.c_int]
         _lib = L
@@ -142,6 +145,30 @@ def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_
     with torch.cuda.device(q.device):
         _check(lib().hyperattn_forward_ex(C.byref(p)), "hyperattn_forward_ex")
     return (out, lse, inter) if debug else (out, lse)
+
+
+class _Grads(C.Structure):
+    _fields_ = [("dout", C.c_void_p), ("dq", C.c_void_p), ("dk", C.c_void_p), ("dv", C.c_void_p), ("grad_dtype", C.c_int)]
+
+
+def backward(q, k, v, out, lse, dout, block, samples, hash_bits, causal=False, n0=0, seed=0, grad_dtype=None, scale=0.0,
+             stream=None):
+    """Backward pass of `forward` (same shape arguments and seed as the forward call; out and lse are its
+    results).  q, k, v, dout: bf16 CUDA tensors [B, H, n, d].  Returns (dq, dk, dv) of grad_dtype (default bf16)."""
+    if not all(t.is_cuda for t in (q, k, v, out, lse, dout)):
+        raise HyperAttnError("all tensors must be CUDA tensors (there is no CPU path)")
+    q, k, v, out, lse, dout = (t.contiguous() for t in (q, k, v, out, lse, dout))
+    B, H, n, d = q.shape
+    grad_dtype = grad_dtype or torch.bfloat16
+    dq, dk, dv = (torch.empty((B, H, n, d), dtype=grad_dtype, device=q.device) for _ in range(3))
+    p = _Params()
+    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, seed, _dtype_code(q.dtype), _dtype_code(out.dtype), scale)
+    p.q, p.k, p.v, p.out, p.lse = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr()
+    p.stream = stream if stream is not None else torch.cuda.current_stream(q.device).cuda_stream
+    g = _Grads(dout.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), _dtype_code(grad_dtype))
+    with torch.cuda.device(q.device):
+        _check(lib().hyperattn_backward(C.byref(p), C.byref(g)), "hyperattn_backward")
+    return dq, dk, dv
 
 
 def forward_host(q, k, v, out, lse, block, samples, hash_bits, causal=False, n0=0, seed=0, scale=0.0, stream=None):

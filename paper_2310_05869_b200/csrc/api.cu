@@ -15,6 +15,9 @@
 namespace hyperattn {
 cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st);
+cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, const float* lse, const void* dout,
+                            float* delta, float* dq, float* dk, float* dv, float scale, cudaStream_t st);
+cudaError_t launch_to_bf16(const float* src, void* dst, size_t count, cudaStream_t st);
 
 namespace {
 
@@ -70,9 +73,11 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
 
 struct Plan {
   size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, part_o, part_lse, total;
+  size_t delta, gacc;   // backward only: <dO, O> per row; fp32 gradient accumulators (bf16 gradients only)
 };
 
-Plan make_plan(const Geometry& g, int is_fp32) {
+// backward: 0 forward plan; 1 backward with fp32 gradients (accumulated in place); 2 backward with bf16 gradients
+Plan make_plan(const Geometry& g, int is_fp32, int backward = 0) {
   Plan pl;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
@@ -91,9 +96,11 @@ Plan make_plan(const Geometry& g, int is_fp32) {
   pl.perm_k = take(g.sorted ? lvl_rows * 4 : 0);
   pl.rank_k = take(g.sorted ? lvl_rows * 4 : 0);
   pl.samples = take((size_t)g.G * g.nodes * g.m * 4);
-  const size_t part_rows = g.L ? (size_t)g.G * g.n + lvl_rows : 0;
+  const size_t part_rows = (g.L && !backward) ? (size_t)g.G * g.n + lvl_rows : 0;
   pl.part_o = take(part_rows * g.d * 4);
   pl.part_lse = take(part_rows * 4);
+  pl.delta = take(backward ? (size_t)g.G * g.n * 4 : 0);
+  pl.gacc = take(backward == 2 ? (size_t)3 * g.G * g.n * g.d * 4 : 0);
   pl.total = off + kAlign;
   return pl;
 }
@@ -165,8 +172,9 @@ int check_ptrs(const hyperattn_params& p) {
 }
 
 // seg0: index of the call's first segment in the caller's whole tensor (not 0 when a caller's batch is
-// processed in several calls: the samples of a segment depend on its index)
-int forward_impl(const hyperattn_params& p, int seg0 = 0) {
+// processed in several calls: the samples of a segment depend on its index).  bw: run the backward
+// pass instead (p->out and p->lse are then the forward pass's results, read only).
+int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads* bw = nullptr) {
   Geometry g;
   int rc = build_geometry(p, g);
   if (rc) return rc;
@@ -175,7 +183,14 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0) {
   if (rc) return rc;
   const int is_fp32 = p.dtype == HYPERATTN_FP32;
   const int out_fp32 = p.out_dtype == HYPERATTN_FP32;
-  const Plan pl = make_plan(g, is_fp32);
+  if (bw) {
+    if (is_fp32) return HYPERATTN_UNSUPPORTED_SHAPE;                 // the backward pass takes bf16 inputs
+    if (!bw->dout || !bw->dq || !bw->dk || !bw->dv) return HYPERATTN_INVALID_ARGUMENT;
+    if (bw->grad_dtype != HYPERATTN_BF16 && bw->grad_dtype != HYPERATTN_FP32) return HYPERATTN_INVALID_ARGUMENT;
+    for (const void* x : {bw->dout, (const void*)bw->dq, (const void*)bw->dk, (const void*)bw->dv})
+      if (reinterpret_cast<uintptr_t>(x) & 15) return HYPERATTN_MISALIGNED;
+  }
+  const Plan pl = make_plan(g, is_fp32, bw ? (bw->grad_dtype == HYPERATTN_FP32 ? 1 : 2) : 0);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
   int dev = 0;
@@ -307,6 +322,25 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0) {
   a.total_tiles = (int)tiles;
   a.level_pair_start[g.levels] = (int)pairs;
   a.total_pairs = (int)pairs;
+  if (bw) {
+    const size_t elems = (size_t)g.G * g.n * g.d;
+    const bool g32 = bw->grad_dtype == HYPERATTN_FP32;
+    float* acc = reinterpret_cast<float*>(base + pl.gacc);
+    float* dq = g32 ? reinterpret_cast<float*>(bw->dq) : acc;
+    float* dk = g32 ? reinterpret_cast<float*>(bw->dk) : acc + elems;
+    float* dv = g32 ? reinterpret_cast<float*>(bw->dv) : acc + 2 * elems;
+    StageScope sc(st, HYPERATTN_STAGE_BACKWARD, 2 + (g32 ? 0 : 3));
+    HA_CHECK(cudaMemsetAsync(dq, 0, elems * 4, st));
+    HA_CHECK(cudaMemsetAsync(dk, 0, elems * 4, st));
+    HA_CHECK(cudaMemsetAsync(dv, 0, elems * 4, st));
+    HA_CHECK(launch_backward(a, p.out, out_fp32, p.lse, bw->dout, reinterpret_cast<float*>(base + pl.delta), dq, dk, dv, scale, st));
+    if (!g32) {
+      HA_CHECK(launch_to_bf16(dq, bw->dq, elems, st));
+      HA_CHECK(launch_to_bf16(dk, bw->dk, elems, st));
+      HA_CHECK(launch_to_bf16(dv, bw->dv, elems, st));
+    }
+    return HYPERATTN_OK;
+  }
   {
     StageScope sc(st, HYPERATTN_STAGE_ATTENTION, 1);
     // bf16 inputs: tcgen05 path; fp32 inputs: split-bf16 logits on the warp-level MMA path
@@ -331,6 +365,20 @@ extern "C" {
 int hyperattn_forward_ex(const hyperattn_params* p) {
   if (!p) return HYPERATTN_INVALID_ARGUMENT;
   return forward_impl(*p);
+}
+
+int hyperattn_backward(const hyperattn_params* p, const hyperattn_grads* grads) {
+  if (!p || !grads) return HYPERATTN_INVALID_ARGUMENT;
+  return forward_impl(*p, 0, grads);
+}
+
+int hyperattn_backward_workspace_bytes(const hyperattn_params* p, int grad_dtype, size_t* bytes) {
+  if (!p || !bytes) return HYPERATTN_INVALID_ARGUMENT;
+  Geometry g;
+  const int rc = build_geometry(*p, g);
+  if (rc) return rc;
+  *bytes = make_plan(g, 0, grad_dtype == HYPERATTN_FP32 ? 1 : 2).total;
+  return HYPERATTN_OK;
 }
 
 int hyperattn_forward(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int n,
