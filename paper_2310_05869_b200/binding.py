@@ -13,8 +13,8 @@ _LIB_PATH = os.environ.get("HYPERATTN_LIB") or os.path.join(os.path.dirname(os.p
 _lib = None
 
 BF16, FP32 = 0, 1
-NUM_STAGES = 7
 STAGE_NAMES = ["convert", "hash", "sample", "sort_scan", "sort_scatter", "attention", "merge", "backward"]
+NUM_STAGES = len(STAGE_NAMES)          # HYPERATTN_NUM_STAGES
 EXPORTS = ["hyperattn_forward", "hyperattn_forward_ex", "hyperattn_forward_host", "hyperattn_workspace_bytes",
            "hyperattn_backward", "hyperattn_backward_workspace_bytes",
            "hyperattn_get_projections", "hyperattn_last_device_status", "hyperattn_profile_enable",

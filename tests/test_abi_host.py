@@ -89,3 +89,15 @@ def test_cuda_tensors_are_required():
     q = torch.zeros(1, 1, 128, 64, dtype=torch.bfloat16)
     with pytest.raises(ha.HyperAttnError):
         ha.forward(q, q, q, 64, 8, 4)
+
+
+def test_binding_mirrors_the_stage_table_of_the_header():
+    """The binding's stage-times structure must have the header's HYPERATTN_NUM_STAGES entries
+    (hyperattn_profile_read writes that many)."""
+    import re
+    hdr = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "hyperattn.h")).read()
+    n = int(re.search(r"HYPERATTN_NUM_STAGES\s*=\s*(\d+)", hdr).group(1))
+    stages = re.findall(r"HYPERATTN_STAGE_(\w+)\s*=\s*(\d+)", hdr)
+    from paper_2310_05869_b200 import binding as Bn
+    assert Bn.NUM_STAGES == n == len(stages)
+    assert [s.lower() for s, _ in sorted(stages, key=lambda t: int(t[1]))] == Bn.STAGE_NAMES
