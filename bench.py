@@ -315,6 +315,27 @@ def gpu_arm(args, w):
     lat = sorted(a0.elapsed_time(a1) for a0, a1 in evs)
     latency = {"median_ms": lat[len(lat) // 2], "min_ms": lat[0], "calls": lat_steps}
 
+    # ---- backward pass (on request): the derivative of the same call, timed on its own ------------
+    backward = None
+    if args.backward and w.dtype == "bf16":
+        out_b, lse_b = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+        dout = torch.randn(q.shape, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        for _ in range(2):
+            ha.backward(q, k, v, out_b, lse_b, dout, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+        bsteps = max(3, min(args.steps, 10))
+        barrier()
+        e0.record(stream)
+        for _ in range(bsteps):
+            ha.backward(q, k, v, out_b, lse_b, dout, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+        e1.record(stream)
+        barrier()
+        bms = RK.max_over_ranks(info, e0.elapsed_time(e1), dev) / bsteps
+        bflops = 2.5 * work_model(w)["attention_flops"]          # five contractions per tile instead of two
+        backward = {"ms_per_call": bms, "flops": bflops, "achieved_tflops": bflops / (bms * 1e-3) / 1e12,
+                    "frac_of_bf16_sustained": bflops / (bms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                    "path": "mma.sync, fp32 global reductions", "steps": bsteps}
+        del out_b, lse_b, dout
+
     # ---- end to end through the host-buffer entry point ---------------------------------------
     hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
     ho = torch.empty(q.shape, dtype=q.dtype).pin_memory()
@@ -405,6 +426,8 @@ def gpu_arm(args, w):
             "e2e": e2e, "gpu_launches": sum(launches.values()) * args.steps, "launches_per_step": launches,
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "clocks": clocks,
             "peaks": peaks}
+    if backward is not None:
+        line["backward"] = backward
     print(json.dumps(line))
     RK.shutdown(info)
 
@@ -419,6 +442,7 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="override H (smaller cases for profiler captures)")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--backward", action="store_true", help="also time the backward pass (an extra key of the JSON line)")
     args = ap.parse_args()
     w = WL.CONFIGS[WORKLOADS[args.workload]]
     if args.n:
