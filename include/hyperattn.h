@@ -136,7 +136,9 @@ int hyperattn_forward_ex(const hyperattn_params* p);
  * synchronises `stream` before reading the results.  Results are bit-identical to
  * hyperattn_forward_ex on device copies of the same tensors.  With debug outputs requested the
  * batch is one group.  The staging area is grown on demand (that call synchronises the device)
- * and kept, like the two streams, until hyperattn_release(). */
+ * and kept, like the two streams, until hyperattn_release().  Calls on one device share the staging
+ * area, the two streams and their events: they must not overlap (issue them from one thread, or
+ * order them yourself). */
 int hyperattn_forward_host(const hyperattn_params* p);
 
 /* Backward pass.  The paper times a backward pass (Sec. 4.2) without writing it down; this is the
