@@ -78,6 +78,7 @@ struct BwdArgs {
   const float* delta;          // [G, n] <dO_i, O_i>
   float *dq, *dk, *dv;         // [G, n, D] fp32 accumulators, zeroed before the launch
   float scale;
+  int table_keys;              // key columns of a node tile's row tables (block and samples, each padded to whole tiles)
 };
 
 template <int D>
@@ -85,7 +86,7 @@ struct Smem {
   static constexpr int kQ = kTileQ * D * 2;
   static constexpr int kKV = TK * D * 2;
   static constexpr int kP = kTileQ * TK * 2;
-  static constexpr int kTotal = 2 * kQ + 4 * kKV + 2 * kP + kMaxNodeKeys * 8 + kTileQ * 12;
+  static constexpr int kFixed = 2 * kQ + 4 * kKV + 2 * kP + kTileQ * 12;   // + 8 bytes per key column of the row tables
 };
 
 // delta_i = <dO_i, O_i>: one warp per row
@@ -106,8 +107,9 @@ __global__ void __launch_bounds__(256) delta_kernel(const __nv_bfloat16* __restr
   if (lane == 0) delta[row] = acc;
 }
 
+// (d = 64: two CTAs per SM - the legacy tensor path needs the warps to hide its latencies)
 template <int D>
-__global__ void __launch_bounds__(256, 1) bwd_kernel(const __grid_constant__ BwdArgs b) {
+__global__ void __launch_bounds__(256, D == 64 ? 2 : 1) bwd_kernel(const __grid_constant__ BwdArgs b) {
   extern __shared__ __align__(1024) uint8_t smem[];
   using SM = Smem<D>;
   const AttnArgs& a = b.a;
@@ -117,11 +119,11 @@ __global__ void __launch_bounds__(256, 1) bwd_kernel(const __grid_constant__ Bwd
   uint8_t* sV = sK + 2 * SM::kKV;                 // [2][TK x D]
   uint8_t* sP = sV + 2 * SM::kKV;                 // [128 x TK] bf16, P of the current key tile
   uint8_t* sdS = sP + SM::kP;                     // [128 x TK] bf16, dS of the current key tile
-  int* s_kidx = reinterpret_cast<int*>(sdS + SM::kP);
-  float* s_kbias = reinterpret_cast<float*>(s_kidx + kMaxNodeKeys);
-  int* s_qrow = reinterpret_cast<int*>(s_kbias + kMaxNodeKeys);
+  int* s_qrow = reinterpret_cast<int*>(sdS + SM::kP);
   float* s_lse2 = reinterpret_cast<float*>(s_qrow + kTileQ);
   float* s_delta = s_lse2 + kTileQ;
+  int* s_kidx = reinterpret_cast<int*>(s_delta + kTileQ);       // [table_keys]
+  float* s_kbias = reinterpret_cast<float*>(s_kidx + b.table_keys);
 
   const Geometry& g = a.g;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -332,14 +334,15 @@ cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, co
   if (e != cudaSuccess || a.total_tiles == 0) return e;
   BwdArgs b;
   b.a = a; b.dout = d16; b.lse = lse; b.delta = delta; b.dq = dq; b.dk = dk; b.dv = dv; b.scale = scale;
+  b.table_keys = a.g.sorted ? (a.g.b + TK - 1) / TK * TK + (a.g.m + TK - 1) / TK * TK : 0;
   auto go = [&](auto kernel, int smem_bytes) {
-    cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes + kMaxNodeKeys * 8);
     if (e2 != cudaSuccess) return e2;
-    kernel<<<a.total_tiles, 256, smem_bytes, st>>>(b);
+    kernel<<<a.total_tiles, 256, smem_bytes + b.table_keys * 8, st>>>(b);
     return cudaGetLastError();
   };
-  if (a.g.d == 64) return go(bwd_kernel<64>, Smem<64>::kTotal);
-  return go(bwd_kernel<128>, Smem<128>::kTotal);
+  if (a.g.d == 64) return go(bwd_kernel<64>, Smem<64>::kFixed);
+  return go(bwd_kernel<128>, Smem<128>::kFixed);
 }
 
 cudaError_t launch_to_bf16(const float* src, void* dst, size_t count, cudaStream_t st) {
