@@ -473,9 +473,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
   const uint32_t bar_qfree = bar0 + 8;                                        // both issuers are done with Q
   auto bar_s = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 3 * i + b); };          // S_i buffer b written
   auto bar_p = [&](int i, int b) { return bar0 + 168 + 8 * (6 * C::NS + 6 + 3 * i + b); };      // P_i buffer b written
-  // P_i V of a key tile finished; two barriers per query tile, used alternately, so that the
-  // (rare) waiter can never mistake "one phase behind" for "done" however far the scores run ahead
-  auto bar_pvd = [&](int i, int b) { return bar0 + 16 + 8 * (2 * i + b); };
   auto bar_o = [&](int i) { return bar0 + 80 + 8 * i; };                      // O_i of the item complete
   auto bar_ofree = [&](int i) { return bar0 + 112 + 8 * i; };                 // O_i has been read out
   auto bar_tabfull = [&](int set) { return bar0 + 128 + 8 * set; };           // row tables of a set written
@@ -505,7 +502,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       mbar_init(bar_ofree(i), 128);
       mbar_init(bar_tabfull(i), 1);
       mbar_init(bar_tabfree(i), 257);                   // 256 softmax threads + the K / V streamer
-      mbar_init(bar_pvd(i, 0), 1); mbar_init(bar_pvd(i, 1), 1);
       for (int b = 0; b < C::kSBufs; ++b) { mbar_init(bar_s(i, b), 1); mbar_init(bar_p(i, b), 128); }
     }
     for (int s = 0; s < C::NS; ++s) {
@@ -539,6 +535,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t colO = C::kColO + C::kOCols * i;
     int ga = 0;                                       // key tiles this warpgroup has processed so far (all items)
+    int gbase = 0;                                    // global index (all items) of the item's first key tile
     int vi = 0;                                       // items in which this query tile existed
     bool ok = true;
     int it = 0;
@@ -660,8 +657,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           { const uint64_t al2 = pack_f2(alpha, alpha); l01 = fmul2(l01, al2); lra *= alpha; lrb *= alpha; }
           // O may only be touched between two PV products: the one of the previous tile must
           // have finished (the one of this tile cannot start before this tile's P is published)
+          // That product's completion is what releases its V stage to the streamer, so the
+          // stage's barrier tells (the issuer has nothing extra to commit for this rare path).  Its
+          // phase cannot run ahead of this warpgroup: the next product on the same stage is NS key
+          // tiles later and needs this warpgroup's P first.
           if (na > 0) {
-            ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_pvd(i, (gw - 1) & 1), ((gw - 1) >> 1) & 1, s_abort, status));
+            const int gjp = gbase + tile_of(q, na - 1);
+            ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_vempty(i, gjp % C::NS), (gjp / C::NS) & 1, s_abort, status));
             if (!ok) break;
             tc_fence_after();
             rescale_row(lane_addr + colO, C::kOCols, alpha);
@@ -798,6 +800,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       mbar_arrive(bar_tabfree(set));
       HA_LACC(a_epi, te);
       ga += total;
+      gbase += t.ntiles;
     }
 #ifdef HA_TC_TIMING
     if (row == 0 && i == 0) {
@@ -895,7 +898,6 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 #pragma unroll
           for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
           umma_commit(bar_vempty(i, s));
-          umma_commit(bar_pvd(i, gw & 1));
           vnext = gj + 1;
           if (a2 == total - 1) umma_commit(bar_o(i));
         };
