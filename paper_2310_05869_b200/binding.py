@@ -69,6 +69,8 @@ def lib() -> C.CDLL:
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.hyperattn_backward.restype = C.c_int
         L.hyperattn_backward.argtypes = [C.POINTER(_Params), C.POINTER(_Grads)]
+        L.hyperattn_backward_workspace_bytes.restype = C.c_int
+        L.hyperattn_backward_workspace_bytes.argtypes = [C.POINTER(_Params), C.c_int, C.POINTER(C.c_size_t)]
         L.hyperattn_status_string.restype = C.c_char_p
         L.hyperattn_status_string.argtypes = [C.c_int]
         _lib = L

@@ -101,3 +101,25 @@ def test_binding_mirrors_the_stage_table_of_the_header():
     from paper_2310_05869_b200 import binding as Bn
     assert Bn.NUM_STAGES == n == len(stages)
     assert [s.lower() for s, _ in sorted(stages, key=lambda t: int(t[1]))] == Bn.STAGE_NAMES
+
+
+def test_backward_rejects_bad_arguments_on_the_host():
+    """Nothing is launched for fp32 inputs, missing or misaligned gradient pointers, or a bad gradient type."""
+    L = ha.lib()
+    fake = 0x800000
+    def grads(**kw):
+        g = B._Grads(fake, fake + 0x100000, fake + 0x200000, fake + 0x300000, B.BF16)
+        for k, v in kw.items():
+            setattr(g, k, v)
+        return g
+    assert L.hyperattn_backward(C.byref(_params(dtype=B.FP32)), C.byref(grads())) == -2
+    assert L.hyperattn_backward(C.byref(_params()), C.byref(grads(dq=0))) == -1
+    assert L.hyperattn_backward(C.byref(_params()), C.byref(grads(grad_dtype=7))) == -1
+    assert L.hyperattn_backward(C.byref(_params()), C.byref(grads(dk=fake + 0x100004))) == -3
+    assert L.hyperattn_backward(None, C.byref(grads())) == -1
+    need_f32, need_bf16, need_fwd = C.c_size_t(0), C.c_size_t(0), C.c_size_t(0)
+    p = _params()
+    assert L.hyperattn_backward_workspace_bytes(C.byref(p), B.FP32, C.byref(need_f32)) == 0
+    assert L.hyperattn_backward_workspace_bytes(C.byref(p), B.BF16, C.byref(need_bf16)) == 0
+    # bf16 gradients are accumulated in fp32 in the workspace: three tensors more than for fp32 gradients
+    assert need_bf16.value - need_f32.value >= 3 * p.B * p.H * p.n * p.d * 4
