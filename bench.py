@@ -333,7 +333,7 @@ def gpu_arm(args, w):
         bflops = 2.5 * work_model(w)["attention_flops"]          # five contractions per tile instead of two
         backward = {"ms_per_call": bms, "flops": bflops, "achieved_tflops": bflops / (bms * 1e-3) / 1e12,
                     "frac_of_bf16_sustained": bflops / (bms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                    "path": "mma.sync, fp32 global reductions", "steps": bsteps}
+                    "path": "tcgen05 / TMEM, fp32 global reductions", "steps": bsteps}
         del out_b, lse_b, dout
 
     # ---- end to end through the host-buffer entry point ---------------------------------------

@@ -16,7 +16,7 @@ namespace hyperattn {
 cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st);
 cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, const float* lse, const void* dout,
-                            float* delta, float* dq, float* dk, float* dv, float scale, cudaStream_t st);
+                            float* delta, float* dq, float* dk, float* dv, float scale, int* status, cudaStream_t st);
 cudaError_t launch_to_bf16(const float* src, void* dst, size_t count, cudaStream_t st);
 
 namespace {
@@ -333,7 +333,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     HA_CHECK(cudaMemsetAsync(dq, 0, elems * 4, st));
     HA_CHECK(cudaMemsetAsync(dk, 0, elems * 4, st));
     HA_CHECK(cudaMemsetAsync(dv, 0, elems * 4, st));
-    HA_CHECK(launch_backward(a, p.out, out_fp32, p.lse, bw->dout, reinterpret_cast<float*>(base + pl.delta), dq, dk, dv, scale, st));
+    HA_CHECK(launch_backward(a, p.out, out_fp32, p.lse, bw->dout, reinterpret_cast<float*>(base + pl.delta), dq, dk, dv, scale, ws.status, st));
     if (!g32) {
       HA_CHECK(launch_to_bf16(dq, bw->dq, elems, st));
       HA_CHECK(launch_to_bf16(dk, bw->dk, elems, st));

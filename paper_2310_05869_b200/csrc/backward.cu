@@ -10,17 +10,15 @@
 // The merge of the causal recursion needs no derivative of its own: the merged output is one
 // softmax over everything a row sees, so every tile of every level uses the FINAL lse and delta.
 //
-// First version, on the warp-level tensor-core path (mma.sync m16n8k16): one CTA per query
-// tile of the forward schedule, the same row tables, S and dP like the forward's S, dQ like
-// its O; P and dS are staged in shared memory so that the transposed products (dV, dK) can
-// read them with ldmatrix.trans, and all three gradients are accumulated in fp32 with global
-// reductions (a key tile is shared by every query tile that samples it).
+// One CTA per query tile of the forward schedule (same row tables, same sort and samples), key
+// tiles of 128, all five products on the tcgen05 tensor cores with accumulators in TMEM (see
+// bwd_tc_kernel); the three gradients are accumulated in fp32 with global reductions (a key
+// tile is shared by every query tile that samples it, a query row by every level it appears in).
 #include "attn_common.cuh"
 
 namespace hyperattn {
 namespace {
 
-constexpr int TK = 64;   // keys per tile
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -31,20 +29,6 @@ __device__ __forceinline__ void st_shared_zero16(uint32_t dst) {
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
@@ -67,9 +51,6 @@ __device__ __forceinline__ void gather_tile(uint32_t dst, const __nv_bfloat16* s
     else st_shared_zero16(d);
   }
 }
-__device__ __forceinline__ void red_add2(float* p, float x, float y) {
-  atomicAdd(reinterpret_cast<float2*>(p), make_float2(x, y));
-}
 
 struct BwdArgs {
   AttnArgs a;
@@ -79,14 +60,6 @@ struct BwdArgs {
   float *dq, *dk, *dv;         // [G, n, D] fp32 accumulators, zeroed before the launch
   float scale;
   int table_keys;              // key columns of a node tile's row tables (block and samples, each padded to whole tiles)
-};
-
-template <int D>
-struct Smem {
-  static constexpr int kQ = kTileQ * D * 2;
-  static constexpr int kKV = TK * D * 2;
-  static constexpr int kP = kTileQ * TK * 2;
-  static constexpr int kFixed = 2 * kQ + 4 * kKV + 2 * kP + kTileQ * 12;   // + 8 bytes per key column of the row tables
 };
 
 // delta_i = <dO_i, O_i>: one warp per row
@@ -107,29 +80,87 @@ __global__ void __launch_bounds__(256) delta_kernel(const __nv_bfloat16* __restr
   if (lane == 0) delta[row] = acc;
 }
 
-// (d = 64: two CTAs per SM - the legacy tensor path needs the warps to hide its latencies)
-template <int D>
-__global__ void __launch_bounds__(256, D == 64 ? 2 : 1) bwd_kernel(const __grid_constant__ BwdArgs b) {
-  extern __shared__ __align__(1024) uint8_t smem[];
-  using SM = Smem<D>;
-  const AttnArgs& a = b.a;
-  uint8_t* sQ = smem;
-  uint8_t* sdO = sQ + SM::kQ;
-  uint8_t* sK = sdO + SM::kQ;                     // [2][TK x D]
-  uint8_t* sV = sK + 2 * SM::kKV;                 // [2][TK x D]
-  uint8_t* sP = sV + 2 * SM::kKV;                 // [128 x TK] bf16, P of the current key tile
-  uint8_t* sdS = sP + SM::kP;                     // [128 x TK] bf16, dS of the current key tile
-  int* s_qrow = reinterpret_cast<int*>(sdS + SM::kP);
-  float* s_lse2 = reinterpret_cast<float*>(s_qrow + kTileQ);
-  float* s_delta = s_lse2 + kTileQ;
-  int* s_kidx = reinterpret_cast<int*>(s_delta + kTileQ);       // [table_keys]
-  float* s_kbias = reinterpret_cast<float*>(s_kidx + b.table_keys);
+// ---------------------------------------------------------------------------------------------
+// One CTA per query tile, key tiles of 128, all five
+// products on the 5th-generation tensor cores with operands in 128-byte-swizzled shared memory:
+//     S  = Q K^T       A = Q  [query][d]   K-major,  B = K  [key][d]   K-major      -> TMEM cols   0..127
+//     dP = dO V^T      A = dO [query][d]   K-major,  B = V  [key][d]   K-major      -> TMEM cols 128..255
+//     dQ += dS K       A = dS [query][key] K-major,  B = K  [key][d]   MN-major     -> TMEM cols 256..256+d
+//     dV  = P^T dO     A = P  [query][key] MN-major, B = dO [query][d]  MN-major     -> over S's columns
+//     dK  = dS^T Q     A = dS [query][key] MN-major, B = Q  [query][d]  MN-major     -> over dP's columns
+// 256 threads: thread t and thread t + 128 share TMEM lane t mod 128 - query row t when P and dS
+// are formed (each takes 64 of the tile's 128 key columns), key row t when dV (threads 0-127) and
+// dK (threads 128-255) leave TMEM.  The phases of a key tile run one after the other (loads, S
+// and dP, P and dS, the three gradient products, reductions): correct first, overlapped later.
+constexpr int TKB = 128;   // keys per tile
+constexpr unsigned long long kBwdWaitNs = 2000000000ull;
 
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// bounded wait: false after two seconds (the caller raises the status word and winds down)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  unsigned long long t0 = 0;
+  for (unsigned it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
+    if (ok) return true;
+    if ((it & 63u) == 63u) {
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kBwdWaitNs) return false;
+    }
+  }
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}\n"
+               ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+               "\ttcgen05.wait::ld.sync.aligned;\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                 "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                 "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+               : "r"(taddr) : "memory");
+}
+
+template <int D>
+struct SmemTc {
+  static constexpr int kQ = 128 * D * 2;              // Q, dO, K, V tiles: [128 rows x D]
+  static constexpr int kP = 128 * TKB * 2;            // P, dS: [128 queries x 128 keys]
+  static constexpr int kOffQ = 0, kOffdO = kQ, kOffK = 2 * kQ, kOffV = 3 * kQ, kOffP = 4 * kQ, kOffdS = 4 * kQ + kP;
+  static constexpr int kOffMisc = 4 * kQ + 2 * kP;    // mbarrier, TMEM address, abort flag
+  static constexpr int kOffRow = kOffMisc + 64;       // s_qrow [128]
+  static constexpr int kFixed = kOffRow + 128 * 4;    // + 8 bytes per key column of the row tables
+};
+
+template <int D>
+__global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ BwdArgs b, int* status) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  using SM = SmemTc<D>;
+  const AttnArgs& a = b.a;
   const Geometry& g = a.g;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int gid = lane >> 2, tig = lane & 3;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int row = tid & 127, half = tid >> 7;            // TMEM lane / tile row of this thread; which half of the work it takes
   const TileDesc t = decode_tile(a, blockIdx.x);
   if (t.nq <= 0) return;
+
+  const uint32_t ubase = smem_u32(smem);
+  const uint32_t uQ = ubase + SM::kOffQ, udO = ubase + SM::kOffdO, uK = ubase + SM::kOffK, uV = ubase + SM::kOffV;
+  const uint32_t uP = ubase + SM::kOffP, udS = ubase + SM::kOffdS;
+  const uint32_t bar = ubase + SM::kOffMisc;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + SM::kOffMisc + 16);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + SM::kOffMisc + 32);
+  int* s_qrow = reinterpret_cast<int*>(smem + SM::kOffRow);
+  int* s_kidx = s_qrow + 128;                                    // [table_keys]
+  float* s_kbias = reinterpret_cast<float*>(s_kidx + b.table_keys);
 
   const size_t seg_row0 = (size_t)t.seg * g.n;
   const __nv_bfloat16* qs = a.q + seg_row0 * D;
@@ -137,10 +168,10 @@ __global__ void __launch_bounds__(256, D == 64 ? 2 : 1) bwd_kernel(const __grid_
   const __nv_bfloat16* vs = a.v + seg_row0 * D;
   const __nv_bfloat16* dos = b.dout + seg_row0 * D;
 
-  // ---- row tables (as in the forward pass) ------------------------------------------------
+  // ---- row tables: key columns padded to whole tiles of 128 ----------------------------------
   int nkeys;
   if (t.mode == 1) {
-    const int bpad = (g.b + TK - 1) / TK * TK, mpad = (g.m + TK - 1) / TK * TK;
+    const int bpad = (g.b + TKB - 1) / TKB * TKB, mpad = (g.m + TKB - 1) / TKB * TKB;
     nkeys = bpad + mpad;
     const float wlog = g.m > 0 ? log2f((float)t.nk / (float)g.m) : 0.f;
     const int32_t* smp = a.samples + ((size_t)t.seg * g.nodes + t.node) * g.m;
@@ -155,156 +186,190 @@ __global__ void __launch_bounds__(256, D == 64 ? 2 : 1) bwd_kernel(const __grid_
       }
       s_kidx[i] = idx; s_kbias[i] = bias;
     }
-    if (tid < kTileQ) s_qrow[tid] = tid < t.nq ? t.qnode0 + a.perm_q[t.slice + t.spos0 + tid] : -1;
+    if (tid < 128) s_qrow[tid] = tid < t.nq ? t.qnode0 + a.perm_q[t.slice + t.spos0 + tid] : -1;
   } else {
     const int lim = t.causal ? min(t.nk, t.qk_off + t.nq) : t.nk;
-    nkeys = (lim + TK - 1) / TK * TK;
-    if (tid < kTileQ) s_qrow[tid] = tid < t.nq ? t.q0 + tid : -1;
+    nkeys = (lim + TKB - 1) / TKB * TKB;
+    if (tid < 128) s_qrow[tid] = tid < t.nq ? t.q0 + tid : -1;
   }
+  if (tid == 0) {
+    *s_abort = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  constexpr int kTmemCols = 512;                       // S 128 | dP 128 | dQ D  (power of two)
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (tid < kTileQ) {
-    const int qr = s_qrow[tid];
-    // (a padding row gets lse = +inf, so that all its weights are zero)
-    s_lse2[tid] = qr >= 0 ? b.lse[seg_row0 + qr] * 1.4426950408889634f : INFINITY;
-    s_delta[tid] = qr >= 0 ? b.delta[seg_row0 + qr] : 0.f;
-  }
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = *s_tmem;
+  const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+  constexpr uint32_t colS = 0, colDP = 128, colDQ = 256;
 
-  const uint32_t uQ = smem_u32(sQ), udO = smem_u32(sdO), uK = smem_u32(sK), uV = smem_u32(sV);
-  const uint32_t uP = smem_u32(sP), udS = smem_u32(sdS);
-  auto qrow_fn = [&](int r) { return s_qrow[r]; };
+  const int my_qrow = s_qrow[row];
+  // (a padding row gets lse = +inf, so that all its weights are zero)
+  const float lse2 = my_qrow >= 0 ? b.lse[seg_row0 + my_qrow] * 1.4426950408889634f : INFINITY;
+  const float delta = my_qrow >= 0 ? b.delta[seg_row0 + my_qrow] : 0.f;
+
   auto krow_of = [&](int i) {          // segment-relative key row of key column i, -1: padding
     if (t.mode == 1) return s_kidx[i];
     return i < t.nk ? t.k0 + i : -1;
   };
-  auto load_kv = [&](int kt, int stage) {
-    auto krow_fn = [&](int r) { return krow_of(kt * TK + r); };
-    gather_tile<D, TK>(uK + stage * SM::kKV, ks, krow_fn, tid);
-    gather_tile<D, TK>(uV + stage * SM::kKV, vs, krow_fn, tid);
+  constexpr int CPR = D / 8;
+  auto gather_rows = [&](uint32_t dst, const __nv_bfloat16* src, auto rowfn) {
+#pragma unroll
+    for (int i = 0; i < CPR / 2; ++i) {
+      const int c = tid + i * 256;
+      const int r = c / CPR, cc = c % CPR;
+      const int gr = rowfn(r);
+      const uint32_t d = dst + tile_off<128>(r, cc);
+      if (gr >= 0) cp_async16(d, src + (size_t)gr * D + cc * 8);
+      else st_shared_zero16(d);
+    }
   };
-  gather_tile<D, kTileQ>(uQ, qs, qrow_fn, tid);
-  gather_tile<D, kTileQ>(udO, dos, qrow_fn, tid);
-  const int ntiles = nkeys / TK;
-  load_kv(0, 0);
-  cp_async_commit();
+  gather_rows(uQ, qs, [&](int r) { return s_qrow[r]; });
+  gather_rows(udO, dos, [&](int r) { return s_qrow[r]; });
 
-  constexpr int KS = D / 16, NO = D / 8;
-  float dq[NO][4];
-#pragma unroll
-  for (int i = 0; i < NO; ++i) { dq[i][0] = dq[i][1] = dq[i][2] = dq[i][3] = 0.f; }
-  const int r_lo = warp * 16 + gid, r_hi = r_lo + 8;      // this lane's two query rows in the tile
+  // descriptors: low word = start >> 4 | (leading byte offset >> 4) << 16, high word = stride 1024 B | version | 128-byte swizzle
+  constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  constexpr uint32_t kSlab = 128 * 128;                // bytes of one [128 rows x 64 columns] slab
+  constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
+  constexpr uint32_t idesc_s = idesc_base | ((128u >> 3) << 17);                              // K-major x K-major, N = 128
+  constexpr uint32_t idesc_dq = idesc_base | (1u << 16) | (((uint32_t)D >> 3) << 17);          // K-major x MN-major, N = D
+  constexpr uint32_t idesc_t = idesc_base | (1u << 15) | (1u << 16) | (((uint32_t)D >> 3) << 17);   // MN-major x MN-major, N = D
+  auto kmajor = [&](uint32_t base, int ks) { return ((base + (ks >> 2) * kSlab + (ks & 3) * 32) >> 4) | (1u << 16); };
+  auto mnmajor = [&](uint32_t base, int kk) { return ((base + kk * 2048) >> 4) | ((kSlab >> 4) << 16); };
 
-  for (int kt = 0; kt < ntiles; ++kt) {
-    const int stage = kt & 1;
-    if (kt + 1 < ntiles) load_kv(kt + 1, stage ^ 1);
+  const int ntiles = nkeys / TKB;
+  uint32_t phase = 0;
+  bool ok = true;
+  auto load_kv = [&](int kt) {
+    gather_rows(uK, ks, [&](int r) { return krow_of(kt * TKB + r); });
+    gather_rows(uV, vs, [&](int r) { return krow_of(kt * TKB + r); });
     cp_async_commit();
-    cp_async_wait<1>();
+  };
+  if (ntiles > 0) load_kv(0);
+  for (int kt = 0; kt < ntiles; ++kt) {
+    // ---- this tile's K and V (requested while the previous tile's dV and dK left TMEM) ----------
+    cp_async_wait<0>();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    const uint32_t kb = uK + stage * SM::kKV, vb = uV + stage * SM::kKV;
-    // S = Q K^T and dP = dO V^T : 16 x 64 per warp each
-    float sc[TK / 8][4], dp[TK / 8][4];
+    // ---- S = Q K^T, dP = dO V^T ----------------------------------------------------------------
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < TK / 8; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; dp[i][0] = dp[i][1] = dp[i][2] = dp[i][3] = 0.f; }
+      for (int s = 0; s < D / 16; ++s) mma_ss(tmem + colS, kmajor(uQ, s), kmajor(uK, s), desc_hi, idesc_s, s > 0);
 #pragma unroll
-    for (int s = 0; s < KS; ++s) {
-      uint32_t qf[4], df[4];
-      ldmatrix_x4(qf, uQ + tile_off<kTileQ>(warp * 16 + (lane & 15), 2 * s + (lane >> 4)));
-      ldmatrix_x4(df, udO + tile_off<kTileQ>(warp * 16 + (lane & 15), 2 * s + (lane >> 4)));
+      for (int s = 0; s < D / 16; ++s) mma_ss(tmem + colDP, kmajor(udO, s), kmajor(uV, s), desc_hi, idesc_s, s > 0);
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    }
+    if (!mbar_wait_bounded(bar, phase)) *s_abort = 1;
+    phase ^= 1;
+    __syncthreads();
+    if (*s_abort) { ok = false; break; }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    // ---- P = C o exp(s - lse), dS = P (dP - delta): thread = query row ---------------------------
+#pragma unroll 1
+    for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+      uint32_t rs[32], rd[32];
+      tmem_ld32(lane_addr + colS + c0, rs);
+      tmem_ld32(lane_addr + colDP + c0, rd);
+      uint32_t pp[16], dd[16];
+      const int colbase = kt * TKB + c0;
+      // dense tiles need the mask only where the tile crosses the diagonal or the end of the keys
+      const bool dense_mask = t.mode != 1 && (colbase + 32 > t.nk || (t.causal && colbase + 31 > t.qk_off));
 #pragma unroll
-      for (int np = 0; np < TK / 16; ++np) {
-        uint32_t bf[4];
-        const uint32_t koff = tile_off<TK>(np * 16 + (lane & 7) + ((lane >> 4) << 3), 2 * s + ((lane >> 3) & 1));
-        ldmatrix_x4(bf, kb + koff);
-        mma_16816(sc[2 * np], qf, bf[0], bf[1]);
-        mma_16816(sc[2 * np + 1], qf, bf[2], bf[3]);
-        ldmatrix_x4(bf, vb + koff);
-        mma_16816(dp[2 * np], df, bf[0], bf[1]);
-        mma_16816(dp[2 * np + 1], df, bf[2], bf[3]);
+      for (int e = 0; e < 32; e += 4) {
+        float4 bias = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t.mode == 1) bias = *reinterpret_cast<const float4*>(s_kbias + colbase + e);
+        const float bb[4] = {bias.x, bias.y, bias.z, bias.w};
+        float p[4], ds[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          float x = fmaf(__uint_as_float(rs[e + h]), a.scale_log2, bb[h] - lse2);
+          if (dense_mask) { const int col = colbase + e + h; if (col >= t.nk || (t.causal && col > t.qk_off + row)) x = -INFINITY; }
+          asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p[h]) : "f"(x));
+          ds[h] = p[h] * (__uint_as_float(rd[e + h]) - delta);
+        }
+        pp[e >> 1] = pack2(p[0], p[1]); pp[(e >> 1) + 1] = pack2(p[2], p[3]);
+        dd[e >> 1] = pack2(ds[0], ds[1]); dd[(e >> 1) + 1] = pack2(ds[2], ds[3]);
+      }
+      // row `tid`, key columns c0 .. c0+31 = 16-byte chunks c0/8 .. c0/8+3 of the [query][key] tiles
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const uint32_t off = tile_off<128>(row, c0 / 8 + q4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(uP + off), "r"(pp[4 * q4]), "r"(pp[4 * q4 + 1]), "r"(pp[4 * q4 + 2]), "r"(pp[4 * q4 + 3]) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(udS + off), "r"(dd[4 * q4]), "r"(dd[4 * q4 + 1]), "r"(dd[4 * q4 + 2]), "r"(dd[4 * q4 + 3]) : "memory");
       }
     }
-    // P = C o exp(s - lse) (the coefficient is an additive bias on the log2 logit), dS = P (dP - delta)
-    uint32_t dsf[TK / 16][4];
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    // ---- dQ += dS K, dV = P^T dO, dK = dS^T Q -------------------------------------------------------
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-    for (int nt = 0; nt < TK / 8; ++nt) {
-      float p[4], ds[4];
+      for (int kk = 0; kk < TKB / 16; ++kk) mma_ss(tmem + colDQ, kmajor(udS, kk), mnmajor(uK, kk), desc_hi, idesc_dq, (kt > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int col = kt * TK + nt * 8 + 2 * tig + (e & 1);
-        const int row = (e & 2) ? r_hi : r_lo;
-        float x = sc[nt][e] * a.scale_log2;
-        if (t.mode == 1) x += s_kbias[col];
-        else if (col >= t.nk || (t.causal && col > t.qk_off + row)) x = -INFINITY;
-        p[e] = exp2f(x - s_lse2[row]);
-        ds[e] = p[e] * (dp[nt][e] - s_delta[row]);
-      }
-      const uint32_t p01 = pack2(p[0], p[1]), p23 = pack2(p[2], p[3]);
-      const uint32_t d01 = pack2(ds[0], ds[1]), d23 = pack2(ds[2], ds[3]);
-      dsf[nt >> 1][(nt & 1) * 2] = d01;
-      dsf[nt >> 1][(nt & 1) * 2 + 1] = d23;
-      // staged [query row][key column] for the transposed products
-      const uint32_t o_lo = tile_off<kTileQ>(r_lo, nt) + 4 * tig, o_hi = tile_off<kTileQ>(r_hi, nt) + 4 * tig;
-      asm volatile("st.shared.b32 [%0], %1;" ::"r"(uP + o_lo), "r"(p01));
-      asm volatile("st.shared.b32 [%0], %1;" ::"r"(uP + o_hi), "r"(p23));
-      asm volatile("st.shared.b32 [%0], %1;" ::"r"(udS + o_lo), "r"(d01));
-      asm volatile("st.shared.b32 [%0], %1;" ::"r"(udS + o_hi), "r"(d23));
+      for (int kk = 0; kk < 128 / 16; ++kk) mma_ss(tmem + colS, mnmajor(uP, kk), mnmajor(udO, kk), desc_hi, idesc_t, kk > 0);
+#pragma unroll
+      for (int kk = 0; kk < 128 / 16; ++kk) mma_ss(tmem + colDP, mnmajor(udS, kk), mnmajor(uQ, kk), desc_hi, idesc_t, kk > 0);
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
     }
-    // dQ += dS K
-#pragma unroll
-    for (int kk = 0; kk < TK / 16; ++kk) {
-#pragma unroll
-      for (int dpi = 0; dpi < NO / 2; ++dpi) {
-        uint32_t bf[4];
-        ldmatrix_x4_trans(bf, kb + tile_off<TK>(kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), 2 * dpi + (lane >> 4)));
-        mma_16816(dq[2 * dpi], dsf[kk], bf[0], bf[1]);
-        mma_16816(dq[2 * dpi + 1], dsf[kk], bf[2], bf[3]);
-      }
-    }
-    __syncthreads();   // P and dS of all 128 rows are staged
-    // Transposed products over the 128 query rows: warps 0-3 dV = P^T dO, warps 4-7 dK = dS^T Q,
-    // 16 keys of the tile per warp.
+    if (!mbar_wait_bounded(bar, phase)) *s_abort = 1;
+    phase ^= 1;
+    __syncthreads();
+    if (*s_abort) { ok = false; break; }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    // ---- dV and dK of this key tile leave TMEM: thread = key row ----------------------------------
     {
-      const int w4 = warp & 3;
-      const uint32_t uA = warp < 4 ? uP : udS;             // [query][key], read transposed
-      const uint32_t uB = warp < 4 ? udO : uQ;             // [query][d]
-      float acc[NO][4];
+      const int kr = krow_of(kt * TKB + row);
+      // every product that read K and V has finished: the next tile's rows can come in meanwhile
+      if (kt + 1 < ntiles) load_kv(kt + 1);
+      const uint32_t col = half ? colDP : colS;             // threads 0-127: dV, threads 128-255: dK
+      const float f = half ? b.scale : 1.f;
+      float* dst = half ? b.dk : b.dv;
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(lane_addr + col + c0, r);
+        if (kr >= 0) {
+          float* pd = dst + (seg_row0 + kr) * D + c0;
 #pragma unroll
-      for (int i = 0; i < NO; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
-#pragma unroll
-      for (int kq = 0; kq < kTileQ / 16; ++kq) {
-        uint32_t af[4];
-        // A (16 keys x 16 queries) = transpose of the staged block: matrix (mi, ki) comes from query rows
-        // 16 kq + 8 ki .., key chunk 2 w4 + mi
-        ldmatrix_x4_trans(af, uA + tile_off<kTileQ>(kq * 16 + ((lane >> 4) << 3) + (lane & 7), 2 * w4 + ((lane >> 3) & 1)));
-#pragma unroll
-        for (int dpi = 0; dpi < NO / 2; ++dpi) {
-          uint32_t bf[4];
-          ldmatrix_x4_trans(bf, uB + tile_off<kTileQ>(kq * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), 2 * dpi + (lane >> 4)));
-          mma_16816(acc[2 * dpi], af, bf[0], bf[1]);
-          mma_16816(acc[2 * dpi + 1], af, bf[2], bf[3]);
+          for (int e = 0; e < 32; e += 4)
+            atomicAdd(reinterpret_cast<float4*>(pd + e), make_float4(__uint_as_float(r[e]) * f, __uint_as_float(r[e + 1]) * f,
+                                                                      __uint_as_float(r[e + 2]) * f, __uint_as_float(r[e + 3]) * f));
         }
       }
-      const float f = warp < 4 ? 1.f : b.scale;
-      float* dst = warp < 4 ? b.dv : b.dk;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();   // S / dP columns and the K, V, P, dS tiles are free again
+  }
+  // ---- dQ: thread = query row (a row collects from every level it appears in) ---------------------
+  if (ok && ntiles > 0) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+    for (int c0 = (D / 2) * half; c0 < (D / 2) * half + D / 2; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld32(lane_addr + colDQ + c0, r);
+      if (my_qrow >= 0) {
+        float* pq = b.dq + (seg_row0 + my_qrow) * D + c0;
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int kr = krow_of(kt * TK + w4 * 16 + gid + 8 * h);
-        if (kr < 0) continue;
-        float* rowp = dst + (seg_row0 + kr) * D;
-#pragma unroll
-        for (int i = 0; i < NO; ++i) red_add2(rowp + i * 8 + 2 * tig, acc[i][2 * h] * f, acc[i][2 * h + 1] * f);
+        for (int e = 0; e < 32; e += 4)
+          atomicAdd(reinterpret_cast<float4*>(pq + e), make_float4(__uint_as_float(r[e]) * b.scale, __uint_as_float(r[e + 1]) * b.scale,
+                                                                    __uint_as_float(r[e + 2]) * b.scale, __uint_as_float(r[e + 3]) * b.scale));
       }
     }
-    __syncthreads();   // everyone is done with this stage and with the staged P / dS
   }
-  cp_async_wait<0>();
-
-  // ---- dQ: rows back to their original places (a row collects from every level it appears in) ----
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const int qr = s_qrow[h ? r_hi : r_lo];
-    if (qr < 0) continue;
-    float* rowp = b.dq + (seg_row0 + qr) * D;
-#pragma unroll
-    for (int i = 0; i < NO; ++i) red_add2(rowp + i * 8 + 2 * tig, dq[i][2 * h] * b.scale, dq[i][2 * h + 1] * b.scale);
+  if (!ok && tid == 0) atomicOr(status, 1 << 30);      // a bounded wait gave up
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -319,7 +384,7 @@ __global__ void to_bf16_kernel(const float4* __restrict__ src, uint2* __restrict
 
 // a: the forward schedule (tile list, permutations, samples); dq/dk/dv accumulators must be zero
 cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, const float* lse, const void* dout,
-                            float* delta, float* dq, float* dk, float* dv, float scale, cudaStream_t st) {
+                            float* delta, float* dq, float* dk, float* dv, float scale, int* status, cudaStream_t st) {
   const size_t rows = (size_t)a.g.G * a.g.n;
   const __nv_bfloat16* d16 = reinterpret_cast<const __nv_bfloat16*>(dout);
   const int dgrid = (int)((rows + 7) / 8);
@@ -334,15 +399,16 @@ cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, co
   if (e != cudaSuccess || a.total_tiles == 0) return e;
   BwdArgs b;
   b.a = a; b.dout = d16; b.lse = lse; b.delta = delta; b.dq = dq; b.dk = dk; b.dv = dv; b.scale = scale;
-  b.table_keys = a.g.sorted ? (a.g.b + TK - 1) / TK * TK + (a.g.m + TK - 1) / TK * TK : 0;
+  b.table_keys = a.g.sorted ? (a.g.b + TKB - 1) / TKB * TKB + (a.g.m + TKB - 1) / TKB * TKB : 0;
+  if (b.table_keys > kMaxNodeKeys) return cudaErrorInvalidValue;
   auto go = [&](auto kernel, int smem_bytes) {
     cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes + kMaxNodeKeys * 8);
     if (e2 != cudaSuccess) return e2;
-    kernel<<<a.total_tiles, 256, smem_bytes + b.table_keys * 8, st>>>(b);
+    kernel<<<a.total_tiles, 256, smem_bytes + b.table_keys * 8, st>>>(b, status);
     return cudaGetLastError();
   };
-  if (a.g.d == 64) return go(bwd_kernel<64>, Smem<64>::kFixed);
-  return go(bwd_kernel<128>, Smem<128>::kFixed);
+  if (a.g.d == 64) return go(bwd_tc_kernel<64>, SmemTc<64>::kFixed);
+  return go(bwd_tc_kernel<128>, SmemTc<128>::kFixed);
 }
 
 cudaError_t launch_to_bf16(const float* src, void* dst, size_t count, cudaStream_t st) {
