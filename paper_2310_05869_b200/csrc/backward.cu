@@ -243,6 +243,30 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
   auto kmajor = [&](uint32_t base, int ks) { return ((base + (ks >> 2) * kSlab + (ks & 3) * 32) >> 4) | (1u << 16); };
   auto mnmajor = [&](uint32_t base, int kk) { return ((base + kk * 2048) >> 4) | ((kSlab >> 4) << 16); };
 
+  // Rows leave TMEM one per thread, but a reduction instruction whose lanes hit 32 different rows costs
+  // the L2 32 half-filled sectors: the warp's 32 rows x 32 columns pass through a 4 KB slice of shared
+  // memory (the P tile's, idle at that point; chunks XOR-swizzled by row) and go out with eight lanes
+  // per row, four rows per instruction.
+  const uint32_t ustage = uP + warp * 4096;
+  auto reduce_rows = [&](const uint32_t (&r)[32], float f, float* base, int grow, int c0) {
+    const int lane = tid & 31;
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+      asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(ustage + lane * 128 + ((c ^ (lane & 7)) << 4)),
+                   "f"(__uint_as_float(r[4 * c]) * f), "f"(__uint_as_float(r[4 * c + 1]) * f),
+                   "f"(__uint_as_float(r[4 * c + 2]) * f), "f"(__uint_as_float(r[4 * c + 3]) * f) : "memory");
+    __syncwarp();
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int rr = 4 * it + (lane >> 3), c = lane & 7;
+      const int gr = __shfl_sync(0xffffffffu, grow, rr);
+      float4 v;
+      asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                   : "r"(ustage + rr * 128 + ((c ^ (rr & 7)) << 4)) : "memory");
+      if (gr >= 0) atomicAdd(reinterpret_cast<float4*>(base + (seg_row0 + gr) * D + c0 + 4 * c), v);
+    }
+    __syncwarp();
+  };
   const int ntiles = nkeys / TKB;
   uint32_t phase = 0;
   bool ok = true;
@@ -336,13 +360,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
       for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(lane_addr + col + c0, r);
-        if (kr >= 0) {
-          float* pd = dst + (seg_row0 + kr) * D + c0;
-#pragma unroll
-          for (int e = 0; e < 32; e += 4)
-            atomicAdd(reinterpret_cast<float4*>(pd + e), make_float4(__uint_as_float(r[e]) * f, __uint_as_float(r[e + 1]) * f,
-                                                                      __uint_as_float(r[e + 2]) * f, __uint_as_float(r[e + 3]) * f));
-        }
+        reduce_rows(r, f, dst, kr, c0);
       }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -355,13 +373,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
     for (int c0 = (D / 2) * half; c0 < (D / 2) * half + D / 2; c0 += 32) {
       uint32_t r[32];
       tmem_ld32(lane_addr + colDQ + c0, r);
-      if (my_qrow >= 0) {
-        float* pq = b.dq + (seg_row0 + my_qrow) * D + c0;
-#pragma unroll
-        for (int e = 0; e < 32; e += 4)
-          atomicAdd(reinterpret_cast<float4*>(pq + e), make_float4(__uint_as_float(r[e]) * b.scale, __uint_as_float(r[e + 1]) * b.scale,
-                                                                    __uint_as_float(r[e + 2]) * b.scale, __uint_as_float(r[e + 3]) * b.scale));
-      }
+      reduce_rows(r, b.scale, b.dq, my_qrow, c0);
     }
   }
   if (!ok && tid == 0) atomicOr(status, 1 << 30);      // a bounded wait gave up
