@@ -1246,7 +1246,10 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// [rows x d] bf16, row-major; one box = 64 columns x box_rows rows (one slab of an operand tile)
+}  // namespace
+
+// [rows x d] bf16, row-major; one box = 64 columns x box_rows rows (one slab of an operand tile).
+// (Also used by the backward pass's launcher.)
 bool encode_rows_map(CUtensorMap* m, const void* base, size_t rows, int d, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
@@ -1258,7 +1261,6 @@ bool encode_rows_map(CUtensorMap* m, const void* base, size_t rows, int d, int b
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-}  // namespace
 
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st) {
   if (a.total_pairs == 0) return cudaSuccess;

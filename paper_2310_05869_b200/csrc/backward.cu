@@ -14,10 +14,21 @@
 // tiles of 128, all five products on the tcgen05 tensor cores with accumulators in TMEM (see
 // bwd_tc_kernel); the three gradients are accumulated in fp32 with global reductions (a key
 // tile is shared by every query tile that samples it, a query row by every level it appears in).
+#include <cuda.h>
 #include "attn_common.cuh"
 
 namespace hyperattn {
+
+bool encode_rows_map(CUtensorMap* m, const void* base, size_t rows, int d, int box_rows);   // attn_tc.cu
+
 namespace {
+
+// K and V as [G * n rows x d] bf16 tensors, 128-byte swizzle, box = 64 columns x 128 rows: key tiles of
+// consecutive rows (causal leaves, unsorted nodes) arrive by TMA instead of through the load/store unit,
+// which the reductions keep busy
+struct alignas(64) BwdMaps {
+  CUtensorMap k, v;
+};
 
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -142,7 +153,7 @@ struct SmemTc {
 };
 
 template <int D>
-__global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ BwdArgs b, int* status) {
+__global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ BwdArgs b, const __grid_constant__ BwdMaps maps, int* status) {
   extern __shared__ __align__(1024) uint8_t smem[];
   using SM = SmemTc<D>;
   const AttnArgs& a = b.a;
@@ -156,6 +167,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
   const uint32_t uQ = ubase + SM::kOffQ, udO = ubase + SM::kOffdO, uK = ubase + SM::kOffK, uV = ubase + SM::kOffV;
   const uint32_t uP = ubase + SM::kOffP, udS = ubase + SM::kOffdS;
   const uint32_t bar = ubase + SM::kOffMisc;
+  const uint32_t bar_kv = ubase + SM::kOffMisc + 8;       // K and V tile of consecutive rows landed (TMA)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + SM::kOffMisc + 16);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + SM::kOffMisc + 32);
   int* s_qrow = reinterpret_cast<int*>(smem + SM::kOffRow);
@@ -195,6 +207,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
   if (tid == 0) {
     *s_abort = 0;
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_kv) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   constexpr int kTmemCols = 512;                       // S 128 | dP 128 | dQ D  (power of two)
@@ -270,15 +283,32 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
   const int ntiles = nkeys / TKB;
   uint32_t phase = 0;
   bool ok = true;
+  const bool dense = t.mode != 1;
   auto load_kv = [&](int kt) {
-    gather_rows(uK, ks, [&](int r) { return krow_of(kt * TKB + r); });
-    gather_rows(uV, vs, [&](int r) { return krow_of(kt * TKB + r); });
+    if (dense) {
+      // consecutive rows: one TMA box per 64 columns (rows past the key range are masked, rows past the tensor are zeros)
+      if (tid == 0) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_kv), "r"((uint32_t)(2 * SM::kQ)) : "memory");
+        const int y = (int)seg_row0 + t.k0 + kt * TKB;
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl) {
+          asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                       ::"r"(uK + sl * kSlab), "l"(&maps.k), "r"(sl * 64), "r"(y), "r"(bar_kv) : "memory");
+          asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                       ::"r"(uV + sl * kSlab), "l"(&maps.v), "r"(sl * 64), "r"(y), "r"(bar_kv) : "memory");
+        }
+      }
+    } else {
+      gather_rows(uK, ks, [&](int r) { return krow_of(kt * TKB + r); });
+      gather_rows(uV, vs, [&](int r) { return krow_of(kt * TKB + r); });
+    }
     cp_async_commit();
   };
   if (ntiles > 0) load_kv(0);
   for (int kt = 0; kt < ntiles; ++kt) {
     // ---- this tile's K and V (requested while the previous tile's dV and dK left TMEM) ----------
     cp_async_wait<0>();
+    if (dense && !mbar_wait_bounded(bar_kv, kt & 1)) *s_abort = 1;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
     // ---- S = Q K^T, dP = dO V^T ----------------------------------------------------------------
@@ -411,12 +441,15 @@ cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, co
   if (e != cudaSuccess || a.total_tiles == 0) return e;
   BwdArgs b;
   b.a = a; b.dout = d16; b.lse = lse; b.delta = delta; b.dq = dq; b.dk = dk; b.dv = dv; b.scale = scale;
+  if (rows > 0x7fffffffull) return cudaErrorInvalidValue;            // TMA row coordinates are 32-bit
+  BwdMaps maps;
+  if (!encode_rows_map(&maps.k, a.k, rows, a.g.d, 128) || !encode_rows_map(&maps.v, a.v, rows, a.g.d, 128)) return cudaErrorInvalidValue;
   b.table_keys = a.g.sorted ? (a.g.b + TKB - 1) / TKB * TKB + (a.g.m + TKB - 1) / TKB * TKB : 0;
   if (b.table_keys > kMaxNodeKeys) return cudaErrorInvalidValue;
   auto go = [&](auto kernel, int smem_bytes) {
     cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes + kMaxNodeKeys * 8);
     if (e2 != cudaSuccess) return e2;
-    kernel<<<a.total_tiles, 256, smem_bytes + b.table_keys * 8, st>>>(b, status);
+    kernel<<<a.total_tiles, 256, smem_bytes + b.table_keys * 8, st>>>(b, maps, status);
     return cudaGetLastError();
   };
   if (a.g.d == 64) return go(bwd_tc_kernel<64>, SmemTc<64>::kFixed);
