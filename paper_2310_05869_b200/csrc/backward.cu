@@ -131,6 +131,37 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t 
                "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}\n"
                ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
 }
+// packed fp32 pairs (two lanes per instruction)
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
+  return d;
+}
+__device__ __forceinline__ uint64_t pk2u(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a); hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
@@ -140,6 +171,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                  "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
                  "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                : "r"(taddr) : "memory");
+}
+// two loads in flight, one wait
+__device__ __forceinline__ void tmem_ld32_pair(uint32_t ta, uint32_t (&a)[32], uint32_t tb, uint32_t (&b)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+               : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]), "=r"(a[4]), "=r"(a[5]), "=r"(a[6]), "=r"(a[7]),
+                 "=r"(a[8]), "=r"(a[9]), "=r"(a[10]), "=r"(a[11]), "=r"(a[12]), "=r"(a[13]), "=r"(a[14]), "=r"(a[15]),
+                 "=r"(a[16]), "=r"(a[17]), "=r"(a[18]), "=r"(a[19]), "=r"(a[20]), "=r"(a[21]), "=r"(a[22]), "=r"(a[23]),
+                 "=r"(a[24]), "=r"(a[25]), "=r"(a[26]), "=r"(a[27]), "=r"(a[28]), "=r"(a[29]), "=r"(a[30]), "=r"(a[31])
+               : "r"(ta) : "memory");
+  tmem_ld32(tb, b);     // (its wait covers both loads)
+#pragma unroll
+  for (int i = 0; i < 32; ++i) asm volatile("" : "+r"(a[i]));    // no use of a[] may be scheduled above the wait
 }
 
 template <int D>
@@ -329,27 +373,32 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
 #pragma unroll 1
     for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
       uint32_t rs[32], rd[32];
-      tmem_ld32(lane_addr + colS + c0, rs);
-      tmem_ld32(lane_addr + colDP + c0, rd);
+      tmem_ld32_pair(lane_addr + colS + c0, rs, lane_addr + colDP + c0, rd);
       uint32_t pp[16], dd[16];
       const int colbase = kt * TKB + c0;
       // dense tiles need the mask only where the tile crosses the diagonal or the end of the keys
       const bool dense_mask = t.mode != 1 && (colbase + 32 > t.nk || (t.causal && colbase + 31 > t.qk_off));
+      const uint64_t sc2 = pk2(a.scale_log2, a.scale_log2), nlse2 = pk2(-lse2, -lse2), ndel2 = pk2(-delta, -delta);
 #pragma unroll
       for (int e = 0; e < 32; e += 4) {
         float4 bias = make_float4(0.f, 0.f, 0.f, 0.f);
         if (t.mode == 1) bias = *reinterpret_cast<const float4*>(s_kbias + colbase + e);
-        const float bb[4] = {bias.x, bias.y, bias.z, bias.w};
-        float p[4], ds[4];
+        const uint64_t off2[2] = {t.mode == 1 ? fadd2(pk2(bias.x, bias.y), nlse2) : nlse2, t.mode == 1 ? fadd2(pk2(bias.z, bias.w), nlse2) : nlse2};
 #pragma unroll
-        for (int h = 0; h < 4; ++h) {
-          float x = fmaf(__uint_as_float(rs[e + h]), a.scale_log2, bb[h] - lse2);
-          if (dense_mask) { const int col = colbase + e + h; if (col >= t.nk || (t.causal && col > t.qk_off + row)) x = -INFINITY; }
-          asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p[h]) : "f"(x));
-          ds[h] = p[h] * (__uint_as_float(rd[e + h]) - delta);
+        for (int h = 0; h < 2; ++h) {
+          float x0, x1, p0, p1, d0, d1;
+          upk2(ffma2(pk2u(rs[e + 2 * h], rs[e + 2 * h + 1]), sc2, off2[h]), x0, x1);
+          if (dense_mask) {
+            const int col = colbase + e + 2 * h;
+            if (col >= t.nk || (t.causal && col > t.qk_off + row)) x0 = -INFINITY;
+            if (col + 1 >= t.nk || (t.causal && col + 1 > t.qk_off + row)) x1 = -INFINITY;
+          }
+          asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p0) : "f"(x0));
+          asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p1) : "f"(x1));
+          upk2(fmul2(pk2(p0, p1), fadd2(pk2u(rd[e + 2 * h], rd[e + 2 * h + 1]), ndel2)), d0, d1);
+          pp[(e >> 1) + h] = pack2(p0, p1);
+          dd[(e >> 1) + h] = pack2(d0, d1);
         }
-        pp[e >> 1] = pack2(p[0], p[1]); pp[(e >> 1) + 1] = pack2(p[2], p[3]);
-        dd[e >> 1] = pack2(ds[0], ds[1]); dd[(e >> 1) + 1] = pack2(ds[2], ds[3]);
       }
       // row `tid`, key columns c0 .. c0+31 = 16-byte chunks c0/8 .. c0/8+3 of the [query][key] tiles
 #pragma unroll
