@@ -16,7 +16,7 @@ namespace hyperattn {
 cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st);
 cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, const float* lse, const void* dout,
-                            float* delta, float* dq, float* dk, float* dv, float scale, int* status, cudaStream_t st);
+                            float* delta, float* dq, float* dk, float* dv, void* dq_final, int dq_mode, float scale, int* status, cudaStream_t st);
 cudaError_t launch_to_bf16(const float* src, void* dst, size_t count, cudaStream_t st);
 
 namespace {
@@ -330,12 +330,14 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     float* dk = g32 ? reinterpret_cast<float*>(bw->dk) : acc + elems;
     float* dv = g32 ? reinterpret_cast<float*>(bw->dv) : acc + 2 * elems;
     StageScope sc(st, HYPERATTN_STAGE_BACKWARD, 2 + (g32 ? 0 : 3));
-    HA_CHECK(cudaMemsetAsync(dq, 0, elems * 4, st));
+    // without the causal recursion every query row belongs to one tile: the kernel writes dQ in its final type
+    const int dq_mode = a.direct ? (g32 ? 1 : 2) : 0;
+    if (!dq_mode) HA_CHECK(cudaMemsetAsync(dq, 0, elems * 4, st));
     HA_CHECK(cudaMemsetAsync(dk, 0, elems * 4, st));
     HA_CHECK(cudaMemsetAsync(dv, 0, elems * 4, st));
-    HA_CHECK(launch_backward(a, p.out, out_fp32, p.lse, bw->dout, reinterpret_cast<float*>(base + pl.delta), dq, dk, dv, scale, ws.status, st));
+    HA_CHECK(launch_backward(a, p.out, out_fp32, p.lse, bw->dout, reinterpret_cast<float*>(base + pl.delta), dq, dk, dv, bw->dq, dq_mode, scale, ws.status, st));
     if (!g32) {
-      HA_CHECK(launch_to_bf16(dq, bw->dq, elems, st));
+      if (!dq_mode) HA_CHECK(launch_to_bf16(dq, bw->dq, elems, st));
       HA_CHECK(launch_to_bf16(dk, bw->dk, elems, st));
       HA_CHECK(launch_to_bf16(dv, bw->dv, elems, st));
     }

@@ -69,6 +69,8 @@ struct BwdArgs {
   const float* lse;            // [G, n] final log-sum-exp of the forward pass (natural log)
   const float* delta;          // [G, n] <dO_i, O_i>
   float *dq, *dk, *dv;         // [G, n, D] fp32 accumulators, zeroed before the launch
+  void* dq_final;              // dq_mode 1 / 2: dQ rows are written here directly (fp32 / bf16) instead of accumulated
+  int dq_mode;                 // 0: a query row collects from several tiles (causal recursion): fp32 reductions into dq
   float scale;
   int table_keys;              // key columns of a node tile's row tables (block and samples, each padded to whole tiles)
 };
@@ -305,7 +307,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
   // memory (the P tile's, idle at that point; chunks XOR-swizzled by row) and go out with eight lanes
   // per row, four rows per instruction.
   const uint32_t ustage = uP + warp * 4096;
-  auto reduce_rows = [&](const uint32_t (&r)[32], float f, float* base, int grow, int c0) {
+  auto reduce_rows = [&](const uint32_t (&r)[32], float f, float* base, int grow, int c0, int store) {
     const int lane = tid & 31;
 #pragma unroll
     for (int c = 0; c < 8; ++c)
@@ -320,7 +322,12 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
       float4 v;
       asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
                    : "r"(ustage + rr * 128 + ((c ^ (rr & 7)) << 4)) : "memory");
-      if (gr >= 0) atomicAdd(reinterpret_cast<float4*>(base + (seg_row0 + gr) * D + c0 + 4 * c), v);
+      if (gr >= 0) {
+        const size_t el = (seg_row0 + gr) * D + c0 + 4 * c;
+        if (store == 0) atomicAdd(reinterpret_cast<float4*>(base + el), v);
+        else if (store == 1) *reinterpret_cast<float4*>(base + el) = v;
+        else *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(base) + el) = make_uint2(pack2(v.x, v.y), pack2(v.z, v.w));
+      }
     }
     __syncwarp();
   };
@@ -439,7 +446,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
       for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(lane_addr + col + c0, r);
-        reduce_rows(r, f, dst, kr, c0);
+        reduce_rows(r, f, dst, kr, c0, 0);
       }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -452,7 +459,8 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
     for (int c0 = (D / 2) * half; c0 < (D / 2) * half + D / 2; c0 += 32) {
       uint32_t r[32];
       tmem_ld32(lane_addr + colDQ + c0, r);
-      reduce_rows(r, b.scale, b.dq, my_qrow, c0);
+      // (without the causal recursion a query row belongs to exactly one tile: its dQ is final)
+      reduce_rows(r, b.scale, b.dq_mode ? reinterpret_cast<float*>(b.dq_final) : b.dq, my_qrow, c0, b.dq_mode);
     }
   }
   if (!ok && tid == 0) atomicOr(status, 1 << 30);      // a bounded wait gave up
@@ -475,7 +483,7 @@ __global__ void to_bf16_kernel(const float4* __restrict__ src, uint2* __restrict
 
 // a: the forward schedule (tile list, permutations, samples); dq/dk/dv accumulators must be zero
 cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, const float* lse, const void* dout,
-                            float* delta, float* dq, float* dk, float* dv, float scale, int* status, cudaStream_t st) {
+                            float* delta, float* dq, float* dk, float* dv, void* dq_final, int dq_mode, float scale, int* status, cudaStream_t st) {
   const size_t rows = (size_t)a.g.G * a.g.n;
   const __nv_bfloat16* d16 = reinterpret_cast<const __nv_bfloat16*>(dout);
   const int dgrid = (int)((rows + 7) / 8);
@@ -489,7 +497,7 @@ cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, co
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || a.total_tiles == 0) return e;
   BwdArgs b;
-  b.a = a; b.dout = d16; b.lse = lse; b.delta = delta; b.dq = dq; b.dk = dk; b.dv = dv; b.scale = scale;
+  b.a = a; b.dout = d16; b.lse = lse; b.delta = delta; b.dq = dq; b.dk = dk; b.dv = dv; b.dq_final = dq_final; b.dq_mode = dq_mode; b.scale = scale;
   if (rows > 0x7fffffffull) return cudaErrorInvalidValue;            // TMA row coordinates are 32-bit
   BwdMaps maps;
   if (!encode_rows_map(&maps.k, a.k, rows, a.g.d, 128) || !encode_rows_map(&maps.v, a.v, rows, a.g.d, 128)) return cudaErrorInvalidValue;
