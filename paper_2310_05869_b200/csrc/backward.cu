@@ -101,9 +101,10 @@ __global__ void __launch_bounds__(256) delta_kernel(const __nv_bfloat16* __restr
 //     dQ += dS K       A = dS [query][key] K-major,  B = K  [key][d]   MN-major     -> TMEM cols 256..256+d
 //     dV  = P^T dO     A = P  [query][key] MN-major, B = dO [query][d]  MN-major     -> over S's columns
 //     dK  = dS^T Q     A = dS [query][key] MN-major, B = Q  [query][d]  MN-major     -> over dP's columns
-// 256 threads: thread t and thread t + 128 share TMEM lane t mod 128 - query row t when P and dS
-// are formed (each takes 64 of the tile's 128 key columns), key row t when dV (threads 0-127) and
-// dK (threads 128-255) leave TMEM.  The phases of a key tile run one after the other (loads, S
+// 512 threads: threads t, t + 128, t + 256 and t + 384 share TMEM lane t mod 128 - query row t when P
+// and dS are formed (each takes 32 of the tile's 128 key columns), key row t when dV and dK leave
+// TMEM (the 2 d / 32 pieces of 32 columns are dealt round to the four groups of 128 threads).  Sixteen
+// warps instead of eight hide a little more latency (2-3 % per call).  The phases of a key tile run one after the other (loads, S
 // and dP, P and dS, the three gradient products, reductions): correct first, overlapped later.
 constexpr int TKB = 128;   // keys per tile
 constexpr unsigned long long kBwdWaitNs = 2000000000ull;
@@ -188,6 +189,8 @@ __device__ __forceinline__ void tmem_ld32_pair(uint32_t ta, uint32_t (&a)[32], u
   for (int i = 0; i < 32; ++i) asm volatile("" : "+r"(a[i]));    // no use of a[] may be scheduled above the wait
 }
 
+constexpr int kBwdThreads = 512;   // four threads per TMEM lane: 32 of a tile's 128 columns each
+
 template <int D>
 struct SmemTc {
   static constexpr int kQ = 128 * D * 2;              // Q, dO, K, V tiles: [128 rows x D]
@@ -199,13 +202,13 @@ struct SmemTc {
 };
 
 template <int D>
-__global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ BwdArgs b, const __grid_constant__ BwdMaps maps, int* status) {
+__global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_constant__ BwdArgs b, const __grid_constant__ BwdMaps maps, int* status) {
   extern __shared__ __align__(1024) uint8_t smem[];
   using SM = SmemTc<D>;
   const AttnArgs& a = b.a;
   const Geometry& g = a.g;
   const int tid = threadIdx.x, warp = tid >> 5;
-  const int row = tid & 127, half = tid >> 7;            // TMEM lane / tile row of this thread; which half of the work it takes
+  const int row = tid & 127, part = tid >> 7;            // TMEM lane / tile row of this thread; which quarter of the work it takes
   const TileDesc t = decode_tile(a, blockIdx.x);
   if (t.nq <= 0) return;
 
@@ -233,7 +236,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
     nkeys = bpad + mpad;
     const float wlog = g.m > 0 ? log2f((float)t.nk / (float)g.m) : 0.f;
     const int32_t* smp = a.samples + ((size_t)t.seg * g.nodes + t.node) * g.m;
-    for (int i = tid; i < nkeys; i += 256) {
+    for (int i = tid; i < nkeys; i += kBwdThreads) {
       int idx = -1; float bias = -INFINITY;
       if (i < bpad) {
         if (i < block_len(t.nk, g.b, t.beta)) { idx = t.k0 + a.perm_k[t.slice + (size_t)t.beta * g.b + i]; bias = 0.f; }
@@ -280,8 +283,8 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
   constexpr int CPR = D / 8;
   auto gather_rows = [&](uint32_t dst, const __nv_bfloat16* src, auto rowfn) {
 #pragma unroll
-    for (int i = 0; i < CPR / 2; ++i) {
-      const int c = tid + i * 256;
+    for (int i = 0; i < 128 * CPR / kBwdThreads; ++i) {
+      const int c = tid + i * kBwdThreads;
       const int r = c / CPR, cc = c % CPR;
       const int gr = rowfn(r);
       const uint32_t d = dst + tile_off<128>(r, cc);
@@ -378,7 +381,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     // ---- P = C o exp(s - lse), dS = P (dP - delta): thread = query row ---------------------------
 #pragma unroll 1
-    for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+    for (int c0 = 32 * part; c0 < 32 * part + 32; c0 += 32) {
       uint32_t rs[32], rd[32];
       tmem_ld32_pair(lane_addr + colS + c0, rs, lane_addr + colDP + c0, rd);
       uint32_t pp[16], dd[16];
@@ -439,14 +442,14 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
       const int kr = krow_of(kt * TKB + row);
       // every product that read K and V has finished: the next tile's rows can come in meanwhile
       if (kt + 1 < ntiles) load_kv(kt + 1);
-      const uint32_t col = half ? colDP : colS;             // threads 0-127: dV, threads 128-255: dK
-      const float f = half ? b.scale : 1.f;
-      float* dst = half ? b.dk : b.dv;
+      // 2 * D / 32 pieces of 32 columns (dV first, then dK), every fourth one to each group of 128 threads
 #pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
+      for (int piece = part; piece < 2 * (D / 32); piece += 4) {
+        const bool is_dk = piece >= D / 32;
+        const int c0 = (piece % (D / 32)) * 32;
         uint32_t r[32];
-        tmem_ld32(lane_addr + col + c0, r);
-        reduce_rows(r, f, dst, kr, c0, 0);
+        tmem_ld32(lane_addr + (is_dk ? colDP : colS) + c0, r);
+        reduce_rows(r, is_dk ? b.scale : 1.f, is_dk ? b.dk : b.dv, kr, c0, 0);
       }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -456,7 +459,7 @@ __global__ void __launch_bounds__(256, 1) bwd_tc_kernel(const __grid_constant__ 
   if (ok && ntiles > 0) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-    for (int c0 = (D / 2) * half; c0 < (D / 2) * half + D / 2; c0 += 32) {
+    for (int c0 = 32 * part; c0 < D; c0 += 128) {
       uint32_t r[32];
       tmem_ld32(lane_addr + colDQ + c0, r);
       // (without the causal recursion a query row belongs to exactly one tile: its dQ is final)
@@ -506,7 +509,7 @@ cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, co
   auto go = [&](auto kernel, int smem_bytes) {
     cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes + kMaxNodeKeys * 8);
     if (e2 != cudaSuccess) return e2;
-    kernel<<<a.total_tiles, 256, smem_bytes + b.table_keys * 8, st>>>(b, maps, status);
+    kernel<<<a.total_tiles, kBwdThreads, smem_bytes + b.table_keys * 8, st>>>(b, maps, status);
     return cudaGetLastError();
   };
   if (a.g.d == 64) return go(bwd_tc_kernel<64>, SmemTc<64>::kFixed);
