@@ -107,8 +107,9 @@ __global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a, SampleArgs s
 }
 
 // One CTA per (side, level, segment, chunk of the level): stable placement of <= 2048 rows.
+template <int R>
 __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
-  __shared__ uint32_t s_cnt[8][kBuckets];   // per-warp running positions
+  __shared__ __align__(16) uint32_t s_cnt[8][kBuckets];   // per-warp running positions
   __shared__ uint8_t s_id[kSortChunk];
   const Geometry& g = a.g;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
 
   const uint8_t* ids = a.ids + ((size_t)side * g.G + seg) * g.n + row0;
   for (int i = tid; i < rows; i += 256) s_id[i] = ids[i];
-  for (int i = tid; i < 8 * kBuckets; i += 256) (&s_cnt[0][0])[i] = 0;
+  for (int i = tid; i < 8 * kBuckets / 4; i += 256) reinterpret_cast<uint4*>(&s_cnt[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   // per-warp histograms of consecutive sub-ranges of 256 rows
   const int wbeg = warp * (kSortChunk / 8);
@@ -158,11 +159,9 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
     // match.any costs several times more)
     uint32_t peers = __ballot_sync(0xffffffffu, act);
 #pragma unroll
-    for (int bit = 0; bit < 8; ++bit) {
-      if (bit < g.r) {                                  // (uniform: ids have r bits)
-        const uint32_t bal = __ballot_sync(0xffffffffu, (id >> bit) & 1u);
-        peers &= ((id >> bit) & 1u) ? bal : ~bal;
-      }
+    for (int bit = 0; bit < R; ++bit) {                 // (ids have R bits)
+      const uint32_t bal = __ballot_sync(0xffffffffu, (id >> bit) & 1u);
+      peers &= ((id >> bit) & 1u) ? bal : ~bal;
     }
     const int before = __popc(peers & ((1u << lane) - 1u));
     uint32_t pos = 0;
@@ -208,7 +207,17 @@ cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_s
 cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st) {
   if (!g.sorted) return cudaSuccess;
   const SortArgs a = make_sort_args(g, ws);
-  sort_scatter_kernel<<<2 * g.levels * g.G * a.chunks_per_level, 256, 0, st>>>(a);
+  const int grid = 2 * g.levels * g.G * a.chunks_per_level;
+  switch (g.r) {                                         // the hash width is a template parameter of the ballot loop
+    case 1: sort_scatter_kernel<1><<<grid, 256, 0, st>>>(a); break;
+    case 2: sort_scatter_kernel<2><<<grid, 256, 0, st>>>(a); break;
+    case 3: sort_scatter_kernel<3><<<grid, 256, 0, st>>>(a); break;
+    case 4: sort_scatter_kernel<4><<<grid, 256, 0, st>>>(a); break;
+    case 5: sort_scatter_kernel<5><<<grid, 256, 0, st>>>(a); break;
+    case 6: sort_scatter_kernel<6><<<grid, 256, 0, st>>>(a); break;
+    case 7: sort_scatter_kernel<7><<<grid, 256, 0, st>>>(a); break;
+    default: sort_scatter_kernel<8><<<grid, 256, 0, st>>>(a); break;
+  }
   return cudaGetLastError();
 }
 
