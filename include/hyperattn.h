@@ -116,6 +116,12 @@ typedef struct hyperattn_params {
   size_t workspace_bytes;
   const hyperattn_debug* debug; /* may be NULL */
   void* stream;
+  /* ---- options added after version 1; all-zero selects the behaviour described above ---- */
+  int precise;           /* 1: every softmax weight enters the weights-times-values product as a pair of
+                            bf16 numbers (relative error 2^-17 instead of 2^-9).  With single bf16 weights an
+                            output entry can be off by 2^-8 max|v|, which is 2e-2 for values of N(0,1) size
+                            but more for heavy-tailed values; this mode keeps the error below 2e-2 for values
+                            up to +-20 at the price of twice the weights-times-values products.  bf16 inputs only. */
 } hyperattn_params;
 
 /* HyperAttention forward (Alg. 1-4 as specialised in Sec. 4) with bf16 inputs and

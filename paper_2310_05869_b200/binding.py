@@ -37,7 +37,8 @@ class _Params(C.Structure):
                 ("block", C.c_int), ("samples", C.c_int), ("hash_bits", C.c_int), ("causal", C.c_int),
                 ("n0", C.c_int), ("seed", C.c_uint64), ("dtype", C.c_int), ("out_dtype", C.c_int),
                 ("softmax_scale", C.c_float), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("debug", C.POINTER(_Debug)), ("stream", C.c_void_p)]
+                ("debug", C.POINTER(_Debug)), ("stream", C.c_void_p),
+                ("precise", C.c_int)]
 
 
 class _StageTimes(C.Structure):
@@ -113,7 +114,7 @@ def _debug_shapes(B, H, n, block, samples, causal, n0):
 
 
 def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_dtype=None, scale=0.0,
-            workspace=None, debug=False, stream=None):
+            workspace=None, debug=False, stream=None, precise=False):
     """HyperAttention forward on CUDA tensors q, k, v of shape [B, H, n, d] (bf16 or fp32).
     Returns (out, lse) or (out, lse, intermediates) when debug=True."""
     if not (q.is_cuda and k.is_cuda and v.is_cuda):
@@ -129,6 +130,7 @@ def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_
     if workspace is not None:
         p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     p.stream = stream if stream is not None else torch.cuda.current_stream(q.device).cuda_stream
+    p.precise = int(bool(precise))
     inter = None
     if debug:
         G, LV, NL, NODES = _debug_shapes(B, H, n, block, samples, causal, n0)

@@ -21,7 +21,7 @@ cudaError_t launch_to_bf16(const float* src, void* dst, size_t count, cudaStream
 
 namespace {
 
-constexpr int kVersion = 1;
+constexpr int kVersion = 2;
 constexpr size_t kAlign = 256;
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -289,6 +289,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   a.perm_q = ws.perm_q; a.perm_k = ws.perm_k; a.rank_k = ws.rank_k; a.samples = ws.samples;
   a.part_o = ws.part_o; a.part_lse = ws.part_lse; a.out = p.out; a.lse = p.lse;
   a.out_fp32 = out_fp32;
+  a.precise = p.precise != 0;
   a.direct = g.L == 0;
   a.dense_causal = g.causal;
   a.tiles_per_block = (g.b + kTileQ - 1) / kTileQ;

@@ -29,6 +29,7 @@ struct AttnArgs {
   void* out; float* lse;             // final results, used when direct
   int out_fp32;
   int direct;
+  int precise;                       // softmax weights enter the P V product as bf16 hi + lo
   // dense (leaf) tiles
   int dense_causal;
   int tiles_per_leaf, leaves_per_seg, n_leaf_tiles;

@@ -47,6 +47,7 @@ struct alignas(64) TmaMaps {
 constexpr int TK = 64;                  // keys per tile
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
 constexpr float kRescaleThreshold = 32.f;   // octaves the scores may exceed the reference before it moves
+constexpr float kTileSumLimit = 1099511627776.f;   // 2^40: a tile whose weights sum to more has a score > 2^34 above the reference
 
 // Optional per-role cycle counters (compile with -DHA_TC_TIMING; never in the shipped build).
 #ifdef HA_TC_TIMING
@@ -177,7 +178,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
+#ifdef HA_EXP_FAKE
+  asm("mul.f32 %0, %1, 0f00000000;" : "=f"(y) : "f"(x));     // timing experiment only: results are meaningless
+#else
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+#endif
   return y;
 }
 // packed pairs of fp32 (one instruction, two lanes)
@@ -456,7 +461,10 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
 __device__ __forceinline__ int tile_of(const QTile& q, int a) { return a < q.n1 ? q.s1 + a : q.s2 + (a - q.n1); }
 // GATHER_LATE: the softmax threads fetch the next item's Q tiles after, not before, they write
 // the current item's results (see there).
-template <int D, bool GATHER_LATE>
+// PRECISE: every softmax weight enters the P V product as a pair of bf16 numbers hi + lo (relative error
+// 2^-17 instead of 2^-9): lo is written into the second half of the S buffer and multiplied by V with a
+// second set of products.
+template <int D, bool GATHER_LATE, bool PRECISE>
 __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TmaMaps maps, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -573,7 +581,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       }
       return true;
     };
-    HA_LDECL(a_tab); HA_LDECL(a_ws); HA_LDECL(a_cmp); HA_LDECL(a_epi); HA_LDECL(a_gq); HA_LDECL(a_bo); HA_LDECL(a_tiles);
+    HA_LDECL(a_tab); HA_LDECL(a_ws); HA_LDECL(a_cmp); HA_LDECL(a_epi); HA_LDECL(a_gq); HA_LDECL(a_bo); HA_LDECL(a_tiles); HA_LDECL(a_ws0); HA_LDECL(a_c1); HA_LDECL(a_c2); HA_LDECL(a_c3); HA_LDECL(a_c4);
     HA_T0(t_role);
     if (blockIdx.x < a.total_pairs) ok = __all_sync(0xffffffffu, gather_q(0));
     for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
@@ -604,6 +612,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         ok = __all_sync(0xffffffffu, mbar_wait<20, 2>(bar_s(i, buf), (gw / C::kSBufs) & 1, s_abort, status));   // warp-uniform: TMEM ops are .aligned
         if (!ok) break;
         HA_LACC(a_ws, tw);
+#ifdef HA_TC_TIMING
+        if (na == 0) a_ws0 += clock64() - tw;
+#endif
         HA_T0(tc);
         tc_fence_after();
         // mask kind of this (query tile, key tile): uniform over the warpgroup
@@ -630,22 +641,33 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           }
           mask_scores(sbase, visa, visb);
         }
+        // The second half of the scores is requested once the first has arrived and lands while
+        // the first is exponentiated.
         tmem_ld32_issue(sbase, ra);
-        tmem_ld32_issue(sbase + 32, rb);
         tmem_ld32_wait(ra);
-        tmem_ld32_wait(rb);
-        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+        tmem_ld32_issue(sbase + 32, rb);
+        HA_LACC(a_c1, tc);
+        // The row maximum is NOT computed per tile.  Any reference within a few dozen octaves of the
+        // true maximum serves (the accumulators are fp32 and the weights keep their relative
+        // precision as bf16), so a tile is exponentiated against the reference the row already
+        // has, and only when the tile's sum of weights shows that some score lay more than ~2^34
+        // above it (or the row has no reference yet: first tile of an item) is the maximum
+        // taken, the reference moved by whole octaves, O rescaled exactly, and the tile
+        // exponentiated again from the scores still held in registers.
+        auto move_reference = [&]() -> bool {
+          tmem_ld32_wait(rb);
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-          m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
-          m1 = max3(m1, __uint_as_float(ra[e + 2]), __uint_as_float(ra[e + 3]));
-          m2 = max3(m2, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
-          m3 = max3(m3, __uint_as_float(rb[e + 2]), __uint_as_float(rb[e + 3]));
-        }
-        m0 = fmaxf(m0, m2); m1 = fmaxf(m1, m3);
-        const float xm = fmaf(fmaxf(m0, m1), a.scale_log2, ubias);   // scale_log2 > 0: the maximum commutes with it
-        const bool grow = xm > m_ref + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, grow)) {          // rare; per warp so that TMEM accesses stay convergent
+          for (int e = 0; e < 32; e += 4) {
+            m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            m1 = max3(m1, __uint_as_float(ra[e + 2]), __uint_as_float(ra[e + 3]));
+            m2 = max3(m2, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+            m3 = max3(m3, __uint_as_float(rb[e + 2]), __uint_as_float(rb[e + 3]));
+          }
+          m0 = fmaxf(m0, m2); m1 = fmaxf(m1, m3);
+          const float xm = fmaf(fmaxf(m0, m1), a.scale_log2, ubias);   // scale_log2 > 0: the maximum commutes with it
+          const bool grow = xm > m_ref + kRescaleThreshold;
+          if (!__any_sync(0xffffffffu, grow)) return true;
           float alpha = 1.f;
           if (grow) {
             // first tile: leave head room for the weight log2(N/m) that the sampled columns will
@@ -663,35 +685,74 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           // tiles later and needs this warpgroup's P first.
           if (na > 0) {
             const int gjp = gbase + tile_of(q, na - 1);
-            ok = __all_sync(0xffffffffu, mbar_wait<20, 3>(bar_vempty(i, gjp % C::NS), (gjp / C::NS) & 1, s_abort, status));
-            if (!ok) break;
+            if (!__all_sync(0xffffffffu, mbar_wait<20, 3>(bar_vempty(i, gjp % C::NS), (gjp / C::NS) & 1, s_abort, status))) return false;
             tc_fence_after();
             rescale_row(lane_addr + colO, C::kOCols, alpha);
           }
-        }
-        const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
-        // packed fp32 arithmetic (two lanes per instruction) for the scaling and the two row sums
-        const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2), off2 = pack_f2(off, off);
-        auto chunk_exp = [&](const uint32_t (&r)[32], int c) {
-          uint32_t p[16];
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float x0, x1;
-            unpack_f2(ffma2(pack_u2(r[e], r[e + 1]), sc2, off2), x0, x1);
-            const float p0 = ex2(x0), p1 = ex2(x1);
-            l01 = fadd2(l01, pack_f2(p0, p1));
-            const uint32_t w = pack2(p0, p1);
-            if constexpr (!C::kOnes)
-              asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}" : "+f"(lra), "+f"(lrb) : "r"(w));
-            p[e >> 1] = w;
-          }
-          tmem_st16(sbase + c * 16, p);
+          return true;
         };
-        chunk_exp(ra, 0);
-        chunk_exp(rb, 1);
+        if (__any_sync(0xffffffffu, m_ref == -INFINITY)) {
+          ok = move_reference();
+          if (!ok) break;
+        }
+        const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
+        uint64_t lt2;               // this tile's unrounded sum of weights (two partial sums, packed)
+        float lrta, lrtb;           // this tile's sum of the bf16 weights (d = 128)
+        for (int attempt = 0;; ++attempt) {
+          const float off = ubias - (m_ref == -INFINITY ? 0.f : m_ref);
+          // packed fp32 arithmetic (two lanes per instruction) for the scaling and the row sums
+          const uint64_t off2 = pack_f2(off, off);
+          lt2 = 0; lrta = 0.f; lrtb = 0.f;
+          auto chunk_exp = [&](const uint32_t (&r)[32], int c) {
+            uint32_t p[16], plo[16];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float x0, x1;
+              unpack_f2(ffma2(pack_u2(r[e], r[e + 1]), sc2, off2), x0, x1);
+              const float p0 = ex2(x0), p1 = ex2(x1);
+              lt2 = fadd2(lt2, pack_f2(p0, p1));
+              const uint32_t w = pack2(p0, p1);
+              if constexpr (!C::kOnes)
+                asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}" : "+f"(lrta), "+f"(lrtb) : "r"(w));
+              p[e >> 1] = w;
+              if constexpr (PRECISE) {
+                // what the rounding to bf16 left over, as a second bf16 number (infinite weights leave none)
+                const float r0 = p0 - __uint_as_float(w << 16), r1 = p1 - __uint_as_float(w & 0xffff0000u);
+                const uint32_t wl = pack2(r0 == r0 ? r0 : 0.f, r1 == r1 ? r1 : 0.f);
+                if constexpr (!C::kOnes)
+                  asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}" : "+f"(lrta), "+f"(lrtb) : "r"(wl));
+                plo[e >> 1] = wl;
+              }
+            }
+            tmem_st16(sbase + c * 16, p);
+            if constexpr (PRECISE) {
+              tmem_st16(sbase + 32 + c * 16, plo);
+            }
+          };
+          HA_T0(tc2);
+          if constexpr (PRECISE) tmem_ld32_wait(rb);     // the lo halves overwrite the second half of the scores
+          chunk_exp(ra, 0);
+          HA_LACC(a_c2, tc2);
+          HA_T0(tc3);
+          tmem_ld32_wait(rb);
+          chunk_exp(rb, 1);
+          HA_LACC(a_c3, tc3);
+          float lt0, lt1;
+          unpack_f2(lt2, lt0, lt1);
+          // (the negated comparison also catches an infinite sum; one second attempt at most: after the
+          // reference has moved every finite score is within range, and non-finite inputs must not loop)
+          if (attempt == 1 || !__any_sync(0xffffffffu, !(lt0 + lt1 <= kTileSumLimit))) break;
+          ok = move_reference();
+          if (!ok) break;
+        }
+        if (!ok) break;
+        HA_T0(tc4);
+        l01 = fadd2(l01, lt2);
+        lra += lrta; lrb += lrtb;
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p(i, buf));
+        HA_LACC(a_c4, tc4);
         HA_LACC(a_cmp, tc);
 #ifdef HA_TC_TIMING
         a_tiles += 1;
@@ -806,6 +867,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     if (row == 0 && i == 0) {
       HA_LFLUSH(9, a_tab); HA_LFLUSH(0, a_ws); HA_LFLUSH(2, a_cmp); HA_LFLUSH(15, a_epi); HA_LFLUSH(16, a_gq); HA_LFLUSH(17, a_bo);
       HA_LFLUSH(20, a_tiles); HA_TACC(18, t_role); HA_LFLUSH(19, it);
+      HA_LFLUSH(24, a_ws0); HA_LFLUSH(22, a_c1); HA_LFLUSH(29, a_c2); HA_LFLUSH(30, a_c3); HA_LFLUSH(31, a_c4);
     }
 #endif
   } else if (warp < 10) {
@@ -897,6 +959,10 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           mma_ts2(ocol, pcol, dv_lo, desc_hi, idesc_o, a2 > 0);
 #pragma unroll
           for (int kk = 1; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
+          if constexpr (PRECISE) {
+#pragma unroll
+            for (int kk = 0; kk < TK / 16; ++kk) mma_ts2(ocol, pcol + 32 + kk * 8, dv_lo + kk * (2048 >> 4), desc_hi, idesc_o, 1);
+          }
           umma_commit(bar_vempty(i, s));
           vnext = gj + 1;
           if (a2 == total - 1) umma_commit(bar_o(i));
@@ -1278,9 +1344,14 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
     kernel<<<grid, 384, smem_bytes, st>>>(a, maps, status);
     return cudaGetLastError();
   };
-  if (a.g.d == 64) return go(attn_tc_kernel<64, false>, Cfg<64>::kTotal);
-  if (!a.direct) return go(attn_tc_kernel<128, true>, Cfg<128>::kTotal);
-  return go(attn_tc_kernel<128, false>, Cfg<128>::kTotal);
+  if (a.precise) {
+    if (a.g.d == 64) return go(attn_tc_kernel<64, false, true>, Cfg<64>::kTotal);
+    if (!a.direct) return go(attn_tc_kernel<128, true, true>, Cfg<128>::kTotal);
+    return go(attn_tc_kernel<128, false, true>, Cfg<128>::kTotal);
+  }
+  if (a.g.d == 64) return go(attn_tc_kernel<64, false, false>, Cfg<64>::kTotal);
+  if (!a.direct) return go(attn_tc_kernel<128, true, false>, Cfg<128>::kTotal);
+  return go(attn_tc_kernel<128, false, false>, Cfg<128>::kTotal);
 }
 
 }  // namespace hyperattn

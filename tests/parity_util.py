@@ -6,11 +6,14 @@ Rules (one per stage of the path):
   samples  bit-exact
   perms    bit-exact given the GPU's own bucket ids (and end to end when no id differs)
   out/lse  oracle evaluated with the GPU's ids injected: max |err| <= 2e-2, mean |err| <= 2e-3,
-           |d lse| <= 1e-3 * max(|lse|, 1).  The output bounds are the stated ones for value
-           rows of N(0,1) size; the weights enter the tensor cores as bf16 (relative error
-           2^-9 each), so the attainable bound grows with the values: |err| <= 2^-9 * sum_j
-           w_j |v_j - out| <= 2^-8 max|v|.  For inputs with max|v| above ~5 (the heavy-tailed
-           workload, clipped at 20) the bounds scale by max|v| / 5.12.
+           |d lse| <= 1e-3 * max(|lse|, 1), all three unscaled, for every workload.  (The
+           softmax weights enter the tensor cores as bf16, relative error 2^-9 each, so an
+           output entry can be off by 2^-9 * sum_j w_j |v_j - out| <= 2^-8 max|v|: 2e-2 for value
+           rows of N(0,1) size, more for the heavy-tailed workload whose values reach 20.  Calls
+           that must meet 2e-2 on such values pass `precise=True`: the weights then enter as a
+           bf16 pair hi + lo, relative error 2^-17.  `check_outputs` never widens a bound; a
+           caller that knowingly runs the single-bf16 weights on heavy values passes
+           `max_abs_bound` explicitly, and that bound is the derived 2^-8 max|v| itself.)
 """
 from __future__ import annotations
 
@@ -26,6 +29,24 @@ OUT_MAX_ABS = 2e-2
 OUT_MEAN_ABS = 2e-3
 LSE_REL = 1e-3
 AMBIGUOUS = 1e-4
+
+
+def heavy_values(w: WL.Workload) -> bool:
+    """Workloads whose value rows are far larger than N(0,1) draws (Student-t clipped at +-20)."""
+    return w.kind == "student_t"
+
+
+def output_policy(w: WL.Workload, arrs):
+    """(precise, max_abs_bound) for a workload.  Everything is held to the stated 2e-2.  bf16 calls on
+    heavy-tailed values meet it with split weights (`precise`); fp32-input calls have no such mode (their
+    kernel rounds the weights to single bf16 numbers), so for heavy-tailed fp32 inputs the bound asserted
+    is the derived 2^-8 max|v| itself, stated here and printed by the caller next to the measured error."""
+    if not heavy_values(w):
+        return False, OUT_MAX_ABS
+    if w.dtype == "bf16":
+        return True, OUT_MAX_ABS
+    vmax = float(np.abs(WL.as_f64(arrs[2])).max())
+    return False, max(OUT_MAX_ABS, vmax / 256.0)
 
 
 def to_device(w: WL.Workload, arrs):
@@ -142,7 +163,8 @@ def oracle_rows(w, Q64, K64, V64, g, rows, ids_q=None, ids_k=None):
                              scale=1.0 / math.sqrt(w.d), rows=rows, ids_q=ids_q, ids_k=ids_k)
 
 
-def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, segs=None, rng_seed=0):
+def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, segs=None, rng_seed=0,
+                  max_abs_bound=None, blocks_per_seg=0):
     """Compares out/lse with the oracle (GPU ids injected when `inter` is given).  With
     rows_per_seg, a pseudo-random subset of rows plus the rows around every leaf / node
     boundary is checked."""
@@ -173,9 +195,8 @@ def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, seg
     stats = {"max_abs": float(err.max()), "mean_abs": float(err.mean()), "lse_rel": float(lerr.max()),
              "rows": int(lerr.size)}
     assert np.isfinite(err).all() and np.isfinite(lerr).all(), stats
-    vscale = max(1.0, max(float(np.abs(V64[g]).max()) for g in segs) / 5.12)      # see the module docstring
-    stats["value_scale"] = vscale
-    assert stats["max_abs"] <= OUT_MAX_ABS * vscale, stats
-    assert stats["mean_abs"] <= OUT_MEAN_ABS * vscale, stats
+    stats["max_abs_bound"] = OUT_MAX_ABS if max_abs_bound is None else float(max_abs_bound)
+    assert stats["max_abs"] <= stats["max_abs_bound"], stats
+    assert stats["mean_abs"] <= OUT_MEAN_ABS, stats
     assert stats["lse_rel"] <= LSE_REL, stats
     return stats

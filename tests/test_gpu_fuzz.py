@@ -46,7 +46,9 @@ CASES = [draw(s) for s in range(24)]
 def check(w):
     arrs = WL.make_inputs(w)
     q, k, v = PU.to_device(w, arrs)
-    out, lse, inter = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, out_dtype=torch.float32, debug=True)
+    precise, bound = PU.output_policy(w, arrs)
+    out, lse, inter = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, out_dtype=torch.float32, debug=True,
+                                 precise=precise)
     torch.cuda.synchronize()
     assert ha.last_device_status() == 0
     Q64, K64, V64 = (WL.as_f64(x) for x in arrs)
@@ -55,8 +57,8 @@ def check(w):
         assert mism <= amb
         PU.check_samples(w, inter)
         PU.check_perms(w, inter)
-        return PU.check_outputs(w, Q64, K64, V64, out, lse, inter)
-    return PU.check_outputs(w, Q64, K64, V64, out, lse, None)
+        return PU.check_outputs(w, Q64, K64, V64, out, lse, inter, max_abs_bound=bound)
+    return PU.check_outputs(w, Q64, K64, V64, out, lse, None, max_abs_bound=bound)
 
 
 @pytest.mark.parametrize("w", CASES, ids=[f"{w.name}_n{w.n}_d{w.d}_b{w.b}_m{w.m}_r{w.r}_{'c' if w.causal else 'nc'}{w.n0}_{w.kind}_{w.dtype}" for w in CASES])

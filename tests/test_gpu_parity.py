@@ -57,11 +57,11 @@ SMALL = [
 ]
 
 
-def run(w, out_dtype=None, debug=True, workspace=None):
+def run(w, out_dtype=None, debug=True, workspace=None, precise=False):
     arrs = WL.make_inputs(w)
     q, k, v = PU.to_device(w, arrs)
     res = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, out_dtype=out_dtype,
-                     debug=debug, workspace=workspace)
+                     debug=debug, workspace=workspace, precise=precise)
     torch.cuda.synchronize()
     assert ha.last_device_status() == 0
     Q64, K64, V64 = (WL.as_f64(x) for x in arrs)
@@ -70,17 +70,41 @@ def run(w, out_dtype=None, debug=True, workspace=None):
 
 @pytest.mark.parametrize("w", SMALL, ids=[w.name for w in SMALL])
 def test_small_configs_every_stage(w):
-    (out, lse, inter), (Q64, K64, V64) = run(w, out_dtype=torch.float32)
+    precise, bound = PU.output_policy(w, WL.make_inputs(w))
+    (out, lse, inter), (Q64, K64, V64) = run(w, out_dtype=torch.float32, precise=precise)
     sorted_any = any(w.b < s for _, s in PU.levels_of(w))
     if sorted_any:
         amb, mism = PU.check_ids(w, Q64, K64, inter)
         PU.check_samples(w, inter)
         PU.check_perms(w, inter)
-        stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter)
+        stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter, max_abs_bound=bound)
         print(w.name, "ambiguous bits", amb, "id mismatches", mism, stats)
     else:
-        stats = PU.check_outputs(w, Q64, K64, V64, out, lse, None)
+        stats = PU.check_outputs(w, Q64, K64, V64, out, lse, None, max_abs_bound=bound)
         print(w.name, stats)
+
+
+def test_heavy_values_single_bf16_weights_meet_the_derived_bound():
+    """Without split weights the attainable bound is 2^-8 max|v| (each weight is a bf16 number, relative
+    error 2^-9, and the output is normalised by the sum of the rounded weights): asserted as such, with
+    the measured error printed; the mean error stays under the stated 2e-3 either way."""
+    w = [x for x in SMALL if x.name == "causal_heavy_tail"][0]
+    (out, lse, inter), (Q64, K64, V64) = run(w, out_dtype=torch.float32, precise=False)
+    vmax = float(np.abs(V64).max())
+    stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter, max_abs_bound=vmax / 256.0)
+    print(w.name, "single bf16 weights: max|v|", vmax, "bound", vmax / 256.0, stats)
+
+
+@pytest.mark.parametrize("d,causal", [(64, False), (128, True)])
+def test_precise_mode_matches_on_gaussian_inputs(d, causal):
+    """Split weights on ordinary inputs: same tolerances, and a smaller error than single weights."""
+    w = W("precise_gauss", 1, 2, 2048, d, "bf16", 128, 96, 6, causal, 512, seed=40 + d)
+    (o1, l1, i1), (Q64, K64, V64) = run(w, out_dtype=torch.float32, precise=True)
+    s1 = PU.check_outputs(w, Q64, K64, V64, o1, l1, i1)
+    (o0, l0, i0), _ = run(w, out_dtype=torch.float32, precise=False)
+    s0 = PU.check_outputs(w, Q64, K64, V64, o0, l0, i0)
+    print("precise", s1, "single", s0)
+    assert s1["mean_abs"] < 0.25 * s0["mean_abs"]
 
 
 def test_bf16_output_and_caller_workspace():
