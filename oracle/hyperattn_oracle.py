@@ -18,6 +18,8 @@ r hash bits; P_Q, P_K the sortLSH permutations; M^H the block mask):
   bucket_ids         sign pattern -> Gray-ordered bucket id (Def. 1, Alg. 1 line 2)
   stable_argsort     permutations P_Q, P_K (Alg. 1 line 3)
   sortlsh_mask       the mask M^H (Alg. 1 line 4)
+  query_block_size   rows per group of sorted queries when queries and keys differ in number
+  causal_grid        leaves and levels of the recursive split for any sequence length
   sample_indices     l_1..l_m ~ Unif([N]) shared by all rows (Alg. 2 line 4, Sec. 4)
   exact_attention    D^-1 A V and its causal form (Sec. 1.1, Sec. 3.1)
   node_forward       block-diagonal part + sampled residual with estimated D
@@ -178,9 +180,21 @@ def stable_argsort(ids):
     return perm, rank
 
 
-def sortlsh_mask(rank_q, rank_k, b):
-    """M^H_ij = 1{ floor(P_Q(i)/b) = floor(P_K(j)/b) }  (Alg. 1 line 4)."""
-    bq = np.asarray(rank_q) // b
+def query_block_size(n_q, n_k, b):
+    """Rows per group of sorted queries.  Alg. 1 line 4 pairs the beta-th group of b sorted queries
+    with the beta-th group of b sorted keys and is written for n_q = n_k.  Reading taken for
+    n_q != n_k (cross attention, or the last off-diagonal problem of a causal sequence whose length
+    the split does not divide): the key groups keep b rows and the query groups get
+    b_q = ceil(b * n_q / n_k) rows, so that group beta of either side covers the same fraction of the
+    sorted order; b_q = b when n_q = n_k, and ceil(n_q / b_q) <= ceil(n_k / b), so every query group
+    has its key group."""
+    return -((-b * n_q) // n_k)
+
+
+def sortlsh_mask(rank_q, rank_k, b, b_q=None):
+    """M^H_ij = 1{ floor(P_Q(i)/b_q) = floor(P_K(j)/b) }  (Alg. 1 line 4; b_q = b when the sides have
+    the same number of rows, see query_block_size)."""
+    bq = np.asarray(rank_q) // (b if b_q is None else b_q)
     bk = np.asarray(rank_k) // b
     return (bq[:, None] == bk[None, :]).astype(np.int64)
 
@@ -211,9 +225,10 @@ def exact_attention(Q, K, V, scale, causal=False, rows=None):
 # One non-causal HyperAttention problem (Alg. 1-3 as specialised in Sec. 4)
 # --------------------------------------------------------------------------------------
 def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
-    """HyperAttention on N queries x N keys.
+    """HyperAttention on n_q queries x N keys (n_q = N in the paper; see query_block_size for the
+    grouping when they differ).
 
-    For query row i in sorted block beta = floor(P_Q(i)/b):
+    For query row i in sorted block beta = floor(P_Q(i)/b_q):
       * masked part: the keys j with floor(P_K(j)/b) = beta, exact exp(s_ij)
         (Alg. 2, "row-sum of masked entries"; Sec. 4 block-diagonal product);
       * residual: (N/m) * sum over samples l_t with M^H_{i,l_t} = 0 of exp(s_{i,l_t})
@@ -230,19 +245,20 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     N = K.shape[0]
-    assert Q.shape[0] == N, "the paper pairs the beta-th group of Q with the beta-th group of K"
+    n_q = Q.shape[0]
     if b >= N:
         return exact_attention(Q, K, V, scale, causal=False, rows=rows)
+    b_q = query_block_size(n_q, N, b)
     # N need not be a multiple of b: Alg. 1 line 4 defines the mask through floor(P(i)/b), so the
     # last sorted block simply has N mod b rows of Q and of K (the slices below end at N)
     perm_q, rank_q = stable_argsort(ids_q)
     perm_k, rank_k = stable_argsort(ids_k)
     samples = np.asarray(samples, dtype=np.int64)
     m = samples.size
-    want = np.arange(N) if rows is None else np.asarray(rows, dtype=np.int64)
+    want = np.arange(n_q) if rows is None else np.asarray(rows, dtype=np.int64)
     out = np.zeros((want.size, V.shape[1]), dtype=np.float64)
     lse = np.zeros(want.size, dtype=np.float64)
-    blk_of_want = rank_q[want] // b
+    blk_of_want = rank_q[want] // b_q
     Ks, Vs = K[samples], V[samples]
     blk_of_sample = rank_k[samples] // b
     for beta in np.unique(blk_of_want):
@@ -271,41 +287,60 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
 # --------------------------------------------------------------------------------------
 # Causal masking by recursion (Alg. 4, Fig. 2), carried through to the outputs
 # --------------------------------------------------------------------------------------
-def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, _node=0):
-    """Causal HyperAttention.  If N <= n0: exact causal attention (the paper recurses
-    until the length falls below a base size and uses an exact kernel there).  Else
-    split in equal halves (Alg. 4 line 2); recurse on (Q1,K1,V1) and (Q2,K2,V2)
-    (line 3); run the non-causal algorithm on (Q2,K1,V1) (line 4); rows of the second
-    half add the two row sums, D~_21 + D~_C22 (line 5), and so their outputs combine
-    with weights proportional to the two estimated row sums ("merging attention
-    outputs", Sec. 4.2).  Recursion nodes are numbered like a binary heap
-    (root 0, children 2v+1 and 2v+2) and the off-diagonal problem of node v draws its
-    samples from stream (g, v).
-    """
-    N = Q.shape[0]
-    want = np.arange(N) if rows is None else np.asarray(rows, dtype=np.int64)
-    if N <= n0:
-        return exact_attention(Q, K, V, scale, causal=True, rows=want)
-    assert N % 2 == 0
-    h = N // 2
+def causal_grid(n, n0):
+    """(L, leaf): Alg. 4 halves the sequence until a part is not longer than n0.  L halvings give
+    2^L leaves of leaf = ceil(n / 2^L) rows.  Reading taken when 2^L does not divide n (Alg. 4 line 2
+    only speaks of equal halves): the split points are those of the length rounded up to leaf * 2^L,
+    i.e. every part is cut at half of its nominal length and the rows that the rounded-up length
+    would have beyond n do not exist - the last leaf is short, and so is the query side of the last
+    off-diagonal problem of a level (queries and keys then differ in number, see query_block_size)."""
+    L = 0
+    while -((-n) >> L) > n0:
+        L += 1
+    return L, -((-n) >> L)
+
+
+def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None):
+    """Causal HyperAttention.  A part that is a single leaf gets exact causal attention (the paper
+    recurses until the length falls below a base size and uses an exact kernel there).  A larger
+    part of nominal length S is split at S/2 (Alg. 4 line 2); the two halves recurse (line 3); the
+    non-causal algorithm runs on (Q2, K1, V1) (line 4); rows of the second half add the two row
+    sums, D~_21 + D~_C22 (line 5), and so their outputs combine with weights proportional to the
+    two estimated row sums ("merging attention outputs", Sec. 4.2).  Recursion nodes are numbered
+    like a binary heap (root 0, children 2v+1 and 2v+2) and the off-diagonal problem of node v
+    draws its samples from stream (g, v).  See causal_grid for lengths that the split does not
+    divide."""
+    n = Q.shape[0]
+    L, leaf = causal_grid(n, n0)
+    want = np.arange(n) if rows is None else np.asarray(rows, dtype=np.int64)
     out = np.zeros((want.size, V.shape[1]), dtype=np.float64)
     lse = np.zeros(want.size, dtype=np.float64)
-    first = np.nonzero(want < h)[0]
-    second = np.nonzero(want >= h)[0]
-    if first.size:
-        o, l = causal_forward(Q[:h], K[:h], V[:h], ids_q[:h], ids_k[:h], b, m, scale, n0, seed, g,
-                              rows=want[first], _node=2 * _node + 1)
-        out[first], lse[first] = o, l
-    if second.size:
-        r2 = want[second] - h
-        o22, l22 = causal_forward(Q[h:], K[h:], V[h:], ids_q[h:], ids_k[h:], b, m, scale, n0, seed, g,
-                                  rows=r2, _node=2 * _node + 2)
-        mm = m if b < h else 0
-        smp = sample_indices(seed, g, _node, mm, h)
-        o21, l21 = node_forward(Q[h:], K[:h], V[:h], ids_q[h:], ids_k[:h], smp, b, scale, rows=r2)
-        l = np.logaddexp(l21, l22)
-        out[second] = o21 * np.exp(l21 - l)[:, None] + o22 * np.exp(l22 - l)[:, None]
-        lse[second] = l
+
+    def part(a, S, node, sel):
+        """rows want[sel] (all inside [a, a + S)) of the causal problem on rows [a, min(a + S, n))"""
+        if sel.size == 0:
+            return
+        e = min(a + S, n)
+        if S == leaf:
+            o, l = exact_attention(Q[a:e], K[a:e], V[a:e], scale, causal=True, rows=want[sel] - a)
+            out[sel], lse[sel] = o, l
+            return
+        h = S // 2
+        first = sel[want[sel] < a + h]
+        second = sel[want[sel] >= a + h]
+        part(a, h, 2 * node + 1, first)
+        if second.size:
+            part(a + h, h, 2 * node + 2, second)
+            r2 = want[second] - (a + h)
+            mm = m if b < h else 0
+            smp = sample_indices(seed, g, node, mm, h)
+            o21, l21 = node_forward(Q[a + h:e], K[a:a + h], V[a:a + h], ids_q[a + h:e], ids_k[a:a + h], smp, b, scale, rows=r2)
+            o22, l22 = out[second].copy(), lse[second].copy()
+            l = np.logaddexp(l21, l22)
+            out[second] = o21 * np.exp(l21 - l)[:, None] + o22 * np.exp(l22 - l)[:, None]
+            lse[second] = l
+
+    part(0, leaf << L, 0, np.arange(want.size))
     return out, lse
 
 
@@ -324,6 +359,7 @@ def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None
     compared even when a sign bit at |projection| ~ 0 was decided differently."""
     Q = np.asarray(Q, dtype=np.float64)
     n, d = Q.shape
+    n_k = np.asarray(K).shape[0]
     if scale is None:
         scale = 1.0 / math.sqrt(d)
     if ids_q is None:
@@ -331,14 +367,15 @@ def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None
     if ids_k is None:
         ids_k, _ = bucket_ids(K, W)
     if causal:
+        assert n_k == n, "the causal mask is defined for a square attention matrix"
         return causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=rows)
-    mm = m if b < n else 0
-    smp = sample_indices(seed, g, 0, mm, n)
+    mm = m if b < n_k else 0
+    smp = sample_indices(seed, g, 0, mm, n_k)
     return node_forward(Q, K, V, ids_q, ids_k, smp, b, scale, rows=rows)
 
 
 def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None):
-    """Q, K, V: (G, n, d).  Returns out (G, n, d) and lse (G, n), fp64."""
+    """Q: (G, n, d); K, V: (G, n_k, d).  Returns out (G, n, d) and lse (G, n), fp64."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
@@ -363,70 +400,64 @@ def _dense_unnormalised(Q, K, ids_q, ids_k, samples, b, scale):
         return A
     _, rank_q = stable_argsort(ids_q)
     _, rank_k = stable_argsort(ids_k)
-    M = sortlsh_mask(rank_q, rank_k, b).astype(np.float64)
+    M = sortlsh_mask(rank_q, rank_k, b, query_block_size(np.asarray(Q).shape[0], N, b)).astype(np.float64)
     c = np.bincount(np.asarray(samples, dtype=np.int64), minlength=N).astype(np.float64)
     m = max(len(samples), 1)
     return (M + (N / m) * c[None, :] * (1.0 - M)) * A
 
 
-def dense_weights(Q, K, ids_q, ids_k, b, m, scale, causal, n0, seed, g, _node=0):
-    """Row-normalised n x n weights W~ with out = W~ V; causal problems are assembled
-    quadrant by quadrant exactly as Fig. 2 / Alg. 4 split the matrix."""
-    def unnorm(Q, K, iq, ik, node):
-        N = Q.shape[0]
-        if N <= n0:
-            A = np.exp(scale * (np.asarray(Q, np.float64) @ np.asarray(K, np.float64).T))
-            return np.tril(A)
-        h = N // 2
-        U = np.zeros((N, N))
-        U[:h, :h] = unnorm(Q[:h], K[:h], iq[:h], ik[:h], 2 * node + 1)
-        U[h:, h:] = unnorm(Q[h:], K[h:], iq[h:], ik[h:], 2 * node + 2)
-        mm = m if b < h else 0
-        smp = sample_indices(seed, g, node, mm, h)
-        U[h:, :h] = _dense_unnormalised(Q[h:], K[:h], iq[h:], ik[:h], smp, b, scale)
-        return U
-
-    if causal:
-        U = unnorm(Q, K, ids_q, ids_k, _node)
-    else:
-        N = Q.shape[0]
-        mm = m if b < N else 0
-        U = _dense_unnormalised(Q, K, ids_q, ids_k, sample_indices(seed, g, 0, mm, N), b, scale)
+def dense_weights(Q, K, ids_q, ids_k, b, m, scale, causal, n0, seed, g):
+    """Row-normalised weights W~ (n x n_k) with out = W~ V; causal problems are assembled quadrant by
+    quadrant exactly as Fig. 2 / Alg. 4 split the matrix (causal_grid for the split points)."""
+    C = dense_coefficients(np.asarray(Q).shape[0], ids_q, ids_k, b, m, causal, n0, seed, g, n_k=np.asarray(K).shape[0])
+    U = C * np.exp(scale * (np.asarray(Q, np.float64) @ np.asarray(K, np.float64).T))
     return U / U.sum(axis=1, keepdims=True)
 
 
 # --------------------------------------------------------------------------------------
 # Backward pass (tiny n only): derivative of the forward map, discrete choices held fixed
 # --------------------------------------------------------------------------------------
-def dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g, _node=0):
-    """C (n x n, entries >= 0) such that the forward pass is out = rownorm(C o A) V,
+def dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g, n_k=None):
+    """C (n x n_k, entries >= 0) such that the forward pass is out = rownorm(C o A) V,
     lse = ln rowsum(C o A), A = exp(scale Q K^T).  C depends on Q and K only through the
     bucket ids: C_ij = 1 on the block mask M^H, (N/m) * multiplicity of j among the
     samples elsewhere (Alg. 2 lines 7 and 9 without caps), the lower triangle of ones in
     an exact causal leaf, zero above the diagonal blocks of the recursion (Alg. 4)."""
-    def coeff(N, iq, ik, node):
-        if causal and N <= n0:
-            return np.tril(np.ones((N, N)))
-        if causal:
-            h = N // 2
-            C = np.zeros((N, N))
-            C[:h, :h] = coeff(h, iq[:h], ik[:h], 2 * node + 1)
-            C[h:, h:] = coeff(h, iq[h:], ik[h:], 2 * node + 2)
-            C[h:, :h] = block(h, iq[h:], ik[:h], node)
-            return C
-        return block(N, iq, ik, node)
+    ids_q, ids_k = np.asarray(ids_q), np.asarray(ids_k)
+    n_k = n if n_k is None else n_k
 
-    def block(N, iq, ik, node):
+    def block(iq, ik, node):
+        N = ik.shape[0]
         if b >= N:
-            return np.ones((N, N))
+            return np.ones((iq.shape[0], N))
         _, rank_q = stable_argsort(iq)
         _, rank_k = stable_argsort(ik)
-        M = sortlsh_mask(rank_q, rank_k, b).astype(np.float64)
+        M = sortlsh_mask(rank_q, rank_k, b, query_block_size(iq.shape[0], N, b)).astype(np.float64)
         smp = sample_indices(seed, g, node, m, N)
         c = np.bincount(np.asarray(smp, dtype=np.int64), minlength=N).astype(np.float64)
         return M + (N / max(m, 1)) * c[None, :] * (1.0 - M)
 
-    return coeff(n, np.asarray(ids_q), np.asarray(ids_k), _node)
+    if not causal:
+        return block(ids_q, ids_k, 0)
+    assert n_k == n
+    L, leaf = causal_grid(n, n0)
+    C = np.zeros((n, n))
+
+    def part(a, S, node):
+        e = min(a + S, n)
+        if e <= a:
+            return
+        if S == leaf:
+            C[a:e, a:e] = np.tril(np.ones((e - a, e - a)))
+            return
+        h = S // 2
+        part(a, h, 2 * node + 1)
+        part(a + h, h, 2 * node + 2)
+        if e > a + h:
+            C[a + h:e, a:a + h] = block(ids_q[a + h:e], ids_k[a:a + h], node)
+
+    part(0, leaf << L, 0)
+    return C
 
 
 def dense_backward(Q, K, V, C, scale, d_out, d_lse=None, with_term_sizes=False):

@@ -443,3 +443,133 @@ def test_dense_coefficients_reproduce_dense_weights():
         U = C * np.exp(0.3 * (Q @ K.T))
         Wt = O.dense_weights(Q, K, ids_q, ids_k, b, m, 0.3, causal, n0, seed, g)
         assert np.allclose(U / U.sum(axis=1, keepdims=True), Wt, rtol=1e-12, atol=1e-15)
+
+
+# ------------------------------------------------------------------ unequal sides, lengths the split does not divide
+def brute_node(Q, K, V, iq, ik, smp, b, b_q, scale):
+    """Alg. 2 lines 7 and 9 (no caps) with explicit loops: query i belongs to group floor(P_Q(i)/b_q), key j
+    to group floor(P_K(j)/b); the positions come from Python's stable sort."""
+    n_q, N = Q.shape[0], K.shape[0]
+    order_q = sorted(range(n_q), key=lambda i: (int(iq[i]), i))
+    order_k = sorted(range(N), key=lambda j: (int(ik[j]), j))
+    pos_q = {i: p for p, i in enumerate(order_q)}
+    pos_k = {j: p for p, j in enumerate(order_k)}
+    m = len(smp)
+    out = np.zeros((n_q, V.shape[1]))
+    lse = np.zeros(n_q)
+    for i in range(n_q):
+        beta = pos_q[i] // b_q
+        den, num = 0.0, np.zeros(V.shape[1])
+        for j in range(N):
+            if pos_k[j] // b == beta:
+                a = math.exp(scale * float(Q[i] @ K[j]))
+                den += a
+                num += a * V[j]
+        for l in smp:
+            if pos_k[int(l)] // b != beta:
+                a = (N / m) * math.exp(scale * float(Q[i] @ K[int(l)]))
+                den += a
+                num += a * V[int(l)]
+        out[i] = num / den
+        lse[i] = math.log(den)
+    return out, lse
+
+
+def test_query_block_size_rule():
+    """b_q = ceil(b n_q / n_k): equal sides keep b; the hand-worked case n_q = 5, n_k = 10, b = 4 gives groups
+    of 2 queries against groups of 4 keys; there is never a query group without a key group."""
+    assert O.query_block_size(10, 10, 4) == 4 and O.query_block_size(37, 37, 8) == 8
+    assert O.query_block_size(5, 10, 4) == 2 and O.query_block_size(20, 10, 4) == 8
+    assert O.query_block_size(4095, 4096, 256) == 256            # the causal case: sides that differ by a few rows
+    rng = np.random.default_rng(0)
+    for _ in range(2000):
+        n_q, n_k, b = int(rng.integers(1, 500)), int(rng.integers(2, 500)), int(rng.integers(1, 300))
+        if b >= n_k:
+            continue
+        b_q = O.query_block_size(n_q, n_k, b)
+        assert b_q >= 1 and -(-n_q // b_q) <= -(-n_k // b)
+    # the hand-worked mask: sorted queries 0..4 -> groups 0 0 1 1 2, sorted keys 0..9 -> groups 0 0 0 0 1 1 1 1 2 2
+    M = O.sortlsh_mask(np.arange(5), np.arange(10), 4, 2)
+    want = np.zeros((5, 10), dtype=int)
+    want[0:2, 0:4] = 1; want[2:4, 4:8] = 1; want[4, 8:10] = 1
+    assert (M == want).all()
+
+
+@pytest.mark.parametrize("n_q,n_k,b,m", [(13, 40, 8, 9), (50, 21, 6, 7), (5, 10, 4, 3), (31, 32, 8, 5)])
+def test_unequal_sides_against_explicit_loops(n_q, n_k, b, m):
+    rng = np.random.default_rng(n_q * 100 + n_k)
+    Q = rng.standard_normal((n_q, 4)); K = rng.standard_normal((n_k, 4)); V = rng.standard_normal((n_k, 3))
+    iq = rng.integers(0, 6, n_q).astype(np.uint8); ik = rng.integers(0, 6, n_k).astype(np.uint8)
+    smp = rng.integers(0, n_k, m)
+    out, lse = O.node_forward(Q, K, V, iq, ik, smp, b, 0.5)
+    bo, bl = brute_node(Q, K, V, iq, ik, smp, b, -(-b * n_q // n_k), 0.5)
+    np.testing.assert_allclose(out, bo, atol=1e-12)
+    np.testing.assert_allclose(lse, bl, atol=1e-12)
+    # a subset of rows gives the same rows
+    rows = np.array(sorted(rng.choice(n_q, size=min(4, n_q), replace=False)))
+    o2, l2 = O.node_forward(Q, K, V, iq, ik, smp, b, 0.5, rows=rows)
+    np.testing.assert_allclose(o2, out[rows], atol=1e-14)
+    np.testing.assert_allclose(l2, lse[rows], atol=1e-14)
+
+
+@pytest.mark.parametrize("n_q,n_k,b", [(13, 40, 8), (50, 21, 6)])
+def test_unequal_sides_full_coverage_is_exact_and_dense_form_is_row_stochastic(n_q, n_k, b):
+    rng = np.random.default_rng(n_q + n_k)
+    Q = rng.standard_normal((n_q, 5)); K = rng.standard_normal((n_k, 5)); V = rng.standard_normal((n_k, 4))
+    W = O.directions(5, 3, 9)
+    iq, _ = O.bucket_ids(Q, W); ik, _ = O.bucket_ids(K, W)
+    out, lse = O.node_forward(Q, K, V, iq, ik, rng.permutation(n_k), b, 0.4)      # every key sampled once
+    bo, bl = brute_attention(Q, K, V, 0.4, False)
+    np.testing.assert_allclose(out, bo, atol=1e-12)
+    np.testing.assert_allclose(lse, bl, atol=1e-12)
+    # the whole forward with its own samples: the implied weights are row-stochastic and give the output
+    o, l = O.segment_forward(Q, K, V, W, b, 7, False, 0, 3, 2, scale=0.4)
+    Wd = O.dense_weights(Q, K, iq, ik, b, 7, 0.4, False, 0, 3, 2)
+    assert Wd.shape == (n_q, n_k)
+    np.testing.assert_allclose(Wd.sum(axis=1), 1.0, atol=1e-12)
+    np.testing.assert_allclose(Wd @ V, o, atol=1e-12)
+
+
+def test_causal_grid():
+    assert O.causal_grid(131072, 4096) == (5, 4096) and O.causal_grid(4096, 4096) == (0, 4096)
+    assert O.causal_grid(6000, 1000) == (3, 750) and O.causal_grid(100003, 4096) == (5, 3126)
+    assert O.causal_grid(5, 2) == (2, 2) and O.causal_grid(7, 1) == (3, 1)
+
+
+@pytest.mark.parametrize("n,n0", [(33, 4), (47, 6), (101, 9), (5, 2), (7, 1), (100, 7), (19, 32)])
+def test_causal_lengths_the_split_does_not_divide_single_block_nodes_are_exact(n, n0):
+    """Any n: with b at least the largest off-diagonal problem every node is one block, and the recursion
+    over a short last leaf and short last nodes must still add up to exact causal attention."""
+    rng = np.random.default_rng(n * 7 + n0)
+    Q, K, V = (x[None] for x in rand_qkv(rng, n, 3))
+    bo, bl = brute_attention(Q[0], K[0], V[0], 0.6, True)
+    out, lse = O.forward(Q, K, V, b=n, m=8, r=4, causal=True, n0=n0, seed=1, scale=0.6)
+    np.testing.assert_allclose(out[0], bo, atol=1e-11)
+    np.testing.assert_allclose(lse[0], bl, atol=1e-11)
+
+
+@pytest.mark.parametrize("n,n0,b,m", [(45, 6, 4, 5), (101, 13, 5, 6), (37, 5, 3, 4)])
+def test_causal_odd_lengths_dense_form_and_rebuilt_last_node(n, n0, b, m):
+    """Sorted nodes with a short last node: the implied weights are row-stochastic, lower triangular and give the
+    output; the rows of the last (short) root-level node are rebuilt by hand from node_forward and the
+    recursion on the second part."""
+    rng = np.random.default_rng(n)
+    Q, K, V = rand_qkv(rng, n, 4)
+    W = O.directions(4, 3, 5)
+    iq, _ = O.bucket_ids(Q, W); ik, _ = O.bucket_ids(K, W)
+    out, lse = O.segment_forward(Q, K, V, W, b, m, True, n0, 11, 1, scale=0.7)
+    Wd = O.dense_weights(Q, K, iq, ik, b, m, 0.7, True, n0, 11, 1)
+    np.testing.assert_allclose(Wd.sum(axis=1), 1.0, atol=1e-12)
+    assert np.abs(np.triu(Wd, 1)).max() == 0.0
+    np.testing.assert_allclose(Wd @ V, out, atol=1e-12)
+    L, leaf = O.causal_grid(n, n0)
+    h = (leaf << L) // 2                                          # the root splits at half of the rounded-up length
+    assert h < n < 2 * h or n == 2 * h
+    smp = O.sample_indices(11, 1, 0, m if b < h else 0, h)
+    o21, l21 = O.node_forward(Q[h:], K[:h], V[:h], iq[h:], ik[:h], smp, b, 0.7)
+    # total row sum of a second-part row = its off-diagonal estimate + everything the recursion gives it inside the second part
+    inside = np.log(np.exp(lse[h:]) - np.exp(l21))
+    C = O.dense_coefficients(n, iq, ik, b, m, True, n0, 11, 1)
+    A = np.exp(0.7 * (Q @ K.T))
+    np.testing.assert_allclose(np.log((C * A)[h:, h:].sum(axis=1)), inside, atol=1e-9)
+    np.testing.assert_allclose(np.log((C * A)[h:, :h].sum(axis=1)), l21, atol=1e-12)
