@@ -34,12 +34,16 @@
  *     block need not divide n (or a recursion node's size): the mask of Alg. 1 line 4 is
  *     floor(P(i) / block), so the last sorted block is short; block >= n makes the problem one
  *     exact block.  Causal: Alg. 4 halves the rows until a part is not longer than n0 (L
- *     halvings, 2^L exact causal leaves of n / 2^L rows; L = 0 if n <= n0); the halves are
- *     equal, so 2^L must divide n (n = n0 * 2^L is the common case; n = 100000 with
- *     n0 = 4096 has 32 leaves of 3125 rows).
+ *     halvings, 2^L exact causal leaves of leaf = ceil(n / 2^L) rows; L = 0 if n <= n0).  Any n
+ *     is accepted: every part is cut at half of its nominal length leaf * 2^k, and when 2^L
+ *     does not divide n the rows beyond n simply do not exist, so the last leaf is short and
+ *     the last off-diagonal problem of a level has fewer queries than keys (it is then grouped
+ *     like a call with n != n_k, see hyperattn_params.n_k).  n = 100003 with n0 = 4096 has 32
+ *     leaves of 3126 rows, the last one of 3097.
  *   - Recursion nodes are numbered like a binary heap: the off-diagonal problem of the
  *     j-th node of level l (root level 0) is node (2^l - 1) + j; it pairs query rows
- *     [(2j+1)s, (2j+2)s) with key rows [2js, (2j+1)s), s = n / 2^(l+1).  A non-causal
+ *     [(2j+1)s, (2j+2)s) with key rows [2js, (2j+1)s), s = leaf * 2^(L-1-l)
+ *     (= n / 2^(l+1) when 2^L divides n; query rows beyond n do not exist).  A non-causal
  *     call has the single node 0 over all rows.
  *   - Random numbers: Philox4x32-10 keyed by `seed`; directions use counter
  *     (c, 0, 0, 1), samples of (segment g, node v) use counter (j >> 2, g, v, 2),
@@ -73,9 +77,11 @@ typedef enum hyperattn_dtype {
 /* Optional device buffers that receive the intermediate results of the integer stages
  * (needed to compare them bit for bit with a reference).  Any member may be NULL.
  * Let G = B*H, LV = number of levels (1 if non-causal or n <= n0, else L),
- * NL = rows per (level, segment, side): n if non-causal, n/2 if causal with L >= 1,
+ * NL = rows per (level, segment, side): max(n, n_k) if non-causal, leaf * 2^(L-1) if causal with
+ * L >= 1 (n/2 when 2^L divides n; entries of rows that do not exist are left untouched),
  * NODES = 1 if non-causal, 2^L - 1 if causal (0 if n <= n0).
- *   q_ids, k_ids : uint8 [G, n]        bucket id of every row (Def. 1)
+ *   q_ids        : uint8 [G, n]        bucket id of every query row (Def. 1)
+ *   k_ids        : uint8 [G, n_k]      bucket id of every key row
  *   perm_q,perm_k: int32 [LV, G, NL]   node j of level l occupies [j*s, (j+1)*s);
  *                                      entry p = row (relative to the node's first query /
  *                                      key row) placed at sorted position p (Alg. 1 line 3)
@@ -122,6 +128,13 @@ typedef struct hyperattn_params {
                             output entry can be off by 2^-8 max|v|, which is 2e-2 for values of N(0,1) size
                             but more for heavy-tailed values; this mode keeps the error below 2e-2 for values
                             up to +-20 at the price of twice the weights-times-values products.  bf16 inputs only. */
+  int n_k;               /* rows of k and v per (batch, head): k, v are [B, H, n_k, d]; 0 means n.  Non-causal
+                            calls only (the causal mask is defined for a square matrix).  Alg. 1 line 4 pairs the
+                            beta-th group of sorted queries with the beta-th group of sorted keys and is written
+                            for n = n_k; with n != n_k the key groups keep `block` rows and the query groups get
+                            ceil(block * n / n_k) rows, so that a group of either side covers the same fraction of
+                            its sorted order (every query group has a key group).  The samples are drawn from the
+                            n_k keys and weigh n_k / samples. */
 } hyperattn_params;
 
 /* HyperAttention forward (Alg. 1-4 as specialised in Sec. 4) with bf16 inputs and

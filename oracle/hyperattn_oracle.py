@@ -21,6 +21,7 @@ r hash bits; P_Q, P_K the sortLSH permutations; M^H the block mask):
   query_block_size   rows per group of sorted queries when queries and keys differ in number
   causal_grid        leaves and levels of the recursive split for any sequence length
   sample_indices     l_1..l_m ~ Unif([N]) shared by all rows (Alg. 2 line 4, Sec. 4)
+  row_subset         the rows T of Alg. 2 line 2 (capped variant only)
   exact_attention    D^-1 A V and its causal form (Sec. 1.1, Sec. 3.1)
   node_forward       block-diagonal part + sampled residual with estimated D
                      (Alg. 2 lines 7 and 9 without caps, Alg. 3, Sec. 4)
@@ -57,6 +58,7 @@ _SHIFT32 = np.uint64(32)
 
 DOMAIN_DIRECTIONS = 1
 DOMAIN_SAMPLES = 2
+DOMAIN_ROW_SUBSET = 3
 
 
 def philox4x32_10(counter, key):
@@ -131,6 +133,23 @@ def sample_indices(seed, g, node, m, N):
     ctr[:, 3] = DOMAIN_SAMPLES
     x = philox4x32_10(ctr, _seed_key(seed)).reshape(-1)[:m].astype(np.uint64)
     return ((x * np.uint64(N)) >> _SHIFT32).astype(np.int64)
+
+
+def row_subset(seed, g, node, m, n_q):
+    """The rows T over which Alg. 2 line 3 takes the maximum unmasked row sum (line 2: "randomly
+    choose a subset T of [n] with |T| = m").  Reading taken: m i.i.d. uniform row indices (a maximum
+    does not care about repeats), drawn like the sampled columns but from their own stream:
+    counter (j >> 2, g, node, 3), word j & 3, index floor(x * n_q / 2^32)."""
+    if m == 0 or n_q == 0:
+        return np.zeros(0, dtype=np.int64)
+    calls = (m + 3) // 4
+    ctr = np.zeros((calls, 4), dtype=np.uint64)
+    ctr[:, 0] = np.arange(calls, dtype=np.uint64)
+    ctr[:, 1] = g
+    ctr[:, 2] = node
+    ctr[:, 3] = DOMAIN_ROW_SUBSET
+    x = philox4x32_10(ctr, _seed_key(seed)).reshape(-1)[:m].astype(np.uint64)
+    return ((x * np.uint64(n_q)) >> _SHIFT32).astype(np.int64)
 
 
 # --------------------------------------------------------------------------------------
@@ -224,7 +243,21 @@ def exact_attention(Q, K, V, scale, causal=False, rows=None):
 # --------------------------------------------------------------------------------------
 # One non-causal HyperAttention problem (Alg. 1-3 as specialised in Sec. 4)
 # --------------------------------------------------------------------------------------
-def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
+def unmasked_row_sum_bound(Q, K, rank_q, rank_k, T, b, b_q, scale):
+    """ln tau of Alg. 2 line 3: tau = max over j in T of <1 - M^H_j, exp(K q_j)>, the largest
+    row sum of the entries outside the mask among the rows of T (minus infinity if T is empty or
+    every row of T has all its keys inside its block)."""
+    ltau = -np.inf
+    for j in np.asarray(T, dtype=np.int64):
+        s = scale * (K @ Q[j])
+        s = s[(rank_k // b) != (rank_q[j] // b_q)]
+        if s.size:
+            mx = s.max()
+            ltau = max(ltau, mx + math.log(np.exp(s - mx).sum()))
+    return ltau
+
+
+def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None):
     """HyperAttention on n_q queries x N keys (n_q = N in the paper; see query_block_size for the
     grouping when they differ).
 
@@ -240,6 +273,16 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
     out_i = numerator_i / d~_i, lse_i = ln d~_i.  If b >= N the whole problem is one
     block and nothing is sampled.  Returns (out, lse) for `rows` (default all rows),
     in original row order.
+
+    caps = (cap_scale, kappa, T) switches on the caps of Alg. 2 (lines 3, 6, 7 and 9 as printed):
+      tau   = max_{j in T} <1 - M^H_j, exp(K q_j)>                                  (line 3)
+      C_i   = cap_scale * m / (N ln N) * (masked_i + tau / kappa)                   (line 6; the paper
+              writes Theta(eps^2 m / (n log n) (...)): the constant times eps^2 is the caller's cap_scale)
+      d_i   = (N/m) sum_t (1 - M^H_{i,l_t}) min(exp(s_{i,l_t}), C_i)                (line 7)
+      d~_i  = masked_i + max(d_i, tau / kappa)                                      (line 9)
+    The numerator is unchanged (Alg. 3 multiplies D~^-1 by the sampled product A V; the caps belong
+    to the row-sum estimate of Alg. 2 only), so with caps the outputs are no longer convex
+    combinations of value rows.  cap_scale = inf and kappa = inf switch both caps off.
     """
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
@@ -261,6 +304,11 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
     blk_of_want = rank_q[want] // b_q
     Ks, Vs = K[samples], V[samples]
     blk_of_sample = rank_k[samples] // b
+    capped = caps is not None and m > 0
+    if capped:
+        cap_scale, kappa, T = caps
+        lfloor = unmasked_row_sum_bound(Q, K, rank_q, rank_k, T, b, b_q, scale) - math.log(kappa)   # ln(tau / kappa)
+        coef = cap_scale * m / (N * math.log(N))
     for beta in np.unique(blk_of_want):
         sel = np.nonzero(blk_of_want == beta)[0]
         qi = want[sel]
@@ -272,13 +320,21 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None):
             s_smp = scale * (Q[qi] @ Ks.T)
             if keep.any():
                 mx = np.maximum(mx, s_smp[:, keep > 0].max(axis=1, keepdims=True))
+            if capped and lfloor > -np.inf:
+                mx = np.maximum(mx, lfloor)
             w = (N / m) * keep[None, :] * np.exp(np.where(keep[None, :] > 0, s_smp - mx, -np.inf))
         a = np.exp(s_blk - mx)
         den = a.sum(axis=1, keepdims=True)
         num = a @ V[J]
         if m > 0:
-            den = den + w.sum(axis=1, keepdims=True)
             num = num + w @ Vs
+            # Alg. 2 line 7: d_i = (N/m) sum_t (1 - M) min(exp(s), C_i); line 9: d~_i = masked + max(d_i, tau / kappa)
+            # (without caps C_i is infinite and tau / kappa is zero)
+            floor = np.exp(lfloor - mx) if capped else 0.0               # tau / kappa in units of exp(mx)
+            cap = coef * (den + floor) if capped else np.inf             # C_i
+            p = np.exp(np.where(keep[None, :] > 0, s_smp - mx, -np.inf))
+            d_i = (N / m) * (keep[None, :] * np.minimum(p, cap)).sum(axis=1, keepdims=True)
+            den = den + np.maximum(d_i, floor)
         out[sel] = num / den
         lse[sel] = (mx + np.log(den))[:, 0]
     return out, lse
@@ -300,7 +356,7 @@ def causal_grid(n, n0):
     return L, -((-n) >> L)
 
 
-def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None):
+def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, caps=None):
     """Causal HyperAttention.  A part that is a single leaf gets exact causal attention (the paper
     recurses until the length falls below a base size and uses an exact kernel there).  A larger
     part of nominal length S is split at S/2 (Alg. 4 line 2); the two halves recurse (line 3); the
@@ -334,7 +390,8 @@ def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None):
             r2 = want[second] - (a + h)
             mm = m if b < h else 0
             smp = sample_indices(seed, g, node, mm, h)
-            o21, l21 = node_forward(Q[a + h:e], K[a:a + h], V[a:a + h], ids_q[a + h:e], ids_k[a:a + h], smp, b, scale, rows=r2)
+            nc = None if caps is None else (caps[0], caps[1], row_subset(seed, g, node, mm, e - (a + h)))
+            o21, l21 = node_forward(Q[a + h:e], K[a:a + h], V[a:a + h], ids_q[a + h:e], ids_k[a:a + h], smp, b, scale, rows=r2, caps=nc)
             o22, l22 = out[second].copy(), lse[second].copy()
             l = np.logaddexp(l21, l22)
             out[second] = o21 * np.exp(l21 - l)[:, None] + o22 * np.exp(l22 - l)[:, None]
@@ -353,10 +410,12 @@ def heap_node(level, j):
 # Whole forward pass
 # --------------------------------------------------------------------------------------
 def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None,
-                    ids_q=None, ids_k=None):
+                    ids_q=None, ids_k=None, caps=None):
     """Forward pass of one (batch, head) segment.  `ids_q` / `ids_k` may be injected
     (e.g. the bucket ids another implementation produced) so that later stages can be
-    compared even when a sign bit at |projection| ~ 0 was decided differently."""
+    compared even when a sign bit at |projection| ~ 0 was decided differently.
+    caps = (cap_scale, kappa) runs Alg. 2 with its caps (see node_forward); every off-diagonal
+    problem then draws its own row subset T."""
     Q = np.asarray(Q, dtype=np.float64)
     n, d = Q.shape
     n_k = np.asarray(K).shape[0]
@@ -368,13 +427,14 @@ def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None
         ids_k, _ = bucket_ids(K, W)
     if causal:
         assert n_k == n, "the causal mask is defined for a square attention matrix"
-        return causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=rows)
+        return causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=rows, caps=caps)
     mm = m if b < n_k else 0
     smp = sample_indices(seed, g, 0, mm, n_k)
-    return node_forward(Q, K, V, ids_q, ids_k, smp, b, scale, rows=rows)
+    nc = None if caps is None else (caps[0], caps[1], row_subset(seed, g, 0, mm, n))
+    return node_forward(Q, K, V, ids_q, ids_k, smp, b, scale, rows=rows, caps=nc)
 
 
-def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None):
+def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None, caps=None):
     """Q: (G, n, d); K, V: (G, n_k, d).  Returns out (G, n, d) and lse (G, n), fp64."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
@@ -384,7 +444,7 @@ def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None):
     out = np.zeros((G, n, d), dtype=np.float64)
     lse = np.zeros((G, n), dtype=np.float64)
     for g in range(G):
-        out[g], lse[g] = segment_forward(Q[g], K[g], V[g], W, b, m, causal, n0, seed, g, scale)
+        out[g], lse[g] = segment_forward(Q[g], K[g], V[g], W, b, m, causal, n0, seed, g, scale, caps=caps)
     return out, lse
 
 

@@ -38,7 +38,7 @@ class _Params(C.Structure):
                 ("n0", C.c_int), ("seed", C.c_uint64), ("dtype", C.c_int), ("out_dtype", C.c_int),
                 ("softmax_scale", C.c_float), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("debug", C.POINTER(_Debug)), ("stream", C.c_void_p),
-                ("precise", C.c_int)]
+                ("precise", C.c_int), ("n_k", C.c_int)]
 
 
 class _StageTimes(C.Structure):
@@ -91,25 +91,28 @@ def _dtype_code(t: torch.dtype) -> int:
     raise HyperAttnError(f"unsupported dtype {t}")
 
 
-def _fill(p: _Params, B, H, n, d, block, samples, hash_bits, causal, n0, seed, dtype, out_dtype, scale):
+def _fill(p: _Params, B, H, n, d, block, samples, hash_bits, causal, n0, seed, dtype, out_dtype, scale, n_k=0):
     p.B, p.H, p.n, p.d = B, H, n, d
+    p.n_k = 0 if n_k == n else n_k
     p.block, p.samples, p.hash_bits, p.causal, p.n0 = block, samples, hash_bits, int(bool(causal)), n0
     p.seed = seed
     p.dtype, p.out_dtype, p.softmax_scale = dtype, out_dtype, float(scale)
 
 
-def _debug_shapes(B, H, n, block, samples, causal, n0):
+def _debug_shapes(B, H, n, block, samples, causal, n0, n_k=None):
     """Shapes of the exported intermediates (see hyperattn_debug in the header)."""
     G = B * H
+    n_k = n if n_k is None else n_k
     if not causal:
-        LV, NL, NODES = 1, n, 1
+        LV, NL, NODES = 1, max(n, n_k), 1
     elif n <= n0:
         LV, NL, NODES = 1, n, 0
     else:
         L = 0
-        while (n >> L) > n0:                      # Alg. 4: halve until a part is not longer than n0
+        while -((-n) >> L) > n0:                  # Alg. 4: halve until a part is not longer than n0
             L += 1
-        LV, NL, NODES = L, n // 2, (1 << L) - 1
+        leaf = -((-n) >> L)
+        LV, NL, NODES = L, (leaf << L) // 2, (1 << L) - 1
     return G, LV, NL, NODES
 
 
@@ -121,11 +124,14 @@ def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_
         raise HyperAttnError("q, k, v must be CUDA tensors (there is no CPU path)")
     q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
     B, H, n, d = q.shape
+    n_k = k.shape[2]
+    if k.shape != (B, H, n_k, d) or v.shape != k.shape:
+        raise HyperAttnError("k and v must be [B, H, n_k, d] with the batch, heads and d of q")
     out_dtype = out_dtype or q.dtype
     out = torch.empty((B, H, n, d), dtype=out_dtype, device=q.device)
     lse = torch.empty((B, H, n), dtype=torch.float32, device=q.device)
     p = _Params()
-    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, seed, _dtype_code(q.dtype), _dtype_code(out_dtype), scale)
+    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, seed, _dtype_code(q.dtype), _dtype_code(out_dtype), scale, n_k)
     p.q, p.k, p.v, p.out, p.lse = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr()
     if workspace is not None:
         p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
@@ -133,11 +139,11 @@ def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_
     p.precise = int(bool(precise))
     inter = None
     if debug:
-        G, LV, NL, NODES = _debug_shapes(B, H, n, block, samples, causal, n0)
+        G, LV, NL, NODES = _debug_shapes(B, H, n, block, samples, causal, n0, n_k)
         dev = q.device
         inter = {
             "q_ids": torch.zeros((G, n), dtype=torch.uint8, device=dev),
-            "k_ids": torch.zeros((G, n), dtype=torch.uint8, device=dev),
+            "k_ids": torch.zeros((G, n_k), dtype=torch.uint8, device=dev),
             "perm_q": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
             "perm_k": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
             "rank_k": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
@@ -180,7 +186,7 @@ def forward_host(q, k, v, out, lse, block, samples, hash_bits, causal=False, n0=
     Enqueues H2D copies, the forward pass and D2H copies on the stream; the caller synchronises."""
     B, H, n, d = q.shape
     p = _Params()
-    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, seed, _dtype_code(q.dtype), _dtype_code(out.dtype), scale)
+    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, seed, _dtype_code(q.dtype), _dtype_code(out.dtype), scale, k.shape[2])
     p.q, p.k, p.v, p.out, p.lse = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr()
     p.stream = stream if stream is not None else torch.cuda.current_stream().cuda_stream
     _check(lib().hyperattn_forward_host(C.byref(p)), "hyperattn_forward_host")
@@ -208,9 +214,9 @@ def sortlsh_noalloc(x, hash_bits, seed=0, stream=None):
     return ids, perm, rank
 
 
-def workspace_bytes(B, H, n, d, block, samples, hash_bits, causal=False, n0=0, dtype=BF16, out_dtype=BF16) -> int:
+def workspace_bytes(B, H, n, d, block, samples, hash_bits, causal=False, n0=0, dtype=BF16, out_dtype=BF16, n_k=0) -> int:
     p = _Params()
-    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, 0, dtype, out_dtype, 0.0)
+    _fill(p, B, H, n, d, block, samples, hash_bits, causal, n0, 0, dtype, out_dtype, 0.0, n_k or n)
     nbytes = C.c_size_t(0)
     _check(lib().hyperattn_workspace_bytes(C.byref(p), C.byref(nbytes)), "hyperattn_workspace_bytes")
     return int(nbytes.value)

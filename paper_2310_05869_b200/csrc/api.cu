@@ -28,36 +28,46 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // ---- geometry / validation ---------------------------------------------------------------
 int build_geometry(const hyperattn_params& p, Geometry& g) {
-  if (p.B <= 0 || p.H <= 0 || p.n <= 0 || p.block <= 0 || p.samples < 0) return HYPERATTN_INVALID_ARGUMENT;
+  if (p.B <= 0 || p.H <= 0 || p.n <= 0 || p.block <= 0 || p.samples < 0 || p.n_k < 0) return HYPERATTN_INVALID_ARGUMENT;
   if (p.dtype != HYPERATTN_BF16 && p.dtype != HYPERATTN_FP32) return HYPERATTN_INVALID_ARGUMENT;
   if (p.out_dtype != HYPERATTN_BF16 && p.out_dtype != HYPERATTN_FP32) return HYPERATTN_INVALID_ARGUMENT;
   if (p.d != 64 && p.d != 128) return HYPERATTN_UNSUPPORTED_SHAPE;
   if (p.hash_bits < 1 || p.hash_bits > 8) return HYPERATTN_UNSUPPORTED_SHAPE;
   if ((long long)p.B * p.H > (1 << 20)) return HYPERATTN_UNSUPPORTED_SHAPE;
-  if (p.n > (1 << 28)) return HYPERATTN_UNSUPPORTED_SHAPE;
+  if (p.n > (1 << 28) || p.n_k > (1 << 28)) return HYPERATTN_UNSUPPORTED_SHAPE;
+  const int nk = p.n_k ? p.n_k : p.n;
+  if (p.causal && nk != p.n) return HYPERATTN_UNSUPPORTED_SHAPE;       // the causal mask is defined for a square matrix
   std::memset(&g, 0, sizeof(g));
   g.seg0 = 0;
-  g.G = p.B * p.H; g.n = p.n; g.d = p.d; g.b = p.block; g.m = p.samples; g.r = p.hash_bits;
+  g.G = p.B * p.H; g.n = p.n; g.nk = nk; g.npad = p.n; g.d = p.d; g.b = p.block; g.m = p.samples; g.r = p.hash_bits;
+  g.bq = p.block;
   if (!p.causal) {
-    g.causal = 0; g.L = 0; g.leaf = p.n; g.unit = p.n;
-    if (p.block < p.n) {
-      g.levels = 1; g.nl = p.n; g.nodes = 1; g.sorted = 1;
+    g.causal = 0; g.L = 0; g.leaf = p.n; g.unit = p.n; g.unit_k = nk;
+    g.nl = p.n > nk ? p.n : nk;
+    if (p.block < nk) {
+      g.levels = 1; g.nodes = 1; g.sorted = 1;
+      g.bq = query_group(p.block, p.n, nk);
     }
   } else {
     if (p.n0 <= 0) return HYPERATTN_INVALID_ARGUMENT;
     g.causal = 1;
-    // Alg. 4 halves the problem until it is not longer than n0: L levels, 2^L equal leaves of
-    // n / 2^L rows (n0 itself when n = n0 2^L); the halves must be equal, so 2^L must divide n
+    // Alg. 4 halves the problem until a part is not longer than n0: L levels, 2^L leaves of
+    // leaf = ceil(n / 2^L) rows.  The recursion cuts every part at half of its nominal length
+    // leaf 2^k; when 2^L does not divide n the rows beyond n do not exist, so the last leaf and
+    // the query side of a level's last node are short.
     int L = 0;
-    while (((long long)p.n >> L) > p.n0 && L <= kMaxLevels) ++L;
-    if (L > kMaxLevels || (p.n & ((1 << L) - 1)) != 0) return HYPERATTN_UNSUPPORTED_SHAPE;
+    while ((((long long)p.n + (1ll << L) - 1) >> L) > p.n0 && L <= kMaxLevels) ++L;
+    if (L > kMaxLevels) return HYPERATTN_UNSUPPORTED_SHAPE;
     g.L = L;
-    g.leaf = p.n >> L;
-    g.unit = g.leaf;
+    g.leaf = (int)(((long long)p.n + (1ll << L) - 1) >> L);
+    if (((long long)g.leaf << L) > (1ll << 29)) return HYPERATTN_UNSUPPORTED_SHAPE;
+    g.npad = g.leaf << L;
+    g.unit = g.leaf; g.unit_k = g.leaf;
+    g.nl = p.n;
     if (L) {
-      g.levels = L; g.nl = p.n / 2; g.nodes = (1 << L) - 1;
+      g.levels = L; g.nl = g.npad / 2; g.nodes = (1 << L) - 1;
       for (int l = 0; l < L; ++l) {
-        const int s = p.n >> (l + 1);
+        const int s = g.npad >> (l + 1);
         if (p.block < s) g.sorted = 1;
       }
     }
@@ -67,7 +77,9 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
     if (2 * bpad + mpad > kMaxNodeKeys) return HYPERATTN_UNSUPPORTED_SHAPE;
   }
   g.chunks_per_unit = (g.unit + kSortChunk - 1) / kSortChunk;
-  g.chunks_per_seg = (g.n / g.unit) * g.chunks_per_unit;
+  g.chunks_per_seg = (g.npad / g.unit) * g.chunks_per_unit;
+  g.chunks_per_unit_k = (g.unit_k + kSortChunk - 1) / kSortChunk;
+  g.chunks_per_seg_k = g.causal ? g.chunks_per_seg : g.chunks_per_unit_k;
   return HYPERATTN_OK;
 }
 
@@ -81,17 +93,17 @@ Plan make_plan(const Geometry& g, int is_fp32, int backward = 0) {
   Plan pl;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
-  const size_t tensor16 = (size_t)g.G * g.n * g.d * 2;
+  const size_t tensor16 = (size_t)g.G * g.n * g.d * 2, tensor16k = (size_t)g.G * g.nk * g.d * 2;
   pl.q16 = take(is_fp32 ? tensor16 : 0);
-  pl.k16 = take(is_fp32 ? tensor16 : 0);
-  pl.v16 = take(is_fp32 ? tensor16 : 0);
+  pl.k16 = take(is_fp32 ? tensor16k : 0);
+  pl.v16 = take(is_fp32 ? tensor16k : 0);
   pl.q16lo = take(is_fp32 ? tensor16 : 0);
-  pl.k16lo = take(is_fp32 ? tensor16 : 0);
+  pl.k16lo = take(is_fp32 ? tensor16k : 0);
   const size_t lvl_rows = (size_t)g.levels * g.G * g.nl;
-  pl.ids = take(g.sorted ? (size_t)2 * g.G * g.n : 0);
-  pl.hist = take(g.sorted ? (size_t)2 * g.G * g.chunks_per_seg * kBuckets * 4 : 0);
-  const size_t chunks_per_level = g.sorted ? (size_t)(g.nl / g.unit) * g.chunks_per_unit : 0;
-  pl.offs = take((size_t)2 * g.levels * g.G * chunks_per_level * kBuckets * 4);
+  pl.ids = take(g.sorted ? (size_t)g.G * ((size_t)g.n + g.nk) : 0);
+  pl.hist = take(g.sorted ? (size_t)g.G * (g.chunks_per_seg + g.chunks_per_seg_k) * kBuckets * 4 : 0);
+  const size_t chunks_per_level = g.sorted ? (size_t)side_cpl(g, 0) + side_cpl(g, 1) : 0;
+  pl.offs = take((size_t)g.levels * g.G * chunks_per_level * kBuckets * 4);
   pl.perm_q = take(g.sorted ? lvl_rows * 4 : 0);
   pl.perm_k = take(g.sorted ? lvl_rows * 4 : 0);
   pl.rank_k = take(g.sorted ? lvl_rows * 4 : 0);
@@ -185,6 +197,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   const int out_fp32 = p.out_dtype == HYPERATTN_FP32;
   if (bw) {
     if (is_fp32) return HYPERATTN_UNSUPPORTED_SHAPE;                 // the backward pass takes bf16 inputs
+    if (g.nk != g.n || g.npad != g.n) return HYPERATTN_UNSUPPORTED_SHAPE;   // equal sides and causal lengths that 2^L divides only
     if (!bw->dout || !bw->dq || !bw->dk || !bw->dv) return HYPERATTN_INVALID_ARGUMENT;
     if (bw->grad_dtype != HYPERATTN_BF16 && bw->grad_dtype != HYPERATTN_FP32) return HYPERATTN_INVALID_ARGUMENT;
     for (const void* x : {bw->dout, (const void*)bw->dq, (const void*)bw->dk, (const void*)bw->dv})
@@ -244,10 +257,10 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
                       *v16 = reinterpret_cast<const __nv_bfloat16*>(p.v);
   if (is_fp32) {
     StageScope sc(st, HYPERATTN_STAGE_CONVERT, 3);
-    const size_t cnt = (size_t)g.G * g.n * g.d;
+    const size_t cnt = (size_t)g.G * g.n * g.d, cnt_k = (size_t)g.G * g.nk * g.d;
     HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.q), ws.q16, ws.q16lo, cnt, st));
-    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.k), ws.k16, ws.k16lo, cnt, st));
-    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.v), ws.v16, nullptr, cnt, st));
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.k), ws.k16, ws.k16lo, cnt_k, st));
+    HA_CHECK(launch_convert(reinterpret_cast<const float*>(p.v), ws.v16, nullptr, cnt_k, st));
     q16 = ws.q16; k16 = ws.k16; v16 = ws.v16;
   }
   if (g.sorted) {
@@ -271,7 +284,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     if (dbg) {
       const size_t lvl_bytes = (size_t)g.levels * g.G * g.nl * 4;
       if (dbg->q_ids) HA_CHECK(cudaMemcpyAsync(dbg->q_ids, ws.ids, (size_t)g.G * g.n, cudaMemcpyDeviceToDevice, st));
-      if (dbg->k_ids) HA_CHECK(cudaMemcpyAsync(dbg->k_ids, ws.ids + (size_t)g.G * g.n, (size_t)g.G * g.n, cudaMemcpyDeviceToDevice, st));
+      if (dbg->k_ids) HA_CHECK(cudaMemcpyAsync(dbg->k_ids, ws.ids + (size_t)g.G * g.n, (size_t)g.G * g.nk, cudaMemcpyDeviceToDevice, st));
       if (dbg->perm_q) HA_CHECK(cudaMemcpyAsync(dbg->perm_q, ws.perm_q, lvl_bytes, cudaMemcpyDeviceToDevice, st));
       if (dbg->perm_k) HA_CHECK(cudaMemcpyAsync(dbg->perm_k, ws.perm_k, lvl_bytes, cudaMemcpyDeviceToDevice, st));
       if (dbg->rank_k) HA_CHECK(cudaMemcpyAsync(dbg->rank_k, ws.rank_k, lvl_bytes, cudaMemcpyDeviceToDevice, st));
@@ -292,11 +305,11 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   a.precise = p.precise != 0;
   a.direct = g.L == 0;
   a.dense_causal = g.causal;
-  a.tiles_per_block = (g.b + kTileQ - 1) / kTileQ;
+  a.tiles_per_block = (g.bq + kTileQ - 1) / kTileQ;
   const bool has_leaves = g.causal || !g.sorted;
   if (has_leaves) {
     a.tiles_per_leaf = (g.leaf + kTileQ - 1) / kTileQ;
-    a.leaves_per_seg = g.n / g.leaf;
+    a.leaves_per_seg = g.npad / g.leaf;
     a.n_leaf_tiles = g.G * a.leaves_per_seg * a.tiles_per_leaf;
     a.pairs_per_leaf = (a.tiles_per_leaf + 1) / 2;
     a.n_leaf_pairs = g.G * a.leaves_per_seg * a.pairs_per_leaf;
@@ -308,7 +321,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     const int nodes_lvl = g.causal ? (1 << l) : 1;
     a.level_start[l] = (int)tiles;
     a.level_sorted[l] = g.b < s;
-    const long long per_node = a.level_sorted[l] ? (long long)node_blocks(s, g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
+    const long long per_node = a.level_sorted[l] ? (long long)node_blocks(s, g.b) * a.tiles_per_block : ((g.causal ? s : g.n) + kTileQ - 1) / kTileQ;
     tiles += per_node * nodes_lvl * g.G;
     if (tiles > 0x7fffffffLL) return HYPERATTN_UNSUPPORTED_SHAPE;
     a.level_pair_start[l] = (int)pairs;
@@ -316,7 +329,9 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     // or when a block is a single tile; other block sizes run one tile per CTA (a pair that
     // straddles two larger blocks would make each tile's issuer skip more key tiles of the
     // other's block than the stage ring holds, which the ring's release order does not allow)
-    a.level_paired[l] = !a.level_sorted[l] || a.tiles_per_block % 2 == 0 || a.tiles_per_block == 1;
+    // (a single query tile per group only pairs up when the groups' key blocks are short as well: with fewer
+    // queries than keys a group of at most 128 queries can face a key block of many tiles)
+    a.level_paired[l] = !a.level_sorted[l] || a.tiles_per_block % 2 == 0 || (a.tiles_per_block == 1 && g.b <= kTileQ);
     pairs += (a.level_paired[l] ? (per_node + 1) / 2 : per_node) * nodes_lvl * g.G;
   }
   a.level_start[g.levels] = (int)tiles;
@@ -404,9 +419,9 @@ int hyperattn_forward_host(const hyperattn_params* hp) {
   int rc = build_geometry(*hp, g);
   if (rc) return rc;
   const size_t es = hp->dtype == HYPERATTN_FP32 ? 4 : 2, eo = hp->out_dtype == HYPERATTN_FP32 ? 4 : 2;
-  const size_t elems = (size_t)g.G * g.n * g.d;
-  const size_t in_b = align_up(elems * es), out_b = align_up(elems * eo), lse_b = align_up((size_t)g.G * g.n * 4);
-  const size_t need = 3 * in_b + out_b + lse_b;
+  const size_t elems = (size_t)g.G * g.n * g.d, elems_k = (size_t)g.G * g.nk * g.d;
+  const size_t in_b = align_up(elems * es), in_bk = align_up(elems_k * es), out_b = align_up(elems * eo), lse_b = align_up((size_t)g.G * g.n * 4);
+  const size_t need = in_b + 2 * in_bk + out_b + lse_b;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   char* stage = nullptr;
@@ -423,8 +438,8 @@ int hyperattn_forward_host(const hyperattn_params* hp) {
     stage = reinterpret_cast<char*>(ds.host_stage);
   }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(hp->stream);
-  char* dq = stage; char* dk = stage + in_b; char* dv = stage + 2 * in_b;
-  char* dout = stage + 3 * in_b; char* dlse = stage + 3 * in_b + out_b;
+  char* dq = stage; char* dk = stage + in_b; char* dv = stage + in_b + in_bk;
+  char* dout = stage + in_b + 2 * in_bk; char* dlse = dout + out_b;
   // Segments are independent, so the batch goes through in groups: the copy of group c + 1 to the
   // device and the copy of group c - 1 back run (on streams of their own, PCIe being full duplex)
   // while group c is computed on the caller's stream.  With debug outputs requested, one group.
@@ -446,7 +461,7 @@ int hyperattn_forward_host(const hyperattn_params* hp) {
   DeviceState& ds = *dsp;
   const int nchunks = hp->debug ? 1 : (g.G < kHostChunks ? g.G : kHostChunks);
   const int per = (g.G + nchunks - 1) / nchunks;
-  const size_t seg_in = (size_t)g.n * g.d * es, seg_out = (size_t)g.n * g.d * eo, seg_lse = (size_t)g.n * 4;
+  const size_t seg_in = (size_t)g.n * g.d * es, seg_ink = (size_t)g.nk * g.d * es, seg_out = (size_t)g.n * g.d * eo, seg_lse = (size_t)g.n * 4;
 #define HA_HOST(x) do { if ((x) != cudaSuccess) { std::fprintf(stderr, "hyperattn: %s failed\n", #x); return HYPERATTN_CUDA_ERROR; } } while (0)
   // the staging buffers may still be in use by work queued earlier on the caller's stream
   HA_HOST(cudaEventRecord(ds.ev_start, st));
@@ -454,15 +469,15 @@ int hyperattn_forward_host(const hyperattn_params* hp) {
   HA_HOST(cudaStreamWaitEvent(ds.copy_out, ds.ev_start, 0));
   for (int c = 0, s0 = 0; s0 < g.G; ++c, s0 += per) {
     const int ns = (g.G - s0) < per ? (g.G - s0) : per;
-    const size_t oi = (size_t)s0 * seg_in, oo = (size_t)s0 * seg_out, ol = (size_t)s0 * seg_lse;
+    const size_t oi = (size_t)s0 * seg_in, oik = (size_t)s0 * seg_ink, oo = (size_t)s0 * seg_out, ol = (size_t)s0 * seg_lse;
     HA_HOST(cudaMemcpyAsync(dq + oi, static_cast<const char*>(hp->q) + oi, ns * seg_in, cudaMemcpyHostToDevice, ds.copy_in));
-    HA_HOST(cudaMemcpyAsync(dk + oi, static_cast<const char*>(hp->k) + oi, ns * seg_in, cudaMemcpyHostToDevice, ds.copy_in));
-    HA_HOST(cudaMemcpyAsync(dv + oi, static_cast<const char*>(hp->v) + oi, ns * seg_in, cudaMemcpyHostToDevice, ds.copy_in));
+    HA_HOST(cudaMemcpyAsync(dk + oik, static_cast<const char*>(hp->k) + oik, ns * seg_ink, cudaMemcpyHostToDevice, ds.copy_in));
+    HA_HOST(cudaMemcpyAsync(dv + oik, static_cast<const char*>(hp->v) + oik, ns * seg_ink, cudaMemcpyHostToDevice, ds.copy_in));
     HA_HOST(cudaEventRecord(ds.ev_in[c], ds.copy_in));
     HA_HOST(cudaStreamWaitEvent(st, ds.ev_in[c], 0));
     hyperattn_params p = *hp;
     p.B = 1; p.H = ns;
-    p.q = dq + oi; p.k = dk + oi; p.v = dv + oi;
+    p.q = dq + oi; p.k = dk + oik; p.v = dv + oik;
     p.out = dout + oo; p.lse = reinterpret_cast<float*>(dlse + ol);
     rc = forward_impl(p, s0);
     if (rc) return rc;

@@ -36,7 +36,7 @@ struct AttnArgs {
   // node tiles, per level
   int level_start[kMaxLevels + 1];   // first tile index of each level (after the leaf tiles)
   int level_sorted[kMaxLevels];      // 1: sortLSH node tiles; 0: single-block node (dense tiles)
-  int tiles_per_block;               // ceil(b / 128)
+  int tiles_per_block;               // ceil(bq / 128): query tiles per group of sorted queries of a full node
   int total_tiles;
   // the same schedule in pairs of neighbouring query tiles (tcgen05 path)
   int pairs_per_leaf, n_leaf_pairs;
@@ -57,6 +57,7 @@ struct TileDesc {
   size_t slice;        // node: offset of this node's slice in perm_q / perm_k / rank_k
   int spos0;           // node: first sorted position of the tile
   int beta;            // node: block index
+  int bq;              // node: rows per group of sorted queries (b, unless the node has fewer / more queries than keys)
   int node;            // node: heap index
   size_t orow_base;    // output row index = orow_base + (segment-relative query row + odelta)
   int odelta;
@@ -74,9 +75,10 @@ __device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
     t.seg = rem / a.leaves_per_seg;
     const int leaf = rem % a.leaves_per_seg;
     t.mode = 0;
-    t.k0 = leaf * g.leaf; t.nk = g.leaf;
+    // a leaf: the rows [k0, k0 + leaf) that exist; a non-causal call that is one block: all n queries against all nk keys
+    t.k0 = leaf * g.leaf; t.nk = g.causal ? max(0, min(g.leaf, g.n - t.k0)) : g.nk;
     t.q0 = t.k0 + tt * kTileQ;
-    t.nq = min(kTileQ, g.leaf - tt * kTileQ);
+    t.nq = max(0, min(kTileQ, (g.causal ? t.nk : g.n) - tt * kTileQ));
     t.causal = a.dense_causal;
     t.qk_off = tt * kTileQ;
     t.orow_base = (size_t)t.seg * g.n; t.odelta = 0;
@@ -96,10 +98,12 @@ __device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
     t.seg = idx / nodes_lvl;
     node_rows(g, level, j, s, q0n, k0n);
     t.mode = 1;
+    const int nqn = node_queries(g, s, q0n);
+    t.bq = query_group(g.b, nqn, s);
     t.beta = tn / a.tiles_per_block;
     const int sub = tn % a.tiles_per_block;
-    t.spos0 = t.beta * g.b + sub * kTileQ;
-    t.nq = max(0, min(kTileQ, block_len(s, g.b, t.beta) - sub * kTileQ));   // 0: the (short) last block has no such tile
+    t.spos0 = t.beta * t.bq + sub * kTileQ;
+    t.nq = t.bq > 0 ? max(0, min(kTileQ, block_len(nqn, t.bq, t.beta) - sub * kTileQ)) : 0;   // 0: the group has no such tile
     t.k0 = k0n; t.nk = s; t.qnode0 = q0n;
     t.slice = ((size_t)level * g.G + t.seg) * g.nl + (g.causal ? (size_t)j * s : 0);
     t.node = g.causal ? (1 << level) - 1 + j : 0;
@@ -107,7 +111,7 @@ __device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
     if (a.direct) { t.orow_base = (size_t)t.seg * g.n; t.odelta = 0; }
     else { t.orow_base = region + (size_t)t.seg * g.nl + (size_t)j * s; t.odelta = -q0n; }
   } else {
-    const int tiles_node = (s + kTileQ - 1) / kTileQ;
+    const int tiles_node = ((g.causal ? s : g.n) + kTileQ - 1) / kTileQ;
     const int tn = idx % tiles_node; idx /= tiles_node;
     const int j = idx % nodes_lvl;
     t.seg = idx / nodes_lvl;
@@ -115,7 +119,7 @@ __device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
     t.mode = 0;
     t.k0 = k0n; t.nk = s;
     t.q0 = q0n + tn * kTileQ;
-    t.nq = min(kTileQ, s - tn * kTileQ);
+    t.nq = max(0, min(kTileQ, node_queries(g, s, q0n) - tn * kTileQ));
     t.causal = 0; t.qk_off = 0;
     if (a.direct) { t.orow_base = (size_t)t.seg * g.n; t.odelta = 0; }
     else { t.orow_base = region + (size_t)t.seg * g.nl + (size_t)j * s; t.odelta = -q0n; }

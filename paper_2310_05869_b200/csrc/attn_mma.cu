@@ -89,10 +89,11 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, tig = lane & 3;
   const TileDesc t = decode_tile(a, blockIdx.x);
+  if (t.nq <= 0) return;                          // (a tile of the schedule whose rows do not exist)
 
   const __nv_bfloat16* qs = a.q + (size_t)t.seg * g.n * D;
-  const __nv_bfloat16* ks = a.k + (size_t)t.seg * g.n * D;
-  const __nv_bfloat16* vs = a.v + (size_t)t.seg * g.n * D;
+  const __nv_bfloat16* ks = a.k + (size_t)t.seg * g.nk * D;
+  const __nv_bfloat16* vs = a.v + (size_t)t.seg * g.nk * D;
 
   // ---- row tables ---------------------------------------------------------------------
   int nkeys;  // padded number of key columns visited
@@ -123,7 +124,7 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
   const uint32_t uQ = smem_u32(sQ), uK = smem_u32(sK), uV = smem_u32(sV);
   const uint32_t uQl = smem_u32(sQl), uKl = smem_u32(sKl);
   const __nv_bfloat16* qls = a.q_lo + (size_t)t.seg * g.n * D;
-  const __nv_bfloat16* kls = a.k_lo + (size_t)t.seg * g.n * D;
+  const __nv_bfloat16* kls = a.k_lo + (size_t)t.seg * g.nk * D;
   auto qrow_fn = [&](int r) { return s_qrow[r]; };
   auto load_kv = [&](int kt, int stage) {
     auto krow_fn = [&](int r) {

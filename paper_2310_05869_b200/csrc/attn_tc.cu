@@ -322,6 +322,7 @@ struct PairDesc {
   int qnode0;          // node: first query row of the node
   size_t slice;        // node: slice offset in perm_q / perm_k / rank_k
   int node;            // node: heap index
+  int nq_node, bq;     // node: query rows of the node, rows per group of sorted queries
   int nbA, nbB, nsmp;  // node: key tiles of block A, of block B (0 if shared), of the samples
   int ntiles;          // key tiles walked
   size_t orow_base; int odelta; int partial;
@@ -388,16 +389,18 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
     t.seg = rem / a.leaves_per_seg;
     const int leaf = rem % a.leaves_per_seg;
     t.mode = 0; t.causal = a.dense_causal;
-    t.k0 = leaf * g.leaf; t.nk = g.leaf;
+    // a leaf: the rows [k0, k0 + leaf) that exist; a non-causal call that is one block: all n queries against all nk keys
+    t.k0 = leaf * g.leaf; t.nk = g.causal ? max(0, min(g.leaf, g.n - t.k0)) : g.nk;
+    const int nq_leaf = g.causal ? t.nk : g.n;
     QTile* qs[2] = {&qa, &qb};
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
       const int tt = 2 * uu + i;
       QTile& q = *qs[i];
-      q.valid = tt < a.tiles_per_leaf;
+      q.valid = tt < a.tiles_per_leaf && tt * kTileQ < nq_leaf;
       q.row0 = tt * kTileQ;
       q.q0 = t.k0 + tt * kTileQ;
-      q.nq = min(kTileQ, g.leaf - tt * kTileQ);
+      q.nq = min(kTileQ, nq_leaf - tt * kTileQ);
       const int lim = t.causal ? min(t.nk, q.row0 + q.nq) : t.nk;
       q.s1 = 0; q.n1 = q.valid ? (lim + TK - 1) / TK : 0; q.s2 = 0; q.n2 = 0;
     }
@@ -410,13 +413,15 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
     const int nodes_lvl = g.causal ? (1 << level) : 1;
     const int sorted = a.level_sorted[level];
     const int paired = a.level_paired[level];
-    const int tiles_node = sorted ? node_blocks(s, g.b) * a.tiles_per_block : (s + kTileQ - 1) / kTileQ;
+    const int tiles_node = sorted ? node_blocks(s, g.b) * a.tiles_per_block : ((g.causal ? s : g.n) + kTileQ - 1) / kTileQ;
     const int pairs_node = paired ? (tiles_node + 1) / 2 : tiles_node;
     const int pn = idx % pairs_node; idx /= pairs_node;
     const int j = idx % nodes_lvl;
     t.seg = idx / nodes_lvl;
     node_rows(g, level, j, s, q0n, k0n);
     t.k0 = k0n; t.nk = s; t.qnode0 = q0n; t.causal = 0;
+    t.nq_node = node_queries(g, s, q0n);
+    t.bq = query_group(g.b, t.nq_node, s);
     t.mode = sorted;
     QTile* qs[2] = {&qa, &qb};
 #pragma unroll
@@ -428,13 +433,14 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
       if (sorted) {
         q.beta = tn / a.tiles_per_block;
         const int sub = tn % a.tiles_per_block;
-        q.spos0 = q.beta * g.b + sub * kTileQ;
-        q.nq = min(kTileQ, block_len(s, g.b, q.beta) - sub * kTileQ);
-        if (q.nq <= 0) q.valid = 0;                       // the (short) last block has no such tile
+        q.spos0 = q.beta * t.bq + sub * kTileQ;
+        q.nq = t.bq > 0 ? min(kTileQ, block_len(t.nq_node, t.bq, q.beta) - sub * kTileQ) : 0;
+        if (q.nq <= 0) q.valid = 0;                       // the group (a short last one, or one past the node's queries) has no such tile
         q.q0 = 0;
       } else {
         q.q0 = q0n + tn * kTileQ;
-        q.nq = min(kTileQ, s - tn * kTileQ);
+        q.nq = min(kTileQ, t.nq_node - tn * kTileQ);
+        if (q.nq <= 0) q.valid = 0;
         q.s1 = 0; q.n1 = q.valid ? (s + TK - 1) / TK : 0; q.s2 = 0; q.n2 = 0;
       }
     }
@@ -1043,7 +1049,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         ItemDesc* de = reinterpret_cast<ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes);
         de->t = t; de->qa = qa; de->qb = qb;
       }
-      const int segrow = t.seg * g.n;                       // row coordinate of the segment's first row
+      const int segrow = t.seg * g.n;                       // row coordinate of the segment's first query row ...
+      const int segrow_k = t.seg * g.nk;                    // ... and of its first key row
       // Key rows as tensor-map row coordinates.  Every global load of a batch is issued before
       // the first one is used; the warp covers 32 consecutive columns per step, so one ballot
       // yields a whole word of the mask tables.  Padding columns point at a valid row (they are
@@ -1073,7 +1080,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             const int c0 = c00 + u * 32;
             if (c0 - lane < nblk) {                       // warp-uniform (nblk is a multiple of 32)
               const unsigned pad = __ballot_sync(0xffffffffu, idx[u] < 0);
-              s_kidx[c0] = segrow + (idx[u] < 0 ? 0 : t.k0 + idx[u]);
+              s_kidx[c0] = segrow_k + (idx[u] < 0 ? 0 : t.k0 + idx[u]);
               if (lane == 0) { s_mask[c0 >> 5] = pad; s_mask[MW + (c0 >> 5)] = pad; }
             }
           }
@@ -1110,7 +1117,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
                 else if (!(m0 || m1)) pos = nblk + nfront + __popc(bf & lt_mask);
                 else pos = nblk + g.m - 1 - (nback + __popc(bb & lt_mask));
                 nfront += __popc(bf); nback += __popc(bb);
-                s_kidx[pos] = segrow + (valid ? t.k0 + l[u] : 0);
+                s_kidx[pos] = segrow_k + (valid ? t.k0 + l[u] : 0);
                 if (m0) atomicOr(&s_mask[pos >> 5], 1u << (pos & 31));
                 if (m1) atomicOr(&s_mask[MW + (pos >> 5)], 1u << (pos & 31));
               }
@@ -1208,7 +1215,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       ok = mbar_wait<100, 18>(bar_tabfull(set), (it >> 1) & 1, s_abort, status);
       if (!ok) break;
       const PairDesc t = reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes)->t;
-      const int segrow = t.seg * g.n;
+      const int segrow = t.seg * g.nk;                      // (keys)
       for (int j = 0; j < t.ntiles && ok; ++j) {
         const int gj = gbase + j;
         const int s = gj % C::NS;
@@ -1330,11 +1337,11 @@ bool encode_rows_map(CUtensorMap* m, const void* base, size_t rows, int d, int b
 
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st) {
   if (a.total_pairs == 0) return cudaSuccess;
-  const size_t rows = (size_t)a.g.G * a.g.n;
-  if (rows > 0x7fffffffull) return cudaErrorInvalidValue;        // row coordinates are 32-bit
+  const size_t rows = (size_t)a.g.G * a.g.n, rows_k = (size_t)a.g.G * a.g.nk;
+  if (rows > 0x7fffffffull || rows_k > 0x7fffffffull) return cudaErrorInvalidValue;        // row coordinates are 32-bit
   TmaMaps maps;
-  if (!encode_rows_map(&maps.q, a.q, rows, a.g.d, 128) || !encode_rows_map(&maps.k, a.k, rows, a.g.d, TK) ||
-      !encode_rows_map(&maps.v, a.v, rows, a.g.d, TK)) return cudaErrorInvalidValue;
+  if (!encode_rows_map(&maps.q, a.q, rows, a.g.d, 128) || !encode_rows_map(&maps.k, a.k, rows_k, a.g.d, TK) ||
+      !encode_rows_map(&maps.v, a.v, rows_k, a.g.d, TK)) return cudaErrorInvalidValue;
   auto go = [&](auto kernel, int smem_bytes) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;

@@ -48,16 +48,22 @@ constexpr uint32_t kDomainDirections = 1, kDomainSamples = 2;
 // rows, or the whole segment.  Units are cut into chunks of at most kSortChunk rows; one
 // hash CTA produces the ids and the 256-bin histogram of one chunk, one scatter CTA places it.
 struct Geometry {
-  int G, n, d;
+  int G, n, d;         // n: query rows per segment
+  int nk;              // key / value rows per segment (n, unless a non-causal call has another number of keys)
+  int npad;            // causal: leaf << L, the length whose halves the recursion cuts (>= n: rows beyond n do
+                       // not exist, so the last leaf and the query side of a level's last node may be short);
+                       // non-causal: n
   int b, m, r;
+  int bq;              // rows per group of sorted queries of a full node: b, or ceil(b n / nk) for unequal sides
   int causal;          // 1: causal with L >= 1 levels or a single causal leaf
   int L;               // number of recursion levels with off-diagonal nodes (0: none)
   int leaf;            // rows per exact leaf (n if L == 0)
-  int unit;            // rows per unit
+  int unit;            // rows per unit (query side; both sides of a causal call)
   int chunks_per_unit;
-  int chunks_per_seg;  // (n / unit) * chunks_per_unit
+  int chunks_per_seg;  // (npad / unit) * chunks_per_unit
+  int unit_k, chunks_per_unit_k, chunks_per_seg_k;   // the same for the key side
   int levels;          // sorted levels: L if causal, else 1 (0 if nothing is sorted)
-  int nl;              // sorted rows per (level, segment, side): n/2 causal, n non-causal
+  int nl;              // sorted rows per (level, segment, side): npad/2 causal, max(n, nk) non-causal
   int nodes;           // off-diagonal nodes per segment (heap-numbered)
   int sorted;          // 1 if any node needs sortLSH (some node has b < its size)
   int seg0;            // index, in the caller's tensor, of this call's first segment (the sampling counters carry it)
@@ -68,21 +74,40 @@ struct Geometry {
 __host__ __device__ inline int node_blocks(int s, int b) { return (s + b - 1) / b; }
 __host__ __device__ inline int block_len(int s, int b, int beta) { return (s - beta * b) < b ? (s - beta * b) : b; }
 
-// node j of level l: size s, first query row, first key row (non-causal: the whole segment)
+// node j of level l: number of keys s, first query row, first key row (non-causal: the whole segment)
 __host__ __device__ inline void node_rows(const Geometry& g, int level, int j, int& s, int& q0, int& k0) {
-  if (!g.causal) { s = g.n; q0 = 0; k0 = 0; return; }
-  s = g.n >> (level + 1);
+  if (!g.causal) { s = g.nk; q0 = 0; k0 = 0; return; }
+  s = g.npad >> (level + 1);
   q0 = (2 * j + 1) * s;
   k0 = 2 * j * s;
 }
+// query rows of a node whose nominal size is s and whose first query row is q0: s, unless the sequence
+// ends inside it (the last node of a causal level) or the call has another number of queries than keys
+__host__ __device__ inline int node_queries(const Geometry& g, int s, int q0) {
+  if (!g.causal) return g.n;
+  const int left = g.n - q0;
+  return left < 0 ? 0 : (left < s ? left : s);
+}
+// rows per group of sorted queries when nq queries meet s keys in groups of b (Alg. 1 line 4 pairs group
+// beta of either side; with nq != s the groups cover the same fraction of the sorted order): ceil(b nq / s)
+__host__ __device__ inline int query_group(int b, int nq, int s) {
+  return (int)(((long long)b * nq + s - 1) / s);
+}
+// per-side chunk geometry (side 0: queries, side 1: keys)
+__host__ __device__ inline int side_rows(const Geometry& g, int side) { return side ? g.nk : g.n; }
+__host__ __device__ inline int side_unit(const Geometry& g, int side) { return side ? g.unit_k : g.unit; }
+__host__ __device__ inline int side_cpu(const Geometry& g, int side) { return side ? g.chunks_per_unit_k : g.chunks_per_unit; }
+__host__ __device__ inline int side_cps(const Geometry& g, int side) { return side ? g.chunks_per_seg_k : g.chunks_per_seg; }
+// chunks of one (level, segment) on a side: every node of the level (causal), or the whole side
+__host__ __device__ inline int side_cpl(const Geometry& g, int side) { return g.causal ? (g.nl / g.unit) * g.chunks_per_unit : side_cps(g, side); }
 
 // ---- stage launchers (each enqueues on `st`; returns cudaGetLastError()) ---------------
 struct Workspace {
   __nv_bfloat16 *q16, *k16, *v16;  // bf16 staging of fp32 inputs (else null)
   __nv_bfloat16 *q16lo, *k16lo;    // second bf16 term of fp32 Q, K: x ~= x16 + x16lo
-  uint8_t* ids;                    // [2, G, n]
-  uint32_t* hist;                  // [2, G, chunks_per_seg, 256]
-  uint32_t* offs;                  // [2, levels, G, chunks per (level,seg,side), 256]
+  uint8_t* ids;                    // queries [G, n], then keys [G, nk]
+  uint32_t* hist;                  // queries [G, chunks_per_seg, 256], then keys [G, chunks_per_seg_k, 256]
+  uint32_t* offs;                  // per side: [levels, G, chunks per (level,seg), 256]
   int32_t *perm_q, *perm_k, *rank_k;  // [levels, G, nl]
   int32_t* samples;                // [G, nodes, m]
   float *part_o, *part_lse;        // causal partials: leaf [G,n,(d)] then per level [G,n/2,(d)]
@@ -91,9 +116,11 @@ struct Workspace {
 
 cudaError_t launch_convert(const float* src, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t count, cudaStream_t st);
 cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
-                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st);
-cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st);
-cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st);
+                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st, int side_mask = 3);
+// side_mask: bit 0 queries, bit 1 keys (3: both)
+cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st, int side_mask = 3);
+cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st, int side_mask = 3);
+// side_mask for the hash as well (a side that is left out is neither read nor written)
 cudaError_t launch_merge(const Geometry& g, const Workspace& ws, void* out, float* lse, int out_fp32,
                          cudaStream_t st);
 

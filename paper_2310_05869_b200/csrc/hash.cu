@@ -47,12 +47,35 @@ __device__ __forceinline__ uint32_t gray_rank8(uint32_t g) {
 struct HashArgs {
   const void* x[2];       // Q, K  [G, n, d]
   float w[128 * 8];       // [d, r] directions, passed by value (<= 4 KB of kernel parameters)
-  uint8_t* ids;           // [2, G, n]
-  uint32_t* hist;         // [2, G, chunks_per_seg, 256]
+  uint8_t* ids;           // queries [G, n], then keys [G, nk]
+  uint32_t* hist;         // queries [G, chunks_per_seg, 256], then keys [G, chunks_per_seg_k, 256]
   unsigned long long* near_zero;
-  int G, n, r;
-  int unit, chunks_per_unit, chunks_per_seg;
+  int G, r;
+  int side_mask;          // bit s set: side s is hashed
+  int n[2];               // rows per segment of either side
+  int unit[2], chunks_per_unit[2], chunks_per_seg[2];
 };
+
+// which chunk a CTA owns: side, segment, first row, number of rows (0: the chunk lies beyond the last row)
+struct ChunkPos { int side, seg, chunk, row0, rows; };
+__device__ __forceinline__ ChunkPos chunk_of_cta(const HashArgs& a, int cta) {
+  ChunkPos c;
+  const int ctas0 = a.G * a.chunks_per_seg[0];
+  c.side = cta >= ctas0;
+  if (c.side) cta -= ctas0;
+  c.chunk = cta % a.chunks_per_seg[c.side];
+  c.seg = cta / a.chunks_per_seg[c.side];
+  const int unit_idx = c.chunk / a.chunks_per_unit[c.side], cu = c.chunk % a.chunks_per_unit[c.side];
+  c.row0 = unit_idx * a.unit[c.side] + cu * kSortChunk;
+  c.rows = max(0, min(min(kSortChunk, a.unit[c.side] - cu * kSortChunk), a.n[c.side] - c.row0));
+  return c;
+}
+__device__ __forceinline__ size_t ids_base(const HashArgs& a, const ChunkPos& c) {
+  return (c.side ? (size_t)a.G * a.n[0] : 0) + (size_t)c.seg * a.n[c.side] + c.row0;
+}
+__device__ __forceinline__ size_t hist_base(const HashArgs& a, const ChunkPos& c) {
+  return ((c.side ? (size_t)a.G * a.chunks_per_seg[0] : 0) + (size_t)c.seg * a.chunks_per_seg[c.side] + c.chunk) * kBuckets;
+}
 
 // One CTA = one chunk (<= kSortChunk rows of one side of one segment).  Each warp walks over
 // groups of 16 rows; the loads of the next group are issued before the MMAs of the current
@@ -68,17 +91,13 @@ __global__ void __launch_bounds__(256, D == 64 ? 4 : 3) hash_bf16_kernel(const _
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, tig = lane & 3;
-  int cta = blockIdx.x;
-  const int chunk = cta % a.chunks_per_seg; cta /= a.chunks_per_seg;
-  const int seg = cta % a.G;
-  const int side = cta / a.G;
-  const int unit_idx = chunk / a.chunks_per_unit, cu = chunk % a.chunks_per_unit;
-  const int row0 = unit_idx * a.unit + cu * kSortChunk;
-  const int rows = min(kSortChunk, a.unit - cu * kSortChunk);
+  const ChunkPos cp = chunk_of_cta(a, blockIdx.x);
+  const int side = cp.side, seg = cp.seg, row0 = cp.row0, rows = cp.rows;
+  if (!((a.side_mask >> side) & 1)) return;
 
   s_hist[tid] = 0;
 
-  const char* base = reinterpret_cast<const char*>(a.x[side]) + ((size_t)seg * a.n + row0) * (D * 2);
+  const char* base = reinterpret_cast<const char*>(a.x[side]) + ((size_t)seg * a.n[side] + row0) * (D * 2);
   unsigned nz = 0;
   const int groups = (rows + 15) >> 4;
   uint4 xa[CPL], xb[CPL];
@@ -160,14 +179,14 @@ __global__ void __launch_bounds__(256, D == 64 ? 4 : 3) hash_bf16_kernel(const _
     if (lane == 0 && nz) atomicAdd(a.near_zero, (unsigned long long)nz);
   }
   __syncthreads();
-  uint8_t* dst = a.ids + ((size_t)side * a.G + seg) * a.n + row0;
+  uint8_t* dst = a.ids + ids_base(a, cp);
   if ((rows & 15) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
     for (int i = tid; i < rows / 16; i += 256)
       reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(s_ids)[i];
   } else {
     for (int i = tid; i < rows; i += 256) dst[i] = s_ids[i];
   }
-  a.hist[(((size_t)side * a.G + seg) * a.chunks_per_seg + chunk) * kBuckets + tid] = s_hist[tid];
+  a.hist[hist_base(a, cp) + tid] = s_hist[tid];
 }
 
 // fp32 rows (small problems): one thread per row, plain fp32 FMA in coordinate order.
@@ -175,18 +194,14 @@ __global__ void __launch_bounds__(256) hash_fp32_kernel(const __grid_constant__ 
   __shared__ float s_w[128 * 8];
   __shared__ uint32_t s_hist[kBuckets];
   const int tid = threadIdx.x;
-  int cta = blockIdx.x;
-  const int chunk = cta % a.chunks_per_seg; cta /= a.chunks_per_seg;
-  const int seg = cta % a.G;
-  const int side = cta / a.G;
-  const int unit_idx = chunk / a.chunks_per_unit, cu = chunk % a.chunks_per_unit;
-  const int row0 = unit_idx * a.unit + cu * kSortChunk;
-  const int rows = min(kSortChunk, a.unit - cu * kSortChunk);
+  const ChunkPos cp = chunk_of_cta(a, blockIdx.x);
+  const int side = cp.side, seg = cp.seg, row0 = cp.row0, rows = cp.rows;
+  if (!((a.side_mask >> side) & 1)) return;
   s_hist[tid] = 0;
   for (int i = tid; i < d * a.r; i += 256) s_w[i] = a.w[i];
   __syncthreads();
-  const float* base = reinterpret_cast<const float*>(a.x[side]) + ((size_t)seg * a.n + row0) * d;
-  uint8_t* dst = a.ids + ((size_t)side * a.G + seg) * a.n + row0;
+  const float* base = reinterpret_cast<const float*>(a.x[side]) + ((size_t)seg * a.n[side] + row0) * d;
+  uint8_t* dst = a.ids + ids_base(a, cp);
   unsigned long long nz = 0;
   for (int row = tid; row < rows; row += 256) {
     float p[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -210,7 +225,7 @@ __global__ void __launch_bounds__(256) hash_fp32_kernel(const __grid_constant__ 
   }
   if (a.near_zero && nz) atomicAdd(a.near_zero, nz);
   __syncthreads();
-  a.hist[(((size_t)side * a.G + seg) * a.chunks_per_seg + chunk) * kBuckets + tid] = s_hist[tid];
+  a.hist[hist_base(a, cp) + tid] = s_hist[tid];
 }
 
 // fp32 -> bf16 staging; `lo` (optional) receives the rounding remainder as a second bf16 term
@@ -239,13 +254,17 @@ cudaError_t launch_convert(const float* src, __nv_bfloat16* hi, __nv_bfloat16* l
 }
 
 cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
-                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st) {
+                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st, int side_mask) {
   HashArgs a;
+  a.side_mask = side_mask;
   for (int i = 0; i < g.d * g.r; ++i) a.w[i] = w_host[i];
   a.x[0] = q; a.x[1] = k; a.ids = ws.ids; a.hist = ws.hist; a.near_zero = near_zero;
-  a.G = g.G; a.n = g.n; a.r = g.r;
-  a.unit = g.unit; a.chunks_per_unit = g.chunks_per_unit; a.chunks_per_seg = g.chunks_per_seg;
-  const int grid = 2 * g.G * g.chunks_per_seg;
+  a.G = g.G; a.r = g.r;
+  for (int s = 0; s < 2; ++s) {
+    a.n[s] = side_rows(g, s); a.unit[s] = side_unit(g, s);
+    a.chunks_per_unit[s] = side_cpu(g, s); a.chunks_per_seg[s] = side_cps(g, s);
+  }
+  const int grid = g.G * (g.chunks_per_seg + g.chunks_per_seg_k);
   if (is_fp32) hash_fp32_kernel<<<grid, 256, 0, st>>>(a, g.d);
   else if (g.d == 64) hash_bf16_kernel<64><<<grid, 256, 0, st>>>(a);
   else hash_bf16_kernel<128><<<grid, 256, 0, st>>>(a);

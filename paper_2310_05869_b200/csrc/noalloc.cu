@@ -18,12 +18,12 @@ namespace {
 
 constexpr int kNoAllocMaxRows = HYPERATTN_NOALLOC_MAX_ROWS;
 constexpr size_t kChunksMax = (kNoAllocMaxRows + kSortChunk - 1) / kSortChunk;
-// layout of the scratch array (bytes): ids of both "sides" | histograms | offsets | perm of side 0
+// layout of the scratch array (bytes): ids | chunk histograms | chunk offsets (the matrix is the "key" side of
+// a one-segment problem that has no query rows)
 constexpr size_t kOffIds = 0;
-constexpr size_t kOffHist = kOffIds + 2 * (size_t)kNoAllocMaxRows;
-constexpr size_t kOffOffs = kOffHist + 2 * kChunksMax * kBuckets * 4;
-constexpr size_t kOffPermQ = kOffOffs + 2 * kChunksMax * kBuckets * 4;
-constexpr size_t kScratchBytes = kOffPermQ + 4 * (size_t)kNoAllocMaxRows;
+constexpr size_t kOffHist = kOffIds + (size_t)kNoAllocMaxRows;
+constexpr size_t kOffOffs = kOffHist + kChunksMax * kBuckets * 4;
+constexpr size_t kScratchBytes = kOffOffs + kChunksMax * kBuckets * 4;
 
 // In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
@@ -67,29 +67,30 @@ extern "C" int hyperattn_sortlsh_noalloc(const void* x, int n, int d, int hash_b
   const int rc = scratch_for_current_device(&scratch);
   if (rc) return rc;
 
-  Geometry g;
-  g.G = 1; g.n = n; g.d = d; g.b = 1; g.m = 0; g.r = hash_bits;
-  g.causal = 0; g.L = 0; g.leaf = n; g.unit = n;
-  g.chunks_per_unit = (n + kSortChunk - 1) / kSortChunk;
-  g.chunks_per_seg = g.chunks_per_unit;
+  // One segment whose key side is the matrix and whose query side has no rows and no chunks: the key side
+  // carries the inverse permutation that callers want, and nothing of the other side is read, hashed or placed.
+  Geometry g = {};
+  g.G = 1; g.n = 0; g.nk = n; g.npad = 0; g.d = d; g.b = 1; g.bq = 1; g.m = 0; g.r = hash_bits;
+  g.causal = 0; g.L = 0; g.leaf = 0; g.unit = 1; g.unit_k = n;
+  g.chunks_per_unit = 0; g.chunks_per_seg = 0;
+  g.chunks_per_unit_k = (n + kSortChunk - 1) / kSortChunk;
+  g.chunks_per_seg_k = g.chunks_per_unit_k;
   g.levels = 1; g.nl = n; g.nodes = 1; g.sorted = 1;
 
   Workspace ws = {};
-  ws.ids = scratch + kOffIds;                                          // [2, 1, n]
+  ws.ids = scratch + kOffIds;                                          // [n]: fully rewritten by the hash kernel
   ws.hist = reinterpret_cast<uint32_t*>(scratch + kOffHist);          // fully rewritten by the hash kernel
   ws.offs = reinterpret_cast<uint32_t*>(scratch + kOffOffs);          // fully rewritten by the scan kernel
-  ws.perm_q = reinterpret_cast<int32_t*>(scratch + kOffPermQ);        // side 0 result, not returned
   ws.perm_k = perm;
   ws.rank_k = rank;
 
   float w[128 * 8];
   hyperattn_get_projections(d, hash_bits, seed, w);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  // the matrix is hashed as both "queries" and "keys" of a one-segment problem; the key side
-  // carries the inverse permutation that callers want
-  if (launch_hash(g, x, x, /*is_fp32=*/0, w, ws, nullptr, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
-  if (launch_sort_scan(g, ws, false, 0, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
-  if (launch_sort_scatter(g, ws, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
-  if (cudaMemcpyAsync(ids, ws.ids + n, (size_t)n, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  constexpr int kKeysOnly = 2;
+  if (launch_hash(g, nullptr, x, /*is_fp32=*/0, w, ws, nullptr, st, kKeysOnly) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  if (launch_sort_scan(g, ws, false, 0, st, kKeysOnly) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  if (launch_sort_scatter(g, ws, st, kKeysOnly) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  if (cudaMemcpyAsync(ids, ws.ids, (size_t)n, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   return HYPERATTN_OK;
 }

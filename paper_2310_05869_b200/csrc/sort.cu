@@ -12,21 +12,26 @@ namespace hyperattn {
 namespace {
 
 struct SortArgs {
-  const uint8_t* ids;     // [2, G, n]
-  const uint32_t* hist;   // [2, G, chunks_per_seg, 256]
-  uint32_t* offs;         // [2, levels, G, chunks_per_level, 256]
+  const uint8_t* ids;     // queries [G, n], then keys [G, nk]
+  const uint32_t* hist;   // queries [G, chunks_per_seg, 256], then keys [G, chunks_per_seg_k, 256]
+  uint32_t* offs;         // queries [levels, G, chunks per (level, segment), 256], then the same for keys
   int32_t *perm_q, *perm_k, *rank_k;  // [levels, G, nl]
   Geometry g;
-  int chunks_per_level;   // chunks per (level, segment, side)
+  int side_mask;          // bit s set: side s is sorted (both, unless a caller wants one side only)
 };
 
 // chunk index (within a segment) of the first chunk of node j's query (side 0) or key (side 1) rows
-__device__ __forceinline__ int node_first_chunk(const Geometry& g, int level, int j, int side, int& nchunks, int& s) {
-  int q0, k0;
+// (chunks that lie beyond the last row have empty histograms and place nothing)
+__device__ __forceinline__ int node_first_chunk(const Geometry& g, int level, int j, int side, int& nchunks) {
+  if (!g.causal) { nchunks = side_cps(g, side); return 0; }
+  int s, q0, k0;
   node_rows(g, level, j, s, q0, k0);
   nchunks = (s / g.unit) * g.chunks_per_unit;
   return ((side == 0 ? q0 : k0) / g.unit) * g.chunks_per_unit;
 }
+__device__ __forceinline__ size_t side_hist_base(const Geometry& g, int side) { return side ? (size_t)g.G * g.chunks_per_seg * kBuckets : 0; }
+__device__ __forceinline__ size_t side_offs_base(const Geometry& g, int side) { return side ? (size_t)g.levels * g.G * side_cpl(g, 0) * kBuckets : 0; }
+__device__ __forceinline__ size_t side_ids_base(const Geometry& g, int side) { return side ? (size_t)g.G * g.n : 0; }
 
 struct SampleArgs {
   int32_t* samples;  // [G, nodes, m]
@@ -45,7 +50,7 @@ __device__ __forceinline__ void samples_body(const SampleArgs& a, int block, int
     const int nd = (int)((i / calls) % g.nodes);
     const int seg = (int)(i / ((size_t)calls * g.nodes));
     const int level = g.causal ? 31 - __clz(nd + 1) : 0;
-    const uint32_t N = g.causal ? (uint32_t)(g.n >> (level + 1)) : (uint32_t)g.n;
+    const uint32_t N = g.causal ? (uint32_t)(g.npad >> (level + 1)) : (uint32_t)g.nk;
     const Philox4 x = philox4x32_10((uint32_t)c, (uint32_t)(g.seg0 + seg), (uint32_t)nd, kDomainSamples, a.k0, a.k1);
     int32_t* dst = a.samples + ((size_t)seg * g.nodes + nd) * g.m;
 #pragma unroll
@@ -67,13 +72,14 @@ __global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a, SampleArgs s
   const int nd = cta % nodes_per; cta /= nodes_per;
   const int seg = cta % g.G;
   const int side = cta / g.G;
+  if (!((a.side_mask >> side) & 1)) return;
   int level = 0, j = nd;
   if (g.causal) { level = 31 - __clz(nd + 1); j = nd + 1 - (1 << level); }
-  int nchunks, s;
-  const int first = node_first_chunk(g, level, j, side, nchunks, s);
-  const uint32_t* h = a.hist + (((size_t)side * g.G + seg) * g.chunks_per_seg + first) * kBuckets;
+  int nchunks;
+  const int first = node_first_chunk(g, level, j, side, nchunks);
+  const uint32_t* h = a.hist + side_hist_base(g, side) + ((size_t)seg * side_cps(g, side) + first) * kBuckets;
   const int lvl_chunk0 = g.causal ? j * nchunks : 0;
-  uint32_t* o = a.offs + ((((size_t)side * g.levels + level) * g.G + seg) * a.chunks_per_level + lvl_chunk0) * kBuckets;
+  uint32_t* o = a.offs + side_offs_base(g, side) + (((size_t)level * g.G + seg) * side_cpl(g, side) + lvl_chunk0) * kBuckets;
   // pass 1: bucket totals of the node (eight loads in flight: the kernel is all latency)
   uint32_t tot = 0;
   for (int c0 = 0; c0 < nchunks; c0 += 8) {
@@ -114,25 +120,31 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
   const Geometry& g = a.g;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   int cta = blockIdx.x;
-  const int lc = cta % a.chunks_per_level; cta /= a.chunks_per_level;
-  const int seg = cta % g.G; cta /= g.G;
-  const int level = cta % g.levels;
-  const int side = cta / g.levels;
+  const int ctas0 = ((a.side_mask & 1) ? g.levels * g.G * side_cpl(g, 0) : 0);
+  const int side = (cta >= ctas0 || !(a.side_mask & 1)) ? 1 : 0;
+  if (side) cta -= ctas0;
+  const int cpl = side_cpl(g, side);
+  const int lc = cta % cpl; cta /= cpl;
+  const int seg = cta % g.G;
+  const int level = cta / g.G;
   // which node and which row range this chunk is
-  int s, q0, k0, j = 0, nchunks_node = a.chunks_per_level;
+  int s, q0, k0, j = 0, nchunks_node = cpl;
   if (g.causal) {
-    s = g.n >> (level + 1);
+    s = g.npad >> (level + 1);
     nchunks_node = (s / g.unit) * g.chunks_per_unit;
     j = lc / nchunks_node;
   }
   node_rows(g, level, j, s, q0, k0);
   const int cn = lc - j * nchunks_node;                  // chunk within the node
-  const int u = cn / g.chunks_per_unit, cu = cn % g.chunks_per_unit;
-  const int local0 = u * g.unit + cu * kSortChunk;       // first row, relative to the node
-  const int rows = min(kSortChunk, g.unit - cu * kSortChunk);
+  const int cpu_s = side_cpu(g, side), unit_s = side_unit(g, side);
+  const int u = cn / cpu_s, cu = cn % cpu_s;
+  const int local0 = u * unit_s + cu * kSortChunk;       // first row, relative to the node
   const int row0 = (side == 0 ? q0 : k0) + local0;       // first row within the segment
+  // (a chunk beyond the last row of the side has nothing to place)
+  const int rows = min(min(kSortChunk, unit_s - cu * kSortChunk), side_rows(g, side) - row0);
+  if (rows <= 0) return;
 
-  const uint8_t* ids = a.ids + ((size_t)side * g.G + seg) * g.n + row0;
+  const uint8_t* ids = a.ids + side_ids_base(g, side) + (size_t)seg * side_rows(g, side) + row0;
   for (int i = tid; i < rows; i += 256) s_id[i] = ids[i];
   for (int i = tid; i < 8 * kBuckets / 4; i += 256) reinterpret_cast<uint4*>(&s_cnt[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
@@ -142,7 +154,7 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
   for (int i = wbeg + lane; i < wend; i += 32) atomicAdd(&s_cnt[warp][s_id[i]], 1u);
   __syncthreads();
   {
-    const uint32_t* o = a.offs + ((((size_t)side * g.levels + level) * g.G + seg) * a.chunks_per_level + lc) * kBuckets;
+    const uint32_t* o = a.offs + side_offs_base(g, side) + (((size_t)level * g.G + seg) * cpl + lc) * kBuckets;
     uint32_t run = o[tid];
 #pragma unroll
     for (int w = 0; w < 8; ++w) { const uint32_t t = s_cnt[w][tid]; s_cnt[w][tid] = run; run += t; }
@@ -178,19 +190,19 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
 
 }  // namespace
 
-static SortArgs make_sort_args(const Geometry& g, const Workspace& ws) {
+static SortArgs make_sort_args(const Geometry& g, const Workspace& ws, int side_mask) {
   SortArgs a;
   a.ids = ws.ids; a.hist = ws.hist; a.offs = ws.offs;
   a.perm_q = ws.perm_q; a.perm_k = ws.perm_k; a.rank_k = ws.rank_k;
   a.g = g;
-  a.chunks_per_level = (g.nl / g.unit) * g.chunks_per_unit;
+  a.side_mask = side_mask;
   return a;
 }
 
 // scan of the chunk histograms; with_samples: the same launch also draws the samples (Alg. 2 line 4)
-cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st) {
+cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st, int side_mask) {
   if (!g.sorted) return cudaSuccess;
-  const SortArgs a = make_sort_args(g, ws);
+  const SortArgs a = make_sort_args(g, ws, side_mask);
   const int nodes_per = g.causal ? g.nodes : 1;
   const int scan_blocks = 2 * g.G * nodes_per;
   SampleArgs sa; sa.samples = ws.samples; sa.g = g; sa.k0 = (uint32_t)seed; sa.k1 = (uint32_t)(seed >> 32);
@@ -204,10 +216,10 @@ cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_s
   return cudaGetLastError();
 }
 
-cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st) {
+cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st, int side_mask) {
   if (!g.sorted) return cudaSuccess;
-  const SortArgs a = make_sort_args(g, ws);
-  const int grid = 2 * g.levels * g.G * a.chunks_per_level;
+  const SortArgs a = make_sort_args(g, ws, side_mask);
+  const int grid = g.levels * g.G * (((side_mask & 1) ? side_cpl(g, 0) : 0) + ((side_mask & 2) ? side_cpl(g, 1) : 0));
   switch (g.r) {                                         // the hash width is a template parameter of the ballot loop
     case 1: sort_scatter_kernel<1><<<grid, 256, 0, st>>>(a); break;
     case 2: sort_scatter_kernel<2><<<grid, 256, 0, st>>>(a); break;

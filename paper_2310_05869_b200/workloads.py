@@ -46,10 +46,15 @@ class Workload:
     kind: str           # "gaussian" | "clustered" | "student_t" | "ramp"
     gen_seed: int
     seed: int = 0       # the library's seed (hash directions and sampled columns)
+    n_k: int = 0        # rows of K and V when they differ from n (0: n)
 
     @property
     def G(self) -> int:
         return self.B * self.H
+
+    @property
+    def nk(self) -> int:
+        return self.n_k or self.n
 
     def scaled(self, **kw) -> "Workload":
         return replace(self, **kw)
@@ -104,11 +109,16 @@ def _ramp(rng, G, n, d):
 
 
 def make_inputs(w: Workload):
-    """Returns Q, K, V as numpy arrays of shape (G, n, d): float32 for "fp32" workloads,
+    """Returns Q (G, n, d) and K, V (G, n_k, d) as numpy arrays: float32 for "fp32" workloads,
     uint16 bf16 bit patterns for "bf16" workloads."""
     rng = np.random.Generator(np.random.PCG64(w.gen_seed))
     gen = {"gaussian": _gaussian, "clustered": _clustered, "student_t": _student_t, "ramp": _ramp}[w.kind]
-    qkv = gen(rng, w.G, w.n, w.d)
+    if w.nk != w.n:
+        # unequal sides: draw max(n, n_k) rows of everything and keep the first n / n_k of each
+        big = gen(rng, w.G, max(w.n, w.nk), w.d)
+        qkv = [np.ascontiguousarray(big[0][:, :w.n]), np.ascontiguousarray(big[1][:, :w.nk]), np.ascontiguousarray(big[2][:, :w.nk])]
+    else:
+        qkv = gen(rng, w.G, w.n, w.d)
     if w.dtype == "bf16":
         return [f32_to_bf16_bits(x) for x in qkv]
     return qkv

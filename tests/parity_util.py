@@ -57,27 +57,26 @@ def to_device(w: WL.Workload, arrs):
             t = torch.from_numpy(x.view(np.int16)).cuda().view(torch.bfloat16)
         else:
             t = torch.from_numpy(x).cuda()
-        outs.append(t.view(w.B, w.H, w.n, w.d))
+        outs.append(t.view(w.B, w.H, x.shape[1], w.d))
     return outs
 
 
 def levels_of(w: WL.Workload):
-    """[(level, node_size)] of the off-diagonal problems; non-causal: one node of n rows."""
+    """[(level, keys per node)] of the off-diagonal problems; non-causal: one node over all keys."""
     if not w.causal:
-        return [(0, w.n)] if w.b < w.n else []
-    if w.n <= w.n0:
-        return []
-    L = 0
-    while (w.n >> L) > w.n0:
-        L += 1
-    return [(l, w.n >> (l + 1)) for l in range(L)]
+        return [(0, w.nk)] if w.b < w.nk else []
+    L, leaf = O.causal_grid(w.n, w.n0)
+    return [(l, leaf << (L - 1 - l)) for l in range(L)]
 
 
 def node_ranges(w: WL.Workload, level: int, j: int):
+    """(first query row, first key row, keys, queries) of node j of a level."""
     if not w.causal:
-        return 0, 0, w.n
-    s = w.n >> (level + 1)
-    return (2 * j + 1) * s, 2 * j * s, s
+        return 0, 0, w.nk, w.n
+    L, leaf = O.causal_grid(w.n, w.n0)
+    s = leaf << (L - 1 - level)
+    q0 = (2 * j + 1) * s
+    return q0, 2 * j * s, s, max(0, min(s, w.n - q0))
 
 
 def check_ids(w, Q64, K64, inter, segs=None):
@@ -134,13 +133,15 @@ def check_perms(w, inter, segs=None):
                 continue
             nodes = (1 << level) if w.causal else 1
             for j in range(nodes):
-                q0, k0, _ = node_ranges(w, level, j)
-                sl = slice(j * s, (j + 1) * s) if w.causal else slice(0, s)
-                perm, _ = O.stable_argsort(gq[g, q0:q0 + s])
-                assert (pq[level, g, sl] == perm).all(), ("perm_q", g, level, j)
+                q0, k0, _, nq = node_ranges(w, level, j)
+                if nq == 0:
+                    continue                             # a node beyond the end of the sequence
+                base = j * s if w.causal else 0
+                perm, _ = O.stable_argsort(gq[g, q0:q0 + nq])
+                assert (pq[level, g, base:base + nq] == perm).all(), ("perm_q", g, level, j)
                 perm, rank = O.stable_argsort(gk[g, k0:k0 + s])
-                assert (pk[level, g, sl] == perm).all(), ("perm_k", g, level, j)
-                assert (rk[level, g, sl] == rank).all(), ("rank_k", g, level, j)
+                assert (pk[level, g, base:base + s] == perm).all(), ("perm_k", g, level, j)
+                assert (rk[level, g, base:base + s] == rank).all(), ("rank_k", g, level, j)
 
 
 class LazySegments:
@@ -181,7 +182,7 @@ def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, seg
         else:
             rows = set(rng.choice(w.n, size=rows_per_seg, replace=False).tolist())
             if w.causal and w.n > w.n0:
-                leaf = w.n >> len(levels_of(w))
+                leaf = O.causal_grid(w.n, w.n0)[1]
                 for edge in range(0, w.n + 1, leaf):
                     rows.update(x for x in (edge - 1, edge, edge + 127, edge + 128) if 0 <= x < w.n)
             rows.update((0, w.n - 1))

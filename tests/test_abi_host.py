@@ -47,7 +47,7 @@ def _params(**kw):
 @pytest.mark.parametrize("kw,code", [
     (dict(d=96), -2), (dict(hash_bits=0), -2), (dict(hash_bits=9), -2),
     (dict(block=0), -1), (dict(samples=-1), -1), (dict(B=0), -1), (dict(dtype=5), -1),
-    (dict(causal=1, n0=0), -1), (dict(causal=1, n0=100, n=1000), -2),
+    (dict(causal=1, n0=0), -1), (dict(causal=1, n0=100, n=1000, n_k=900), -2), (dict(n_k=-5), -1),
     (dict(n=4096, block=1024, samples=256), -2),
 ])
 def test_bad_shapes_are_rejected_on_the_host(kw, code):

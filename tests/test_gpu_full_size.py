@@ -18,7 +18,11 @@ pytestmark = pytest.mark.gpu
 # beyond the benchmark sizes: a million rows (eight recursion levels over 256 leaves) and half a million rows of d = 128
 LONG = [WL.Workload("long_n1m_causal", 1, 2, 1048576, 64, "bf16", 256, 256, 7, True, 4096, "gaussian", 1010),
         WL.Workload("long_n512k_d128", 1, 1, 524288, 128, "bf16", 256, 256, 7, False, 0, "gaussian", 1011)]
-FULL = [WL.CONFIGS[1], WL.CONFIGS[2], WL.CONFIGS[3], WL.CONFIGS[4]] + LONG
+# lengths that nothing divides, at size: a causal sequence of 100003 rows (32 leaves of 3126 rows, the last of 3097) and
+# 50000 queries against 131072 keys
+RAGGED = [WL.Workload("ragged_n100003_causal", 1, 4, 100003, 64, "bf16", 256, 256, 7, True, 4096, "gaussian", 1012),
+          WL.Workload("ragged_cross_50000x131072", 1, 4, 50000, 64, "bf16", 256, 256, 7, False, 0, "gaussian", 1013, 0, 131072)]
+FULL = [WL.CONFIGS[1], WL.CONFIGS[2], WL.CONFIGS[3], WL.CONFIGS[4]] + LONG + RAGGED
 
 
 @pytest.mark.parametrize("w", FULL, ids=[w.name for w in FULL])

@@ -19,6 +19,8 @@ def draw(seed: int) -> WL.Workload:
     dtype = "fp32" if rng.random() < 0.1 else "bf16"
     B, H = int(rng.integers(1, 3)), int(rng.integers(1, 4))
     causal = bool(rng.random() < 0.5)
+    n_k = 0
+    ragged = 24 <= seed < 1000 and seed % 2 == 0      # (the draws above 1000 feed the backward tests: equal sides, lengths that 2^L divides)
     if causal:
         # 2^L leaves of any size: Alg. 4 halves until a part is not longer than n0
         leaf = int(np.exp(rng.uniform(np.log(3), np.log(1000))))
@@ -27,9 +29,13 @@ def draw(seed: int) -> WL.Workload:
             L -= 1
         n = leaf << L
         n0 = int(rng.integers(leaf, 2 * leaf))
+        if ragged:
+            n = max(2, n - int(rng.integers(1, 1 << L)) if L else n)     # lengths that 2^L does not divide
     else:
         n0 = 0
         n = int(np.exp(rng.uniform(np.log(33), np.log(6000))))
+        if ragged:
+            n_k = int(np.exp(rng.uniform(np.log(33), np.log(6000))))     # queries and keys of different number
     while True:
         b = int(np.exp(rng.uniform(0, np.log(700))))
         m = int(rng.choice([0, int(np.exp(rng.uniform(0, np.log(600))))], p=[0.1, 0.9]))
@@ -37,10 +43,10 @@ def draw(seed: int) -> WL.Workload:
             break
     r = int(rng.integers(1, 9))
     kind = str(rng.choice(["gaussian", "clustered", "student_t", "ramp"], p=[0.4, 0.2, 0.2, 0.2]))
-    return WL.Workload(f"fuzz{seed}", B, H, n, d, dtype, b, m, r, causal, n0, kind, 500 + seed, seed)
+    return WL.Workload(f"fuzz{seed}", B, H, n, d, dtype, b, m, r, causal, n0, kind, 500 + seed, seed, n_k)
 
 
-CASES = [draw(s) for s in range(24)]
+CASES = [draw(s) for s in range(40)]
 
 
 def check(w):
@@ -61,6 +67,6 @@ def check(w):
     return PU.check_outputs(w, Q64, K64, V64, out, lse, None, max_abs_bound=bound)
 
 
-@pytest.mark.parametrize("w", CASES, ids=[f"{w.name}_n{w.n}_d{w.d}_b{w.b}_m{w.m}_r{w.r}_{'c' if w.causal else 'nc'}{w.n0}_{w.kind}_{w.dtype}" for w in CASES])
+@pytest.mark.parametrize("w", CASES, ids=[f"{w.name}_n{w.n}_k{w.nk}_d{w.d}_b{w.b}_m{w.m}_r{w.r}_{'c' if w.causal else 'nc'}{w.n0}_{w.kind}_{w.dtype}" for w in CASES])
 def test_random_shapes(w):
     print(w, check(w))

@@ -11,8 +11,8 @@ import parity_util as PU
 pytestmark = pytest.mark.gpu
 
 
-def W(name, B, H, n, d, dtype, b, m, r, causal, n0, kind="gaussian", gen_seed=7, seed=0):
-    return WL.Workload(name, B, H, n, d, dtype, b, m, r, causal, n0, kind, gen_seed, seed)
+def W(name, B, H, n, d, dtype, b, m, r, causal, n0, kind="gaussian", gen_seed=7, seed=0, n_k=0):
+    return WL.Workload(name, B, H, n, d, dtype, b, m, r, causal, n0, kind, gen_seed, seed, n_k)
 
 
 SMALL = [
@@ -54,6 +54,20 @@ SMALL = [
     W("causal_leaves_of_125_rows", 1, 2, 4000, 64, "bf16", 96, 64, 6, True, 128, seed=27),
     W("causal_leaves_of_750_rows_d128", 1, 2, 6000, 128, "bf16", 256, 128, 7, True, 1000, seed=28),
     W("causal_leaves_of_3_rows", 1, 1, 768, 64, "bf16", 16, 8, 4, True, 5, seed=29),
+    # causal lengths that 2^L does not divide: the last leaf and the last node of every level are short
+    W("ragged_causal_n4099", 1, 2, 4099, 64, "bf16", 128, 64, 7, True, 512, seed=50),
+    W("ragged_causal_n2049_d128", 2, 1, 2049, 128, "bf16", 64, 32, 6, True, 256, seed=51),
+    W("ragged_causal_n5000_leaf157", 1, 2, 5000, 128, "bf16", 96, 40, 7, True, 300, seed=52),
+    W("ragged_causal_last_leaf_of_one_row", 1, 1, 1025, 64, "bf16", 64, 16, 5, True, 128, seed=53),
+    W("ragged_causal_fp32_n1111", 1, 1, 1111, 64, "fp32", 48, 24, 6, True, 128, seed=54),
+    W("ragged_causal_unsorted_levels", 1, 2, 1500, 64, "bf16", 256, 32, 7, True, 100, seed=55),
+    # queries and keys of different number
+    W("ragged_cross_more_keys", 1, 2, 1000, 64, "bf16", 256, 256, 7, False, 0, seed=56, n_k=3000),
+    W("ragged_cross_more_queries_d128", 1, 2, 5000, 128, "bf16", 128, 96, 7, False, 0, seed=57, n_k=1200),
+    W("ragged_cross_single_block", 1, 2, 700, 64, "bf16", 512, 16, 4, False, 0, seed=58, n_k=300),
+    W("ragged_cross_seven_queries", 1, 1, 7, 64, "bf16", 256, 64, 6, False, 0, seed=59, n_k=1000),
+    W("ragged_cross_fp32", 1, 1, 900, 64, "fp32", 64, 32, 6, False, 0, seed=60, n_k=400),
+    W("ragged_cross_long_queries_short_keys", 1, 1, 9000, 64, "bf16", 256, 128, 7, False, 0, seed=61, n_k=2304),
 ]
 
 

@@ -573,3 +573,115 @@ def test_causal_odd_lengths_dense_form_and_rebuilt_last_node(n, n0, b, m):
     A = np.exp(0.7 * (Q @ K.T))
     np.testing.assert_allclose(np.log((C * A)[h:, h:].sum(axis=1)), inside, atol=1e-9)
     np.testing.assert_allclose(np.log((C * A)[h:, :h].sum(axis=1)), l21, atol=1e-12)
+
+
+# ------------------------------------------------------------------ Alg. 2 with its caps
+def brute_capped(Q, K, V, iq, ik, smp, T, b, scale, cap_scale, kappa):
+    """Alg. 2 lines 3, 6, 7, 9 with explicit loops, in plain exp arithmetic (small logits)."""
+    n_q, N = Q.shape[0], K.shape[0]
+    b_q = -(-b * n_q // N)
+    order_q = sorted(range(n_q), key=lambda i: (int(iq[i]), i))
+    order_k = sorted(range(N), key=lambda j: (int(ik[j]), j))
+    pos_q = {i: p for p, i in enumerate(order_q)}
+    pos_k = {j: p for p, j in enumerate(order_k)}
+    m = len(smp)
+    A = [[math.exp(scale * float(Q[i] @ K[j])) for j in range(N)] for i in range(n_q)]
+    inside = lambda i, j: pos_k[j] // b == pos_q[i] // b_q
+    tau = max([sum(A[j][k] for k in range(N) if not inside(j, k)) for j in T], default=0.0)       # line 3
+    out = np.zeros((n_q, V.shape[1]))
+    lse = np.zeros(n_q)
+    for i in range(n_q):
+        masked = sum(A[i][j] for j in range(N) if inside(i, j))
+        C = cap_scale * m / (N * math.log(N)) * (masked + tau / kappa)                                # line 6
+        d = (N / m) * sum(min(A[i][int(l)], C) for l in smp if not inside(i, int(l)))                 # line 7
+        dt = masked + max(d, tau / kappa)                                                             # line 9
+        num = sum(A[i][j] * V[j] for j in range(N) if inside(i, j))
+        num = num + (N / m) * sum((A[i][int(l)] * V[int(l)] for l in smp if not inside(i, int(l))), np.zeros(V.shape[1]))
+        out[i] = num / dt
+        lse[i] = math.log(dt)
+    return out, lse, tau
+
+
+@pytest.mark.parametrize("cap_scale,kappa", [(3.0, 2.0), (40.0, 50.0), (0.5, 1000.0)])
+def test_capped_row_sums_against_explicit_loops(cap_scale, kappa):
+    rng = np.random.default_rng(int(cap_scale * 10 + kappa))
+    N, b, m, d = 36, 6, 9, 4
+    Q, K, V = rand_qkv(rng, N, d)
+    iq = rng.integers(0, 8, N).astype(np.uint8); ik = rng.integers(0, 8, N).astype(np.uint8)
+    smp = rng.integers(0, N, m); T = rng.integers(0, N, m)
+    out, lse = O.node_forward(Q, K, V, iq, ik, smp, b, 0.8, caps=(cap_scale, kappa, T))
+    bo, bl, tau = brute_capped(Q, K, V, iq, ik, smp, T, b, 0.8, cap_scale, kappa)
+    np.testing.assert_allclose(lse, bl, atol=1e-11)
+    np.testing.assert_allclose(out, bo, atol=1e-11)
+    # and the caps did something in at least one of the parameter sets: the result differs from the uncapped one
+    o0, l0 = O.node_forward(Q, K, V, iq, ik, smp, b, 0.8)
+    if cap_scale < 10:
+        assert np.abs(l0 - lse).max() > 1e-6
+
+
+def test_caps_switched_off_reproduce_the_uncapped_path_bit_for_bit():
+    rng = np.random.default_rng(77)
+    Q, K, V = (x[None] for x in rand_qkv(rng, 96, 5))
+    for causal, n0 in ((False, 0), (True, 12)):
+        o0, l0 = O.forward(Q, K, V, b=8, m=10, r=4, causal=causal, n0=n0, seed=3, scale=0.5)
+        o1, l1 = O.forward(Q, K, V, b=8, m=10, r=4, causal=causal, n0=n0, seed=3, scale=0.5, caps=(math.inf, math.inf))
+        assert np.array_equal(o0, o1) and np.array_equal(l0, l1)
+
+
+def test_capped_zero_logits_closed_form_with_a_binding_cap_and_the_lower_cap():
+    """Q = 0: every entry is 1, the masked sum of a row is its block's size, tau = N - (smallest block size among
+    the rows of T), and a cap below 1 binds on every sampled entry."""
+    rng = np.random.default_rng(8)
+    N, b, m, d = 37, 8, 12, 3                                      # blocks of 8, 8, 8, 8, 5
+    K = rng.standard_normal((N, d)); V = np.ones((N, d))
+    iq = rng.integers(0, 16, N).astype(np.uint8); ik = rng.integers(0, 16, N).astype(np.uint8)
+    smp = rng.integers(0, N, m); T = np.arange(N)                   # every row: tau = N - 5 (a row of the short block)
+    cap_scale, kappa = 0.3, 4.0
+    out, lse = O.node_forward(np.zeros((N, d)), K, V, iq, ik, smp, b, 1.0, caps=(cap_scale, kappa, T))
+    order_q = sorted(range(N), key=lambda i: (int(iq[i]), i))
+    order_k = sorted(range(N), key=lambda i: (int(ik[i]), i))
+    tau = N - 5
+    for i in range(N):
+        beta = order_q.index(i) // b
+        blk = min(b, N - beta * b)
+        outside = sum(1 for l in smp if order_k.index(int(l)) // b != beta)
+        C = cap_scale * m / (N * math.log(N)) * (blk + tau / kappa)
+        assert C < 1.0                                              # the cap binds
+        want = blk + max((N / m) * outside * C, tau / kappa)
+        assert abs(lse[i] - math.log(want)) < 1e-12
+        np.testing.assert_allclose(out[i], (blk + (N / m) * outside) / want, atol=1e-12)     # numerator uncapped
+    # every sample inside the row's block: the estimate is the lower cap tau / kappa
+    one_block = np.array([order_k[0]] * 5)                          # five copies of a key of block 0
+    out, lse = O.node_forward(np.zeros((N, d)), K, V, iq, ik, one_block, b, 1.0, caps=(cap_scale, kappa, T))
+    for i in order_q[:b]:
+        assert abs(lse[i] - math.log(b + tau / kappa)) < 1e-12
+
+
+def test_row_subset_stream_is_separate_and_in_range():
+    a = O.row_subset(5, 2, 3, 64, 1000)
+    bb = O.sample_indices(5, 2, 3, 64, 1000)
+    assert a.min() >= 0 and a.max() < 1000 and not np.array_equal(a, bb)
+    x = O.philox4x32_10(np.array([[0, 2, 3, 3]], dtype=np.uint64), (5, 0))[0]
+    assert a[0] == (int(x[0]) * 1000) >> 32 and a[3] == (int(x[3]) * 1000) >> 32
+
+
+def test_caps_reduce_the_variance_of_the_row_sum_on_heavy_tailed_logits():
+    """What the caps are for (Lemma 1's proof bounds the estimator's variance through them): with a few huge
+    off-block entries the uncapped estimate of the row sum swings with whether a sample hits them; the capped one
+    does not.  Heavy-tailed Q, K (Student-t, 3 d.o.f.), 400 sample sets."""
+    rng = np.random.default_rng(1234)
+    N, b, m, d = 256, 16, 32, 8
+    Q = np.clip(rng.standard_t(3.0, (N, d)), -20, 20); K = np.clip(rng.standard_t(3.0, (N, d)), -20, 20)
+    V = rng.standard_normal((N, d))
+    W = O.directions(d, 4, 1)
+    iq, _ = O.bucket_ids(Q, W); ik, _ = O.bucket_ids(K, W)
+    T = rng.integers(0, N, m)
+    l_un, l_cap = [], []
+    for t in range(400):
+        smp = rng.integers(0, N, m)
+        l_un.append(O.node_forward(Q, K, V, iq, ik, smp, b, 0.35)[1])
+        l_cap.append(O.node_forward(Q, K, V, iq, ik, smp, b, 0.35, caps=(8.0, 16.0, T))[1])
+    var_un = np.var(np.array(l_un), axis=0).mean()
+    var_cap = np.var(np.array(l_cap), axis=0).mean()
+    print("mean variance of ln d~ over rows: uncapped", var_un, "capped", var_cap)
+    assert var_cap < 0.5 * var_un
