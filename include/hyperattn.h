@@ -97,6 +97,11 @@ typedef struct hyperattn_debug {
   int32_t* rank_k;
   int32_t* samples;
   unsigned long long* near_zero_bits;
+  /* capped calls only (hyperattn_params.capped): */
+  int32_t* row_subset;   /* int32 [G, NODES, m]: the probe rows T of Alg. 2 line 2, as positions in the node's
+                            sorted query order */
+  float* log2_tau;       /* float [G, NODES]: log2 of tau (Alg. 2 line 3) with the softmax scale applied, i.e.
+                            ln(tau) / ln 2; minus infinity for a node without probe rows or unmasked entries */
 } hyperattn_debug;
 
 typedef struct hyperattn_params {
@@ -135,6 +140,20 @@ typedef struct hyperattn_params {
                             ceil(block * n / n_k) rows, so that a group of either side covers the same fraction of
                             its sorted order (every query group has a key group).  The samples are drawn from the
                             n_k keys and weigh n_k / samples. */
+  int capped;            /* 1: the row-sum estimate of every sorted node carries the caps of Alg. 2 as printed:
+                              tau  = max over a random set T of m probe rows of the row sum outside the mask (line 3;
+                                     T = m i.i.d. uniform positions of the node's sorted query order, Philox counter
+                                     (j >> 2, g, v, 3)),
+                              C_i  = cap_scale * m / (N ln N) * (masked_i + tau / kappa)          (line 6),
+                              d_i  = (N/m) sum_t (1 - M_{i,l_t}) min(exp(s_{i,l_t}), C_i)         (line 7),
+                              d~_i = masked_i + max(d_i, tau / kappa)                             (line 9),
+                            masked_i the exact row sum inside the block.  The numerator keeps the uncapped sampled
+                            weights (Alg. 3), so out_i = numerator_i / d~_i is no longer a convex combination of
+                            value rows.  The paper gives the constant of line 6 only as Theta(eps^2 ...): the caller
+                            supplies it.  Costs one extra pass of m rows against all keys of every node.  bf16
+                            inputs, forward only, not together with `precise`. */
+  float cap_scale;       /* the constant (times eps^2) of Alg. 2 line 6; > 0 when capped */
+  float kappa;           /* kappa of Alg. 2; > 0 when capped */
 } hyperattn_params;
 
 /* HyperAttention forward (Alg. 1-4 as specialised in Sec. 4) with bf16 inputs and

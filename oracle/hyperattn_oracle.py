@@ -137,9 +137,10 @@ def sample_indices(seed, g, node, m, N):
 
 def row_subset(seed, g, node, m, n_q):
     """The rows T over which Alg. 2 line 3 takes the maximum unmasked row sum (line 2: "randomly
-    choose a subset T of [n] with |T| = m").  Reading taken: m i.i.d. uniform row indices (a maximum
-    does not care about repeats), drawn like the sampled columns but from their own stream:
-    counter (j >> 2, g, node, 3), word j & 3, index floor(x * n_q / 2^32)."""
+    choose a subset T of [n] with |T| = m"), given as POSITIONS in the sorted order of the queries
+    (position p stands for row P_Q^-1(p); a uniform position is a uniform row).  Reading taken: m
+    i.i.d. uniform positions (a maximum does not care about repeats), drawn like the sampled columns
+    but from their own stream: counter (j >> 2, g, node, 3), word j & 3, index floor(x * n_q / 2^32)."""
     if m == 0 or n_q == 0:
         return np.zeros(0, dtype=np.int64)
     calls = (m + 3) // 4
@@ -274,7 +275,8 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None)
     block and nothing is sampled.  Returns (out, lse) for `rows` (default all rows),
     in original row order.
 
-    caps = (cap_scale, kappa, T) switches on the caps of Alg. 2 (lines 3, 6, 7 and 9 as printed):
+    caps = (cap_scale, kappa, T) switches on the caps of Alg. 2 (lines 3, 6, 7 and 9 as printed; T holds
+    positions of the sorted query order, see row_subset):
       tau   = max_{j in T} <1 - M^H_j, exp(K q_j)>                                  (line 3)
       C_i   = cap_scale * m / (N ln N) * (masked_i + tau / kappa)                   (line 6; the paper
               writes Theta(eps^2 m / (n log n) (...)): the constant times eps^2 is the caller's cap_scale)
@@ -306,8 +308,8 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None)
     blk_of_sample = rank_k[samples] // b
     capped = caps is not None and m > 0
     if capped:
-        cap_scale, kappa, T = caps
-        lfloor = unmasked_row_sum_bound(Q, K, rank_q, rank_k, T, b, b_q, scale) - math.log(kappa)   # ln(tau / kappa)
+        cap_scale, kappa, T = caps                                       # T: positions in the sorted query order
+        lfloor = unmasked_row_sum_bound(Q, K, rank_q, rank_k, perm_q[np.asarray(T, dtype=np.int64)], b, b_q, scale) - math.log(kappa)   # ln(tau / kappa)
         coef = cap_scale * m / (N * math.log(N))
     for beta in np.unique(blk_of_want):
         sel = np.nonzero(blk_of_want == beta)[0]

@@ -15,6 +15,7 @@
 namespace hyperattn {
 cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st);
+cudaError_t launch_tau(const AttnArgs& at, const int32_t* tpos, float* ltau, cudaStream_t st);
 cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, const float* lse, const void* dout,
                             float* delta, float* dq, float* dk, float* dv, void* dq_final, int dq_mode, float scale, int* status, cudaStream_t st);
 cudaError_t launch_to_bf16(const float* src, void* dst, size_t count, cudaStream_t st);
@@ -84,12 +85,12 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
 }
 
 struct Plan {
-  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, part_o, part_lse, total;
+  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, tpos, ltau, part_o, part_lse, total;
   size_t delta, gacc;   // backward only: <dO, O> per row; fp32 gradient accumulators (bf16 gradients only)
 };
 
 // backward: 0 forward plan; 1 backward with fp32 gradients (accumulated in place); 2 backward with bf16 gradients
-Plan make_plan(const Geometry& g, int is_fp32, int backward = 0) {
+Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = false) {
   Plan pl;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
@@ -108,6 +109,8 @@ Plan make_plan(const Geometry& g, int is_fp32, int backward = 0) {
   pl.perm_k = take(g.sorted ? lvl_rows * 4 : 0);
   pl.rank_k = take(g.sorted ? lvl_rows * 4 : 0);
   pl.samples = take((size_t)g.G * g.nodes * g.m * 4);
+  pl.tpos = take(capped ? (size_t)g.G * g.nodes * g.m * 4 : 0);
+  pl.ltau = take(capped ? (size_t)g.G * g.nodes * 4 : 0);
   const size_t part_rows = (g.L && !backward) ? (size_t)g.G * g.n + lvl_rows : 0;
   pl.part_o = take(part_rows * g.d * 4);
   pl.part_lse = take(part_rows * 4);
@@ -203,7 +206,14 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     for (const void* x : {bw->dout, (const void*)bw->dq, (const void*)bw->dk, (const void*)bw->dv})
       if (reinterpret_cast<uintptr_t>(x) & 15) return HYPERATTN_MISALIGNED;
   }
-  const Plan pl = make_plan(g, is_fp32, bw ? (bw->grad_dtype == HYPERATTN_FP32 ? 1 : 2) : 0);
+  // Alg. 2 with its caps: sorted nodes with samples only (elsewhere there is nothing to cap)
+  const bool capped = p.capped != 0 && g.sorted && g.m > 0;
+  if (p.capped != 0) {
+    if (!(p.cap_scale > 0.f) || !(p.kappa > 0.f)) return HYPERATTN_INVALID_ARGUMENT;
+    if (is_fp32 || bw || p.precise) return HYPERATTN_UNSUPPORTED_SHAPE;     // bf16 forward with single bf16 weights only
+  }
+  if (p.precise && is_fp32) return HYPERATTN_UNSUPPORTED_SHAPE;
+  const Plan pl = make_plan(g, is_fp32, bw ? (bw->grad_dtype == HYPERATTN_FP32 ? 1 : 2) : 0, capped);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
   int dev = 0;
@@ -243,6 +253,8 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   ws.perm_k = reinterpret_cast<int32_t*>(base + pl.perm_k);
   ws.rank_k = reinterpret_cast<int32_t*>(base + pl.rank_k);
   ws.samples = reinterpret_cast<int32_t*>(base + pl.samples);
+  ws.tpos = capped ? reinterpret_cast<int32_t*>(base + pl.tpos) : nullptr;
+  ws.ltau = capped ? reinterpret_cast<float*>(base + pl.ltau) : nullptr;
   ws.part_o = reinterpret_cast<float*>(base + pl.part_o);
   ws.part_lse = reinterpret_cast<float*>(base + pl.part_lse);
   ws.status = ds.status;
@@ -303,6 +315,8 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   a.part_o = ws.part_o; a.part_lse = ws.part_lse; a.out = p.out; a.lse = p.lse;
   a.out_fp32 = out_fp32;
   a.precise = p.precise != 0;
+  a.capped = capped;
+  a.cap_scale = p.cap_scale; a.log2_kappa = capped ? std::log2(p.kappa) : 0.f; a.ltau = ws.ltau;
   a.direct = g.L == 0;
   a.dense_causal = g.causal;
   a.tiles_per_block = (g.bq + kTileQ - 1) / kTileQ;
@@ -358,6 +372,13 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
       HA_CHECK(launch_to_bf16(dv, bw->dv, elems, st));
     }
     return HYPERATTN_OK;
+  }
+  if (capped) {
+    // Alg. 2 line 3: the largest unmasked row sum among the probe rows of every node
+    StageScope sc(st, HYPERATTN_STAGE_ATTENTION, 1);
+    HA_CHECK(launch_tau(a, ws.tpos, ws.ltau, st));
+    if (dbg && dbg->row_subset) HA_CHECK(cudaMemcpyAsync(dbg->row_subset, ws.tpos, (size_t)g.G * g.nodes * g.m * 4, cudaMemcpyDeviceToDevice, st));
+    if (dbg && dbg->log2_tau) HA_CHECK(cudaMemcpyAsync(dbg->log2_tau, ws.ltau, (size_t)g.G * g.nodes * 4, cudaMemcpyDeviceToDevice, st));
   }
   {
     StageScope sc(st, HYPERATTN_STAGE_ATTENTION, 1);
@@ -498,7 +519,7 @@ int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes) {
   Geometry g;
   const int rc = build_geometry(*p, g);
   if (rc) return rc;
-  *bytes = make_plan(g, p->dtype == HYPERATTN_FP32).total;
+  *bytes = make_plan(g, p->dtype == HYPERATTN_FP32, 0, p->capped != 0 && g.sorted && g.m > 0).total;
   return HYPERATTN_OK;
 }
 

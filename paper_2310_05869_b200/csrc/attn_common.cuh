@@ -30,6 +30,11 @@ struct AttnArgs {
   int out_fp32;
   int direct;
   int precise;                       // softmax weights enter the P V product as bf16 hi + lo
+  // Alg. 2 with its caps (lines 3, 6, 7, 9): capped != 0 switches them on for the sorted nodes
+  int capped;
+  float cap_scale;                   // the constant of line 6: C_i = cap_scale m / (N ln N) (masked_i + tau / kappa)
+  float log2_kappa;
+  const float* ltau;                 // [G, nodes] log2 tau in the scaled domain
   // dense (leaf) tiles
   int dense_causal;
   int tiles_per_leaf, leaves_per_seg, n_leaf_tiles;

@@ -470,7 +470,8 @@ __device__ __forceinline__ int tile_of(const QTile& q, int a) { return a < q.n1 
 // PRECISE: every softmax weight enters the P V product as a pair of bf16 numbers hi + lo (relative error
 // 2^-17 instead of 2^-9): lo is written into the second half of the S buffer and multiplied by V with a
 // second set of products.
-template <int D, bool GATHER_LATE, bool PRECISE>
+// CAPPED: the sampled part of a sorted node's row sum carries the caps of Alg. 2 (lines 6, 7 and 9).
+template <int D, bool GATHER_LATE, bool PRECISE, bool CAPPED>
 __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TmaMaps maps, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -610,6 +611,17 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       float m_ref = -INFINITY;
       uint64_t l01 = 0;             // l: unrounded row sum (two partial sums, packed)
       float lra = 0.f, lrb = 0.f;   // lr: sum of the bf16 weights (two partial sums; the mixed-precision add takes the bf16 halves as they are)
+      // Alg. 2 with caps (sorted nodes only): the masked row sum (block part) is complete when the first
+      // sampled tile starts; from then on every sampled weight enters the row sum as min(weight, (N/m) C_i),
+      // C_i = cap_scale m / (N ln N) (masked_i + tau / kappa), while the numerator keeps the weight itself.
+      const bool capped_item = CAPPED && t.mode == 1 && g.m > 0;
+      float lblk = 0.f;             // masked row sum in units of 2^m_ref
+      bool in_samples = false;
+      float capfac = 0.f, lfloor = -INFINITY;     // (N/m) cap_scale m / (N ln N); log2(tau / kappa)
+      if (capped_item) {
+        capfac = a.cap_scale / (logf((float)t.nk));
+        lfloor = a.ltau[(size_t)t.seg * g.nodes + t.node] - a.log2_kappa;
+      }
       for (int na = 0; na < total && ok; ++na) {
         const int j = tile_of(q, na);
         const int gw = ga + na;
@@ -682,7 +694,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             if (m_ref == -INFINITY) { m_ref = xm + (wlog - ubias); alpha = 0.f; }
             else { const float k = ceilf(xm - m_ref); m_ref += k; alpha = ex2(-k); }
           }
-          { const uint64_t al2 = pack_f2(alpha, alpha); l01 = fmul2(l01, al2); lra *= alpha; lrb *= alpha; }
+          { const uint64_t al2 = pack_f2(alpha, alpha); l01 = fmul2(l01, al2); lra *= alpha; lrb *= alpha; lblk *= alpha; }
           // O may only be touched between two PV products: the one of the previous tile must
           // have finished (the one of this tile cannot start before this tile's P is published)
           // That product's completion is what releases its V stage to the streamer, so the
@@ -700,6 +712,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         if (__any_sync(0xffffffffu, m_ref == -INFINITY)) {
           ok = move_reference();
           if (!ok) break;
+        }
+        const bool capped_tile = capped_item && j >= t.nbA + t.nbB;
+        if (capped_tile && !in_samples) {            // the block part is complete: its row sum is the masked sum of line 6
+          float b0, b1;
+          unpack_f2(l01, b0, b1);
+          lblk = b0 + b1;
+          in_samples = true;
         }
         const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
         uint64_t lt2;               // this tile's unrounded sum of weights (two partial sums, packed)
@@ -735,16 +754,32 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
               tmem_st16(sbase + 32 + c * 16, plo);
             }
           };
+          // capped tiles: the row sum takes min(weight, cap), the check below and P take the weight itself
+          uint64_t ltu2 = 0;
+          const float capw = capped_tile ? capfac * (lblk + (m_ref == -INFINITY ? 0.f : ex2(lfloor - m_ref))) : 0.f;
+          auto chunk_exp_capped = [&](const uint32_t (&r)[32], int c) {
+            uint32_t p[16];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float x0, x1;
+              unpack_f2(ffma2(pack_u2(r[e], r[e + 1]), sc2, off2), x0, x1);
+              const float p0 = ex2(x0), p1 = ex2(x1);
+              ltu2 = fadd2(ltu2, pack_f2(p0, p1));
+              lt2 = fadd2(lt2, pack_f2(fminf(p0, capw), fminf(p1, capw)));
+              p[e >> 1] = pack2(p0, p1);
+            }
+            tmem_st16(sbase + c * 16, p);
+          };
           HA_T0(tc2);
           if constexpr (PRECISE) tmem_ld32_wait(rb);     // the lo halves overwrite the second half of the scores
-          chunk_exp(ra, 0);
+          if (CAPPED && capped_tile) chunk_exp_capped(ra, 0); else chunk_exp(ra, 0);
           HA_LACC(a_c2, tc2);
           HA_T0(tc3);
           tmem_ld32_wait(rb);
-          chunk_exp(rb, 1);
+          if (CAPPED && capped_tile) chunk_exp_capped(rb, 1); else chunk_exp(rb, 1);
           HA_LACC(a_c3, tc3);
           float lt0, lt1;
-          unpack_f2(lt2, lt0, lt1);
+          unpack_f2((CAPPED && capped_tile) ? ltu2 : lt2, lt0, lt1);
           // (the negated comparison also catches an infinite sum; one second attempt at most: after the
           // reference has moved every finite score is within range, and non-finite inputs must not loop)
           if (attempt == 1 || !__any_sync(0xffffffffu, !(lt0 + lt1 <= kTileSumLimit))) break;
@@ -792,8 +827,16 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];\n\ttcgen05.wait::ld.sync.aligned;\n" : "=r"(sumw) : "r"(lane_addr + colO + D) : "memory");
           lr0 = __uint_as_float(sumw); lr1 = 0.f;
         }
-        const float inv = 1.f / (lr0 + lr1);
-        const float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
+        float inv = 1.f / (lr0 + lr1);
+        float lse = (m_ref + log2f(l0 + l1)) * 0.69314718055994531f;
+        if (capped_item) {
+          // line 9: d~_i = masked_i + max(d_i, tau / kappa), d_i the sum of the capped sampled weights
+          if (!in_samples) lblk = l0 + l1;
+          const float fl = m_ref == -INFINITY ? 0.f : ex2(lfloor - m_ref);
+          const float dt = lblk + fmaxf((l0 + l1) - lblk, fl);
+          inv = 1.f / dt;
+          lse = (m_ref + log2f(dt)) * 0.69314718055994531f;
+        }
         const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
         {
           // O leaves TMEM in pieces of 16 columns (thread = row), is normalised (and rounded to
@@ -1351,14 +1394,20 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
     kernel<<<grid, 384, smem_bytes, st>>>(a, maps, status);
     return cudaGetLastError();
   };
-  if (a.precise) {
-    if (a.g.d == 64) return go(attn_tc_kernel<64, false, true>, Cfg<64>::kTotal);
-    if (!a.direct) return go(attn_tc_kernel<128, true, true>, Cfg<128>::kTotal);
-    return go(attn_tc_kernel<128, false, true>, Cfg<128>::kTotal);
+  if (a.capped) {
+    if (a.precise) return cudaErrorInvalidValue;
+    if (a.g.d == 64) return go(attn_tc_kernel<64, false, false, true>, Cfg<64>::kTotal);
+    if (!a.direct) return go(attn_tc_kernel<128, true, false, true>, Cfg<128>::kTotal);
+    return go(attn_tc_kernel<128, false, false, true>, Cfg<128>::kTotal);
   }
-  if (a.g.d == 64) return go(attn_tc_kernel<64, false, false>, Cfg<64>::kTotal);
-  if (!a.direct) return go(attn_tc_kernel<128, true, false>, Cfg<128>::kTotal);
-  return go(attn_tc_kernel<128, false, false>, Cfg<128>::kTotal);
+  if (a.precise) {
+    if (a.g.d == 64) return go(attn_tc_kernel<64, false, true, false>, Cfg<64>::kTotal);
+    if (!a.direct) return go(attn_tc_kernel<128, true, true, false>, Cfg<128>::kTotal);
+    return go(attn_tc_kernel<128, false, true, false>, Cfg<128>::kTotal);
+  }
+  if (a.g.d == 64) return go(attn_tc_kernel<64, false, false, false>, Cfg<64>::kTotal);
+  if (!a.direct) return go(attn_tc_kernel<128, true, false, false>, Cfg<128>::kTotal);
+  return go(attn_tc_kernel<128, false, false, false>, Cfg<128>::kTotal);
 }
 
 }  // namespace hyperattn

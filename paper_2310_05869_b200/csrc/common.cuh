@@ -41,7 +41,7 @@ __host__ __device__ inline Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
   Philox4 r; r.x[0] = c0; r.x[1] = c1; r.x[2] = c2; r.x[3] = c3;
   return r;
 }
-constexpr uint32_t kDomainDirections = 1, kDomainSamples = 2;
+constexpr uint32_t kDomainDirections = 1, kDomainSamples = 2, kDomainRowSubset = 3;
 
 // ---- geometry of one forward call, shared by all stages --------------------------------
 // "unit" = the largest row range that never straddles a recursion node: a causal leaf of n0
@@ -110,6 +110,8 @@ struct Workspace {
   uint32_t* offs;                  // per side: [levels, G, chunks per (level,seg), 256]
   int32_t *perm_q, *perm_k, *rank_k;  // [levels, G, nl]
   int32_t* samples;                // [G, nodes, m]
+  int32_t* tpos;                   // capped row sums: [G, nodes, m] probe positions (else null)
+  float* ltau;                     // capped row sums: [G, nodes] log2 of the largest unmasked probe row sum
   float *part_o, *part_lse;        // causal partials: leaf [G,n,(d)] then per level [G,n/2,(d)]
   int* status;                     // device status word
 };

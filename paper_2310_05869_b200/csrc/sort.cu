@@ -35,6 +35,8 @@ __device__ __forceinline__ size_t side_ids_base(const Geometry& g, int side) { r
 
 struct SampleArgs {
   int32_t* samples;  // [G, nodes, m]
+  int32_t* tpos;     // capped row sums only (else null): [G, nodes, m] probe positions of Alg. 2 line 2
+  float* ltau;       // capped row sums only: [G, nodes], set to -inf here (the probe pass takes a maximum into it)
   Geometry g;
   uint32_t k0, k1;
 };
@@ -56,6 +58,19 @@ __device__ __forceinline__ void samples_body(const SampleArgs& a, int block, int
 #pragma unroll
     for (int w = 0; w < 4; ++w)
       if (4 * c + w < g.m) dst[4 * c + w] = (int32_t)__umulhi(x.x[w], N);
+    if (a.tpos) {
+      // Alg. 2 line 2: the probe rows T, m i.i.d. uniform positions of the node's sorted query order, from a
+      // stream of their own (the node may have fewer queries than keys; none: nothing is read later)
+      int s, q0, k0;
+      node_rows(g, level, g.causal ? nd + 1 - (1 << level) : 0, s, q0, k0);
+      const uint32_t NQ = (uint32_t)node_queries(g, s, q0);
+      const Philox4 y = philox4x32_10((uint32_t)c, (uint32_t)(g.seg0 + seg), (uint32_t)nd, kDomainRowSubset, a.k0, a.k1);
+      int32_t* dt = a.tpos + ((size_t)seg * g.nodes + nd) * g.m;
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+        if (4 * c + w < g.m) dt[4 * c + w] = (int32_t)__umulhi(y.x[w], NQ);
+      if (c == 0) a.ltau[(size_t)seg * g.nodes + nd] = -INFINITY;
+    }
   }
 }
 
@@ -201,11 +216,12 @@ static SortArgs make_sort_args(const Geometry& g, const Workspace& ws, int side_
 
 // scan of the chunk histograms; with_samples: the same launch also draws the samples (Alg. 2 line 4)
 cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st, int side_mask) {
+  // (ws.tpos non-null: the launch also draws the probe rows of the capped row-sum estimate)
   if (!g.sorted) return cudaSuccess;
   const SortArgs a = make_sort_args(g, ws, side_mask);
   const int nodes_per = g.causal ? g.nodes : 1;
   const int scan_blocks = 2 * g.G * nodes_per;
-  SampleArgs sa; sa.samples = ws.samples; sa.g = g; sa.k0 = (uint32_t)seed; sa.k1 = (uint32_t)(seed >> 32);
+  SampleArgs sa; sa.samples = ws.samples; sa.tpos = ws.tpos; sa.ltau = ws.ltau; sa.g = g; sa.k0 = (uint32_t)seed; sa.k1 = (uint32_t)(seed >> 32);
   int sample_blocks = 0;
   if (with_samples && g.nodes > 0 && g.m > 0) {
     const size_t total = (size_t)g.G * g.nodes * ((g.m + 3) / 4);

@@ -158,17 +158,19 @@ class LazySegments:
         return self.cache[g]
 
 
-def oracle_rows(w, Q64, K64, V64, g, rows, ids_q=None, ids_k=None):
+def oracle_rows(w, Q64, K64, V64, g, rows, ids_q=None, ids_k=None, caps=None):
     W = O.directions(w.d, w.r, w.seed)
     return O.segment_forward(Q64[g], K64[g], V64[g], W, w.b, w.m, w.causal, w.n0, w.seed, g,
-                             scale=1.0 / math.sqrt(w.d), rows=rows, ids_q=ids_q, ids_k=ids_k)
+                             scale=1.0 / math.sqrt(w.d), rows=rows, ids_q=ids_q, ids_k=ids_k, caps=caps)
 
 
 def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, segs=None, rng_seed=0,
-                  max_abs_bound=None, blocks_per_seg=0):
+                  max_abs_bound=None, blocks_per_seg=0, caps=None, row_scale=None):
     """Compares out/lse with the oracle (GPU ids injected when `inter` is given).  With
     rows_per_seg, a pseudo-random subset of rows plus the rows around every leaf / node
-    boundary is checked."""
+    boundary is checked.  `row_scale` (G x n, >= 1) divides the output errors row by row before they meet the
+    bounds: with capped row sums a row's output is its uncapped output times (uncapped row sum / capped
+    row sum), and so are its rounding errors."""
     out = out.float().cpu().numpy().reshape(w.G, w.n, w.d)
     lse = lse.float().cpu().numpy().reshape(w.G, w.n)
     gq = inter["q_ids"].cpu().numpy() if inter is not None else None
@@ -188,8 +190,11 @@ def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, seg
             rows.update((0, w.n - 1))
             rows = np.array(sorted(rows))
         ref_o, ref_l = oracle_rows(w, Q64, K64, V64, g, rows,
-                                   None if gq is None else gq[g], None if gk is None else gk[g])
-        errs.append(np.abs(out[g, rows] - ref_o))
+                                   None if gq is None else gq[g], None if gk is None else gk[g], caps=caps)
+        e = np.abs(out[g, rows] - ref_o)
+        if row_scale is not None:                   # capped row sums: errors measured in units of the row's own scale
+            e = e / row_scale[g, rows][:, None]
+        errs.append(e)
         lerrs.append(np.abs(lse[g, rows] - ref_l) / np.maximum(np.abs(ref_l), 1.0))
     err = np.concatenate([e.reshape(-1) for e in errs])
     lerr = np.concatenate(lerrs)

@@ -587,7 +587,7 @@ def brute_capped(Q, K, V, iq, ik, smp, T, b, scale, cap_scale, kappa):
     m = len(smp)
     A = [[math.exp(scale * float(Q[i] @ K[j])) for j in range(N)] for i in range(n_q)]
     inside = lambda i, j: pos_k[j] // b == pos_q[i] // b_q
-    tau = max([sum(A[j][k] for k in range(N) if not inside(j, k)) for j in T], default=0.0)       # line 3
+    tau = max([sum(A[order_q[p]][k] for k in range(N) if not inside(order_q[p], k)) for p in T], default=0.0)       # line 3 (T: sorted positions)
     out = np.zeros((n_q, V.shape[1]))
     lse = np.zeros(n_q)
     for i in range(n_q):
