@@ -266,6 +266,20 @@ int hyperattn_profile_read(hyperattn_stage_times* out);
 int hyperattn_sortlsh_noalloc(const void* x, int n, int d, int hash_bits, uint64_t seed,
                               uint8_t* ids, int32_t* perm, int32_t* rank, void* stream);
 
+/* The quantity the paper's guarantee is stated in (Theorem 1; measured on real models in Sec. 4.3):
+ *     alpha = n * max_j || D^-1 A e_j ||_2^2,
+ * n times the largest squared column norm of the EXACT softmax matrix of every (batch, head), with the
+ * causal mask M^C if causal != 0; the first skip_cols columns are left out of the maximum (Sec. 4.3 leaves
+ * out the first 32 columns of causal language models, which hold heavy entries).  A diagnostic: it evaluates
+ * the whole n x n_k matrix twice, so it is meant for a few thousand rows.
+ *   q        device, bf16 [B, H, n, d];  k  device, bf16 [B, H, n_k, d] (n_k = 0 means n; causal needs n_k = n)
+ *   alpha    device, float [B * H], written
+ *   workspace device scratch of hyperattn_alpha_workspace_bytes(...) bytes, owned by the caller
+ * softmax_scale <= 0 selects 1/sqrt(d).  Enqueued on `stream`; does not synchronise or allocate. */
+int hyperattn_alpha(const void* q, const void* k, int B, int H, int n, int n_k, int d, float softmax_scale,
+                    int causal, int skip_cols, float* alpha, void* workspace, size_t workspace_bytes, void* stream);
+int hyperattn_alpha_workspace_bytes(int B, int H, int n, int n_k, size_t* bytes);
+
 /* Frees the private workspaces and profiling events of every device. */
 int hyperattn_release(void);
 

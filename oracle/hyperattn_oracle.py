@@ -27,6 +27,7 @@ r hash bits; P_Q, P_K the sortLSH permutations; M^H the block mask):
                      (Alg. 2 lines 7 and 9 without caps, Alg. 3, Sec. 4)
   causal_forward     recursive split (Alg. 4) carried through to outputs
   forward            all (batch, head) segments
+  alpha_diagnostic   n times the largest squared column norm of the exact softmax matrix (Theorem 1, Sec. 4.3)
   dense_weights      the implied n x n row-stochastic weight matrix (tiny n only)
   dense_coefficients the matrix C with W~ = rownorm(C o exp(scale Q K^T)) (tiny n only)
   dense_backward     gradients of (out, lse) with respect to Q, K, V with the sortLSH
@@ -239,6 +240,20 @@ def exact_attention(Q, K, V, scale, causal=False, rows=None):
     out = (a @ V) / den
     lse = (mx + np.log(den))[:, 0]
     return out, lse
+
+
+def alpha_diagnostic(Q, K, scale, causal=False, skip_cols=0):
+    """alpha = n * max_j ||D^-1 A e_j||_2^2 (Theorem 1; Sec. 4.3): n times the largest squared column
+    norm of the exact softmax matrix, the first skip_cols columns left out of the maximum."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    n = Q.shape[0]
+    s = scale * (Q @ K.T)
+    if causal:
+        s = np.where(np.arange(n)[:, None] >= np.arange(K.shape[0])[None, :], s, -np.inf)
+    P = np.exp(s - s.max(axis=1, keepdims=True))
+    P /= P.sum(axis=1, keepdims=True)
+    return n * float((P * P).sum(axis=0)[skip_cols:].max())
 
 
 # --------------------------------------------------------------------------------------

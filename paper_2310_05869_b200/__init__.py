@@ -1,6 +1,7 @@
 """B200-native HyperAttention forward (arXiv 2310.05869): thin binding over libhyperattn.so."""
 from .binding import (  # noqa: F401
     HyperAttnError,
+    alpha,
     backward,
     forward,
     forward_host,

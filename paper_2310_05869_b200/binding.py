@@ -19,7 +19,8 @@ EXPORTS = ["hyperattn_forward", "hyperattn_forward_ex", "hyperattn_forward_host"
            "hyperattn_backward", "hyperattn_backward_workspace_bytes",
            "hyperattn_get_projections", "hyperattn_last_device_status", "hyperattn_profile_enable",
            "hyperattn_profile_reset", "hyperattn_profile_read", "hyperattn_release",
-           "hyperattn_status_string", "hyperattn_version", "hyperattn_sortlsh_noalloc"]
+           "hyperattn_status_string", "hyperattn_version", "hyperattn_sortlsh_noalloc",
+           "hyperattn_alpha", "hyperattn_alpha_workspace_bytes"]
 
 
 class HyperAttnError(RuntimeError):
@@ -69,6 +70,11 @@ def lib() -> C.CDLL:
         L.hyperattn_sortlsh_noalloc.restype = C.c_int
         L.hyperattn_sortlsh_noalloc.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_uint64,
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.hyperattn_alpha.restype = C.c_int
+        L.hyperattn_alpha.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_int, C.c_int,
+                                      C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hyperattn_alpha_workspace_bytes.restype = C.c_int
+        L.hyperattn_alpha_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_size_t)]
         L.hyperattn_backward.restype = C.c_int
         L.hyperattn_backward.argtypes = [C.POINTER(_Params), C.POINTER(_Grads)]
         L.hyperattn_backward_workspace_bytes.restype = C.c_int
@@ -218,6 +224,25 @@ def sortlsh_noalloc(x, hash_bits, seed=0, stream=None):
         _check(lib().hyperattn_sortlsh_noalloc(x.data_ptr(), n, d, hash_bits, seed, ids.data_ptr(), perm.data_ptr(),
                                                rank.data_ptr(), s), "hyperattn_sortlsh_noalloc")
     return ids, perm, rank
+
+
+def alpha(q, k, causal=False, skip_cols=0, scale=0.0, stream=None):
+    """n times the largest squared column norm of the exact softmax matrix of every (batch, head) (the alpha
+    of the paper's Theorem 1): CUDA bf16 tensors q [B, H, n, d], k [B, H, n_k, d] -> float tensor [B, H]."""
+    if not (q.is_cuda and k.is_cuda) or q.dtype != torch.bfloat16 or k.dtype != torch.bfloat16:
+        raise HyperAttnError("q and k must be CUDA bf16 tensors")
+    q, k = q.contiguous(), k.contiguous()
+    B, H, n, d = q.shape
+    n_k = k.shape[2]
+    nbytes = C.c_size_t(0)
+    _check(lib().hyperattn_alpha_workspace_bytes(B, H, n, n_k, C.byref(nbytes)), "hyperattn_alpha_workspace_bytes")
+    ws = torch.empty(int(nbytes.value), dtype=torch.uint8, device=q.device)
+    out = torch.empty((B, H), dtype=torch.float32, device=q.device)
+    s = stream if stream is not None else torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        _check(lib().hyperattn_alpha(q.data_ptr(), k.data_ptr(), B, H, n, 0 if n_k == n else n_k, d, float(scale), int(bool(causal)),
+                                     int(skip_cols), out.data_ptr(), ws.data_ptr(), ws.numel(), s), "hyperattn_alpha")
+    return out
 
 
 def workspace_bytes(B, H, n, d, block, samples, hash_bits, causal=False, n0=0, dtype=BF16, out_dtype=BF16, n_k=0) -> int:

@@ -685,3 +685,33 @@ def test_caps_reduce_the_variance_of_the_row_sum_on_heavy_tailed_logits():
     var_cap = np.var(np.array(l_cap), axis=0).mean()
     print("mean variance of ln d~ over rows: uncapped", var_un, "capped", var_cap)
     assert var_cap < 0.5 * var_un
+
+
+# ------------------------------------------------------------------ the alpha of Theorem 1 / Sec. 4.3
+def test_alpha_closed_forms_and_explicit_loops():
+    n, d = 24, 4
+    rng = np.random.default_rng(3)
+    K = rng.standard_normal((n, d))
+    # uniform attention: every entry 1/n, a column's squared norm is 1/n, alpha = 1
+    assert abs(O.alpha_diagnostic(np.zeros((n, d)), K, 1.0) - 1.0) < 1e-12
+    # causal uniform attention: P_ij = 1/(i+1) for j <= i; the first column is the heaviest: n * sum_i 1/(i+1)^2
+    want = n * sum(1.0 / (i + 1) ** 2 for i in range(n))
+    assert abs(O.alpha_diagnostic(np.zeros((n, d)), K, 1.0, causal=True) - want) < 1e-12
+    # ... and without the first 3 columns: column 3 is the heaviest of the rest
+    want3 = n * sum(1.0 / (i + 1) ** 2 for i in range(3, n))
+    assert abs(O.alpha_diagnostic(np.zeros((n, d)), K, 1.0, causal=True, skip_cols=3) - want3) < 1e-12
+    # every query looks at one key only: that column is all ones, alpha = n^2
+    Kone = np.zeros((n, d)); Kone[5, 0] = 1.0
+    Qbig = np.zeros((n, d)); Qbig[:, 0] = 800.0
+    assert abs(O.alpha_diagnostic(Qbig, Kone, 1.0) - n * n) < 1e-6
+    # explicit loops on random inputs
+    Q = rng.standard_normal((n, d))
+    for causal in (False, True):
+        col = [0.0] * n
+        for i in range(n):
+            js = [j for j in range(n) if (not causal or j <= i)]
+            e = [math.exp(0.7 * float(Q[i] @ K[j])) for j in js]
+            tot = sum(e)
+            for j, x in zip(js, e):
+                col[j] += (x / tot) ** 2
+        assert abs(O.alpha_diagnostic(Q, K, 0.7, causal=causal) - n * max(col)) < 1e-10
