@@ -22,6 +22,8 @@ r hash bits; P_Q, P_K the sortLSH permutations; M^H the block mask):
   causal_grid        leaves and levels of the recursive split for any sequence length
   sample_indices     l_1..l_m ~ Unif([N]) shared by all rows (Alg. 2 line 4, Sec. 4)
   row_subset         the rows T of Alg. 2 line 2 (capped variant only)
+  value_norm_weights, sample_by_value_norms
+                     sampling by squared row norms of V with weights 1 / (m p_l) (Lemma 2)
   exact_attention    D^-1 A V and its causal form (Sec. 1.1, Sec. 3.1)
   node_forward       block-diagonal part + sampled residual with estimated D
                      (Alg. 2 lines 7 and 9 without caps, Alg. 3, Sec. 4)
@@ -154,6 +156,49 @@ def row_subset(seed, g, node, m, n_q):
     return ((x * np.uint64(n_q)) >> _SHIFT32).astype(np.int64)
 
 
+VALUE_NORM_SHIFT = 12
+
+
+def value_norm_weights(V):
+    """Integer sampling weights floor(||V_l||^2 * 2^12) for Lemma 2's distribution p_l = ||V_l||^2 / ||V||_F^2.
+    The squared norm is accumulated in fp32 in coordinate order (for bf16 values every square is exact in
+    fp32, so only the additions round) and then cut to a multiple of 2^-12: integers, so that the
+    cumulative sums and the sampled indices below are exactly reproducible on any machine.  (A row
+    whose squared norm is below 2^-12 is never sampled.)"""
+    V = np.asarray(V, dtype=np.float32)
+    acc = np.zeros(V.shape[0], dtype=np.float32)
+    for c in range(V.shape[1]):
+        acc = (acc + V[:, c] * V[:, c]).astype(np.float32)
+    return np.floor(acc.astype(np.float64) * float(1 << VALUE_NORM_SHIFT)).astype(np.uint64)
+
+
+def sample_by_value_norms(seed, g, node, m, wq):
+    """Lemma 2: m i.i.d. indices with probability p_l = wq_l / sum(wq) (wq from value_norm_weights, for the N
+    keys of one node) and their weights 1 / (m p_l), which make sum_t w_t a_{l_t} v_{l_t} an unbiased
+    estimate of sum_l a_l v_l (Lemma 2's S^T S) and sum_t w_t a_{l_t} one of the row sum.  Sample j uses
+    the same Philox word x as the uniform sampler; the index is the first l whose cumulative weight
+    exceeds floor(x * total / 2^32).  All weights zero: uniform sampling with weights N / m."""
+    wq = np.asarray(wq, dtype=np.uint64)
+    N = wq.size
+    if m == 0:
+        return np.zeros(0, dtype=np.int64), np.zeros(0, dtype=np.float64)
+    calls = (m + 3) // 4
+    ctr = np.zeros((calls, 4), dtype=np.uint64)
+    ctr[:, 0] = np.arange(calls, dtype=np.uint64)
+    ctr[:, 1] = g
+    ctr[:, 2] = node
+    ctr[:, 3] = DOMAIN_SAMPLES
+    x = philox4x32_10(ctr, _seed_key(seed)).reshape(-1)[:m]
+    total = int(wq.sum())
+    if total == 0:
+        idx = np.array([(int(v) * N) >> 32 for v in x], dtype=np.int64)
+        return idx, np.full(m, N / m, dtype=np.float64)
+    cum = np.cumsum(wq)
+    target = np.array([(int(v) * total) >> 32 for v in x], dtype=np.uint64)
+    idx = np.searchsorted(cum, target, side="right").astype(np.int64)
+    return idx, total / (m * wq[idx].astype(np.float64))
+
+
 # --------------------------------------------------------------------------------------
 # sortLSH (Def. 1, Alg. 1)
 # --------------------------------------------------------------------------------------
@@ -273,7 +318,7 @@ def unmasked_row_sum_bound(Q, K, rank_q, rank_k, T, b, b_q, scale):
     return ltau
 
 
-def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None):
+def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None, sample_weights=None):
     """HyperAttention on n_q queries x N keys (n_q = N in the paper; see query_block_size for the
     grouping when they differ).
 
@@ -300,6 +345,10 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None)
     The numerator is unchanged (Alg. 3 multiplies D~^-1 by the sampled product A V; the caps belong
     to the row-sum estimate of Alg. 2 only), so with caps the outputs are no longer convex
     combinations of value rows.  cap_scale = inf and kappa = inf switch both caps off.
+
+    sample_weights (one per sample) replaces the uniform weight N/m: with samples drawn from another
+    distribution p the weight of sample t is 1 / (m p_{l_t}) (Lemma 2; sample_by_value_norms), in
+    the numerator and in the row sum alike.
     """
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
@@ -339,7 +388,11 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None)
                 mx = np.maximum(mx, s_smp[:, keep > 0].max(axis=1, keepdims=True))
             if capped and lfloor > -np.inf:
                 mx = np.maximum(mx, lfloor)
-            w = (N / m) * keep[None, :] * np.exp(np.where(keep[None, :] > 0, s_smp - mx, -np.inf))
+            if sample_weights is None:
+                w = (N / m) * keep[None, :] * np.exp(np.where(keep[None, :] > 0, s_smp - mx, -np.inf))
+            else:
+                sw = np.asarray(sample_weights, dtype=np.float64)
+                w = sw[None, :] * keep[None, :] * np.exp(np.where(keep[None, :] > 0, s_smp - mx, -np.inf))
         a = np.exp(s_blk - mx)
         den = a.sum(axis=1, keepdims=True)
         num = a @ V[J]
@@ -350,7 +403,10 @@ def node_forward(Q, K, V, ids_q, ids_k, samples, b, scale, rows=None, caps=None)
             floor = np.exp(lfloor - mx) if capped else 0.0               # tau / kappa in units of exp(mx)
             cap = coef * (den + floor) if capped else np.inf             # C_i
             p = np.exp(np.where(keep[None, :] > 0, s_smp - mx, -np.inf))
-            d_i = (N / m) * (keep[None, :] * np.minimum(p, cap)).sum(axis=1, keepdims=True)
+            if sample_weights is None:
+                d_i = (N / m) * (keep[None, :] * np.minimum(p, cap)).sum(axis=1, keepdims=True)
+            else:
+                d_i = (sw[None, :] * keep[None, :] * np.minimum(p, cap)).sum(axis=1, keepdims=True)
             den = den + np.maximum(d_i, floor)
         out[sel] = num / den
         lse[sel] = (mx + np.log(den))[:, 0]
@@ -373,7 +429,14 @@ def causal_grid(n, n0):
     return L, -((-n) >> L)
 
 
-def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, caps=None):
+def draw_samples(seed, g, node, m, N, wq=None):
+    """(indices, weights or None): uniform (Sec. 4) or, given the keys' integer weights, by value norms (Lemma 2)."""
+    if wq is None:
+        return sample_indices(seed, g, node, m, N), None
+    return sample_by_value_norms(seed, g, node, m, wq)
+
+
+def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, caps=None, wq=None):
     """Causal HyperAttention.  A part that is a single leaf gets exact causal attention (the paper
     recurses until the length falls below a base size and uses an exact kernel there).  A larger
     part of nominal length S is split at S/2 (Alg. 4 line 2); the two halves recurse (line 3); the
@@ -406,9 +469,10 @@ def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, c
             part(a + h, h, 2 * node + 2, second)
             r2 = want[second] - (a + h)
             mm = m if b < h else 0
-            smp = sample_indices(seed, g, node, mm, h)
+            smp, sw = draw_samples(seed, g, node, mm, h, None if wq is None else wq[a:a + h])
             nc = None if caps is None else (caps[0], caps[1], row_subset(seed, g, node, mm, e - (a + h)))
-            o21, l21 = node_forward(Q[a + h:e], K[a:a + h], V[a:a + h], ids_q[a + h:e], ids_k[a:a + h], smp, b, scale, rows=r2, caps=nc)
+            o21, l21 = node_forward(Q[a + h:e], K[a:a + h], V[a:a + h], ids_q[a + h:e], ids_k[a:a + h], smp, b, scale, rows=r2, caps=nc,
+                                    sample_weights=sw)
             o22, l22 = out[second].copy(), lse[second].copy()
             l = np.logaddexp(l21, l22)
             out[second] = o21 * np.exp(l21 - l)[:, None] + o22 * np.exp(l22 - l)[:, None]
@@ -427,12 +491,13 @@ def heap_node(level, j):
 # Whole forward pass
 # --------------------------------------------------------------------------------------
 def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None,
-                    ids_q=None, ids_k=None, caps=None):
+                    ids_q=None, ids_k=None, caps=None, value_norm_sampling=False):
     """Forward pass of one (batch, head) segment.  `ids_q` / `ids_k` may be injected
     (e.g. the bucket ids another implementation produced) so that later stages can be
     compared even when a sign bit at |projection| ~ 0 was decided differently.
     caps = (cap_scale, kappa) runs Alg. 2 with its caps (see node_forward); every off-diagonal
-    problem then draws its own row subset T."""
+    problem then draws its own row subset T.  value_norm_sampling draws the sampled columns by
+    squared row norms of V (Lemma 2) instead of uniformly (Sec. 4)."""
     Q = np.asarray(Q, dtype=np.float64)
     n, d = Q.shape
     n_k = np.asarray(K).shape[0]
@@ -442,16 +507,17 @@ def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None
         ids_q, _ = bucket_ids(Q, W)
     if ids_k is None:
         ids_k, _ = bucket_ids(K, W)
+    wq = value_norm_weights(V) if value_norm_sampling else None
     if causal:
         assert n_k == n, "the causal mask is defined for a square attention matrix"
-        return causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=rows, caps=caps)
+        return causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=rows, caps=caps, wq=wq)
     mm = m if b < n_k else 0
-    smp = sample_indices(seed, g, 0, mm, n_k)
+    smp, sw = draw_samples(seed, g, 0, mm, n_k, wq)
     nc = None if caps is None else (caps[0], caps[1], row_subset(seed, g, 0, mm, n))
-    return node_forward(Q, K, V, ids_q, ids_k, smp, b, scale, rows=rows, caps=nc)
+    return node_forward(Q, K, V, ids_q, ids_k, smp, b, scale, rows=rows, caps=nc, sample_weights=sw)
 
 
-def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None, caps=None):
+def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None, caps=None, value_norm_sampling=False):
     """Q: (G, n, d); K, V: (G, n_k, d).  Returns out (G, n, d) and lse (G, n), fp64."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
@@ -461,7 +527,8 @@ def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None, caps=None)
     out = np.zeros((G, n, d), dtype=np.float64)
     lse = np.zeros((G, n), dtype=np.float64)
     for g in range(G):
-        out[g], lse[g] = segment_forward(Q[g], K[g], V[g], W, b, m, causal, n0, seed, g, scale, caps=caps)
+        out[g], lse[g] = segment_forward(Q[g], K[g], V[g], W, b, m, causal, n0, seed, g, scale, caps=caps,
+                                         value_norm_sampling=value_norm_sampling)
     return out, lse
 
 
@@ -483,10 +550,10 @@ def _dense_unnormalised(Q, K, ids_q, ids_k, samples, b, scale):
     return (M + (N / m) * c[None, :] * (1.0 - M)) * A
 
 
-def dense_weights(Q, K, ids_q, ids_k, b, m, scale, causal, n0, seed, g):
+def dense_weights(Q, K, ids_q, ids_k, b, m, scale, causal, n0, seed, g, wq=None):
     """Row-normalised weights W~ (n x n_k) with out = W~ V; causal problems are assembled quadrant by
     quadrant exactly as Fig. 2 / Alg. 4 split the matrix (causal_grid for the split points)."""
-    C = dense_coefficients(np.asarray(Q).shape[0], ids_q, ids_k, b, m, causal, n0, seed, g, n_k=np.asarray(K).shape[0])
+    C = dense_coefficients(np.asarray(Q).shape[0], ids_q, ids_k, b, m, causal, n0, seed, g, n_k=np.asarray(K).shape[0], wq=wq)
     U = C * np.exp(scale * (np.asarray(Q, np.float64) @ np.asarray(K, np.float64).T))
     return U / U.sum(axis=1, keepdims=True)
 
@@ -494,28 +561,33 @@ def dense_weights(Q, K, ids_q, ids_k, b, m, scale, causal, n0, seed, g):
 # --------------------------------------------------------------------------------------
 # Backward pass (tiny n only): derivative of the forward map, discrete choices held fixed
 # --------------------------------------------------------------------------------------
-def dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g, n_k=None):
+def dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g, n_k=None, wq=None):
     """C (n x n_k, entries >= 0) such that the forward pass is out = rownorm(C o A) V,
     lse = ln rowsum(C o A), A = exp(scale Q K^T).  C depends on Q and K only through the
     bucket ids: C_ij = 1 on the block mask M^H, (N/m) * multiplicity of j among the
     samples elsewhere (Alg. 2 lines 7 and 9 without caps), the lower triangle of ones in
-    an exact causal leaf, zero above the diagonal blocks of the recursion (Alg. 4)."""
+    an exact causal leaf, zero above the diagonal blocks of the recursion (Alg. 4).  wq: the keys'
+    integer weights when the columns are sampled by value norms (then the coefficient of a sampled key
+    is the sum of the weights 1 / (m p) of the samples that hit it)."""
     ids_q, ids_k = np.asarray(ids_q), np.asarray(ids_k)
     n_k = n if n_k is None else n_k
 
-    def block(iq, ik, node):
+    def block(iq, ik, node, wq_node=None):
         N = ik.shape[0]
         if b >= N:
             return np.ones((iq.shape[0], N))
         _, rank_q = stable_argsort(iq)
         _, rank_k = stable_argsort(ik)
         M = sortlsh_mask(rank_q, rank_k, b, query_block_size(iq.shape[0], N, b)).astype(np.float64)
-        smp = sample_indices(seed, g, node, m, N)
-        c = np.bincount(np.asarray(smp, dtype=np.int64), minlength=N).astype(np.float64)
-        return M + (N / max(m, 1)) * c[None, :] * (1.0 - M)
+        smp, sw = draw_samples(seed, g, node, m, N, wq_node)
+        if sw is None:
+            c = (N / max(m, 1)) * np.bincount(np.asarray(smp, dtype=np.int64), minlength=N).astype(np.float64)
+        else:
+            c = np.bincount(np.asarray(smp, dtype=np.int64), weights=sw, minlength=N)       # sum of the weights of the samples that hit a key
+        return M + c[None, :] * (1.0 - M)
 
     if not causal:
-        return block(ids_q, ids_k, 0)
+        return block(ids_q, ids_k, 0, wq)
     assert n_k == n
     L, leaf = causal_grid(n, n0)
     C = np.zeros((n, n))
@@ -531,7 +603,7 @@ def dense_coefficients(n, ids_q, ids_k, b, m, causal, n0, seed, g, n_k=None):
         part(a, h, 2 * node + 1)
         part(a + h, h, 2 * node + 2)
         if e > a + h:
-            C[a + h:e, a:a + h] = block(ids_q[a + h:e], ids_k[a:a + h], node)
+            C[a + h:e, a:a + h] = block(ids_q[a + h:e], ids_k[a:a + h], node, None if wq is None else wq[a:a + h])
 
     part(0, leaf << L, 0)
     return C

@@ -715,3 +715,82 @@ def test_alpha_closed_forms_and_explicit_loops():
             for j, x in zip(js, e):
                 col[j] += (x / tot) ** 2
         assert abs(O.alpha_diagnostic(Q, K, 0.7, causal=causal) - n * max(col)) < 1e-10
+
+
+# ------------------------------------------------------------------ sampling by value norms (Lemma 2)
+def test_value_norm_weights_are_cut_squared_norms():
+    rng = np.random.default_rng(4)
+    from paper_2310_05869_b200 import workloads as WL
+    V = WL.bf16_bits_to_f32(WL.f32_to_bf16_bits(rng.standard_normal((50, 64)).astype(np.float32)))     # bf16 values
+    wq = O.value_norm_weights(V)
+    exact = (V.astype(np.float64) ** 2).sum(axis=1)
+    assert wq.dtype == np.uint64
+    assert (np.abs(wq.astype(np.float64) / 4096.0 - exact) <= 64 * 2.0 ** -24 * exact + 1.0 / 4096.0).all()
+    assert O.value_norm_weights(np.zeros((3, 8)))[0] == 0
+    # coordinate order matters in fp32 and is the stated one: an explicit scalar loop gives the same integers
+    for i in range(5):
+        acc = np.float32(0.0)
+        for c in range(64):
+            acc = np.float32(acc + np.float32(V[i, c] * V[i, c]))
+        assert int(wq[i]) == int(math.floor(float(acc) * 4096.0))
+
+
+def test_value_norm_sampler_tiny_case_and_distribution():
+    # weights 1, 0, 3: cumulative 1, 1, 4; target floor(x * 4 / 2^32) in {0, 1, 2, 3} -> index 0 for 0, index 2 otherwise
+    idx, w = O.sample_by_value_norms(7, 1, 2, 4000, np.array([1, 0, 3], dtype=np.uint64))
+    assert set(idx.tolist()) == {0, 2}
+    assert abs((idx == 0).mean() - 0.25) < 0.03
+    np.testing.assert_allclose(w[idx == 0], 4.0 / (4000 * 1.0))
+    np.testing.assert_allclose(w[idx == 2], 4.0 / (4000 * 3.0))
+    x = O.philox4x32_10(np.array([[0, 1, 2, 2]], dtype=np.uint64), (7, 0))[0]
+    assert idx[0] == (0 if (int(x[0]) * 4) >> 32 == 0 else 2)
+    # all weights zero: the uniform sampler
+    i0, w0 = O.sample_by_value_norms(7, 1, 2, 16, np.zeros(10, dtype=np.uint64))
+    assert (i0 == O.sample_indices(7, 1, 2, 16, 10)).all() and (w0 == 10 / 16).all()
+    # chi-square against p_l = wq_l / total
+    rng = np.random.default_rng(9)
+    wq = rng.integers(0, 1000, 40).astype(np.uint64)
+    counts = np.zeros(40)
+    for seed in range(50):
+        counts += np.bincount(O.sample_by_value_norms(seed, 0, 0, 2000, wq)[0], minlength=40)
+    expect = 100000 * wq.astype(np.float64) / wq.sum()
+    nz = expect > 0
+    assert counts[~nz].sum() == 0
+    chi2 = ((counts[nz] - expect[nz]) ** 2 / expect[nz]).sum()
+    assert chi2 < 39 + 5 * math.sqrt(2 * 39)
+
+
+def test_value_norm_sampling_is_unbiased_and_dense_form_holds():
+    """E[sum_t w_t (1 - M) a_t v_t] = off-block numerator and E[sum_t w_t (1 - M) a_t] = off-block row sum
+    (Lemma 2 with w = 1 / (m p)); and for one seed the implied weights reproduce the output."""
+    rng = np.random.default_rng(21)
+    N, b, m, d = 32, 8, 6, 4
+    Q, K, _ = rand_qkv(rng, N, d)
+    V = rng.standard_normal((N, d)) * rng.uniform(0.2, 3.0, (N, 1))        # rows of very different norms
+    W = O.directions(d, 3, 2)
+    iq, _ = O.bucket_ids(Q, W); ik, _ = O.bucket_ids(K, W)
+    wq = O.value_norm_weights(V)
+    _, rank_q = O.stable_argsort(iq); _, rank_k = O.stable_argsort(ik)
+    M = O.sortlsh_mask(rank_q, rank_k, b)
+    A = np.exp(0.5 * (Q @ K.T))
+    off_sum = ((1 - M) * A).sum(axis=1)
+    off_num = ((1 - M) * A) @ V
+    blk_sum = (M * A).sum(axis=1)
+    blk_num = (M * A) @ V
+    dens, nums = [], []
+    trials = 6000
+    for seed in range(trials):
+        smp, sw = O.sample_by_value_norms(seed, 0, 0, m, wq)
+        o, l = O.node_forward(Q, K, V, iq, ik, smp, b, 0.5, sample_weights=sw)
+        dens.append(np.exp(l) - blk_sum)
+        nums.append(o * np.exp(l)[:, None] - blk_num)
+    dens, nums = np.array(dens), np.array(nums)
+    se = dens.std(axis=0) / math.sqrt(trials)
+    assert (np.abs(dens.mean(axis=0) - off_sum) <= 4.5 * se + 1e-12).all()
+    se = nums.std(axis=0) / math.sqrt(trials)
+    assert (np.abs(nums.mean(axis=0) - off_num) <= 4.5 * se + 1e-12).all()
+    for causal, n0 in ((False, 0), (True, 8)):
+        o, l = O.segment_forward(Q, K, V, W, b, m, causal, n0, 5, 1, scale=0.5, value_norm_sampling=True)
+        Wd = O.dense_weights(Q, K, iq, ik, b, m, 0.5, causal, n0, 5, 1, wq=wq)
+        np.testing.assert_allclose(Wd.sum(axis=1), 1.0, atol=1e-12)
+        np.testing.assert_allclose(Wd @ V, o, atol=1e-12)
