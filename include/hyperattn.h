@@ -102,6 +102,8 @@ typedef struct hyperattn_debug {
                             sorted query order */
   float* log2_tau;       /* float [G, NODES]: log2 of tau (Alg. 2 line 3) with the softmax scale applied, i.e.
                             ln(tau) / ln 2; minus infinity for a node without probe rows or unmasked entries */
+  /* sampling by value norms only (hyperattn_params.sampling): */
+  float* sample_log2w;   /* float [G, NODES, m]: log2 of the weight 1 / (m p_l) of every drawn column */
 } hyperattn_debug;
 
 typedef struct hyperattn_params {
@@ -154,7 +156,22 @@ typedef struct hyperattn_params {
                             inputs, forward only, not together with `precise`. */
   float cap_scale;       /* the constant (times eps^2) of Alg. 2 line 6; > 0 when capped */
   float kappa;           /* kappa of Alg. 2; > 0 when capped */
+  int sampling;          /* hyperattn_sampling: how the m residual columns of a sorted node are drawn.
+                            HYPERATTN_SAMPLE_UNIFORM (Sec. 4): uniformly, weight N/m each.
+                            HYPERATTN_SAMPLE_VALUE_NORMS (Lemma 2): key l with probability p_l proportional to
+                            ||V_l||^2 over the node's keys, weight 1 / (m p_l) in the numerator and in the row sum.
+                            The distribution is made of integers so that the indices are reproducible: the squared
+                            norm is accumulated in fp32 in coordinate order and cut to a multiple of 2^-12; draw j is
+                            the first key whose cumulative weight exceeds floor(x * total / 2^32), x the Philox word
+                            of the uniform sampler (counter (j >> 2, g, v, 2), word j & 3); all weights zero falls
+                            back to uniform.  Costs one more pass over V.  bf16 inputs, forward only, samples <= 512,
+                            not together with `precise` or `capped`. */
 } hyperattn_params;
+
+typedef enum hyperattn_sampling {
+  HYPERATTN_SAMPLE_UNIFORM = 0,
+  HYPERATTN_SAMPLE_VALUE_NORMS = 1
+} hyperattn_sampling;
 
 /* HyperAttention forward (Alg. 1-4 as specialised in Sec. 4) with bf16 inputs and
  * output, softmax scale 1/sqrt(d) and the library's private workspace. */

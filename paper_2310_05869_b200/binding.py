@@ -30,7 +30,7 @@ class HyperAttnError(RuntimeError):
 class _Debug(C.Structure):
     _fields_ = [("q_ids", C.c_void_p), ("k_ids", C.c_void_p), ("perm_q", C.c_void_p), ("perm_k", C.c_void_p),
                 ("rank_k", C.c_void_p), ("samples", C.c_void_p), ("near_zero_bits", C.c_void_p),
-                ("row_subset", C.c_void_p), ("log2_tau", C.c_void_p)]
+                ("row_subset", C.c_void_p), ("log2_tau", C.c_void_p), ("sample_log2w", C.c_void_p)]
 
 
 class _Params(C.Structure):
@@ -40,7 +40,8 @@ class _Params(C.Structure):
                 ("n0", C.c_int), ("seed", C.c_uint64), ("dtype", C.c_int), ("out_dtype", C.c_int),
                 ("softmax_scale", C.c_float), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("debug", C.POINTER(_Debug)), ("stream", C.c_void_p),
-                ("precise", C.c_int), ("n_k", C.c_int), ("capped", C.c_int), ("cap_scale", C.c_float), ("kappa", C.c_float)]
+                ("precise", C.c_int), ("n_k", C.c_int), ("capped", C.c_int), ("cap_scale", C.c_float), ("kappa", C.c_float),
+                ("sampling", C.c_int)]
 
 
 class _StageTimes(C.Structure):
@@ -124,7 +125,7 @@ def _debug_shapes(B, H, n, block, samples, causal, n0, n_k=None):
 
 
 def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_dtype=None, scale=0.0,
-            workspace=None, debug=False, stream=None, precise=False, caps=None):
+            workspace=None, debug=False, stream=None, precise=False, caps=None, value_norm_sampling=False):
     """HyperAttention forward on CUDA tensors q [B, H, n, d] and k, v [B, H, n_k, d] (bf16 or fp32).
     caps = (cap_scale, kappa) runs the row-sum estimate with the caps of Alg. 2.
     Returns (out, lse) or (out, lse, intermediates) when debug=True."""
@@ -147,6 +148,7 @@ def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_
     p.precise = int(bool(precise))
     if caps is not None:
         p.capped, p.cap_scale, p.kappa = 1, float(caps[0]), float(caps[1])
+    p.sampling = int(bool(value_norm_sampling))
     inter = None
     if debug:
         G, LV, NL, NODES = _debug_shapes(B, H, n, block, samples, causal, n0, n_k)
@@ -161,6 +163,7 @@ def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_
             "near_zero_bits": torch.zeros(1, dtype=torch.int64, device=dev),
             "row_subset": torch.full((G, max(NODES, 1), max(samples, 1)), -1, dtype=torch.int32, device=dev),
             "log2_tau": torch.full((G, max(NODES, 1)), float("nan"), dtype=torch.float32, device=dev),
+            "sample_log2w": torch.full((G, max(NODES, 1), max(samples, 1)), float("nan"), dtype=torch.float32, device=dev),
         }
         dbg = _Debug(*(inter[f].data_ptr() for f, _ in _Debug._fields_))
         p.debug = C.pointer(dbg)

@@ -8,7 +8,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libhyperattn.so")
-SOURCES = ["api.cu", "hash.cu", "sort.cu", "attn_mma.cu", "attn_tc.cu", "merge.cu", "noalloc.cu", "backward.cu", "caps.cu", "alpha.cu"]
+SOURCES = ["api.cu", "hash.cu", "sort.cu", "attn_mma.cu", "attn_tc.cu", "merge.cu", "noalloc.cu", "backward.cu", "caps.cu", "alpha.cu", "vnorm.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

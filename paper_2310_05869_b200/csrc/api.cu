@@ -15,6 +15,8 @@
 namespace hyperattn {
 cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st);
+cudaError_t launch_vnorm_sampling(const Geometry& g, const __nv_bfloat16* v, uint32_t* wq, unsigned long long* cum, int32_t* samples,
+                                  float* wlog, uint64_t seed, cudaStream_t st);
 cudaError_t launch_tau(const AttnArgs& at, const int32_t* tpos, float* ltau, cudaStream_t st);
 cudaError_t launch_backward(const AttnArgs& a, const void* out, int out_fp32, const float* lse, const void* dout,
                             float* delta, float* dq, float* dk, float* dv, void* dq_final, int dq_mode, float scale, int* status, cudaStream_t st);
@@ -85,12 +87,12 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
 }
 
 struct Plan {
-  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, tpos, ltau, part_o, part_lse, total;
+  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, tpos, ltau, vwq, vcum, swlog, part_o, part_lse, total;
   size_t delta, gacc;   // backward only: <dO, O> per row; fp32 gradient accumulators (bf16 gradients only)
 };
 
 // backward: 0 forward plan; 1 backward with fp32 gradients (accumulated in place); 2 backward with bf16 gradients
-Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = false) {
+Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = false, bool vnorm = false) {
   Plan pl;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
@@ -111,6 +113,9 @@ Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = f
   pl.samples = take((size_t)g.G * g.nodes * g.m * 4);
   pl.tpos = take(capped ? (size_t)g.G * g.nodes * g.m * 4 : 0);
   pl.ltau = take(capped ? (size_t)g.G * g.nodes * 4 : 0);
+  pl.vwq = take(vnorm ? (size_t)g.G * g.nk * 4 : 0);
+  pl.vcum = take(vnorm ? (size_t)g.G * ((size_t)g.nk + 1) * 8 : 0);
+  pl.swlog = take(vnorm ? (size_t)g.G * g.nodes * g.m * 4 : 0);
   const size_t part_rows = (g.L && !backward) ? (size_t)g.G * g.n + lvl_rows : 0;
   pl.part_o = take(part_rows * g.d * 4);
   pl.part_lse = take(part_rows * 4);
@@ -213,7 +218,14 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     if (is_fp32 || bw || p.precise) return HYPERATTN_UNSUPPORTED_SHAPE;     // bf16 forward with single bf16 weights only
   }
   if (p.precise && is_fp32) return HYPERATTN_UNSUPPORTED_SHAPE;
-  const Plan pl = make_plan(g, is_fp32, bw ? (bw->grad_dtype == HYPERATTN_FP32 ? 1 : 2) : 0, capped);
+  // sampled columns by squared row norms of V (Lemma 2) instead of uniformly (Sec. 4)
+  if (p.sampling != HYPERATTN_SAMPLE_UNIFORM && p.sampling != HYPERATTN_SAMPLE_VALUE_NORMS) return HYPERATTN_INVALID_ARGUMENT;
+  const bool vnorm = p.sampling == HYPERATTN_SAMPLE_VALUE_NORMS && g.sorted && g.m > 0;
+  if (p.sampling == HYPERATTN_SAMPLE_VALUE_NORMS) {
+    if (is_fp32 || bw || p.precise || p.capped) return HYPERATTN_UNSUPPORTED_SHAPE;
+    if (g.m > kMaxWeightedSamples) return HYPERATTN_UNSUPPORTED_SHAPE;
+  }
+  const Plan pl = make_plan(g, is_fp32, bw ? (bw->grad_dtype == HYPERATTN_FP32 ? 1 : 2) : 0, capped, vnorm);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
   int dev = 0;
@@ -287,7 +299,14 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     {
       // (the samples of Alg. 2 line 4 are drawn by extra blocks of this launch)
       StageScope sc(st, HYPERATTN_STAGE_SORT_SCAN, 1);
-      HA_CHECK(launch_sort_scan(g, ws, true, p.seed, st));
+      HA_CHECK(launch_sort_scan(g, ws, !vnorm, p.seed, st));
+    }
+    if (vnorm) {
+      StageScope sc(st, HYPERATTN_STAGE_SAMPLE, 3);
+      HA_CHECK(launch_vnorm_sampling(g, v16, reinterpret_cast<uint32_t*>(base + pl.vwq), reinterpret_cast<unsigned long long*>(base + pl.vcum),
+                                     ws.samples, reinterpret_cast<float*>(base + pl.swlog), p.seed, st));
+      if (dbg && dbg->sample_log2w)
+        HA_CHECK(cudaMemcpyAsync(dbg->sample_log2w, base + pl.swlog, (size_t)g.G * g.nodes * g.m * 4, cudaMemcpyDeviceToDevice, st));
     }
     {
       StageScope sc(st, HYPERATTN_STAGE_SORT_SCATTER, 1);
@@ -317,6 +336,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   a.precise = p.precise != 0;
   a.capped = capped;
   a.cap_scale = p.cap_scale; a.log2_kappa = capped ? std::log2(p.kappa) : 0.f; a.ltau = ws.ltau;
+  a.sample_wlog = vnorm ? reinterpret_cast<const float*>(base + pl.swlog) : nullptr;
   a.direct = g.L == 0;
   a.dense_causal = g.causal;
   a.tiles_per_block = (g.bq + kTileQ - 1) / kTileQ;
@@ -519,7 +539,8 @@ int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes) {
   Geometry g;
   const int rc = build_geometry(*p, g);
   if (rc) return rc;
-  *bytes = make_plan(g, p->dtype == HYPERATTN_FP32, 0, p->capped != 0 && g.sorted && g.m > 0).total;
+  *bytes = make_plan(g, p->dtype == HYPERATTN_FP32, 0, p->capped != 0 && g.sorted && g.m > 0,
+                     p->sampling == HYPERATTN_SAMPLE_VALUE_NORMS && g.sorted && g.m > 0).total;
   return HYPERATTN_OK;
 }
 

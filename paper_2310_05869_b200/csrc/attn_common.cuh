@@ -17,6 +17,7 @@
 namespace hyperattn {
 
 constexpr int kMaxLevels = 24;
+constexpr int kMaxWeightedSamples = 512;   // sampled columns with weights of their own (sampling by value norms): table size
 constexpr int kMaxNodeKeys = 2048;   // 2 * (b rounded up to 128) + (m rounded up to 128) must fit the key table
 
 struct AttnArgs {
@@ -35,6 +36,9 @@ struct AttnArgs {
   float cap_scale;                   // the constant of line 6: C_i = cap_scale m / (N ln N) (masked_i + tau / kappa)
   float log2_kappa;
   const float* ltau;                 // [G, nodes] log2 tau in the scaled domain
+  // sampled columns drawn with probabilities of their own (Lemma 2): log2 of the weight 1 / (m p) of every draw,
+  // [G, nodes, m]; null: uniform sampling, weight N / m
+  const float* sample_wlog;
   // dense (leaf) tiles
   int dense_causal;
   int tiles_per_leaf, leaves_per_seg, n_leaf_tiles;

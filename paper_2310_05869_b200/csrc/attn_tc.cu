@@ -324,6 +324,7 @@ struct PairDesc {
   int node;            // node: heap index
   int nq_node, bq;     // node: query rows of the node, rows per group of sorted queries
   int nbA, nbB, nsmp;  // node: key tiles of block A, of block B (0 if shared), of the samples
+  float bias_max;      // node, weighted sampling: the largest log2 weight among the samples
   int ntiles;          // key tiles walked
   size_t orow_base; int odelta; int partial;
 };
@@ -368,7 +369,8 @@ struct Cfg {
   static constexpr int kOffDesc = (kOffMisc + 16 + 15) / 16 * 16;   // ItemDesc [2], one per table set
   static constexpr int kOffStage = (kOffDesc + 2 * kDescBytes + 127) / 128 * 128;
   static constexpr int kOffOnes = (kOffStage + ((D == 64) ? 8 : 4) * kStageWarp + 1023) / 1024 * 1024;   // [TK keys x 128 B] of bf16 1.0
-  static constexpr int kTotal = kOnes ? kOffOnes + TK * 128 : kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;
+  static constexpr int kOffBias = kOnes ? kOffOnes + TK * 128 : kOffStage + ((D == 64) ? 8 : 4) * kStageWarp;   // float [2][kMaxWeightedSamples]: log2 weight of every sampled column (weighted sampling only)
+  static constexpr int kTotal = kOffBias + 2 * kMaxWeightedSamples * 4;
   static_assert(kTotal <= 232448, "shared memory");
   static_assert(D == 64 || 4 * kStageWarp <= kMaxNodeKeys * 4, "staging of query tile 0 must fit one key-row table");
   static constexpr int kTmemCols = 512;
@@ -614,10 +616,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       // Alg. 2 with caps (sorted nodes only): the masked row sum (block part) is complete when the first
       // sampled tile starts; from then on every sampled weight enters the row sum as min(weight, (N/m) C_i),
       // C_i = cap_scale m / (N ln N) (masked_i + tau / kappa), while the numerator keeps the weight itself.
-      const bool capped_item = CAPPED && t.mode == 1 && g.m > 0;
+      const bool capped_item = CAPPED && t.mode == 1 && g.m > 0 && a.capped;
       float lblk = 0.f;             // masked row sum in units of 2^m_ref
       bool in_samples = false;
       float capfac = 0.f, lfloor = -INFINITY;     // (N/m) cap_scale m / (N ln N); log2(tau / kappa)
+      // weighted sampling (columns drawn by value norms): every sampled column carries its own log2 weight
+      const bool weighted_item = CAPPED && t.mode == 1 && a.sample_wlog != nullptr;
+      const float* s_bias = reinterpret_cast<const float*>(smem + C::kOffBias) + set * kMaxWeightedSamples;
       if (capped_item) {
         capfac = a.cap_scale / (logf((float)t.nk));
         lfloor = a.ltau[(size_t)t.seg * g.nodes + t.node] - a.log2_kappa;
@@ -637,7 +642,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         tc_fence_after();
         // mask kind of this (query tile, key tile): uniform over the warpgroup
         const bool table = (tile_masked >> j) & 1u;
-        const float ubias = (t.mode == 1 && j >= t.nbA + t.nbB) ? wlog : 0.f;
+        // (weighted sampling: the tile's columns have weights of their own; the largest one stands in where one number is needed)
+        const bool weighted_tile = weighted_item && j >= t.nbA + t.nbB;
+        const float ubias = (t.mode == 1 && j >= t.nbA + t.nbB) ? (weighted_tile ? t.bias_max : wlog) : 0.f;
         const bool dense_mask = t.mode != 1 && ((j * TK + TK > t.nk) || (t.causal && j * TK + TK - 1 > q.row0));
         // The 64 scores of this row are read from TMEM once; then (1) the row maximum, (2)
         // exponentials, row sums and the bf16 P written over the first half of the S buffer.
@@ -770,13 +777,32 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
             }
             tmem_st16(sbase + c * 16, p);
           };
+          // weighted tiles: x = score * scale + (the column's log2 weight - reference)
+          const float* bias_tile = s_bias + (j - (t.nbA + t.nbB)) * TK;
+          const uint64_t nref2 = pack_f2(off - ubias, off - ubias);
+          auto chunk_exp_weighted = [&](const uint32_t (&r)[32], int c) {
+            uint32_t p[16];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float2 bb = *reinterpret_cast<const float2*>(bias_tile + c * 32 + e);
+              float x0, x1;
+              unpack_f2(ffma2(pack_u2(r[e], r[e + 1]), sc2, fadd2(pack_f2(bb.x, bb.y), nref2)), x0, x1);
+              const float p0 = ex2(x0), p1 = ex2(x1);
+              lt2 = fadd2(lt2, pack_f2(p0, p1));
+              const uint32_t w = pack2(p0, p1);
+              if constexpr (!C::kOnes)
+                asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}" : "+f"(lrta), "+f"(lrtb) : "r"(w));
+              p[e >> 1] = w;
+            }
+            tmem_st16(sbase + c * 16, p);
+          };
           HA_T0(tc2);
           if constexpr (PRECISE) tmem_ld32_wait(rb);     // the lo halves overwrite the second half of the scores
-          if (CAPPED && capped_tile) chunk_exp_capped(ra, 0); else chunk_exp(ra, 0);
+          if (CAPPED && capped_tile) chunk_exp_capped(ra, 0); else if (CAPPED && weighted_tile) chunk_exp_weighted(ra, 0); else chunk_exp(ra, 0);
           HA_LACC(a_c2, tc2);
           HA_T0(tc3);
           tmem_ld32_wait(rb);
-          if (CAPPED && capped_tile) chunk_exp_capped(rb, 1); else chunk_exp(rb, 1);
+          if (CAPPED && capped_tile) chunk_exp_capped(rb, 1); else if (CAPPED && weighted_tile) chunk_exp_weighted(rb, 1); else chunk_exp(rb, 1);
           HA_LACC(a_c3, tc3);
           float lt0, lt1;
           unpack_f2((CAPPED && capped_tile) ? ltu2 : lt2, lt0, lt1);
@@ -1136,6 +1162,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           for (int wd = (nblk >> 5) + lane; wd < (ncols >> 5); wd += 32) { s_mask[wd] = 0; s_mask[MW + wd] = 0; }
           __syncwarp();
           int nfront = 0, nback = 0;                      // unmasked samples placed from the front, masked ones from the back
+          float* s_bias = reinterpret_cast<float*>(smem + C::kOffBias) + set * kMaxWeightedSamples;
+          const float* swl = a.sample_wlog ? a.sample_wlog + ((size_t)t.seg * g.nodes + t.node) * g.m : nullptr;
+          float bmax = -INFINITY;
           const unsigned lt_mask = (1u << lane) - 1u;
           for (int c00 = lane; c00 < ncols - nblk; c00 += 32 * UB) {
             int l[UB], blk[UB];
@@ -1161,10 +1190,20 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
                 else pos = nblk + g.m - 1 - (nback + __popc(bb & lt_mask));
                 nfront += __popc(bf); nback += __popc(bb);
                 s_kidx[pos] = segrow_k + (valid ? t.k0 + l[u] : 0);
+                if (CAPPED && swl) {                      // weighted sampling: the column's own log2 weight travels with it
+                  const float wl = valid ? swl[c] : 0.f;
+                  s_bias[pos - nblk] = wl;
+                  if (valid) bmax = fmaxf(bmax, wl);
+                }
                 if (m0) atomicOr(&s_mask[pos >> 5], 1u << (pos & 31));
                 if (m1) atomicOr(&s_mask[MW + (pos >> 5)], 1u << (pos & 31));
               }
             }
+          }
+          if (CAPPED && swl) {
+#pragma unroll
+            for (int o = 16; o; o >>= 1) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, o));
+            if (lane == 0) reinterpret_cast<ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes)->t.bias_max = bmax;
           }
         }
       }
@@ -1394,8 +1433,8 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
     kernel<<<grid, 384, smem_bytes, st>>>(a, maps, status);
     return cudaGetLastError();
   };
-  if (a.capped) {
-    if (a.precise) return cudaErrorInvalidValue;
+  if (a.capped || a.sample_wlog) {
+    if (a.precise || (a.capped && a.sample_wlog)) return cudaErrorInvalidValue;
     if (a.g.d == 64) return go(attn_tc_kernel<64, false, false, true>, Cfg<64>::kTotal);
     if (!a.direct) return go(attn_tc_kernel<128, true, false, true>, Cfg<128>::kTotal);
     return go(attn_tc_kernel<128, false, false, true>, Cfg<128>::kTotal);
