@@ -92,7 +92,7 @@ def _seed_key(seed):
     return (seed & 0xFFFFFFFF, seed >> 32)
 
 
-def directions(d, r, seed):
+def directions(d, r, seed, node=0):
     """The r random directions of the Hamming-sorted LSH (Def. 1; Alg. 1 line 2).
 
     The paper cites the construction without printing it; the reading taken is r
@@ -102,11 +102,15 @@ def directions(d, r, seed):
     key = seed) gives words x0..x3; u_i = (x_i + 0.5) / 2^32; Box-Muller on (u0, u1)
     and on (u2, u3) gives normals 4c .. 4c+3 as (rho cos, rho sin) pairs.  The fp64
     result is rounded once to fp32 (the precision the directions are stored in).
+    `node` (variant with fresh directions for every recursion node, which the paper neither
+    prescribes nor excludes): the stream of node v has counter (c, 0, v, 1); node 0 is the
+    shared set.
     """
     total = d * r
     calls = (total + 3) // 4
     ctr = np.zeros((calls, 4), dtype=np.uint64)
     ctr[:, 0] = np.arange(calls, dtype=np.uint64)
+    ctr[:, 2] = node
     ctr[:, 3] = DOMAIN_DIRECTIONS
     x = philox4x32_10(ctr, _seed_key(seed)).astype(np.float64)
     u = (x + 0.5) * 2.0 ** -32
@@ -436,6 +440,29 @@ def draw_samples(seed, g, node, m, N, wq=None):
     return sample_by_value_norms(seed, g, node, m, wq)
 
 
+def node_bucket_ids(Q, K, d, r, seed, n0):
+    """Bucket ids when every recursion node of a causal call hashes with directions of its own
+    (directions(.., node=v)): two (L, n) arrays; entry (l, i) of the first is the id of query row i
+    in the level-l node whose second half holds it, entry (l, i) of the second the id of key row i in
+    the level-l node whose first half holds it (a row is on one side of exactly one node per level;
+    the other entries are left at zero)."""
+    n = Q.shape[0]
+    L, leaf = causal_grid(n, n0)
+    iq = np.zeros((L, n), dtype=np.uint8)
+    ik = np.zeros((L, n), dtype=np.uint8)
+    for level in range(L):
+        s = leaf << (L - 1 - level)
+        for j in range(1 << level):
+            q0, k0 = (2 * j + 1) * s, 2 * j * s
+            e = min(q0 + s, n)
+            if e <= q0:
+                continue
+            W = directions(d, r, seed, node=heap_node(level, j))
+            iq[level, q0:e] = bucket_ids(Q[q0:e], W)[0]
+            ik[level, k0:k0 + s] = bucket_ids(K[k0:k0 + s], W)[0]
+    return iq, ik
+
+
 def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, caps=None, wq=None):
     """Causal HyperAttention.  A part that is a single leaf gets exact causal attention (the paper
     recurses until the length falls below a base size and uses an exact kernel there).  A larger
@@ -451,6 +478,8 @@ def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, c
     want = np.arange(n) if rows is None else np.asarray(rows, dtype=np.int64)
     out = np.zeros((want.size, V.shape[1]), dtype=np.float64)
     lse = np.zeros(want.size, dtype=np.float64)
+    ids_q, ids_k = np.asarray(ids_q), np.asarray(ids_k)
+    per_level = ids_q.ndim == 2                       # (L, n): ids from directions of the node's own (node_bucket_ids)
 
     def part(a, S, node, sel):
         """rows want[sel] (all inside [a, a + S)) of the causal problem on rows [a, min(a + S, n))"""
@@ -471,7 +500,10 @@ def causal_forward(Q, K, V, ids_q, ids_k, b, m, scale, n0, seed, g, rows=None, c
             mm = m if b < h else 0
             smp, sw = draw_samples(seed, g, node, mm, h, None if wq is None else wq[a:a + h])
             nc = None if caps is None else (caps[0], caps[1], row_subset(seed, g, node, mm, e - (a + h)))
-            o21, l21 = node_forward(Q[a + h:e], K[a:a + h], V[a:a + h], ids_q[a + h:e], ids_k[a:a + h], smp, b, scale, rows=r2, caps=nc,
+            level = (node + 1).bit_length() - 1
+            iq = ids_q[level, a + h:e] if per_level else ids_q[a + h:e]
+            ik = ids_k[level, a:a + h] if per_level else ids_k[a:a + h]
+            o21, l21 = node_forward(Q[a + h:e], K[a:a + h], V[a:a + h], iq, ik, smp, b, scale, rows=r2, caps=nc,
                                     sample_weights=sw)
             o22, l22 = out[second].copy(), lse[second].copy()
             l = np.logaddexp(l21, l22)
@@ -491,22 +523,29 @@ def heap_node(level, j):
 # Whole forward pass
 # --------------------------------------------------------------------------------------
 def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None,
-                    ids_q=None, ids_k=None, caps=None, value_norm_sampling=False):
+                    ids_q=None, ids_k=None, caps=None, value_norm_sampling=False, node_directions=False):
     """Forward pass of one (batch, head) segment.  `ids_q` / `ids_k` may be injected
     (e.g. the bucket ids another implementation produced) so that later stages can be
     compared even when a sign bit at |projection| ~ 0 was decided differently.
     caps = (cap_scale, kappa) runs Alg. 2 with its caps (see node_forward); every off-diagonal
     problem then draws its own row subset T.  value_norm_sampling draws the sampled columns by
-    squared row norms of V (Lemma 2) instead of uniformly (Sec. 4)."""
+    squared row norms of V (Lemma 2) instead of uniformly (Sec. 4).  node_directions (causal calls
+    with at least one level): every recursion node hashes with directions of its own, and injected
+    ids are (L, n) arrays as node_bucket_ids returns them."""
     Q = np.asarray(Q, dtype=np.float64)
     n, d = Q.shape
     n_k = np.asarray(K).shape[0]
     if scale is None:
         scale = 1.0 / math.sqrt(d)
-    if ids_q is None:
-        ids_q, _ = bucket_ids(Q, W)
-    if ids_k is None:
-        ids_k, _ = bucket_ids(K, W)
+    if node_directions and causal and causal_grid(n, n0)[0] > 0:
+        if ids_q is None or ids_k is None:
+            r = np.asarray(W).shape[1]
+            ids_q, ids_k = node_bucket_ids(Q, np.asarray(K, dtype=np.float64), d, r, seed, n0)
+    else:
+        if ids_q is None:
+            ids_q, _ = bucket_ids(Q, W)
+        if ids_k is None:
+            ids_k, _ = bucket_ids(K, W)
     wq = value_norm_weights(V) if value_norm_sampling else None
     if causal:
         assert n_k == n, "the causal mask is defined for a square attention matrix"
@@ -517,7 +556,8 @@ def segment_forward(Q, K, V, W, b, m, causal, n0, seed, g, scale=None, rows=None
     return node_forward(Q, K, V, ids_q, ids_k, smp, b, scale, rows=rows, caps=nc, sample_weights=sw)
 
 
-def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None, caps=None, value_norm_sampling=False):
+def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None, caps=None, value_norm_sampling=False,
+            node_directions=False):
     """Q: (G, n, d); K, V: (G, n_k, d).  Returns out (G, n, d) and lse (G, n), fp64."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
@@ -528,7 +568,7 @@ def forward(Q, K, V, b, m, r, causal=False, n0=0, seed=0, scale=None, caps=None,
     lse = np.zeros((G, n), dtype=np.float64)
     for g in range(G):
         out[g], lse[g] = segment_forward(Q[g], K[g], V[g], W, b, m, causal, n0, seed, g, scale, caps=caps,
-                                         value_norm_sampling=value_norm_sampling)
+                                         value_norm_sampling=value_norm_sampling, node_directions=node_directions)
     return out, lse
 
 

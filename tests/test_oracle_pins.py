@@ -794,3 +794,42 @@ def test_value_norm_sampling_is_unbiased_and_dense_form_holds():
         Wd = O.dense_weights(Q, K, iq, ik, b, m, 0.5, causal, n0, 5, 1, wq=wq)
         np.testing.assert_allclose(Wd.sum(axis=1), 1.0, atol=1e-12)
         np.testing.assert_allclose(Wd @ V, o, atol=1e-12)
+
+
+# ------------------------------------------------------------------ directions of the node's own
+def test_node_directions_streams_and_bookkeeping():
+    """Node 0 is the shared set; other nodes are independent standard normals; with single-block nodes the ids do not
+    matter and the recursion is still exact; with sorted nodes the result is the one rebuilt by hand from node_forward
+    on the root's own ids."""
+    assert np.array_equal(O.directions(16, 5, 3, node=0), O.directions(16, 5, 3))
+    w1, w2 = O.directions(64, 8, 3, node=1), O.directions(64, 8, 3, node=2)
+    assert not np.array_equal(w1, w2) and abs(np.corrcoef(w1.ravel(), w2.ravel())[0, 1]) < 0.15
+    assert abs(w1.mean()) < 0.15 and abs(w1.std() - 1.0) < 0.15
+    x = O.philox4x32_10(np.array([[0, 0, 2, 1]], dtype=np.uint64), (3, 0))[0].astype(np.float64)
+    u = (x + 0.5) * 2.0 ** -32
+    assert abs(float(w2.ravel()[0]) - math.sqrt(-2.0 * math.log(u[0])) * math.cos(2.0 * math.pi * u[1])) < 1e-6
+    rng = np.random.default_rng(12)
+    n, n0, d = 64, 8, 5
+    Q, K, V = rand_qkv(rng, n, d)
+    bo, bl = brute_attention(Q, K, V, 0.5, True)
+    o, l = O.forward(Q[None], K[None], V[None], b=n, m=4, r=3, causal=True, n0=n0, seed=2, scale=0.5, node_directions=True)
+    np.testing.assert_allclose(o[0], bo, atol=1e-11)
+    # sorted nodes: the ids of level l, node j come from directions(.., node) and nothing else
+    iq, ik = O.node_bucket_ids(Q, K, d, 3, 2, n0)
+    L, leaf = O.causal_grid(n, n0)
+    assert iq.shape == (L, n)
+    W3 = O.directions(d, 3, 2, node=O.heap_node(1, 1))                 # level 1, second node: queries [48, 64), keys [32, 48)
+    assert np.array_equal(iq[1, 48:64], O.bucket_ids(Q[48:64], W3)[0]) and np.array_equal(ik[1, 32:48], O.bucket_ids(K[32:48], W3)[0])
+    # one level, rebuilt by hand: second-half rows merge the node's estimate (root's own ids) with exact causal attention
+    n1 = 2 * n0
+    o, l = O.segment_forward(Q[:n1], K[:n1], V[:n1], O.directions(d, 3, 2), 2, 5, True, n0, 2, 0, scale=0.5, node_directions=True)
+    iq1, ik1 = O.node_bucket_ids(Q[:n1], K[:n1], d, 3, 2, n0)
+    o21, l21 = O.node_forward(Q[n0:n1], K[:n0], V[:n0], iq1[0, n0:], ik1[0, :n0], O.sample_indices(2, 0, 0, 5, n0), 2, 0.5)
+    o22, l22 = brute_attention(Q[n0:n1], K[n0:n1], V[n0:n1], 0.5, True)
+    lm = np.logaddexp(l21, l22)
+    np.testing.assert_allclose(l[n0:], lm, atol=1e-12)
+    np.testing.assert_allclose(o[n0:], o21 * np.exp(l21 - lm)[:, None] + o22 * np.exp(l22 - lm)[:, None], atol=1e-12)
+    np.testing.assert_allclose(o[:n0], brute_attention(Q[:n0], K[:n0], V[:n0], 0.5, True)[0], atol=1e-12)
+    # and deeper recursions differ from the shared-directions result (the nodes below the root hash differently)
+    o_nd = O.segment_forward(Q, K, V, O.directions(d, 3, 2), 4, 5, True, n0, 2, 0, scale=0.5, node_directions=True)[0]
+    assert not np.allclose(o_nd, O.segment_forward(Q, K, V, O.directions(d, 3, 2), 4, 5, True, n0, 2, 0, scale=0.5)[0])
