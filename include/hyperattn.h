@@ -166,6 +166,13 @@ typedef struct hyperattn_params {
                             of the uniform sampler (counter (j >> 2, g, v, 2), word j & 3); all weights zero falls
                             back to uniform.  Costs one more pass over V.  bf16 inputs, forward only, samples <= 512,
                             not together with `precise` or `capped`. */
+  int node_directions;   /* 1 (causal calls): every recursion node hashes its queries and keys with directions of its own
+                            (Philox counter (c, 0, v, 1) for node v; node 0 is the shared set) instead of one set per
+                            call.  The paper is silent on this; one shared set is the default.  Every row is then hashed
+                            once per level, and the exported bucket ids are [LV, G, n]: entry (l, g, i) of q_ids is the id
+                            of query row i in the level-l node whose second half holds it, of k_ids the id of key row i in
+                            the level-l node whose first half holds it (other entries are not written).  Forward only, at
+                            most 4095 nodes. */
 } hyperattn_params;
 
 typedef enum hyperattn_sampling {
@@ -228,6 +235,8 @@ int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes);
 /* Host-side: writes the d x hash_bits direction matrix of Def. 1's hash (row-major,
  * entry [k*hash_bits + t] = coordinate k of direction t) that a call with this seed uses. */
 int hyperattn_get_projections(int d, int hash_bits, uint64_t seed, float* host_out);
+/* The same for the directions of recursion node `node`'s own (hyperattn_params.node_directions). */
+int hyperattn_get_node_projections(int d, int hash_bits, uint64_t seed, int node, float* host_out);
 
 /* Synchronises `stream` and reports the device status word (0, or
  * HYPERATTN_DEVICE_TIMEOUT if a kernel's bounded wait gave up since the last query) and

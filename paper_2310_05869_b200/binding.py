@@ -20,7 +20,7 @@ EXPORTS = ["hyperattn_forward", "hyperattn_forward_ex", "hyperattn_forward_host"
            "hyperattn_get_projections", "hyperattn_last_device_status", "hyperattn_profile_enable",
            "hyperattn_profile_reset", "hyperattn_profile_read", "hyperattn_release",
            "hyperattn_status_string", "hyperattn_version", "hyperattn_sortlsh_noalloc",
-           "hyperattn_alpha", "hyperattn_alpha_workspace_bytes"]
+           "hyperattn_alpha", "hyperattn_alpha_workspace_bytes", "hyperattn_get_node_projections"]
 
 
 class HyperAttnError(RuntimeError):
@@ -41,7 +41,7 @@ class _Params(C.Structure):
                 ("softmax_scale", C.c_float), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("debug", C.POINTER(_Debug)), ("stream", C.c_void_p),
                 ("precise", C.c_int), ("n_k", C.c_int), ("capped", C.c_int), ("cap_scale", C.c_float), ("kappa", C.c_float),
-                ("sampling", C.c_int)]
+                ("sampling", C.c_int), ("node_directions", C.c_int)]
 
 
 class _StageTimes(C.Structure):
@@ -64,6 +64,8 @@ def lib() -> C.CDLL:
         L.hyperattn_workspace_bytes.argtypes = [C.POINTER(_Params), C.POINTER(C.c_size_t)]
         L.hyperattn_get_projections.restype = C.c_int
         L.hyperattn_get_projections.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_void_p]
+        L.hyperattn_get_node_projections.restype = C.c_int
+        L.hyperattn_get_node_projections.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_int, C.c_void_p]
         L.hyperattn_last_device_status.restype = C.c_int
         L.hyperattn_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
         L.hyperattn_profile_enable.argtypes = [C.c_int]
@@ -125,7 +127,8 @@ def _debug_shapes(B, H, n, block, samples, causal, n0, n_k=None):
 
 
 def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_dtype=None, scale=0.0,
-            workspace=None, debug=False, stream=None, precise=False, caps=None, value_norm_sampling=False):
+            workspace=None, debug=False, stream=None, precise=False, caps=None, value_norm_sampling=False,
+            node_directions=False):
     """HyperAttention forward on CUDA tensors q [B, H, n, d] and k, v [B, H, n_k, d] (bf16 or fp32).
     caps = (cap_scale, kappa) runs the row-sum estimate with the caps of Alg. 2.
     Returns (out, lse) or (out, lse, intermediates) when debug=True."""
@@ -149,13 +152,15 @@ def forward(q, k, v, block, samples, hash_bits, causal=False, n0=0, seed=0, out_
     if caps is not None:
         p.capped, p.cap_scale, p.kappa = 1, float(caps[0]), float(caps[1])
     p.sampling = int(bool(value_norm_sampling))
+    p.node_directions = int(bool(node_directions))
     inter = None
     if debug:
         G, LV, NL, NODES = _debug_shapes(B, H, n, block, samples, causal, n0, n_k)
         dev = q.device
+        id_sets = (LV,) if (node_directions and causal and NODES > 0) else ()
         inter = {
-            "q_ids": torch.zeros((G, n), dtype=torch.uint8, device=dev),
-            "k_ids": torch.zeros((G, n_k), dtype=torch.uint8, device=dev),
+            "q_ids": torch.zeros(id_sets + (G, n), dtype=torch.uint8, device=dev),
+            "k_ids": torch.zeros(id_sets + (G, n_k), dtype=torch.uint8, device=dev),
             "perm_q": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
             "perm_k": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
             "rank_k": torch.full((LV, G, NL), -1, dtype=torch.int32, device=dev),
@@ -256,9 +261,12 @@ def workspace_bytes(B, H, n, d, block, samples, hash_bits, causal=False, n0=0, d
     return int(nbytes.value)
 
 
-def get_projections(d: int, hash_bits: int, seed: int) -> np.ndarray:
+def get_projections(d: int, hash_bits: int, seed: int, node: int = 0) -> np.ndarray:
     w = np.zeros((d, hash_bits), dtype=np.float32)
-    _check(lib().hyperattn_get_projections(d, hash_bits, seed, w.ctypes.data), "hyperattn_get_projections")
+    if node:
+        _check(lib().hyperattn_get_node_projections(d, hash_bits, C.c_uint64(seed), node, w.ctypes.data), "hyperattn_get_node_projections")
+    else:
+        _check(lib().hyperattn_get_projections(d, hash_bits, seed, w.ctypes.data), "hyperattn_get_projections")
     return w
 
 

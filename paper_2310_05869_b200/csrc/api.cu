@@ -87,7 +87,7 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
 }
 
 struct Plan {
-  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, tpos, ltau, vwq, vcum, swlog, part_o, part_lse, total;
+  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, tpos, ltau, vwq, vcum, swlog, wnodes, part_o, part_lse, total;
   size_t delta, gacc;   // backward only: <dO, O> per row; fp32 gradient accumulators (bf16 gradients only)
 };
 
@@ -103,8 +103,10 @@ Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = f
   pl.q16lo = take(is_fp32 ? tensor16 : 0);
   pl.k16lo = take(is_fp32 ? tensor16k : 0);
   const size_t lvl_rows = (size_t)g.levels * g.G * g.nl;
-  pl.ids = take(g.sorted ? (size_t)g.G * ((size_t)g.n + g.nk) : 0);
-  pl.hist = take(g.sorted ? (size_t)g.G * (g.chunks_per_seg + g.chunks_per_seg_k) * kBuckets * 4 : 0);
+  const size_t id_sets = g.node_dirs ? g.levels : 1;     // directions of the nodes' own: ids and histograms once per level
+  pl.ids = take(g.sorted ? id_sets * g.G * ((size_t)g.n + g.nk) : 0);
+  pl.hist = take(g.sorted ? id_sets * g.G * (g.chunks_per_seg + g.chunks_per_seg_k) * kBuckets * 4 : 0);
+  pl.wnodes = take(g.node_dirs ? (size_t)g.nodes * g.d * g.r * 4 : 0);
   const size_t chunks_per_level = g.sorted ? (size_t)side_cpl(g, 0) + side_cpl(g, 1) : 0;
   pl.offs = take((size_t)g.levels * g.G * chunks_per_level * kBuckets * 4);
   pl.perm_q = take(g.sorted ? lvl_rows * 4 : 0);
@@ -126,11 +128,12 @@ Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = f
 }
 
 // ---- direction matrix (Def. 1): Philox + Box-Muller in fp64, rounded once to fp32 -------------
-void make_directions(int d, int r, uint64_t seed, float* w) {
+// node: 0 for the shared set; v for the directions of recursion node v's own (counter word 2)
+void make_directions(int d, int r, uint64_t seed, float* w, uint32_t node = 0) {
   const int total = d * r, calls = (total + 3) / 4;
   const double two_pi = 6.283185307179586476925286766559;
   for (int c = 0; c < calls; ++c) {
-    const Philox4 x = philox4x32_10((uint32_t)c, 0u, 0u, kDomainDirections, (uint32_t)seed, (uint32_t)(seed >> 32));
+    const Philox4 x = philox4x32_10((uint32_t)c, 0u, node, kDomainDirections, (uint32_t)seed, (uint32_t)(seed >> 32));
     double u[4], z[4];
     for (int i = 0; i < 4; ++i) u[i] = ((double)x.x[i] + 0.5) * (1.0 / 4294967296.0);
     for (int a = 0; a < 4; a += 2) {
@@ -163,6 +166,10 @@ std::vector<StageEvents> g_events;
 std::vector<cudaEvent_t> g_event_pool;
 int g_profile_calls = 0;
 struct { int d = 0, r = 0; uint64_t seed = 0; bool valid = false; float w[128 * 8]; } g_wcache;
+// directions of the recursion nodes' own, [nodes, d, r]; kept on the host (it is copied to the device by every call that
+// uses it, possibly from inside a captured graph, so the buffer only ever grows and is never freed before release)
+struct { int d = 0, r = 0, nodes = 0; uint64_t seed = 0; std::vector<float> w; } g_wnodes;
+constexpr int kMaxNodesOwnDirections = 4095;
 
 cudaEvent_t take_event() {
   if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
@@ -201,6 +208,9 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   g.seg0 = seg0;
   rc = check_ptrs(p);
   if (rc) return rc;
+  // directions of every recursion node's own: only causal calls with sorted levels have more than one node
+  g.node_dirs = p.node_directions != 0 && g.causal && g.L > 0 && g.sorted;
+  if (g.node_dirs && (g.nodes > kMaxNodesOwnDirections || bw)) return HYPERATTN_UNSUPPORTED_SHAPE;
   const int is_fp32 = p.dtype == HYPERATTN_FP32;
   const int out_fp32 = p.out_dtype == HYPERATTN_FP32;
   if (bw) {
@@ -292,9 +302,20 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
       make_directions(g.d, g.r, p.seed, g_wcache.w);
       g_wcache.d = g.d; g_wcache.r = g.r; g_wcache.seed = p.seed; g_wcache.valid = true;
     }
+    const float* w_nodes = nullptr;
+    if (g.node_dirs) {
+      const size_t per = (size_t)g.d * g.r;
+      if (g_wnodes.d != g.d || g_wnodes.r != g.r || g_wnodes.seed != p.seed || g_wnodes.nodes < g.nodes) {
+        if (g_wnodes.w.size() < per * kMaxNodesOwnDirections) g_wnodes.w.resize(per * kMaxNodesOwnDirections);   // once: the address stays
+        for (int v = 0; v < g.nodes; ++v) make_directions(g.d, g.r, p.seed, g_wnodes.w.data() + v * per, (uint32_t)v);
+        g_wnodes.d = g.d; g_wnodes.r = g.r; g_wnodes.seed = p.seed; g_wnodes.nodes = g.nodes;
+      }
+      HA_CHECK(cudaMemcpyAsync(base + pl.wnodes, g_wnodes.w.data(), per * g.nodes * 4, cudaMemcpyHostToDevice, st));
+      w_nodes = reinterpret_cast<const float*>(base + pl.wnodes);
+    }
     {
       StageScope sc(st, HYPERATTN_STAGE_HASH, 1);
-      HA_CHECK(launch_hash(g, p.q, p.k, is_fp32, g_wcache.w, ws, dbg ? dbg->near_zero_bits : nullptr, st));
+      HA_CHECK(launch_hash(g, p.q, p.k, is_fp32, g_wcache.w, ws, dbg ? dbg->near_zero_bits : nullptr, st, 3, w_nodes));
     }
     {
       // (the samples of Alg. 2 line 4 are drawn by extra blocks of this launch)
@@ -314,8 +335,13 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     }
     if (dbg) {
       const size_t lvl_bytes = (size_t)g.levels * g.G * g.nl * 4;
-      if (dbg->q_ids) HA_CHECK(cudaMemcpyAsync(dbg->q_ids, ws.ids, (size_t)g.G * g.n, cudaMemcpyDeviceToDevice, st));
-      if (dbg->k_ids) HA_CHECK(cudaMemcpyAsync(dbg->k_ids, ws.ids + (size_t)g.G * g.n, (size_t)g.G * g.nk, cudaMemcpyDeviceToDevice, st));
+      // (directions of the nodes' own: one set of ids per level, [LV, G, n] each)
+      const int sets = g.node_dirs ? g.levels : 1;
+      for (int l = 0; l < sets; ++l) {
+        const uint8_t* src = ws.ids + l * ids_level_stride(g);
+        if (dbg->q_ids) HA_CHECK(cudaMemcpyAsync(dbg->q_ids + (size_t)l * g.G * g.n, src, (size_t)g.G * g.n, cudaMemcpyDeviceToDevice, st));
+        if (dbg->k_ids) HA_CHECK(cudaMemcpyAsync(dbg->k_ids + (size_t)l * g.G * g.nk, src + (size_t)g.G * g.n, (size_t)g.G * g.nk, cudaMemcpyDeviceToDevice, st));
+      }
       if (dbg->perm_q) HA_CHECK(cudaMemcpyAsync(dbg->perm_q, ws.perm_q, lvl_bytes, cudaMemcpyDeviceToDevice, st));
       if (dbg->perm_k) HA_CHECK(cudaMemcpyAsync(dbg->perm_k, ws.perm_k, lvl_bytes, cudaMemcpyDeviceToDevice, st));
       if (dbg->rank_k) HA_CHECK(cudaMemcpyAsync(dbg->rank_k, ws.rank_k, lvl_bytes, cudaMemcpyDeviceToDevice, st));
@@ -539,6 +565,7 @@ int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes) {
   Geometry g;
   const int rc = build_geometry(*p, g);
   if (rc) return rc;
+  g.node_dirs = p->node_directions != 0 && g.causal && g.L > 0 && g.sorted;
   *bytes = make_plan(g, p->dtype == HYPERATTN_FP32, 0, p->capped != 0 && g.sorted && g.m > 0,
                      p->sampling == HYPERATTN_SAMPLE_VALUE_NORMS && g.sorted && g.m > 0).total;
   return HYPERATTN_OK;
@@ -547,6 +574,12 @@ int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes) {
 int hyperattn_get_projections(int d, int hash_bits, uint64_t seed, float* host_out) {
   if (!host_out || d <= 0 || d > 128 || hash_bits < 1 || hash_bits > 8) return HYPERATTN_INVALID_ARGUMENT;
   make_directions(d, hash_bits, seed, host_out);
+  return HYPERATTN_OK;
+}
+
+int hyperattn_get_node_projections(int d, int hash_bits, uint64_t seed, int node, float* host_out) {
+  if (!host_out || d <= 0 || d > 128 || hash_bits < 1 || hash_bits > 8 || node < 0) return HYPERATTN_INVALID_ARGUMENT;
+  make_directions(d, hash_bits, seed, host_out, (uint32_t)node);
   return HYPERATTN_OK;
 }
 

@@ -67,7 +67,12 @@ struct Geometry {
   int nodes;           // off-diagonal nodes per segment (heap-numbered)
   int sorted;          // 1 if any node needs sortLSH (some node has b < its size)
   int seg0;            // index, in the caller's tensor, of this call's first segment (the sampling counters carry it)
+  int node_dirs;       // 1: every recursion node hashes with directions of its own: ids and chunk histograms exist
+                       // once per level (a row is on one side of exactly one node per level)
 };
+// ids / histograms of a level start this many elements after those of level 0 (0: one set shared by all levels)
+__host__ __device__ inline size_t ids_level_stride(const Geometry& g) { return g.node_dirs ? (size_t)g.G * ((size_t)g.n + g.nk) : 0; }
+__host__ __device__ inline size_t hist_level_stride(const Geometry& g) { return g.node_dirs ? (size_t)g.G * (g.chunks_per_seg + g.chunks_per_seg_k) * kBuckets : 0; }
 
 // sorted blocks of a node of s rows: ceil(s / b) of them, the last one with the remaining rows
 // (Alg. 1 line 4: row i belongs to block floor(P(i) / b))
@@ -117,8 +122,10 @@ struct Workspace {
 };
 
 cudaError_t launch_convert(const float* src, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t count, cudaStream_t st);
+// w_host: the shared direction matrix; w_nodes (device, [nodes, d, r], g.node_dirs only): the nodes' own
 cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
-                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st, int side_mask = 3);
+                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st, int side_mask = 3,
+                        const float* w_nodes = nullptr);
 // side_mask: bit 0 queries, bit 1 keys (3: both)
 cudaError_t launch_sort_scan(const Geometry& g, const Workspace& ws, bool with_samples, uint64_t seed, cudaStream_t st, int side_mask = 3);
 cudaError_t launch_sort_scatter(const Geometry& g, const Workspace& ws, cudaStream_t st, int side_mask = 3);

@@ -54,12 +54,20 @@ struct HashArgs {
   int side_mask;          // bit s set: side s is hashed
   int n[2];               // rows per segment of either side
   int unit[2], chunks_per_unit[2], chunks_per_seg[2];
+  // directions of every recursion node's own (causal calls): the grid covers every level; a chunk belongs to
+  // node j = unit / (2 u) of its level (u units per half) and is hashed there if it lies on the side's half
+  const float* w_nodes;   // [nodes, d, r] or null
+  int levels, L, d;
+  size_t ids_level_stride, hist_level_stride;
 };
 
 // which chunk a CTA owns: side, segment, first row, number of rows (0: the chunk lies beyond the last row)
-struct ChunkPos { int side, seg, chunk, row0, rows; };
+struct ChunkPos { int side, seg, chunk, row0, rows, level, node; };
 __device__ __forceinline__ ChunkPos chunk_of_cta(const HashArgs& a, int cta) {
   ChunkPos c;
+  const int per_level = a.G * (a.chunks_per_seg[0] + a.chunks_per_seg[1]);
+  c.level = cta / per_level; cta -= c.level * per_level;
+  c.node = 0;
   const int ctas0 = a.G * a.chunks_per_seg[0];
   c.side = cta >= ctas0;
   if (c.side) cta -= ctas0;
@@ -68,13 +76,21 @@ __device__ __forceinline__ ChunkPos chunk_of_cta(const HashArgs& a, int cta) {
   const int unit_idx = c.chunk / a.chunks_per_unit[c.side], cu = c.chunk % a.chunks_per_unit[c.side];
   c.row0 = unit_idx * a.unit[c.side] + cu * kSortChunk;
   c.rows = max(0, min(min(kSortChunk, a.unit[c.side] - cu * kSortChunk), a.n[c.side] - c.row0));
+  if (a.w_nodes) {
+    // level l: nodes of 2 u units, u = 2^(L - 1 - l); queries live in the second half, keys in the first
+    const int u = 1 << (a.L - 1 - c.level);
+    const int j = unit_idx / (2 * u);
+    const bool second = (unit_idx / u) & 1;
+    c.node = (1 << c.level) - 1 + j;
+    if (second != (c.side == 0)) c.rows = -1;          // this side of the level does not hold the chunk: nothing to do
+  }
   return c;
 }
 __device__ __forceinline__ size_t ids_base(const HashArgs& a, const ChunkPos& c) {
-  return (c.side ? (size_t)a.G * a.n[0] : 0) + (size_t)c.seg * a.n[c.side] + c.row0;
+  return c.level * a.ids_level_stride + (c.side ? (size_t)a.G * a.n[0] : 0) + (size_t)c.seg * a.n[c.side] + c.row0;
 }
 __device__ __forceinline__ size_t hist_base(const HashArgs& a, const ChunkPos& c) {
-  return ((c.side ? (size_t)a.G * a.chunks_per_seg[0] : 0) + (size_t)c.seg * a.chunks_per_seg[c.side] + c.chunk) * kBuckets;
+  return c.level * a.hist_level_stride + ((c.side ? (size_t)a.G * a.chunks_per_seg[0] : 0) + (size_t)c.seg * a.chunks_per_seg[c.side] + c.chunk) * kBuckets;
 }
 
 // One CTA = one chunk (<= kSortChunk rows of one side of one segment).  Each warp walks over
@@ -93,7 +109,8 @@ __global__ void __launch_bounds__(256, D == 64 ? 4 : 3) hash_bf16_kernel(const _
   const int gid = lane >> 2, tig = lane & 3;
   const ChunkPos cp = chunk_of_cta(a, blockIdx.x);
   const int side = cp.side, seg = cp.seg, row0 = cp.row0, rows = cp.rows;
-  if (!((a.side_mask >> side) & 1)) return;
+  if (!((a.side_mask >> side) & 1) || rows < 0) return;
+  const float* wsrc = a.w_nodes ? a.w_nodes + (size_t)cp.node * (D * a.r) : a.w;
 
   s_hist[tid] = 0;
 
@@ -123,7 +140,7 @@ __global__ void __launch_bounds__(256, D == 64 ? 4 : 3) hash_bf16_kernel(const _
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const int coord = 8 * (lt + 4 * (s >> 1)) + 2 * (2 * (s & 1) + h) + e;
-        const float w = (lg < a.r) ? a.w[coord * a.r + lg] : 0.f;
+        const float w = (lg < a.r) ? wsrc[coord * a.r + lg] : 0.f;
         t1[e] = __bfloat162float(__float2bfloat16_rn(w));
         const float r1 = w - t1[e];
         t2[e] = __bfloat162float(__float2bfloat16_rn(r1));
@@ -196,9 +213,10 @@ __global__ void __launch_bounds__(256) hash_fp32_kernel(const __grid_constant__ 
   const int tid = threadIdx.x;
   const ChunkPos cp = chunk_of_cta(a, blockIdx.x);
   const int side = cp.side, seg = cp.seg, row0 = cp.row0, rows = cp.rows;
-  if (!((a.side_mask >> side) & 1)) return;
+  if (!((a.side_mask >> side) & 1) || rows < 0) return;
+  const float* wsrc = a.w_nodes ? a.w_nodes + (size_t)cp.node * (d * a.r) : a.w;
   s_hist[tid] = 0;
-  for (int i = tid; i < d * a.r; i += 256) s_w[i] = a.w[i];
+  for (int i = tid; i < d * a.r; i += 256) s_w[i] = wsrc[i];
   __syncthreads();
   const float* base = reinterpret_cast<const float*>(a.x[side]) + ((size_t)seg * a.n[side] + row0) * d;
   uint8_t* dst = a.ids + ids_base(a, cp);
@@ -254,9 +272,12 @@ cudaError_t launch_convert(const float* src, __nv_bfloat16* hi, __nv_bfloat16* l
 }
 
 cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_fp32, const float* w_host,
-                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st, int side_mask) {
+                        const Workspace& ws, unsigned long long* near_zero, cudaStream_t st, int side_mask, const float* w_nodes) {
   HashArgs a;
   a.side_mask = side_mask;
+  a.w_nodes = g.node_dirs ? w_nodes : nullptr;
+  a.levels = g.node_dirs ? g.levels : 1; a.L = g.L; a.d = g.d;
+  a.ids_level_stride = ids_level_stride(g); a.hist_level_stride = hist_level_stride(g);
   for (int i = 0; i < g.d * g.r; ++i) a.w[i] = w_host[i];
   a.x[0] = q; a.x[1] = k; a.ids = ws.ids; a.hist = ws.hist; a.near_zero = near_zero;
   a.G = g.G; a.r = g.r;
@@ -264,7 +285,7 @@ cudaError_t launch_hash(const Geometry& g, const void* q, const void* k, int is_
     a.n[s] = side_rows(g, s); a.unit[s] = side_unit(g, s);
     a.chunks_per_unit[s] = side_cpu(g, s); a.chunks_per_seg[s] = side_cps(g, s);
   }
-  const int grid = g.G * (g.chunks_per_seg + g.chunks_per_seg_k);
+  const int grid = a.levels * g.G * (g.chunks_per_seg + g.chunks_per_seg_k);
   if (is_fp32) hash_fp32_kernel<<<grid, 256, 0, st>>>(a, g.d);
   else if (g.d == 64) hash_bf16_kernel<64><<<grid, 256, 0, st>>>(a);
   else hash_bf16_kernel<128><<<grid, 256, 0, st>>>(a);

@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(256) sort_scan_kernel(SortArgs a, SampleArgs s
   if (g.causal) { level = 31 - __clz(nd + 1); j = nd + 1 - (1 << level); }
   int nchunks;
   const int first = node_first_chunk(g, level, j, side, nchunks);
-  const uint32_t* h = a.hist + side_hist_base(g, side) + ((size_t)seg * side_cps(g, side) + first) * kBuckets;
+  const uint32_t* h = a.hist + level * hist_level_stride(g) + side_hist_base(g, side) + ((size_t)seg * side_cps(g, side) + first) * kBuckets;
   const int lvl_chunk0 = g.causal ? j * nchunks : 0;
   uint32_t* o = a.offs + side_offs_base(g, side) + (((size_t)level * g.G + seg) * side_cpl(g, side) + lvl_chunk0) * kBuckets;
   // pass 1: bucket totals of the node (eight loads in flight: the kernel is all latency)
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(256) sort_scatter_kernel(SortArgs a) {
   const int rows = min(min(kSortChunk, unit_s - cu * kSortChunk), side_rows(g, side) - row0);
   if (rows <= 0) return;
 
-  const uint8_t* ids = a.ids + side_ids_base(g, side) + (size_t)seg * side_rows(g, side) + row0;
+  const uint8_t* ids = a.ids + level * ids_level_stride(g) + side_ids_base(g, side) + (size_t)seg * side_rows(g, side) + row0;
   for (int i = tid; i < rows; i += 256) s_id[i] = ids[i];
   for (int i = tid; i < 8 * kBuckets / 4; i += 256) reinterpret_cast<uint4*>(&s_cnt[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();

@@ -123,3 +123,10 @@ def test_backward_rejects_bad_arguments_on_the_host():
     assert L.hyperattn_backward_workspace_bytes(C.byref(p), B.BF16, C.byref(need_bf16)) == 0
     # bf16 gradients are accumulated in fp32 in the workspace: three tensors more than for fp32 gradients
     assert need_bf16.value - need_f32.value >= 3 * p.B * p.H * p.n * p.d * 4
+
+
+def test_node_projections_match_the_oracle():
+    for node in (0, 1, 7, 30):
+        w = ha.get_projections(64, 7, 5, node=node)
+        assert np.array_equal(w, O.directions(64, 7, 5, node=node))
+    assert not np.array_equal(ha.get_projections(64, 7, 5, node=1), ha.get_projections(64, 7, 5))
