@@ -87,12 +87,12 @@ int build_geometry(const hyperattn_params& p, Geometry& g) {
 }
 
 struct Plan {
-  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, tpos, ltau, vwq, vcum, swlog, wnodes, part_o, part_lse, total;
+  size_t q16, k16, v16, q16lo, k16lo, ids, hist, offs, perm_q, perm_k, rank_k, samples, tpos, ltau, vwq, vcum, swlog, wnodes, sched, part_o, part_lse, total;
   size_t delta, gacc;   // backward only: <dO, O> per row; fp32 gradient accumulators (bf16 gradients only)
 };
 
 // backward: 0 forward plan; 1 backward with fp32 gradients (accumulated in place); 2 backward with bf16 gradients
-Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = false, bool vnorm = false) {
+Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = false, bool vnorm = false, bool part_bf16 = false) {
   Plan pl;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
@@ -113,13 +113,14 @@ Plan make_plan(const Geometry& g, int is_fp32, int backward = 0, bool capped = f
   pl.perm_k = take(g.sorted ? lvl_rows * 4 : 0);
   pl.rank_k = take(g.sorted ? lvl_rows * 4 : 0);
   pl.samples = take((size_t)g.G * g.nodes * g.m * 4);
+  pl.sched = take(256);
   pl.tpos = take(capped ? (size_t)g.G * g.nodes * g.m * 4 : 0);
   pl.ltau = take(capped ? (size_t)g.G * g.nodes * 4 : 0);
   pl.vwq = take(vnorm ? (size_t)g.G * g.nk * 4 : 0);
   pl.vcum = take(vnorm ? (size_t)g.G * ((size_t)g.nk + 1) * 8 : 0);
   pl.swlog = take(vnorm ? (size_t)g.G * g.nodes * g.m * 4 : 0);
   const size_t part_rows = (g.L && !backward) ? (size_t)g.G * g.n + lvl_rows : 0;
-  pl.part_o = take(part_rows * g.d * 4);
+  pl.part_o = take(part_rows * g.d * (part_bf16 ? 2 : 4));
   pl.part_lse = take(part_rows * 4);
   pl.delta = take(backward ? (size_t)g.G * g.n * 4 : 0);
   pl.gacc = take(backward == 2 ? (size_t)3 * g.G * g.n * g.d * 4 : 0);
@@ -235,7 +236,9 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     if (is_fp32 || bw || p.precise || p.capped) return HYPERATTN_UNSUPPORTED_SHAPE;
     if (g.m > kMaxWeightedSamples) return HYPERATTN_UNSUPPORTED_SHAPE;
   }
-  const Plan pl = make_plan(g, is_fp32, bw ? (bw->grad_dtype == HYPERATTN_FP32 ? 1 : 2) : 0, capped, vnorm);
+  // partial results of the causal recursion travel in the type of the final output (bf16 inputs only)
+  const bool part_bf16 = !is_fp32 && !out_fp32 && g.L > 0;
+  const Plan pl = make_plan(g, is_fp32, bw ? (bw->grad_dtype == HYPERATTN_FP32 ? 1 : 2) : 0, capped, vnorm, part_bf16);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
   int dev = 0;
@@ -277,7 +280,8 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   ws.samples = reinterpret_cast<int32_t*>(base + pl.samples);
   ws.tpos = capped ? reinterpret_cast<int32_t*>(base + pl.tpos) : nullptr;
   ws.ltau = capped ? reinterpret_cast<float*>(base + pl.ltau) : nullptr;
-  ws.part_o = reinterpret_cast<float*>(base + pl.part_o);
+  ws.part_o = base + pl.part_o;
+  ws.part_bf16 = part_bf16;
   ws.part_lse = reinterpret_cast<float*>(base + pl.part_lse);
   ws.status = ds.status;
 
@@ -357,7 +361,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   if (is_fp32) { a.q_lo = ws.q16lo; a.k_lo = ws.k16lo; }
   a.scale_log2 = scale * 1.4426950408889634f;
   a.perm_q = ws.perm_q; a.perm_k = ws.perm_k; a.rank_k = ws.rank_k; a.samples = ws.samples;
-  a.part_o = ws.part_o; a.part_lse = ws.part_lse; a.out = p.out; a.lse = p.lse;
+  a.part_o = ws.part_o; a.part_lse = ws.part_lse; a.part_bf16 = part_bf16; a.out = p.out; a.lse = p.lse;
   a.out_fp32 = out_fp32;
   a.precise = p.precise != 0;
   a.capped = capped;
@@ -430,7 +434,11 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     StageScope sc(st, HYPERATTN_STAGE_ATTENTION, 1);
     // bf16 inputs: tcgen05 path; fp32 inputs: split-bf16 logits on the warp-level MMA path
     if (is_fp32) HA_CHECK(launch_attention_mma(a, st));
-    else HA_CHECK(launch_attention_tc(a, ws.status, st));
+    else {
+      a.sched = reinterpret_cast<int*>(base + pl.sched);
+      HA_CHECK(cudaMemsetAsync(a.sched, 0, 4, st));
+      HA_CHECK(launch_attention_tc(a, ws.status, st));
+    }
   }
   if (g.L) {
     StageScope sc(st, HYPERATTN_STAGE_MERGE, 1);
@@ -567,7 +575,8 @@ int hyperattn_workspace_bytes(const hyperattn_params* p, size_t* bytes) {
   if (rc) return rc;
   g.node_dirs = p->node_directions != 0 && g.causal && g.L > 0 && g.sorted;
   *bytes = make_plan(g, p->dtype == HYPERATTN_FP32, 0, p->capped != 0 && g.sorted && g.m > 0,
-                     p->sampling == HYPERATTN_SAMPLE_VALUE_NORMS && g.sorted && g.m > 0).total;
+                     p->sampling == HYPERATTN_SAMPLE_VALUE_NORMS && g.sorted && g.m > 0,
+                     p->dtype != HYPERATTN_FP32 && p->out_dtype != HYPERATTN_FP32 && g.L > 0).total;
   return HYPERATTN_OK;
 }
 

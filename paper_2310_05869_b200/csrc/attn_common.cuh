@@ -26,7 +26,8 @@ struct AttnArgs {
   Geometry g;
   float scale_log2;                  // softmax scale * log2(e)
   const int32_t *perm_q, *perm_k, *rank_k, *samples;
-  float *part_o, *part_lse;          // partial results (fp32), used when !direct
+  void* part_o; float* part_lse;     // partial results, used when !direct: rows of fp32, or of bf16 when part_bf16
+  int part_bf16;                     // (partials are kept in the type of the final output; their log-sum-exp always in fp32)
   void* out; float* lse;             // final results, used when direct
   int out_fp32;
   int direct;
@@ -52,6 +53,7 @@ struct AttnArgs {
   int level_pair_start[kMaxLevels + 1];
   int level_paired[kMaxLevels];      // 1: CTAs of this level own two query tiles, 0: one
   int total_pairs;
+  int* sched;                        // work counter of the launch (global memory, zero at launch): next item to hand out
 };
 
 struct TileDesc {

@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(256, 1) attn_mma_kernel(const __grid_constant_
     const float lse = (mrow[h] + log2f(lrow[h])) * 0.69314718055994531f;
     const size_t orow = t.orow_base + (size_t)(qr + t.odelta);
     if (t.partial) {
-      float* dst = a.part_o + orow * D;
+      float* dst = reinterpret_cast<float*>(a.part_o) + orow * D;     // (this path keeps fp32 partials)
 #pragma unroll
       for (int i = 0; i < NO; ++i)
         *reinterpret_cast<float2*>(dst + i * 8 + 2 * tig) = make_float2(o[i][2 * h] * inv, o[i][2 * h + 1] * inv);

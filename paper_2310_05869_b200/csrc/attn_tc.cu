@@ -385,9 +385,11 @@ __device__ __forceinline__ void decode_pair(const AttnArgs& a, int pair, PairDes
   t.nbA = t.nbB = t.nsmp = 0;
   int s, q0n, k0n;
   if (pair < a.n_leaf_pairs) {
-    const int per = g.G * a.leaves_per_seg;
-    const int uu = a.pairs_per_leaf - 1 - pair / per;       // heavy pairs first
-    const int rem = pair % per;
+    // Leaf after leaf, the pairs of a leaf from the heaviest (last rows, most keys) to the lightest: items are
+    // handed out in this order, so the CTAs that run at the same time work on a handful of neighbouring leaves
+    // and find each other's K / V tiles in L2, and the list still ends with light items.
+    const int uu = a.pairs_per_leaf - 1 - pair % a.pairs_per_leaf;
+    const int rem = pair / a.pairs_per_leaf;
     t.seg = rem / a.leaves_per_seg;
     const int leaf = rem % a.leaves_per_seg;
     t.mode = 0; t.causal = a.dense_causal;
@@ -563,10 +565,12 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     // item preparer; then the arrival here is immediate.)
     auto gather_q = [&](int nit) {
       bool good = mbar_wait<20, 19>(bar_tabfull(nit & 1), (nit >> 1) & 1, s_abort, status);
-      if (good && nit >= 1) good = mbar_wait<20, 20>(bar_qfree, (nit - 1) & 1, s_abort, status);
       if (!good) return false;
       const ItemDesc& de = *reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + (nit & 1) * C::kDescBytes);
       const PairDesc& t = de.t;
+      if (t.mode < 0) return true;                        // the end of the work list: nothing to fetch
+      if (nit >= 1) good = mbar_wait<20, 20>(bar_qfree, (nit - 1) & 1, s_abort, status);
+      if (!good) return false;
       const QTile &qa = de.qa, &qb = de.qb;
       if (t.mode == 1) {
         constexpr int CPR = D / 8;
@@ -592,8 +596,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     };
     HA_LDECL(a_tab); HA_LDECL(a_ws); HA_LDECL(a_cmp); HA_LDECL(a_epi); HA_LDECL(a_gq); HA_LDECL(a_bo); HA_LDECL(a_tiles); HA_LDECL(a_ws0); HA_LDECL(a_c1); HA_LDECL(a_c2); HA_LDECL(a_c3); HA_LDECL(a_c4);
     HA_T0(t_role);
-    if (blockIdx.x < a.total_pairs) ok = __all_sync(0xffffffffu, gather_q(0));
-    for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+    ok = __all_sync(0xffffffffu, gather_q(0));
+    for (; ok; ++it) {
       const int set = it & 1;
       const uint32_t* s_mask = s_mask_all + (set * 2 + i) * MW;
       const int* s_qrow = s_qrow_all + (set * 2 + i) * 128;
@@ -604,6 +608,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       HA_LACC(a_tab, tt);
       const ItemDesc& de = *reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes);
       const PairDesc t = de.t;
+      if (t.mode < 0) break;                              // the work list is exhausted
       const QTile q = i ? de.qb : de.qa;
       const int total = q.n1 + q.n2;
       const float wlog = (t.mode == 1 && g.m > 0) ? log2f((float)t.nk / (float)g.m) : 0.f;   // log2(N/m): weight of a sampled column
@@ -832,7 +837,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       // copies in the load/store unit (measured: 5 % faster with the gather after them, while
       // bf16 results are 5 % slower that way).
       HA_T0(tg);
-      if (!GATHER_LATE && item + (int)gridDim.x < a.total_pairs) {
+      if (!GATHER_LATE) {
         ok = __all_sync(0xffffffffu, gather_q(it + 1));
         if (!ok) break;
       }
@@ -872,8 +877,8 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           constexpr int RB = C::kStageRow;
           constexpr int LPR = RB / 16, RPI = 32 / LPR, NI = 32 / RPI;
           constexpr int NP = D / 16;
-          const bool f32o = t.partial || a.out_fp32;
-          char* obase = f32o ? reinterpret_cast<char*>(t.partial ? a.part_o : reinterpret_cast<float*>(a.out)) : reinterpret_cast<char*>(a.out);
+          const bool f32o = t.partial ? !a.part_bf16 : a.out_fp32;
+          char* obase = reinterpret_cast<char*>(t.partial ? a.part_o : a.out);
           const long long myoff = qr >= 0 ? (long long)(orow * (size_t)(D * (f32o ? 4 : 2))) : -1;
           long long roff[NI];
 #pragma unroll
@@ -929,7 +934,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
         ++vi;
       }
-      if (GATHER_LATE && item + (int)gridDim.x < a.total_pairs) {
+      if (GATHER_LATE) {
         ok = __all_sync(0xffffffffu, gather_q(it + 1));
         if (!ok) break;
       }
@@ -995,10 +1000,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       int it = 0;
       HA_LDECL(b_q); HA_LDECL(b_p); HA_LDECL(b_v); HA_LDECL(b_k);
       HA_T0(tloop);
-      for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+      for (; ok; ++it) {
         ok = wait_fast<22>(bar_tabfull(it & 1), (it >> 1) & 1, s_abort, status);
         if (!ok) break;
         const ItemDesc& de = *reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + (it & 1) * C::kDescBytes);
+        if (de.t.mode < 0) break;
         const QTile q = i ? de.qb : de.qa;
         const int total = q.n1 + q.n2;
         const int ntiles = de.t.ntiles;
@@ -1099,10 +1105,17 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     // dependent global lookups below overlap with the computation of the item in between.
     bool ok = true;
     int it = 0;
-    for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+    for (; ok; ++it) {
       HA_T0(tdec);
-      PairDesc t; QTile qa, qb;
-      decode_pair(a, item, t, qa, qb);
+      // Work items are handed out by a counter in global memory, in list order (heavy first): whichever CTA
+      // is free takes the next one.
+      int item = 0;
+      if (lane == 0) item = atomicAdd(a.sched, 1);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      const bool end = item >= a.total_pairs;
+      PairDesc t = {}; QTile qa = {}, qb = {};
+      if (!end) decode_pair(a, item, t, qa, qb);
+      else t.mode = -1;                                   // tells every role that the list is exhausted
       if (lane == 0) HA_TACC(26, tdec);
       const int set = it & 1;
       int* s_kidx = s_kidx_all + set * kMaxNodeKeys;
@@ -1117,6 +1130,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       if (lane == 0) {
         ItemDesc* de = reinterpret_cast<ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes);
         de->t = t; de->qa = qa; de->qb = qb;
+      }
+      if (end) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tabfull(set));
+        break;
       }
       const int segrow = t.seg * g.n;                       // row coordinate of the segment's first query row ...
       const int segrow_k = t.seg * g.nk;                    // ... and of its first key row
@@ -1291,12 +1309,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       doff[e] = (uint32_t)((cc >> 3) * (TK * 128) + (4 * rq + e) * 128 + (((cc & 7) ^ ((4 * rq + e) & 7)) << 4));
     const char* ksrc = reinterpret_cast<const char*>(a.k) + cc * 16;
     const char* vsrc = reinterpret_cast<const char*>(a.v) + cc * 16;
-    for (int item = blockIdx.x; item < a.total_pairs && ok; item += gridDim.x, ++it) {
+    for (; ok; ++it) {
       const int set = it & 1;
       const int* s_kidx = s_kidx_all + set * kMaxNodeKeys;
       ok = mbar_wait<100, 18>(bar_tabfull(set), (it >> 1) & 1, s_abort, status);
       if (!ok) break;
       const PairDesc t = reinterpret_cast<const ItemDesc*>(smem + C::kOffDesc + set * C::kDescBytes)->t;
+      if (t.mode < 0) break;
       const int segrow = t.seg * g.nk;                      // (keys)
       for (int j = 0; j < t.ntiles && ok; ++j) {
         const int gj = gbase + j;
@@ -1436,16 +1455,16 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
   if (a.capped || a.sample_wlog) {
     if (a.precise || (a.capped && a.sample_wlog)) return cudaErrorInvalidValue;
     if (a.g.d == 64) return go(attn_tc_kernel<64, false, false, true>, Cfg<64>::kTotal);
-    if (!a.direct) return go(attn_tc_kernel<128, true, false, true>, Cfg<128>::kTotal);
+    if (!a.direct && !a.part_bf16) return go(attn_tc_kernel<128, true, false, true>, Cfg<128>::kTotal);
     return go(attn_tc_kernel<128, false, false, true>, Cfg<128>::kTotal);
   }
   if (a.precise) {
     if (a.g.d == 64) return go(attn_tc_kernel<64, false, true, false>, Cfg<64>::kTotal);
-    if (!a.direct) return go(attn_tc_kernel<128, true, true, false>, Cfg<128>::kTotal);
+    if (!a.direct && !a.part_bf16) return go(attn_tc_kernel<128, true, true, false>, Cfg<128>::kTotal);
     return go(attn_tc_kernel<128, false, true, false>, Cfg<128>::kTotal);
   }
   if (a.g.d == 64) return go(attn_tc_kernel<64, false, false, false>, Cfg<64>::kTotal);
-  if (!a.direct) return go(attn_tc_kernel<128, true, false, false>, Cfg<128>::kTotal);
+  if (!a.direct && !a.part_bf16) return go(attn_tc_kernel<128, true, false, false>, Cfg<128>::kTotal);
   return go(attn_tc_kernel<128, false, false, false>, Cfg<128>::kTotal);
 }
 

@@ -117,7 +117,8 @@ struct Workspace {
   int32_t* samples;                // [G, nodes, m]
   int32_t* tpos;                   // capped row sums: [G, nodes, m] probe positions (else null)
   float* ltau;                     // capped row sums: [G, nodes] log2 of the largest unmasked probe row sum
-  float *part_o, *part_lse;        // causal partials: leaf [G,n,(d)] then per level [G,n/2,(d)]
+  void* part_o; float* part_lse;   // causal partials: leaf [G,n,(d)] then per level [G,nl,(d)]; rows of fp32 or bf16
+  int part_bf16;
   int* status;                     // device status word
 };
 
