@@ -164,11 +164,36 @@ def oracle_rows(w, Q64, K64, V64, g, rows, ids_q=None, ids_k=None, caps=None):
                              scale=1.0 / math.sqrt(w.d), rows=rows, ids_q=ids_q, ids_k=ids_k, caps=caps)
 
 
+def whole_block_rows(w, inter, g, count, rng):
+    """Query rows of `count` whole sorted blocks of segment g, drawn over all sorted nodes (a block's rows through
+    the GPU's own permutation, which check_perms compares with the oracle's)."""
+    nodes = []
+    for level, s in levels_of(w):
+        if w.b >= s:
+            continue
+        for j in range((1 << level) if w.causal else 1):
+            q0, _, s_, nq = node_ranges(w, level, j)
+            if nq > 0:
+                nodes.append((level, j, q0, s_, nq))
+    if not nodes:
+        return []
+    pq = inter["perm_q"]
+    rows = []
+    for _ in range(count):
+        level, j, q0, s, nq = nodes[int(rng.integers(len(nodes)))]
+        bq = O.query_block_size(nq, s, w.b)
+        beta = int(rng.integers(-(-nq // bq)))
+        base = j * s if w.causal else 0
+        lo, hi = base + beta * bq, base + min((beta + 1) * bq, nq)
+        rows.extend((q0 + pq[level, g, lo:hi].cpu().numpy()).tolist())
+    return rows
+
+
 def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, segs=None, rng_seed=0,
                   max_abs_bound=None, blocks_per_seg=0, caps=None, row_scale=None):
     """Compares out/lse with the oracle (GPU ids injected when `inter` is given).  With
     rows_per_seg, a pseudo-random subset of rows plus the rows around every leaf / node
-    boundary is checked.  `row_scale` (G x n, >= 1) divides the output errors row by row before they meet the
+    boundary is checked, plus (blocks_per_seg) the rows of that many whole sorted blocks.  `row_scale` (G x n, >= 1) divides the output errors row by row before they meet the
     bounds: with capped row sums a row's output is its uncapped output times (uncapped row sum / capped
     row sum), and so are its rounding errors."""
     out = out.float().cpu().numpy().reshape(w.G, w.n, w.d)
@@ -183,6 +208,8 @@ def check_outputs(w, Q64, K64, V64, out, lse, inter=None, rows_per_seg=None, seg
             rows = np.arange(w.n)
         else:
             rows = set(rng.choice(w.n, size=rows_per_seg, replace=False).tolist())
+            if blocks_per_seg and inter is not None:
+                rows.update(whole_block_rows(w, inter, g, blocks_per_seg, rng))
             if w.causal and w.n > w.n0:
                 leaf = O.causal_grid(w.n, w.n0)[1]
                 for edge in range(0, w.n + 1, leaf):

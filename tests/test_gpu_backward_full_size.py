@@ -7,7 +7,10 @@ computed row by row and what holds at any size:
   bucket ids (hence the permutations) and the samples fixed, dQ_i is the gradient of
   f(q_i) = <dO_i, out_i(q_i)> in q_i, and out_i can be evaluated for one row;
 * every row of P sums to one (the saved lse is the logarithm of the row's weighted sum), so
-  sum_j dV_j = sum_i dO_i, and sum_j dS_ij = <dO_i, O_i> - delta_i = 0, so sum_j dK_j = 0.
+  sum_j dV_j = sum_i dO_i, and sum_j dS_ij = <dO_i, O_i> - delta_i = 0, so sum_j dK_j = 0;
+* dV_j and dK_j of a few keys j element by element (the two smaller workloads): the oracle's forward pass, given
+  one-hot "values" e_j, returns column j of P for every row, and dV_j = sum_i P_ij dO_i,
+  dK_j = scale sum_i P_ij (<dO_i, v_j> - <dO_i, O_i>) q_i need nothing else.
 
 Tolerances: P and dS are rounded to bf16 before the tensor-core products and O enters delta in
 bf16, so, as in the small-size parity test, a dQ entry may be off by 2^-6 of the summed absolute
@@ -98,5 +101,24 @@ def test_backward_full_size_rows_and_sums(w):
         err = np.abs(got[i] - want)
         worst = max(worst, float((err / (terms + 1e-30)).max()))
         assert (err <= TERMS_REL * terms + 1e-6).all(), (w.name, i, float((err / (terms + 1e-30)).max()))
+    # ---- dV_j, dK_j of a few keys, element by element (one segment of the two smaller workloads) ------------
+    if w.n <= 32768:
+        keys = [3, w.n // 2 - 7, w.n // 2 + 250, w.n - 2] + [int(x) for x in inter["samples"][g, 0, :2].cpu().numpy()]   # two of them sampled columns of the root
+        onehot = np.zeros((w.n, len(keys)))
+        onehot[keys, np.arange(len(keys))] = 1.0
+        Pcols, _ = O.segment_forward(Q64, K64, onehot, W, w.b, w.m, w.causal, w.n0, w.seed, g, scale=scale, ids_q=ids_q, ids_k=ids_k)
+        O_all, _ = O.segment_forward(Q64, K64, V64, W, w.b, w.m, w.causal, w.n0, w.seed, g, scale=scale, ids_q=ids_q, ids_k=ids_k)
+        delta = (dO * O_all).sum(axis=1)
+        gv = dv.double().reshape(w.G, w.n, w.d)[g].cpu().numpy()
+        gk = dk.double().reshape(w.G, w.n, w.d)[g].cpu().numpy()
+        for c, j in enumerate(keys):
+            P = Pcols[:, c]
+            want_v = P @ dO
+            size_v = P @ np.abs(dO)
+            dS = P * (dO @ V64[j] - delta)
+            want_k = scale * (dS @ Q64)
+            size_k = scale * ((P * (np.abs(dO @ V64[j]) + np.abs(delta) + (np.abs(dO) * np.abs(O_all)).sum(axis=1))) @ np.abs(Q64))
+            assert (np.abs(gv[j] - want_v) <= TERMS_REL * size_v + 1e-6).all(), (w.name, "dV", j)
+            assert (np.abs(gk[j] - want_k) <= TERMS_REL * size_k + 1e-6).all(), (w.name, "dK", j)
     print(w.name, "dQ rows vs central differences: worst error / summed term sizes", worst,
           "sum dV error / size", sum_err / sum_size, "sum dK / size", dk_err / max(dk_size, 1e-30))

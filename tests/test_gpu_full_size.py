@@ -2,8 +2,9 @@
 
 The oracle cannot evaluate these workloads as a whole, so two segments (the first and the
 last (batch, head) pair) are checked per workload: bucket ids and permutations in full, the
-outputs on sampled rows plus the rows around every leaf boundary; every output of every
-segment must be finite."""
+sampled columns of every segment, the outputs on the rows of 64 whole sorted blocks per checked
+segment, on sampled rows and on the rows around every leaf boundary; every output of every
+segment must be finite.  The 32768-row configuration is also compared row by row, all of it."""
 import numpy as np
 import pytest
 import torch
@@ -40,5 +41,25 @@ def test_full_size_sampled_segments(w):
     amb, mism = PU.check_ids(w, Q64, K64, inter, segs=segs)
     assert mism <= amb
     PU.check_perms(w, inter, segs=segs)
-    stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter, rows_per_seg=48, segs=segs, rng_seed=1, max_abs_bound=bound)
+    PU.check_samples(w, inter)
+    stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter, rows_per_seg=48, segs=segs, rng_seed=1, max_abs_bound=bound,
+                             blocks_per_seg=64)
+    print(w.name, stats, "ambiguous hash bits", amb, "rows that differ", mism)
+
+
+def test_c2_every_row_of_every_segment():
+    """The 32768-row configuration (32 heads, d = 128) against the oracle on all of its 1 048 576 rows."""
+    w = WL.CONFIGS[1]
+    arrs = WL.make_inputs(w)
+    q, k, v = PU.to_device(w, arrs)
+    out, lse, inter = ha.forward(q, k, v, w.b, w.m, w.r, seed=w.seed, debug=True, out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    assert ha.last_device_status() == 0
+    Q64, K64, V64 = (PU.LazySegments(x) for x in arrs)
+    amb, mism = PU.check_ids(w, Q64, K64, inter)
+    assert mism <= amb
+    PU.check_samples(w, inter)
+    PU.check_perms(w, inter)
+    stats = PU.check_outputs(w, Q64, K64, V64, out, lse, inter)
+    assert stats["rows"] == w.G * w.n
     print(w.name, stats, "ambiguous hash bits", amb, "rows that differ", mism)
