@@ -52,5 +52,24 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
+WAIT_TEST_LIB = os.path.join(PKG_DIR, "libhyperattn_waittest.so")
+
+
+def build_wait_test_library(force: bool = False) -> str:
+    """A second copy of the library for ONE test (tests/test_gpu_wait_limit.py): the attention kernel compiled with
+    a 20 ms limit on its waits and a switch that makes one K / V tile never arrive, once, so that the path on which
+    a wait gives up (status word, draining, TMEM release) can be run.  Never loaded by the package itself."""
+    if not force and os.path.exists(WAIT_TEST_LIB) and os.path.getmtime(WAIT_TEST_LIB) >= os.path.getmtime(build_library()):
+        return WAIT_TEST_LIB
+    build_library()
+    obj = os.path.join(CSRC, "attn_tc_waittest.o")
+    subprocess.check_call([_nvcc(), *NVCC_FLAGS, "-DHA_WAIT_LIMIT_NS=20000000ull", "-DHA_TEST_DROP_ARRIVAL", "-c",
+                           os.path.join(CSRC, "attn_tc.cu"), "-o", obj])
+    objs = [os.path.join(CSRC, src.replace(".cu", ".o")) for src in SOURCES if src != "attn_tc.cu"] + [obj]
+    subprocess.check_call([_nvcc(), "-shared", "-o", WAIT_TEST_LIB, *objs, "-lcudart"])
+    return WAIT_TEST_LIB
+
+
 if __name__ == "__main__":
     print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_wait_test_library(force="--force" in sys.argv))

@@ -45,7 +45,16 @@ struct alignas(64) TmaMaps {
 };
 
 constexpr int TK = 64;                  // keys per tile
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
+#ifndef HA_WAIT_LIMIT_NS
+#define HA_WAIT_LIMIT_NS 2000000000ull
+#endif
+constexpr unsigned long long kWaitLimitNs = HA_WAIT_LIMIT_NS;   // every mbarrier wait gives up after 2 s
+// Test build only (-DHA_TEST_DROP_ARRIVAL, never in the shipped library): when armed, the K / V streamer of one CTA
+// leaves out the copies of one V tile once, so that the wait for that tile runs out and the give-up path can be
+// exercised without any fault.
+#ifdef HA_TEST_DROP_ARRIVAL
+__device__ int g_test_drop_armed;
+#endif
 constexpr float kRescaleThreshold = 32.f;   // octaves the scores may exceed the reference before it moves
 constexpr float kTileSumLimit = 1099511627776.f;   // 2^40: a tile whose weights sum to more has a score > 2^34 above the reference
 
@@ -1366,6 +1375,13 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
         }
         if (lane == 0) HA_TACC(11, tle2);
         HA_T0(tgv);
+#ifdef HA_TEST_DROP_ARRIVAL
+        {
+          int drop = 0;
+          if (lane == 0 && gj == 1) drop = atomicExch(&g_test_drop_armed, 0);
+          if (__shfl_sync(0xffffffffu, drop, 0)) { v_armed = gj; continue; }     // nothing issued, nothing will arrive
+        }
+#endif
         fill(ubase + C::kOffV + s * C::kTile, &maps.v, vsrc, bar_vfull(s));
         v_armed = gj + 1;
         if (lane == 0) HA_TACC(1, tgv);
@@ -1394,6 +1410,12 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
 }
 
 }  // namespace
+
+#ifdef HA_TEST_DROP_ARRIVAL
+extern "C" int hyperattn_test_arm_drop(int on) {
+  return cudaMemcpyToSymbol(g_test_drop_armed, &on, sizeof(int)) == cudaSuccess ? 0 : -5;
+}
+#endif
 
 #ifdef HA_TC_TIMING
 extern "C" int hyperattn_debug_tc_timing(unsigned long long* host16, int reset) {
