@@ -124,8 +124,15 @@ typedef struct hyperattn_params {
   float softmax_scale;   /* <= 0 selects 1/sqrt(d) */
   void* workspace;       /* device scratch owned by the caller, or NULL: the library then
                             uses a private per-device buffer that it grows on demand (the
-                            growing call synchronises the device) and keeps until
-                            hyperattn_release(); calls that share it must not overlap */
+                            growing call synchronises the device, frees the old buffer and
+                            allocates a new one) and keeps until hyperattn_release(); calls
+                            that share it must not overlap.  Stream capture: a call made while
+                            `stream` is being captured never allocates or synchronises; it
+                            returns HYPERATTN_WORKSPACE_TOO_SMALL if it has no caller's workspace
+                            and the private one is missing or too small.  A captured graph holds
+                            the workspace's address: capture with a caller-owned workspace, or
+                            know that a graph captured on the private buffer is invalidated by
+                            any later call that grows it and by hyperattn_release(). */
   size_t workspace_bytes;
   const hyperattn_debug* debug; /* may be NULL */
   void* stream;
@@ -270,24 +277,25 @@ int hyperattn_profile_enable(int on);
 int hyperattn_profile_reset(void);
 int hyperattn_profile_read(hyperattn_stage_times* out);
 
-/* sortLSH of ONE bf16 matrix x[n, d] with no allocation of any kind (the paper has no
- * counterpart; the computation is Def. 1 + Alg. 1 lines 2-3 exactly as in hyperattn_forward).
- * For callers that must not allocate device memory while running (a server that partitions HBM
- * at start-up, a plug-in in someone else's process, a loop that may not take the driver's
- * allocation locks): the scratch memory is a fixed array inside the library image, about
- * 2.1 MB, which every GPU that loads the library holds until the process exits.
+/* sortLSH of ONE bf16 matrix x[n, d] by an entry point that allocates nothing (the paper has no
+ * counterpart to this entry point; what it computes is the hash and the argsort of
+ * hyperattn_forward, for one matrix).  It is for callers that must not allocate device memory while
+ * they run: a server that partitions HBM at start-up, a plug-in inside someone else's process, a loop
+ * that may not take the driver's allocation locks.  Its scratch memory is a fixed array inside the
+ * library image, 0.5 MB, which every GPU that loads the library holds until the process exits.
  *   x     device, [n, d] bf16 row-major, 16-byte aligned; d in {64, 128}; 1 <= hash_bits <= 8
  *   ids   device, uint8[n]  : bucket id of every row
  *   perm  device, int32[n]  : perm[p] = row at sorted position p (stable, ascending bucket id)
  *   rank  device, int32[n]  : inverse of perm
  * n may not exceed HYPERATTN_NOALLOC_MAX_ROWS; larger n returns HYPERATTN_UNSUPPORTED_SHAPE and
  * nothing is launched.  The caller owns x, ids, perm, rank.  Work is enqueued on `stream`; the
- * call does not synchronise, does not call cudaMalloc / cudaFree or any allocating routine.
- * The first call on each device (with that device current) looks up the array's device
- * address; make that first call outside any stream capture.  All calls share the one array:
- * it keeps the previous call's contents (every word that is read is rewritten first, so
- * nothing needs clearing), and two calls whose kernels overlap on the GPU race on it --
- * issue them on one stream or order them with events. */
+ * call does not synchronise and calls neither cudaMalloc / cudaFree nor any other allocating routine,
+ * on the device or on the host.  The matrix is read once (it is hashed as the key side of a problem
+ * without queries).  The first call on each device (with that device current) looks up the array's
+ * device address and keeps it in a fixed table; make that first call outside any stream capture.
+ * All calls share the one array: it keeps the previous call's contents (every word that is read is
+ * rewritten first, so nothing needs clearing), and two calls whose kernels overlap on the GPU race
+ * on it -- issue them on one stream or order them with events. */
 #define HYPERATTN_NOALLOC_MAX_ROWS 262144
 int hyperattn_sortlsh_noalloc(const void* x, int n, int d, int hash_bits, uint64_t seed,
                               uint8_t* ids, int32_t* perm, int32_t* rank, void* stream);

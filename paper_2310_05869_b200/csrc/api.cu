@@ -245,7 +245,13 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
   if (cudaGetDevice(&dev) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   std::lock_guard<std::mutex> lock(g_mu);
   DeviceState& ds = g_dev[dev];
+  // While the stream is being captured into a graph nothing may be allocated or synchronised: the status word
+  // and (without a caller's workspace) a large enough private workspace must exist already.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+  const bool capturing = cap != cudaStreamCaptureStatusNone;
   if (!ds.status) {
+    if (capturing) return HYPERATTN_WORKSPACE_TOO_SMALL;
     if (cudaMalloc(&ds.status, 256) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
     if (cudaMemset(ds.status, 0, 256) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
   }
@@ -254,6 +260,7 @@ int forward_impl(const hyperattn_params& p, int seg0 = 0, const hyperattn_grads*
     if (p.workspace_bytes < pl.total) return HYPERATTN_WORKSPACE_TOO_SMALL;
     base = reinterpret_cast<char*>(p.workspace);
   } else {
+    if (ds.ws_bytes < pl.total && capturing) return HYPERATTN_WORKSPACE_TOO_SMALL;
     if (ds.ws_bytes < pl.total) {
       cudaDeviceSynchronize();
       if (ds.ws) cudaFree(ds.ws);

@@ -7,7 +7,6 @@
 // one entry point whose scratch memory is a fixed array that is part of the library image.
 // The price: every GPU that loads the library holds the array (kScratchBytes) until the
 // process exits, the problem size is capped, and all calls share the one array.
-#include <map>
 #include <mutex>
 
 #include "../../include/hyperattn.h"
@@ -28,24 +27,25 @@ constexpr size_t kScratchBytes = kOffOffs + kChunksMax * kBuckets * 4;
 // In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
+constexpr int kMaxDevices = 64;
 std::mutex g_mu;
-std::map<int, unsigned char*> g_scratch_ptr;   // device ordinal -> device address of g_scratch
+unsigned char* g_scratch_ptr[kMaxDevices];     // device ordinal -> device address of g_scratch (a fixed table: no heap)
 
 // First call on a device: resolve the array's device address (with that device current).
 int scratch_for_current_device(unsigned char** out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return HYPERATTN_CUDA_ERROR;
+  if (dev < 0 || dev >= kMaxDevices) return HYPERATTN_UNSUPPORTED_SHAPE;
   std::lock_guard<std::mutex> lock(g_mu);
-  auto it = g_scratch_ptr.find(dev);
-  if (it == g_scratch_ptr.end()) {
+  if (!g_scratch_ptr[dev]) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_scratch) != cudaSuccess || p == nullptr) {
       cudaGetLastError();
       return HYPERATTN_CUDA_ERROR;
     }
-    it = g_scratch_ptr.emplace(dev, static_cast<unsigned char*>(p)).first;
+    g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
   }
-  *out = it->second;
+  *out = g_scratch_ptr[dev];
   return HYPERATTN_OK;
 }
 

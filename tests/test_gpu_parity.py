@@ -189,25 +189,32 @@ def test_stage_profile_counts_launches():
 
 
 def test_forward_can_be_captured_in_a_cuda_graph():
-    """The entry point only enqueues work on the caller's stream (workspace from the stream-ordered
-    pool, no synchronisation), so a forward call can be captured once and replayed."""
+    """The entry point only enqueues work on the caller's stream, so a forward call can be captured once and
+    replayed - with a caller-owned workspace (a graph keeps the workspace's address).  Without one, a call
+    under capture that would have to grow the private workspace is refused instead of allocating."""
     w = W("graph_capture", 1, 4, 2048, 64, "bf16", 128, 64, 7, True, 512, seed=31)
     arrs = WL.make_inputs(w)
     q, k, v = PU.to_device(w, arrs)
     out, lse = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
     torch.cuda.synchronize()
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):                      # warm the pool on the capture stream
-        ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
-    torch.cuda.current_stream().wait_stream(side)
+    ws = torch.empty(ha.workspace_bytes(w.B, w.H, w.n, w.d, w.b, w.m, w.r, w.causal, w.n0), dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        out2, lse2 = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)
+        out2, lse2 = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, workspace=ws)
     for _ in range(3):
         out2.zero_()
         graph.replay()
     torch.cuda.synchronize()
     assert ha.last_device_status() == 0
     assert torch.equal(out2, out) and torch.equal(lse2, lse)
+    # a shape whose workspace the private buffer cannot hold yet, under capture and without a workspace: refused
+    big = W("graph_capture_big", 1, 8, 16384, 64, "bf16", 128, 64, 7, True, 512, seed=31)
+    qb, kb, vb = PU.to_device(big, WL.make_inputs(big))
+    ha.release()                                        # (drops the private buffer)
+    ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed)      # small private buffer and status word exist again
+    torch.cuda.synchronize()
+    g2 = torch.cuda.CUDAGraph()
+    with pytest.raises(ha.HyperAttnError, match="workspace too small"):
+        with torch.cuda.graph(g2):
+            ha.forward(qb, kb, vb, big.b, big.m, big.r, causal=True, n0=big.n0, seed=0)
