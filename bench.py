@@ -40,9 +40,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the attention kernel,
 # from the ncu captures summarised under profiles/ (taken on 4 / 8 heads and scaled to the
 # workload's 32 heads: the traffic is proportional to the number of segments).
-NCU_TRAFFIC_BYTES = {"c3_n131k_causal": 8 * 1.760e9, "c2_n32k_d128": 4 * 0.2456e9}
+NCU_TRAFFIC_BYTES = {"c3_n131k_causal": 8 * 0.9292e9, "c2_n32k_d128": 4 * 0.2456e9}
 # sm__pipe_tensor_cycles_active (% of peak sustained active) of the attention kernel in the same captures
-NCU_TENSOR_PIPE_PCT = {"c3_n131k_causal": 24.6, "c2_n32k_d128": 27.0}
+NCU_TENSOR_PIPE_PCT = {"c3_n131k_causal": 26.0, "c2_n32k_d128": 27.0}
 
 
 def load_peaks():
@@ -95,7 +95,8 @@ def work_model(w: WL.Workload):
         L = 0
         while (n >> L) > w.n0:
             L += 1
-        merge_bytes = G * n * ((1 + L / 2.0) * (4 * d + 4) + d * e + 4)
+        # partial rows travel in the output's type (bf16 here), their log-sum-exp in fp32
+        merge_bytes = G * n * ((1 + L / 2.0) * (e * d + 4) + d * e + 4)
     dense_flops = G * (4.0 * n * n * d) * (0.5 if w.causal else 1.0)
     return {"attention_flops": flops, "hash_bytes": hash_bytes, "sort_bytes": float(sort_bytes),
             "merge_bytes": merge_bytes, "dense_attention_flops": dense_flops}
@@ -154,7 +155,7 @@ def oracle_sample_plan(w: WL.Workload, leg: str):
     if w.n <= 2048:
         return {"segments": spread(w.G), "rows": None}
     if w.causal:
-        return {"segments": spread(4 if leg == "baseline" else 2), "rows": 8192 if leg == "baseline" else 4096}
+        return {"segments": spread(8 if leg == "baseline" else 2), "rows": 16384 if leg == "baseline" else 4096}
     per_seg_cost = w.n / 32768.0
     k = max(1, int((32 if leg == "baseline" else 4) / per_seg_cost))
     return {"segments": spread(k), "rows": None}

@@ -60,7 +60,7 @@ constexpr float kTileSumLimit = 1099511627776.f;   // 2^40: a tile whose weights
 
 // Optional per-role cycle counters (compile with -DHA_TC_TIMING; never in the shipped build).
 #ifdef HA_TC_TIMING
-__device__ unsigned long long g_tc_timing[32];
+__device__ unsigned long long g_tc_timing[48];
 #define HA_T0(var) const long long var = clock64()
 #define HA_TACC(slot, var) atomicAdd(&g_tc_timing[slot], (unsigned long long)(clock64() - var))
 #define HA_LDECL(name) long long name = 0
@@ -603,7 +603,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
       }
       return true;
     };
-    HA_LDECL(a_tab); HA_LDECL(a_ws); HA_LDECL(a_cmp); HA_LDECL(a_epi); HA_LDECL(a_gq); HA_LDECL(a_bo); HA_LDECL(a_tiles); HA_LDECL(a_ws0); HA_LDECL(a_c1); HA_LDECL(a_c2); HA_LDECL(a_c3); HA_LDECL(a_c4);
+    HA_LDECL(a_tab); HA_LDECL(a_ws); HA_LDECL(a_cmp); HA_LDECL(a_epi); HA_LDECL(a_gq); HA_LDECL(a_bo); HA_LDECL(a_tiles); HA_LDECL(a_ws0); HA_LDECL(a_c1); HA_LDECL(a_c2); HA_LDECL(a_c3); HA_LDECL(a_c4); HA_LDECL(a_e1); HA_LDECL(a_e2); HA_LDECL(a_e3);
     HA_T0(t_role);
     ok = __all_sync(0xffffffffu, gather_q(0));
     for (; ok; ++it) {
@@ -898,9 +898,11 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
           const int crow = lane / LPR, cc = lane % LPR;
           const int lg_pps = f32o ? (RB == 128 ? 1 : 0) : (RB == 128 ? 2 : 1);   // log2(pieces per staging step)
           uint32_t r[16];
+          HA_LACC(a_e1, te);
           tmem_ld16_issue(lane_addr + colO, r);
 #pragma unroll 1
           for (int pc = 0; pc < NP; ++pc) {
+            HA_T0(te2);
             tmem_ld16_wait(r);
             float f[16];
 #pragma unroll
@@ -921,7 +923,9 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
                              "r"(pack2(f[8 * c], f[8 * c + 1])), "r"(pack2(f[8 * c + 2], f[8 * c + 3])),
                              "r"(pack2(f[8 * c + 4], f[8 * c + 5])), "r"(pack2(f[8 * c + 6], f[8 * c + 7])) : "memory");
             }
+            HA_LACC(a_e2, te2);
             if (pin == (1 << lg_pps) - 1) {
+              HA_T0(te3);
               __syncwarp();
               const int step = pc >> lg_pps;
 #pragma unroll
@@ -934,6 +938,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
                 if (roff[k] >= 0) *reinterpret_cast<uint4*>(obase + roff[k] + step * RB + cc * 16) = w;
               }
               __syncwarp();
+              HA_LACC(a_e3, te3);
             }
           }
         }
@@ -956,7 +961,7 @@ __global__ void __launch_bounds__(384, 1) attn_tc_kernel(const __grid_constant__
     if (row == 0 && i == 0) {
       HA_LFLUSH(9, a_tab); HA_LFLUSH(0, a_ws); HA_LFLUSH(2, a_cmp); HA_LFLUSH(15, a_epi); HA_LFLUSH(16, a_gq); HA_LFLUSH(17, a_bo);
       HA_LFLUSH(20, a_tiles); HA_TACC(18, t_role); HA_LFLUSH(19, it);
-      HA_LFLUSH(24, a_ws0); HA_LFLUSH(22, a_c1); HA_LFLUSH(29, a_c2); HA_LFLUSH(30, a_c3); HA_LFLUSH(31, a_c4);
+      HA_LFLUSH(40, a_e1); HA_LFLUSH(41, a_e2); HA_LFLUSH(42, a_e3); HA_LFLUSH(24, a_ws0); HA_LFLUSH(22, a_c1); HA_LFLUSH(29, a_c2); HA_LFLUSH(30, a_c3); HA_LFLUSH(31, a_c4);
     }
 #endif
   } else if (warp < 10) {
@@ -1419,8 +1424,8 @@ extern "C" int hyperattn_test_arm_drop(int on) {
 
 #ifdef HA_TC_TIMING
 extern "C" int hyperattn_debug_tc_timing(unsigned long long* host16, int reset) {
-  if (cudaMemcpyFromSymbol(host16, g_tc_timing, sizeof(unsigned long long) * 32) != cudaSuccess) return -5;
-  if (reset) { unsigned long long z[32] = {0}; cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)); }
+  if (cudaMemcpyFromSymbol(host16, g_tc_timing, sizeof(unsigned long long) * 48) != cudaSuccess) return -5;
+  if (reset) { unsigned long long z[48] = {0}; cudaMemcpyToSymbol(g_tc_timing, z, sizeof(z)); }
   return 0;
 }
 #endif
