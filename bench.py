@@ -40,9 +40,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the attention kernel,
 # from the ncu captures summarised under profiles/ (taken on 4 / 8 heads and scaled to the
 # workload's 32 heads: the traffic is proportional to the number of segments).
-NCU_TRAFFIC_BYTES = {"c3_n131k_causal": 8 * 0.9292e9, "c2_n32k_d128": 4 * 0.2456e9}
+NCU_TRAFFIC_BYTES = {"c3_n131k_causal": 8 * 0.9292e9, "c2_n32k_d128": 4 * 0.2453e9}
 # sm__pipe_tensor_cycles_active (% of peak sustained active) of the attention kernel in the same captures
-NCU_TENSOR_PIPE_PCT = {"c3_n131k_causal": 26.0, "c2_n32k_d128": 27.0}
+NCU_TENSOR_PIPE_PCT = {"c3_n131k_causal": 26.0, "c2_n32k_d128": 27.1}
 
 
 def load_peaks():
