@@ -2,7 +2,7 @@
 // the outputs): a row of the second half of a recursion node adds the estimated row sums
 // D~_21 + D~_C22, so its output is the sum of the partial outputs weighted by their share of
 // the total row sum.  Every row owns one exact-leaf partial and one partial per recursion
-// level at which it sits in a second half.  HBM-bound: reads the fp32 partials once, writes
+// level at which it sits in a second half.  HBM-bound: reads the partials once, writes
 // the final rows once.
 #include <type_traits>
 
@@ -19,105 +19,152 @@ struct MergeArgs {
   int out_fp32;
 };
 
-// EPT consecutive entries of partial row k, starting at column EPT c (one 16-byte load, or 8 bytes for four bf16)
-template <int D, bool PB, int EPT>
-__device__ __forceinline__ void load_part(const void* base, size_t k, int c, float (&x)[EPT]) {
-  if constexpr (PB && EPT == 8) {
-    const uint4 w = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(base) + k * D) + c);
-    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) { x[2 * e] = __uint_as_float(u[e] << 16); x[2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u); }
-  } else if constexpr (PB) {
-    const uint2 w = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(base) + k * D) + c);
-    x[0] = __uint_as_float(w.x << 16); x[1] = __uint_as_float(w.x & 0xffff0000u);
-    x[2] = __uint_as_float(w.y << 16); x[3] = __uint_as_float(w.y & 0xffff0000u);
-  } else {
-    const float4 w = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(base) + k * D) + c);
-    x[0] = w.x; x[1] = w.y; x[2] = w.z; x[3] = w.w;
-  }
-}
-
-// LM: compile-time bound on the recursion depth (the loads of all levels are unrolled); PB: bf16 partials (then every
-// thread owns eight columns, so that its loads stay 16 bytes wide; four for the deepest variant, to bound the registers)
+// LM: compile-time bound on the recursion depth; PB: bf16 partials and results (else fp32).
+// A warp owns 32 consecutive rows.  First lane = row: the row's log-sum-exp values (its leaf partial and one partial
+// per level at which it sits in a second half), its weights and where its partial rows are - once per row.  Then the
+// data: LPR lanes per row, whole rows per warp instruction on every side, the weights and row offsets handed round by
+// shuffles; KB row groups and all their levels are in flight together.  (One thread per 16 bytes of a row doing all
+// of this on its own - the layout before - spent 385 instructions per thread, 56 % of the issue slots, and reached
+// 60 % of the memory bandwidth.)
+// (Occupancy matters more than loads in flight per thread: C3 0.416 ms with four resident CTAs of 64 registers,
+// 0.52 ms with the compiler's 88; d = 128 does best with three and two row groups.)
 template <int D, int LM, bool PB>
-__global__ void __launch_bounds__(256) merge_kernel(MergeArgs a) {
-  constexpr int EPT = (PB && LM <= 8) ? 8 : 4;
-  constexpr int TPR = D / EPT;                     // threads per row
+__global__ void __launch_bounds__(256, LM <= 8 ? (D == 64 ? 4 : 3) : 1) merge_kernel(MergeArgs a) {
+  constexpr int ES = PB ? 2 : 4, RBY = D * ES;     // bytes per element and per row
+  constexpr int LPR = RBY / 16 < 32 ? RBY / 16 : 32;   // lanes per row
+  constexpr int CI = RBY / 16 / LPR;               // 16-byte chunks per lane and row (2 for fp32 rows of d = 128)
+  constexpr int RPS = 32 / LPR;                    // rows per warp instruction
+  constexpr int KB = (CI == 1 && LPR > 8) ? 2 : 1; // row groups in flight together (rows of 128 bytes do best one group at a time)
+  constexpr int NE = 16 / ES;                      // entries per chunk
+  constexpr int LG = LM <= 5 ? LM : 4;             // levels whose rows are in flight together
   const Geometry& g = a.g;
-  // grid: x over the rows of a segment, y = segment
   const int seg = blockIdx.y;
-  const int gt = blockIdx.x * blockDim.x + threadIdx.x;
-  const int i = gt / TPR;
-  const int c = gt % TPR;
-  // (rows are never split between warps - TPR divides 32 - and a warp's rows past the end just idle: the shuffles
-  // below name the row's own lanes only)
-  const bool live = i < g.n;
-  const unsigned rowmask = TPR >= 32 ? 0xffffffffu : (((1u << TPR) - 1u) << ((threadIdx.x & 31) / TPR * TPR));
-  if (!live) return;
-  const size_t row = (size_t)seg * g.n + i;
-  // a node of level `level` has s = leaf << (L - 1 - level) rows, so the row's place in every level follows
+  const int lane = threadIdx.x & 31;
+  const int row0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32;
+  if (row0 >= g.n) return;
+  const int nr = min(32, g.n - row0);              // rows of this warp
+  // ---- lane = row ---------------------------------------------------------------------------------------
+  const int i = row0 + lane;
+  const bool live = lane < nr;
+  // a node of level `level` has s = leaf << (L - 1 - level) rows per half, so the row's place in every level follows
   // from its leaf number by shifts
   const int leaf_no = i / g.leaf;
   const int in_leaf = i - leaf_no * g.leaf;
-  // All loads of a row (its leaf partial and one partial per level at which it sits in a second
-  // half) are issued before any is used: the kernel has nothing to hide their latency behind.
-  float l[LM + 1];
-  float x[LM + 1][EPT];
-  // the row's log-sum-exp values are fetched by one lane each (lane t of the row takes partial t) and passed round
-  float lmine = -INFINITY;
-  if (c == 0) lmine = __ldcs(a.part_lse + row);
-  load_part<D, PB, EPT>(a.part_o, row, c, x[0]);
+  unsigned present = 0;
+  uint32_t off[LM];                                // the row's partial row at a level, counted from the segment's first row of that level
+  float w[LM];
+  float wself = live ? __ldcs(a.part_lse + (size_t)seg * g.n + i) : 0.f;
+  float mx = wself;
 #pragma unroll
   for (int level = 0; level < LM; ++level) {
-    const int sh = g.L - 1 - level;                 // s = leaf << sh
-    l[level + 1] = -INFINITY;
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) x[level + 1][e] = 0.f;
-    if (level < g.L && ((leaf_no >> sh) & 1)) {
-      const int j = leaf_no >> (sh + 1);
-      const int in_node = (leaf_no & ((1 << sh) - 1)) * g.leaf + in_leaf;      // i % s
-      const size_t k = (size_t)g.G * g.n + ((size_t)level * g.G + seg) * g.nl + ((size_t)j << sh) * g.leaf + in_node;
-      if (c == (level + 1) % TPR) lmine = (level + 1 < TPR) ? __ldcs(a.part_lse + k) : lmine;
-      if (level + 1 >= TPR) l[level + 1] = __ldcs(a.part_lse + k);      // (more partials than lanes per row: fetched by every lane)
-      load_part<D, PB, EPT>(a.part_o, k, c, x[level + 1]);
+    w[level] = -INFINITY; off[level] = 0;
+    const int sh = g.L - 1 - level;
+    if (live && level < g.L && ((leaf_no >> sh) & 1)) {
+      present |= 1u << level;
+      off[level] = (uint32_t)(((size_t)(leaf_no >> (sh + 1)) << sh) * g.leaf + (size_t)(leaf_no & ((1 << sh) - 1)) * g.leaf + in_leaf);
+      w[level] = __ldcs(a.part_lse + (size_t)g.G * g.n + ((size_t)level * g.G + seg) * g.nl + off[level]);
+      mx = fmaxf(mx, w[level]);
     }
   }
+  wself = __expf(wself - mx);
+  float tot = wself;
 #pragma unroll
-  for (int t = 0; t <= LM; ++t)
-    if (t < TPR) l[t] = __shfl_sync(rowmask, lmine, (int)((threadIdx.x & 31) / TPR * TPR) + t);
-  float mx = l[0];
-#pragma unroll
-  for (int t = 1; t <= LM; ++t) mx = fmaxf(mx, l[t]);
-  float tot = 0.f;
-#pragma unroll
-  for (int t = 0; t <= LM; ++t) { l[t] = __expf(l[t] - mx); tot += l[t]; }   // exp(-inf) = 0 for the absent ones
+  for (int level = 0; level < LM; ++level) { w[level] = __expf(w[level] - mx); tot += w[level]; }   // exp(-inf) = 0 for the absent ones
   const float inv = 1.f / tot;
-  float acc[EPT];
+  wself *= inv;
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) acc[e] = 0.f;
+  for (int level = 0; level < LM; ++level) w[level] *= inv;
+  if (live) a.lse[(size_t)seg * g.n + i] = mx + __logf(tot);
+  const unsigned any_present = __reduce_or_sync(0xffffffffu, present);
+  // ---- LPR lanes per row ----------------------------------------------------------------------------------
+  const int crow = lane / LPR, cc = lane % LPR;
+  const char* pself = reinterpret_cast<const char*>(a.part_o) + ((size_t)seg * g.n + row0) * RBY + cc * 16;
+  auto unpack = [&](const uint4& v, float (&x)[NE]) {
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-  for (int t = 0; t <= LM; ++t) {
-    const float w = l[t] * inv;
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) acc[e] += w * x[t][e];
-  }
-  if (a.out_fp32) {
-#pragma unroll
-    for (int q4 = 0; q4 < EPT / 4; ++q4)
-      __stcs(reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + row * D + EPT * c) + q4,
-             make_float4(acc[4 * q4], acc[4 * q4 + 1], acc[4 * q4 + 2], acc[4 * q4 + 3]));
-  } else {
-    uint32_t o[EPT / 2];
-#pragma unroll
-    for (int e = 0; e < EPT / 2; ++e) {
-      __nv_bfloat162 t2 = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
-      o[e] = *reinterpret_cast<uint32_t*>(&t2);
+    for (int e = 0; e < 4; ++e) {
+      if (PB) { x[2 * e] = __uint_as_float(u[e] << 16); x[2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u); }
+      else x[e] = __uint_as_float(u[e]);
     }
-    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.out) + row * D + EPT * c;
-    if constexpr (EPT == 8) __stcs(reinterpret_cast<uint4*>(dst), make_uint4(o[0], o[1], o[2], o[3]));
-    else __stcs(reinterpret_cast<uint2*>(dst), make_uint2(o[0], o[1]));
+  };
+  const int oes = (PB || a.out_fp32) ? ES : 2;     // bytes per entry of the results (fp32 partials may end as bf16 rows)
+  char* pout = reinterpret_cast<char*>(a.out) + ((size_t)seg * g.n + row0) * (size_t)(D * oes);
+#pragma unroll 1
+  for (int sb = 0; sb * RPS < nr; sb += KB) {
+#pragma unroll
+    for (int ci = 0; ci < CI; ++ci) {
+      uint4 xs[KB];
+      float acc[KB][NE];
+      int rl[KB];                                    // the row of the warp this lane works on
+#pragma unroll
+      for (int kk = 0; kk < KB; ++kk) {
+        rl[kk] = (sb + kk) * RPS + crow;
+        xs[kk] = rl[kk] < nr ? __ldcs(reinterpret_cast<const uint4*>(pself + (size_t)rl[kk] * RBY + ci * (LPR * 16))) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int l0 = 0; l0 < LM; l0 += LG) {
+        if (l0 > 0 && ((any_present >> l0) & ((1u << LG) - 1u)) == 0) continue;
+        uint4 x[KB][LG];
+        float wl[KB][LG];
+#pragma unroll
+        for (int kk = 0; kk < KB; ++kk) {
+          const unsigned pr = __shfl_sync(0xffffffffu, present, rl[kk] & 31);
+#pragma unroll
+          for (int lv = 0; lv < LG; ++lv) {
+            const int level = l0 + lv;
+            if (level >= LM || !((any_present >> level) & 1u)) continue;
+            wl[kk][lv] = __shfl_sync(0xffffffffu, w[level], rl[kk] & 31);
+            const uint32_t o = __shfl_sync(0xffffffffu, off[level], rl[kk] & 31);
+            x[kk][lv] = make_uint4(0, 0, 0, 0);
+            if (rl[kk] < nr && ((pr >> level) & 1u))
+              x[kk][lv] = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(a.part_o)
+                                 + ((size_t)g.G * g.n + ((size_t)level * g.G + seg) * g.nl + o) * RBY + cc * 16 + ci * (LPR * 16)));
+          }
+        }
+        if (l0 == 0) {
+#pragma unroll
+          for (int kk = 0; kk < KB; ++kk) {
+            const float ws = __shfl_sync(0xffffffffu, wself, rl[kk] & 31);
+            float v[NE];
+            unpack(xs[kk], v);
+#pragma unroll
+            for (int e = 0; e < NE; ++e) acc[kk][e] = ws * v[e];
+          }
+        }
+#pragma unroll
+        for (int kk = 0; kk < KB; ++kk) {
+#pragma unroll
+          for (int lv = 0; lv < LG; ++lv) {
+            const int level = l0 + lv;
+            if (level >= LM || !((any_present >> level) & 1u)) continue;
+            float v[NE];
+            unpack(x[kk][lv], v);
+#pragma unroll
+            for (int e = 0; e < NE; ++e) acc[kk][e] = fmaf(wl[kk][lv], v[e], acc[kk][e]);
+          }
+        }
+      }
+#pragma unroll
+      for (int kk = 0; kk < KB; ++kk) {
+        if (rl[kk] >= nr) continue;
+        char* dst = pout + ((size_t)rl[kk] * D + (size_t)(ci * LPR + cc) * NE) * oes;
+        if (PB) {
+          uint32_t q[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 t2 = __floats2bfloat162_rn(acc[kk][2 * e], acc[kk][2 * e + 1]);
+            q[e] = *reinterpret_cast<uint32_t*>(&t2);
+          }
+          __stcs(reinterpret_cast<uint4*>(dst), make_uint4(q[0], q[1], q[2], q[3]));
+        } else if (a.out_fp32) {
+          __stcs(reinterpret_cast<float4*>(dst), make_float4(acc[kk][0], acc[kk][1], acc[kk][2], acc[kk][3]));
+        } else {
+          __nv_bfloat162 t0 = __floats2bfloat162_rn(acc[kk][0], acc[kk][1]), t1 = __floats2bfloat162_rn(acc[kk][2], acc[kk][3]);
+          __stcs(reinterpret_cast<uint2*>(dst), make_uint2(*reinterpret_cast<uint32_t*>(&t0), *reinterpret_cast<uint32_t*>(&t1)));
+        }
+      }
+    }
   }
-  if (c == 0) a.lse[row] = mx + __logf(tot);
 }
 
 }  // namespace
@@ -125,9 +172,9 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs a) {
 cudaError_t launch_merge(const Geometry& g, const Workspace& ws, void* out, float* lse, int out_fp32,
                          cudaStream_t st) {
   MergeArgs a; a.part_o = ws.part_o; a.part_lse = ws.part_lse; a.out = out; a.lse = lse; a.g = g; a.out_fp32 = out_fp32;
-  const int ept = (ws.part_bf16 && g.L <= 8) ? 8 : 4;                   // columns per thread (see the kernel)
-  const size_t threads = (size_t)g.n * (g.d / ept);
-  const dim3 blocks((unsigned)((threads + 255) / 256), (unsigned)g.G);
+  if (ws.part_bf16 && out_fp32) return cudaErrorInvalidValue;                   // bf16 partials are only kept for bf16 results
+  const size_t warps = ((size_t)g.n + 31) / 32;                                 // a warp per 32 rows
+  const dim3 blocks((unsigned)((warps + 7) / 8), (unsigned)g.G);
   if (g.G > 65535) return cudaErrorInvalidValue;
   auto go = [&](auto kernel) { kernel<<<blocks, 256, 0, st>>>(a); };
   auto pick = [&](auto dtag, auto pbtag) {
