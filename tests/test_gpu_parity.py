@@ -121,6 +121,19 @@ def test_precise_mode_matches_on_gaussian_inputs(d, causal):
     assert s1["mean_abs"] < 0.25 * s0["mean_abs"]
 
 
+@pytest.mark.parametrize("dtype,out_dtype,d", [("bf16", None, 64), ("bf16", None, 128), ("bf16", torch.float32, 128),
+                                               ("fp32", torch.bfloat16, 64), ("fp32", torch.float32, 128)])
+def test_causal_merge_in_every_pair_of_partial_and_output_types(dtype, out_dtype, d):
+    """The merge of the causal recursion keeps partial rows as bf16 for bf16 inputs and outputs and as fp32 otherwise, and
+    writes bf16 or fp32 rows; n and the leaf size (1237) are odd, so the 32 rows a warp owns straddle leaves, whose rows
+    sit in second halves at different levels."""
+    w = W("merge_types", 1, 2, 4948, d, dtype, 64, 32, 6, True, 1300, seed=70 + d)
+    (out, lse, inter), (Q64, K64, V64) = run(w, out_dtype=out_dtype)
+    assert out.dtype == (out_dtype or torch.bfloat16)
+    assert len(PU.levels_of(w)) >= 2
+    PU.check_outputs(w, Q64, K64, V64, out, lse, inter)
+
+
 def test_bf16_output_and_caller_workspace():
     w = SMALL[1]
     nbytes = ha.workspace_bytes(w.B, w.H, w.n, w.d, w.b, w.m, w.r, w.causal, w.n0)
