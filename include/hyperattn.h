@@ -198,7 +198,7 @@ int hyperattn_forward_ex(const hyperattn_params* p);
 
 /* The same computation for HOST buffers: q, k, v, out, lse of *p are host pointers (pinned
  * memory makes the copies asynchronous).  The (batch, head) segments are independent, so they
- * go through a private device staging area in up to eight groups: the copy of the next group to
+ * go through a private device staging area in up to sixteen groups: the copy of the next group to
  * the device and the copy of the previous group's out / lse back run on two streams of the
  * library while a group is computed on `stream`.  Everything is ordered after the work already
  * queued on `stream`, and `stream` is made to wait for the last copy back: the caller

@@ -148,7 +148,7 @@ void make_directions(int d, int r, uint64_t seed, float* w, uint32_t node = 0) {
 }
 
 // ---- per-process state ---------------------------------------------------------------------
-constexpr int kHostChunks = 8;          // the host-buffer entry point pipelines copies and compute over this many groups of segments
+constexpr int kHostChunks = 16;          // the host-buffer entry point pipelines copies and compute over this many groups of segments
 struct DeviceState {
   void* ws = nullptr; size_t ws_bytes = 0;
   void* host_stage = nullptr; size_t host_stage_bytes = 0;   // device staging for the host-buffer entry
