@@ -53,7 +53,9 @@ def check(w):
     arrs = WL.make_inputs(w)
     q, k, v = PU.to_device(w, arrs)
     precise, bound = PU.output_policy(w, arrs)
-    out, lse, inter = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, out_dtype=torch.float32, debug=True,
+    # every third draw asks for bf16 results (for bf16 inputs that also makes the partial rows of the causal recursion bf16)
+    out_dtype = None if (w.seed % 3 == 0 and not precise) else torch.float32
+    out, lse, inter = ha.forward(q, k, v, w.b, w.m, w.r, causal=w.causal, n0=w.n0, seed=w.seed, out_dtype=out_dtype, debug=True,
                                  precise=precise)
     torch.cuda.synchronize()
     assert ha.last_device_status() == 0
