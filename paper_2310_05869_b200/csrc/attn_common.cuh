@@ -80,9 +80,11 @@ __device__ __forceinline__ TileDesc decode_tile(const AttnArgs& a, int tile) {
   TileDesc t;
   t.partial = !a.direct;
   if (tile < a.n_leaf_tiles) {
-    const int per = g.G * a.leaves_per_seg;
-    const int tt = a.tiles_per_leaf - 1 - tile / per;      // heavy tiles first
-    const int rem = tile % per;
+    // leaf after leaf, the tiles of a leaf from the heaviest (last rows, most keys) to the lightest: the CTAs that run
+    // at the same time work on a handful of neighbouring leaves, whose K / V rows - and, in the backward pass, whose
+    // dK / dV accumulator rows, which every query tile of the leaf adds to - then stay in L2
+    const int tt = a.tiles_per_leaf - 1 - tile % a.tiles_per_leaf;
+    const int rem = tile / a.tiles_per_leaf;
     t.seg = rem / a.leaves_per_seg;
     const int leaf = rem % a.leaves_per_seg;
     t.mode = 0;
